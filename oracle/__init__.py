@@ -1,0 +1,161 @@
+"""ctypes front end of the CPU oracle (oracle/rago_oracle.cpp).
+
+TEST INFRASTRUCTURE ONLY: imported by tests/, by the smoke check and by the
+benchmark's cpu_baseline / reference arm.  The product package never imports
+this module, and this module never imports the product package.
+
+Inputs and outputs are numpy arrays (bf16 data travels as uint16 bit
+patterns).  `build()` compiles the shared object with g++ when it is missing
+or older than its source.
+"""
+
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "rago_oracle.cpp")
+_LIB = os.path.join(_HERE, "librago_oracle.so")
+_lib = None
+
+L2, IP = 0, 1
+_METRIC = {"l2": L2, "ip": IP, L2: L2, IP: IP}
+
+
+def build(force: bool = False) -> str:
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["g++", "-O2", "-std=c++17", "-fPIC", "-shared", "-pthread", "-o", _LIB, _SRC]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        build()
+        _lib = ctypes.CDLL(_LIB)
+    return _lib
+
+
+def _p(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _c(a, dtype):
+    a = np.ascontiguousarray(a, dtype=dtype)
+    return a
+
+
+def default_threads() -> int:
+    try:
+        return max(1, len(os.sched_getaffinity(0)))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+class Index:
+    """Borrowed views of an IVF-PQ index in host memory."""
+
+    def __init__(self, centroids, codebooks, codes, list_offsets, ids, metric, coarse_bf16=False):
+        self.coarse_bf16 = bool(coarse_bf16)
+        self.centroids = _c(centroids, np.uint16 if coarse_bf16 else np.float32)
+        self.codebooks = _c(codebooks, np.float32)
+        self.codes = _c(codes, np.uint8)
+        self.offsets = _c(list_offsets, np.int64)
+        self.ids = _c(ids, np.int64)
+        self.metric = _METRIC[metric]
+        self.nlist, self.d = self.centroids.shape
+        self.M = self.codebooks.shape[0]
+        assert self.codebooks.shape == (self.M, 256, self.d // self.M)
+        self.N = int(self.offsets[-1])
+        assert self.codes.shape == (self.N, self.M) and self.ids.shape == (self.N,)
+
+    def _head(self):
+        return (_p(self.centroids), ctypes.c_int(self.coarse_bf16), _p(self.codebooks), _p(self.codes))
+
+
+def coarse(centroids, queries, nprobe, metric, coarse_bf16=False, nthreads=1):
+    cen = _c(centroids, np.uint16 if coarse_bf16 else np.float32)
+    q = _c(queries, np.float32)
+    nq, d = q.shape
+    lists = np.empty((nq, nprobe), np.int32)
+    scores = np.empty((nq, nprobe), np.float64)
+    rc = lib().oracle_coarse(_p(cen), ctypes.c_int(bool(coarse_bf16)), d, cen.shape[0], _METRIC[metric], _p(q), nq,
+                             nprobe, _p(lists), _p(scores), nthreads)
+    if rc:
+        raise ValueError("oracle_coarse: bad arguments")
+    return lists, scores
+
+
+def ivfpq_search(ix: Index, queries, nprobe, k, nthreads=1, want_probes=False):
+    q = _c(queries, np.float32)
+    nq = q.shape[0]
+    ids = np.empty((nq, k), np.int64)
+    dists = np.empty((nq, k), np.float32)
+    probes = np.empty((nq, nprobe), np.int32) if want_probes else None
+    rc = lib().oracle_ivfpq_search(*ix._head(), _p(ix.offsets), _p(ix.ids), ctypes.c_int64(ix.N), ix.d, ix.nlist,
+                                   ix.M, ix.metric, _p(q), nq, nprobe, k, _p(ids), _p(dists), _p(probes), nthreads)
+    if rc:
+        raise ValueError("oracle_ivfpq_search: bad arguments")
+    return (ids, dists, probes) if want_probes else (ids, dists)
+
+
+def adc_score(ix: Index, query, list_no, pos) -> float:
+    q = _c(query, np.float32)
+    out = ctypes.c_double()
+    rc = lib().oracle_adc_score(*ix._head(), ix.d, ix.nlist, ix.M, ix.metric, _p(q), int(list_no),
+                                ctypes.c_int64(int(pos)), ctypes.byref(out))
+    if rc:
+        raise ValueError("oracle_adc_score: bad arguments")
+    return out.value
+
+
+def decode_score(ix: Index, query, list_no, pos, want_decoded=False):
+    q = _c(query, np.float32)
+    out = ctypes.c_double()
+    dec = np.empty(ix.d, np.float64) if want_decoded else None
+    rc = lib().oracle_decode_score(*ix._head(), ix.d, ix.nlist, ix.M, ix.metric, _p(q), int(list_no),
+                                   ctypes.c_int64(int(pos)), ctypes.byref(out), _p(dec))
+    if rc:
+        raise ValueError("oracle_decode_score: bad arguments")
+    return (out.value, dec) if want_decoded else out.value
+
+
+def flat_search(db_bits, query_bits, k, nthreads=1):
+    db = _c(db_bits, np.uint16)
+    q = _c(query_bits, np.uint16)
+    nq, d = q.shape
+    ids = np.empty((nq, k), np.int64)
+    sc = np.empty((nq, k), np.float32)
+    rc = lib().oracle_flat_search(_p(db), ctypes.c_int64(db.shape[0]), d, _p(q), nq, k, _p(ids), _p(sc), nthreads)
+    if rc:
+        raise ValueError("oracle_flat_search: bad arguments")
+    return ids, sc
+
+
+def flat_scores(db_bits, query_bits, rows):
+    db = _c(db_bits, np.uint16)
+    q = _c(query_bits, np.uint16)
+    rows = _c(rows, np.int64)
+    out = np.empty(rows.shape[0], np.float64)
+    lib().oracle_flat_scores(_p(db), db.shape[1], _p(q), _p(rows), rows.shape[0], _p(out))
+    return out
+
+
+def f32_to_bf16_bits(x):
+    x = _c(x, np.float32)
+    out = np.empty(x.shape, np.uint16)
+    lib().oracle_f32_to_bf16(_p(x), _p(out), ctypes.c_int64(x.size))
+    return out
+
+
+def locate(ix: Index, ident: int):
+    """(list, position) of the vector with id `ident` (linear search; small inputs only)."""
+    pos = int(np.nonzero(ix.ids == ident)[0][0])
+    lst = int(np.searchsorted(ix.offsets, pos, side="right") - 1)
+    return lst, pos

@@ -1,0 +1,51 @@
+"""Shared test helpers: tolerant comparison of result lists and host views of synthetic data."""
+
+import numpy as np
+import torch
+
+
+def host_index(oracle, data):
+    """oracle.Index over the CPU copies of a synth.IvfPqData."""
+    cen = data.centroids
+    if cen.dtype == torch.bfloat16:
+        cen_h = cen.cpu().view(torch.uint16).numpy()
+    else:
+        cen_h = cen.cpu().numpy()
+    return oracle.Index(cen_h, data.codebooks.cpu().numpy(), data.codes.cpu().numpy(),
+                        data.list_offsets.cpu().numpy(), data.ids.cpu().numpy(), data.metric,
+                        coarse_bf16=cen.dtype == torch.bfloat16)
+
+
+def match_results(ids_a, d_a, ids_o, d_o, rel=1e-4, floor=1e-6):
+    """Compare one query's result list (a) with the oracle's (o).
+
+    Distances must agree position by position within `rel` (relative, with an
+    absolute floor); ids must be equal except inside groups of oracle
+    distances that tie within the same tolerance, where any order and any
+    member of the tie group at the list's tail is accepted.
+    Returns a list of problems (empty = match).
+    """
+    problems = []
+    k = len(ids_o)
+    scale = max(floor, float(np.max(np.abs(d_o[np.isfinite(d_o)]))) if np.isfinite(d_o).any() else floor)
+    for t in range(k):
+        if np.isinf(d_o[t]) or np.isinf(d_a[t]):
+            if not (d_o[t] == d_a[t] and ids_a[t] == ids_o[t]):
+                problems.append((t, "pad", int(ids_a[t]), float(d_a[t]), int(ids_o[t]), float(d_o[t])))
+            continue
+        tol = rel * max(abs(float(d_o[t])), floor * scale)
+        if abs(float(d_a[t]) - float(d_o[t])) > tol:
+            problems.append((t, "dist", int(ids_a[t]), float(d_a[t]), int(ids_o[t]), float(d_o[t])))
+            continue
+        if ids_a[t] != ids_o[t]:
+            # accept when the oracle has this id at a position whose distance ties with position t,
+            # or when position t ties with the last oracle entry (tie group cut by k)
+            where = np.nonzero(ids_o == ids_a[t])[0]
+            ok = False
+            if where.size and abs(float(d_o[where[0]]) - float(d_o[t])) <= 2 * tol:
+                ok = True
+            elif not where.size and abs(float(d_o[k - 1]) - float(d_o[t])) <= 2 * tol:
+                ok = True
+            if not ok:
+                problems.append((t, "id", int(ids_a[t]), float(d_a[t]), int(ids_o[t]), float(d_o[t])))
+    return problems
