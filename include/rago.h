@@ -1,0 +1,170 @@
+/*
+ * rago.h -- C ABI of the B200 (sm_100a) retrieval library.
+ *
+ * The library implements the retrieval stage that retrieval-augmented generation adds to LLM
+ * serving, as the RAGO paper states it (Background, "Vector search for retrieval"): return the K
+ * database vectors most similar to a D-dimensional query under L2 distance or cosine / inner
+ * product, either approximately with IVF-PQ (an inverted file over product-quantised vectors,
+ * one byte per sub-space) or exactly by brute force for small databases (case study II).  The
+ * paper's cost model for the stage is the number of bytes of quantised vectors scanned per query
+ * (RAGSchema section, "Retrieval component").
+ *
+ * Conventions for every call
+ *   - "dev" pointers are CUDA device pointers in the current device's address space; "host"
+ *     pointers are ordinary host memory.  Nothing here takes or returns a framework type.
+ *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL = default stream)
+ *     and the call returns without synchronising, unless stated otherwise.
+ *   - The caller owns every buffer it passes.  An index BORROWS its arrays: they must stay valid
+ *     and unchanged until rago_index_free.  Scratch memory is caller-provided ("workspace"); the
+ *     search calls allocate nothing.
+ *   - Errors are return codes.  Argument errors are found on the host before anything is
+ *     launched.  rago_last_error() returns a thread-local description of the last failure.
+ *   - L2 means SQUARED Euclidean distance, smaller is better, results ascending.  IP means inner
+ *     product, larger is better, results descending.  Missing results (fewer than k candidates)
+ *     are id -1 with +INFINITY (L2) or -INFINITY (IP).
+ *   - 8-bit product quantisation only (256 codewords per sub-space).
+ */
+#ifndef RAGO_H
+#define RAGO_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct rago_index rago_index; /* opaque */
+
+typedef enum {
+    RAGO_OK = 0,
+    RAGO_EINVAL = 1,       /* null pointer, non-positive size, k or nprobe out of range, bad offsets */
+    RAGO_EALIGN = 2,       /* a pointer is not aligned as documented */
+    RAGO_EUNSUPPORTED = 3, /* shape outside the supported envelope (see rago_index_load) */
+    RAGO_ENOMEM = 4,       /* workspace too small, or an allocation at index load failed */
+    RAGO_ECUDA = 5,        /* a CUDA runtime call failed */
+    RAGO_ETIMEOUT = 6      /* a bounded device-side wait expired (reported by rago_check) */
+} rago_status;
+
+typedef enum { RAGO_L2 = 0, RAGO_IP = 1 } rago_metric;
+typedef enum { RAGO_F32 = 0, RAGO_BF16 = 1 } rago_dtype;
+
+/* Number of per-stage timings rago_profile_read returns:
+ * 0 coarse distances, 1 probe selection, 2 work planning, 3 table build + scan, 4 merge. */
+#define RAGO_NUM_STAGES 5
+
+/*
+ * Build a search handle over an IVF-PQ index that already lives in device memory
+ * (IVF-PQ: Background, "Vector search for retrieval"; storage is the usual inverted file:
+ * vectors of one list stored contiguously, lists addressed by offsets).
+ *
+ *   coarse_centroids  dev [nlist][d], row-major, RAGO_F32 or RAGO_BF16 (16-byte aligned)
+ *   pq_codebooks      dev [M][256][d/M] fp32: codeword j of sub-space m
+ *   codes             dev [N][M] uint8, 16-byte aligned; vectors of list l occupy rows
+ *                     list_offsets[l] .. list_offsets[l+1]-1.  A code quantises the RESIDUAL
+ *                     (vector - its list's centroid); one codebook set serves all lists.
+ *   list_offsets      dev [nlist+1] int64, offsets[0]=0, non-decreasing, offsets[nlist]=N
+ *   ids               dev [N] int64, caller-chosen ids reported in results
+ *   N, d, nlist, M    sizes; d % M == 0
+ *   metric            RAGO_L2 or RAGO_IP.  For IP the score of a vector is
+ *                     <q, centroid> + sum over sub-spaces of <q_m, codeword>.
+ *
+ * Supported envelope: M a multiple of 16 with M <= 192 and M not in {112, 144, 176};
+ * d <= 4096; N < 2^32; nlist < 2^31.  Anything else returns RAGO_EUNSUPPORTED.
+ *
+ * This call synchronises: it copies list_offsets to the host to validate them, allocates the
+ * small derived arrays the library owns (centroid norms, a transposed codebook) and fills them.
+ * On success *out receives the handle.
+ */
+rago_status rago_index_load(rago_index** out, const void* coarse_centroids, rago_dtype coarse_dtype,
+                            const float* pq_codebooks, const uint8_t* codes, const int64_t* list_offsets,
+                            const int64_t* ids, int64_t N, int32_t d, int32_t nlist, int32_t M,
+                            rago_metric metric, void* cuda_stream);
+
+/* Release the handle and the arrays the library allocated for it (never the borrowed ones).
+ * Synchronises the device first.  NULL is accepted. */
+rago_status rago_index_free(rago_index* index);
+
+/* Bytes of device scratch rago_search / rago_search_probes / rago_search_host need for a batch
+ * of up to nq queries with these nprobe and k (1 <= nprobe <= nlist, 1 <= k <= 1024). */
+rago_status rago_search_workspace_bytes(const rago_index* index, int32_t nq, int32_t nprobe, int32_t k,
+                                        size_t* out_bytes);
+
+/*
+ * Batched IVF-PQ search (the whole hot path): coarse query-to-centroid distances with nprobe
+ * selection, per-(query, list) lookup tables, table-sum scan of the probed lists, k best.
+ *
+ *   queries    dev [nq][d] fp32, 16-byte aligned
+ *   out_ids    dev [nq][k] int64, best first
+ *   out_dists  dev [nq][k] fp32: squared L2 distance, or inner-product score
+ *   workspace  dev, 256-byte aligned, at least rago_search_workspace_bytes(...) bytes; contents
+ *              are scratch.  Two searches that overlap on the GPU need distinct workspaces.
+ *
+ * With a RAGO_BF16 coarse quantiser the query is rounded to bf16 (nearest-even) for the coarse
+ * step only; tables are built from the fp32 query.  Ties are broken by storage position.
+ * nq == 0 is a no-op.
+ */
+rago_status rago_search(const rago_index* index, const float* queries, int32_t nq, int32_t nprobe, int32_t k,
+                        int64_t* out_ids, float* out_dists, void* workspace, size_t workspace_bytes,
+                        void* cuda_stream);
+
+/*
+ * The coarse step alone (test hook for the first stage of rago_search).
+ *   out_lists   dev [nq][nprobe] int32 list numbers, best first
+ *   out_coarse  dev [nq][nprobe] fp32: squared L2 distance to the centroid, or <q, centroid>
+ */
+rago_status rago_search_probes(const rago_index* index, const float* queries, int32_t nq, int32_t nprobe,
+                               int32_t* out_lists, float* out_coarse, void* workspace, size_t workspace_bytes,
+                               void* cuda_stream);
+
+/*
+ * rago_search for callers whose queries and results live in HOST memory: copies the queries to
+ * the device, searches, copies ids and distances back, all on `cuda_stream`, then synchronises
+ * that stream.  `workspace` must be 256-byte aligned and hold
+ * rago_search_workspace_bytes(...) + rago_host_staging_bytes(...) bytes.  Pinned host buffers
+ * make the copies asynchronous; pageable ones work too.
+ */
+rago_status rago_search_host(const rago_index* index, const float* host_queries, int32_t nq, int32_t nprobe,
+                             int32_t k, int64_t* host_out_ids, float* host_out_dists, void* workspace,
+                             size_t workspace_bytes, void* cuda_stream);
+rago_status rago_host_staging_bytes(const rago_index* index, int32_t nq, int32_t k, size_t* out_bytes);
+
+/*
+ * Exact (brute-force) search for small databases: score = <q, y_i> over bf16 inputs with fp32
+ * accumulation, k largest, best first.  For cosine similarity pass unit-norm rows and queries.
+ *
+ *   db          dev [N][d] bf16 row-major, 16-byte aligned; d a multiple of 64, d <= 4096
+ *   queries     dev [nq][d] bf16, 16-byte aligned
+ *   out_ids     dev [nq][k] int64 row numbers; out_scores dev [nq][k] fp32
+ *   workspace   dev, 256-byte aligned, rago_flat_workspace_bytes(...) bytes
+ *   1 <= k <= 1024, N < 2^32.
+ */
+rago_status rago_flat_search(const void* db, int64_t N, int32_t d, const void* queries, int32_t nq, int32_t k,
+                             int64_t* out_ids, float* out_scores, void* workspace, size_t workspace_bytes,
+                             void* cuda_stream);
+rago_status rago_flat_workspace_bytes(int64_t N, int32_t d, int32_t nq, int32_t k, size_t* out_bytes);
+
+/*
+ * Synchronise `cuda_stream` and report whether any kernel launched through `workspace` since
+ * the last check recorded a device-side error (RAGO_ETIMEOUT: a bounded wait on a copy or on the
+ * tensor pipe gave up; the results of that call are then undefined).  Device waits never spin
+ * without a limit.
+ */
+rago_status rago_check(void* workspace, void* cuda_stream);
+
+/* Per-stage device timings of rago_search.  When enabled, rago_search records CUDA events on the
+ * caller's stream around each stage; rago_profile_read synchronises and returns the last call's
+ * stage times in milliseconds (out_ms[RAGO_NUM_STAGES]). */
+rago_status rago_profile_enable(rago_index* index, int32_t enable);
+rago_status rago_profile_read(rago_index* index, float* out_ms);
+
+/* Number of kernels the library has launched in this process since it was loaded. */
+int64_t rago_kernel_launches(void);
+
+/* Description of the calling thread's last error ("" if none).  Static storage. */
+const char* rago_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RAGO_H */

@@ -1,0 +1,357 @@
+// C ABI of the retrieval library: argument checks, workspace layout, stage launches.
+#include <atomic>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+
+namespace rago {
+
+static std::atomic<long long> g_launches{0};
+static thread_local char g_err[512] = "";
+
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+void set_error(const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+}
+
+static rago_status fail(rago_status st, const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return st;
+}
+
+static rago_status cuda_fail(cudaError_t e, const char* what) {
+    return fail(RAGO_ECUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+static bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+// Workspace carving.  Every region starts on a 256-byte boundary; the first 256 bytes hold the
+// device error word.
+struct Layout {
+    size_t err, probe_list, probe_term, scores, pair_tiles, work_prefix, qthresh, slot_cnt, slot_keys, total;
+    size_t nslots;
+};
+
+static Layout make_layout(const IndexImpl* ix, int nq, int nprobe, int k) {
+    Layout L;
+    size_t o = 0;
+    auto take = [&](size_t bytes) {
+        const size_t at = o;
+        o += align_up(bytes ? bytes : 1, 256);
+        return at;
+    };
+    const size_t npairs = (size_t)nq * nprobe;
+    L.nslots = npairs + (size_t)ix->plan.ctas;
+    L.err = take(256);
+    L.probe_list = take(npairs * 4);
+    L.probe_term = take(npairs * 4);
+    L.scores = take((size_t)nq * ix->nlist * 4);
+    L.pair_tiles = take(npairs * 4);
+    L.work_prefix = take((npairs + 1) * 8);
+    L.qthresh = take((size_t)nq * 8);
+    L.slot_cnt = take(L.nslots * 4);
+    L.slot_keys = take(L.nslots * (size_t)k * 8);
+    L.total = o;
+    return L;
+}
+
+static rago_status check_search_args(const IndexImpl* ix, int nq, int nprobe, int k) {
+    if (!ix) return fail(RAGO_EINVAL, "index is null");
+    if (nq < 0) return fail(RAGO_EINVAL, "nq = %d is negative", nq);
+    if (nprobe < 1 || nprobe > ix->nlist) return fail(RAGO_EINVAL, "nprobe = %d outside [1, nlist = %d]", nprobe, ix->nlist);
+    if (nprobe > MAX_K) return fail(RAGO_EUNSUPPORTED, "nprobe = %d exceeds %d", nprobe, MAX_K);
+    if (k < 1) return fail(RAGO_EINVAL, "k = %d must be at least 1", k);
+    if (k > MAX_K) return fail(RAGO_EUNSUPPORTED, "k = %d exceeds %d", k, MAX_K);
+    if ((long long)nq * nprobe > 0x7fffffffLL - 4096) return fail(RAGO_EUNSUPPORTED, "nq * nprobe too large");
+    return RAGO_OK;
+}
+
+static void record(IndexImpl* ix, int i, cudaStream_t s) {
+    if (ix->profile) cudaEventRecord(ix->ev[i], s);
+}
+
+static rago_status run_coarse(const IndexImpl* ix, const float* queries, int nq, int nprobe, uint8_t* ws,
+                              const Layout& L, cudaStream_t s) {
+    IndexImpl* mix = const_cast<IndexImpl*>(ix);
+    cudaError_t e;
+    record(mix, 0, s);
+    e = launch_coarse_scores(ix, queries, nq, reinterpret_cast<float*>(ws + L.scores), s);
+    if (e != cudaSuccess) return cuda_fail(e, "coarse score kernel");
+    record(mix, 1, s);
+    e = launch_select_probes(ix, queries, reinterpret_cast<float*>(ws + L.scores), nq, nprobe,
+                             reinterpret_cast<int32_t*>(ws + L.probe_list),
+                             reinterpret_cast<float*>(ws + L.probe_term), s);
+    if (e != cudaSuccess) return cuda_fail(e, "probe selection kernel");
+    record(mix, 2, s);
+    return RAGO_OK;
+}
+
+}  // namespace rago
+
+using namespace rago;
+
+extern "C" {
+
+const char* rago_last_error(void) { return g_err; }
+int64_t rago_kernel_launches(void) { return g_launches.load(); }
+
+rago_status rago_index_load(rago_index** out, const void* coarse_centroids, rago_dtype coarse_dtype,
+                            const float* pq_codebooks, const uint8_t* codes, const int64_t* list_offsets,
+                            const int64_t* ids, int64_t N, int32_t d, int32_t nlist, int32_t M, rago_metric metric,
+                            void* cuda_stream) {
+    if (!out) return fail(RAGO_EINVAL, "out is null");
+    *out = nullptr;
+    if (!coarse_centroids || !pq_codebooks || !list_offsets) return fail(RAGO_EINVAL, "null index array");
+    if (N < 0 || d <= 0 || nlist <= 0 || M <= 0) return fail(RAGO_EINVAL, "sizes must be positive");
+    if (N > 0 && (!codes || !ids)) return fail(RAGO_EINVAL, "codes / ids are null but N > 0");
+    if (metric != RAGO_L2 && metric != RAGO_IP) return fail(RAGO_EINVAL, "unknown metric %d", (int)metric);
+    if (coarse_dtype != RAGO_F32 && coarse_dtype != RAGO_BF16) return fail(RAGO_EINVAL, "unknown coarse dtype");
+    if (d % M != 0) return fail(RAGO_EINVAL, "d = %d is not a multiple of M = %d", d, M);
+    if (!scan_supported(M)) return fail(RAGO_EUNSUPPORTED, "M = %d: supported sub-space counts are 16,32,48,64,80,96,128", M);
+    if (d > 4096) return fail(RAGO_EUNSUPPORTED, "d = %d exceeds 4096", d);
+    if (N >= (1LL << 32)) return fail(RAGO_EUNSUPPORTED, "N = %lld needs more than 32-bit positions", (long long)N);
+    if (!aligned(coarse_centroids, 16) || !aligned(pq_codebooks, 16) || !aligned(codes, 16) ||
+        !aligned(list_offsets, 8) || !aligned(ids, 8))
+        return fail(RAGO_EALIGN, "index arrays must be 16-byte aligned (offsets and ids 8-byte)");
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+
+    std::vector<int64_t> off((size_t)nlist + 1);
+    cudaError_t e = cudaMemcpyAsync(off.data(), list_offsets, off.size() * 8, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return cuda_fail(e, "reading list_offsets");
+    if (off[0] != 0 || off[nlist] != N) return fail(RAGO_EINVAL, "list_offsets must start at 0 and end at N");
+    for (int l = 0; l < nlist; ++l)
+        if (off[l + 1] < off[l]) return fail(RAGO_EINVAL, "list_offsets decrease at list %d", l);
+
+    IndexImpl* ix = new (std::nothrow) IndexImpl();
+    if (!ix) return fail(RAGO_ENOMEM, "host allocation failed");
+    std::memset(ix, 0, sizeof(*ix));
+    ix->centroids = coarse_centroids;
+    ix->coarse_bf16 = coarse_dtype == RAGO_BF16;
+    ix->codebooks = pq_codebooks;
+    ix->codes = codes;
+    ix->list_offsets = list_offsets;
+    ix->ids = ids;
+    ix->N = N; ix->d = d; ix->nlist = nlist; ix->M = M; ix->dsub = d / M; ix->metric = metric;
+    e = cudaGetDevice(&ix->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ix->num_sms, cudaDevAttrMultiProcessorCount, ix->device);
+    if (e == cudaSuccess) e = cudaMalloc(&ix->cnorm, (size_t)nlist * 4);
+    if (e == cudaSuccess) e = cudaMalloc(&ix->cbT, (size_t)KSUB * d * 4);
+    if (e != cudaSuccess) {
+        rago_status st = e == cudaErrorMemoryAllocation ? fail(RAGO_ENOMEM, "device allocation failed")
+                                                         : cuda_fail(e, "index setup");
+        rago_index_free(reinterpret_cast<rago_index*>(ix));
+        return st;
+    }
+    for (int i = 0; i <= RAGO_NUM_STAGES && e == cudaSuccess; ++i) e = cudaEventCreate(&ix->ev[i]);
+    if (e == cudaSuccess) { ix->ev_valid = 1; e = scan_plan(ix, &ix->plan); }
+    if (e == cudaSuccess) e = launch_centroid_norms(coarse_centroids, ix->coarse_bf16, nlist, d, ix->cnorm, s);
+    if (e == cudaSuccess) e = launch_transpose_codebook(pq_codebooks, M, ix->dsub, ix->cbT, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) {
+        rago_status st = cuda_fail(e, "index setup kernels");
+        rago_index_free(reinterpret_cast<rago_index*>(ix));
+        return st;
+    }
+    *out = reinterpret_cast<rago_index*>(ix);
+    return RAGO_OK;
+}
+
+rago_status rago_index_free(rago_index* index) {
+    if (!index) return RAGO_OK;
+    IndexImpl* ix = reinterpret_cast<IndexImpl*>(index);
+    cudaDeviceSynchronize();
+    if (ix->cnorm) cudaFree(ix->cnorm);
+    if (ix->cbT) cudaFree(ix->cbT);
+    if (ix->ev_valid)
+        for (int i = 0; i <= RAGO_NUM_STAGES; ++i) cudaEventDestroy(ix->ev[i]);
+    delete ix;
+    return RAGO_OK;
+}
+
+rago_status rago_search_workspace_bytes(const rago_index* index, int32_t nq, int32_t nprobe, int32_t k,
+                                        size_t* out_bytes) {
+    const IndexImpl* ix = reinterpret_cast<const IndexImpl*>(index);
+    if (!out_bytes) return fail(RAGO_EINVAL, "out_bytes is null");
+    rago_status st = check_search_args(ix, nq, nprobe, k);
+    if (st != RAGO_OK) return st;
+    *out_bytes = make_layout(ix, nq, nprobe, k).total;
+    return RAGO_OK;
+}
+
+rago_status rago_host_staging_bytes(const rago_index* index, int32_t nq, int32_t k, size_t* out_bytes) {
+    const IndexImpl* ix = reinterpret_cast<const IndexImpl*>(index);
+    if (!ix || !out_bytes || nq < 0 || k < 1) return fail(RAGO_EINVAL, "bad arguments");
+    *out_bytes = align_up((size_t)nq * ix->d * 4, 256) + align_up((size_t)nq * k * 8, 256) +
+                 align_up((size_t)nq * k * 4, 256);
+    return RAGO_OK;
+}
+
+rago_status rago_search_probes(const rago_index* index, const float* queries, int32_t nq, int32_t nprobe,
+                               int32_t* out_lists, float* out_coarse, void* workspace, size_t workspace_bytes,
+                               void* cuda_stream) {
+    const IndexImpl* ix = reinterpret_cast<const IndexImpl*>(index);
+    rago_status st = check_search_args(ix, nq, nprobe, 1);
+    if (st != RAGO_OK) return st;
+    if (nq == 0) return RAGO_OK;
+    if (!queries || !out_lists || !out_coarse || !workspace) return fail(RAGO_EINVAL, "null pointer");
+    if (!aligned(queries, 16) || !aligned(workspace, 256)) return fail(RAGO_EALIGN, "queries need 16-byte, workspace 256-byte alignment");
+    const Layout L = make_layout(ix, nq, nprobe, 1);
+    if (workspace_bytes < L.total) return fail(RAGO_ENOMEM, "workspace holds %zu bytes, %zu needed", workspace_bytes, L.total);
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    st = run_coarse(ix, queries, nq, nprobe, ws, L, s);
+    if (st != RAGO_OK) return st;
+    const size_t bytes = (size_t)nq * nprobe * 4;
+    cudaError_t e = cudaMemcpyAsync(out_lists, ws + L.probe_list, bytes, cudaMemcpyDeviceToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(out_coarse, ws + L.probe_term, bytes, cudaMemcpyDeviceToDevice, s);
+    if (e != cudaSuccess) return cuda_fail(e, "copying probe table");
+    return RAGO_OK;
+}
+
+rago_status rago_search(const rago_index* index, const float* queries, int32_t nq, int32_t nprobe, int32_t k,
+                        int64_t* out_ids, float* out_dists, void* workspace, size_t workspace_bytes,
+                        void* cuda_stream) {
+    const IndexImpl* ix = reinterpret_cast<const IndexImpl*>(index);
+    rago_status st = check_search_args(ix, nq, nprobe, k);
+    if (st != RAGO_OK) return st;
+    if (nq == 0) return RAGO_OK;
+    if (!queries || !out_ids || !out_dists || !workspace) return fail(RAGO_EINVAL, "null pointer");
+    if (!aligned(queries, 16) || !aligned(workspace, 256) || !aligned(out_ids, 8) || !aligned(out_dists, 4))
+        return fail(RAGO_EALIGN, "queries need 16-byte, workspace 256-byte alignment");
+    const Layout L = make_layout(ix, nq, nprobe, k);
+    if (workspace_bytes < L.total) return fail(RAGO_ENOMEM, "workspace holds %zu bytes, %zu needed", workspace_bytes, L.total);
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    IndexImpl* mix = const_cast<IndexImpl*>(ix);
+    const int npairs = nq * nprobe;
+
+    cudaError_t e = cudaMemsetAsync(ws + L.err, 0, 256, s);
+    if (e != cudaSuccess) return cuda_fail(e, "clearing the error word");
+    st = run_coarse(ix, queries, nq, nprobe, ws, L, s);
+    if (st != RAGO_OK) return st;
+
+    int32_t* probe_list = reinterpret_cast<int32_t*>(ws + L.probe_list);
+    float* probe_term = reinterpret_cast<float*>(ws + L.probe_term);
+    int64_t* work_prefix = reinterpret_cast<int64_t*>(ws + L.work_prefix);
+    unsigned long long* qthresh = reinterpret_cast<unsigned long long*>(ws + L.qthresh);
+    int32_t* slot_cnt = reinterpret_cast<int32_t*>(ws + L.slot_cnt);
+    unsigned long long* slot_keys = reinterpret_cast<unsigned long long*>(ws + L.slot_keys);
+
+    e = launch_plan_work(ix, probe_list, npairs, ix->plan.tile_vecs, reinterpret_cast<int32_t*>(ws + L.pair_tiles),
+                         work_prefix, s);
+    if (e == cudaSuccess) e = launch_fill_u64(qthresh, (size_t)nq, KEY_MAX, s);
+    if (e == cudaSuccess) e = cudaMemsetAsync(slot_cnt, 0, L.nslots * 4, s);
+    if (e != cudaSuccess) return cuda_fail(e, "work planning");
+    record(mix, 3, s);
+    e = launch_scan(ix, ix->plan, queries, probe_list, probe_term, work_prefix, nq, nprobe, k, qthresh, slot_cnt,
+                    slot_keys, reinterpret_cast<uint32_t*>(ws + L.err), s);
+    if (e != cudaSuccess) return cuda_fail(e, "scan kernel");
+    record(mix, 4, s);
+    e = launch_merge(ix, work_prefix, nq, nprobe, k, ix->plan.ctas, slot_cnt, slot_keys, out_ids, out_dists, s);
+    if (e != cudaSuccess) return cuda_fail(e, "merge kernel");
+    record(mix, 5, s);
+    return RAGO_OK;
+}
+
+rago_status rago_search_host(const rago_index* index, const float* host_queries, int32_t nq, int32_t nprobe,
+                             int32_t k, int64_t* host_out_ids, float* host_out_dists, void* workspace,
+                             size_t workspace_bytes, void* cuda_stream) {
+    const IndexImpl* ix = reinterpret_cast<const IndexImpl*>(index);
+    rago_status st = check_search_args(ix, nq, nprobe, k);
+    if (st != RAGO_OK) return st;
+    if (nq == 0) return RAGO_OK;
+    if (!host_queries || !host_out_ids || !host_out_dists || !workspace) return fail(RAGO_EINVAL, "null pointer");
+    if (!aligned(workspace, 256)) return fail(RAGO_EALIGN, "workspace needs 256-byte alignment");
+    const Layout L = make_layout(ix, nq, nprobe, k);
+    size_t staging = 0;
+    rago_host_staging_bytes(index, nq, k, &staging);
+    if (workspace_bytes < L.total + staging)
+        return fail(RAGO_ENOMEM, "workspace holds %zu bytes, %zu needed", workspace_bytes, L.total + staging);
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    uint8_t* st0 = ws + L.total;
+    float* dq = reinterpret_cast<float*>(st0);
+    int64_t* dids = reinterpret_cast<int64_t*>(st0 + align_up((size_t)nq * ix->d * 4, 256));
+    float* ddist = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(dids) + align_up((size_t)nq * k * 8, 256));
+    cudaError_t e = cudaMemcpyAsync(dq, host_queries, (size_t)nq * ix->d * 4, cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) return cuda_fail(e, "copying queries to the device");
+    st = rago_search(index, dq, nq, nprobe, k, dids, ddist, workspace, L.total, cuda_stream);
+    if (st != RAGO_OK) return st;
+    e = cudaMemcpyAsync(host_out_ids, dids, (size_t)nq * k * 8, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(host_out_dists, ddist, (size_t)nq * k * 4, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return cuda_fail(e, "copying results to the host");
+    return RAGO_OK;
+}
+
+rago_status rago_flat_workspace_bytes(int64_t N, int32_t d, int32_t nq, int32_t k, size_t* out_bytes) {
+    if (!out_bytes) return fail(RAGO_EINVAL, "out_bytes is null");
+    if (N < 0 || d <= 0 || nq < 0 || k < 1) return fail(RAGO_EINVAL, "bad sizes");
+    if (k > MAX_K) return fail(RAGO_EUNSUPPORTED, "k = %d exceeds %d", k, MAX_K);
+    *out_bytes = flat_workspace_bytes(N, nq, k);
+    return RAGO_OK;
+}
+
+rago_status rago_flat_search(const void* db, int64_t N, int32_t d, const void* queries, int32_t nq, int32_t k,
+                             int64_t* out_ids, float* out_scores, void* workspace, size_t workspace_bytes,
+                             void* cuda_stream) {
+    if (N < 0 || d <= 0 || nq < 0) return fail(RAGO_EINVAL, "bad sizes");
+    if (k < 1) return fail(RAGO_EINVAL, "k = %d must be at least 1", k);
+    if (k > MAX_K) return fail(RAGO_EUNSUPPORTED, "k = %d exceeds %d", k, MAX_K);
+    if (d % 64 != 0 || d > 4096) return fail(RAGO_EUNSUPPORTED, "d = %d must be a multiple of 64, at most 4096", d);
+    if (N >= (1LL << 32)) return fail(RAGO_EUNSUPPORTED, "N needs more than 32-bit row numbers");
+    if (nq == 0) return RAGO_OK;
+    if ((N > 0 && !db) || !queries || !out_ids || !out_scores || !workspace) return fail(RAGO_EINVAL, "null pointer");
+    if (!aligned(db, 16) || !aligned(queries, 16) || !aligned(workspace, 256))
+        return fail(RAGO_EALIGN, "db and queries need 16-byte, workspace 256-byte alignment");
+    const size_t need = flat_workspace_bytes(N, nq, k);
+    if (workspace_bytes < need) return fail(RAGO_ENOMEM, "workspace holds %zu bytes, %zu needed", workspace_bytes, need);
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e = cudaMemsetAsync(workspace, 0, 256, s);
+    if (e == cudaSuccess) e = launch_flat_search(db, N, d, queries, nq, k, out_ids, out_scores, workspace, s);
+    if (e != cudaSuccess) return cuda_fail(e, "flat search");
+    return RAGO_OK;
+}
+
+rago_status rago_check(void* workspace, void* cuda_stream) {
+    if (!workspace) return fail(RAGO_EINVAL, "workspace is null");
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    uint32_t w = 0;
+    cudaError_t e = cudaMemcpyAsync(&w, workspace, 4, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return cuda_fail(e, "reading the error word");
+    if (w == ERR_WAIT_TIMEOUT) return fail(RAGO_ETIMEOUT, "a bounded device-side wait expired");
+    if (w != ERR_NONE) return fail(RAGO_ECUDA, "device error word = %u", w);
+    return RAGO_OK;
+}
+
+rago_status rago_profile_enable(rago_index* index, int32_t enable) {
+    if (!index) return fail(RAGO_EINVAL, "index is null");
+    reinterpret_cast<IndexImpl*>(index)->profile = enable ? 1 : 0;
+    return RAGO_OK;
+}
+
+rago_status rago_profile_read(rago_index* index, float* out_ms) {
+    IndexImpl* ix = reinterpret_cast<IndexImpl*>(index);
+    if (!ix || !out_ms) return fail(RAGO_EINVAL, "null pointer");
+    if (!ix->profile) return fail(RAGO_EINVAL, "profiling is not enabled");
+    cudaError_t e = cudaEventSynchronize(ix->ev[RAGO_NUM_STAGES]);
+    for (int i = 0; i < RAGO_NUM_STAGES && e == cudaSuccess; ++i)
+        e = cudaEventElapsedTime(&out_ms[i], ix->ev[i], ix->ev[i + 1]);
+    if (e != cudaSuccess) return cuda_fail(e, "reading stage timings");
+    return RAGO_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,173 @@
+// Shared device/host helpers of the retrieval library (sm_100a).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/rago.h"
+
+namespace rago {
+
+constexpr int KSUB = 256;            // codewords per sub-space (8-bit codes)
+constexpr int TOPK_CAP = 2048;       // candidate buffer of the block-level selector (keys)
+constexpr int MAX_K = 1024;          // k and nprobe limit: TOPK_CAP must hold k plus one batch of pushes
+constexpr int PROBE_GUARD = 8;       // extra coarse candidates re-scored exactly before the final nprobe cut
+constexpr unsigned long long KEY_MAX = 0xFFFFFFFFFFFFFFFFull;
+
+// Device-side error word (first word of every workspace).
+enum : uint32_t { ERR_NONE = 0, ERR_WAIT_TIMEOUT = 1 };
+
+// Launch shape of the table-build + scan kernel for one index (fixed at index load).
+struct ScanPlan {
+    int tile_vecs;     // vectors per code tile
+    int stages;        // tiles in flight per CTA
+    int ctas;          // persistent CTAs (one per SM)
+    size_t smem_bytes;
+};
+
+// Index handle.  Borrowed pointers first, then what the library owns.
+struct IndexImpl {
+    const void* centroids;
+    int coarse_bf16;
+    const float* codebooks;
+    const uint8_t* codes;
+    const int64_t* list_offsets;
+    const int64_t* ids;
+    int64_t N;
+    int32_t d, nlist, M, dsub, metric;
+    // owned
+    float* cnorm;  // [nlist] squared centroid norms (L2 coarse ranking)
+    float* cbT;    // [256][M][dsub] codebook with the codeword index outermost
+    int device, num_sms;
+    ScanPlan plan;
+    int profile;
+    cudaEvent_t ev[RAGO_NUM_STAGES + 1];
+    float last_ms[RAGO_NUM_STAGES];
+    int ev_valid;
+};
+
+// ---- order-preserving float <-> uint32 ------------------------------------------------------
+__host__ __device__ inline uint32_t f32_orderable(float f) {
+#ifdef __CUDA_ARCH__
+    uint32_t u = __float_as_uint(f);
+#else
+    union { float f; uint32_t u; } c; c.f = f; uint32_t u = c.u;
+#endif
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__host__ __device__ inline float orderable_f32(uint32_t o) {
+    uint32_t u = (o & 0x80000000u) ? (o & 0x7FFFFFFFu) : ~o;
+#ifdef __CUDA_ARCH__
+    return __uint_as_float(u);
+#else
+    union { float f; uint32_t u; } c; c.u = u; return c.f;
+#endif
+}
+__host__ __device__ inline unsigned long long make_key(float score_smaller_is_better, uint32_t payload) {
+    return ((unsigned long long)f32_orderable(score_smaller_is_better) << 32) | payload;
+}
+
+__host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+#ifdef __CUDACC__
+// ---- shared-memory address / mbarrier / bulk-copy wrappers ----------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up after ~2^22 polls (with back-off) or as soon as *abort_flag is set by
+// another warp.  On give-up it raises the CTA abort flag and the global error word; callers keep
+// their control flow (so CTA-wide barriers still match) but the data is garbage.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                          uint32_t* err_word) {
+    if (mbar_try_wait(bar, parity)) return true;
+    for (uint32_t it = 0; it < (1u << 22); ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (it > 64) __nanosleep(it > 4096 ? 256 : 32);
+        if ((it & 63) == 63 && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    atomicExch(err_word, (uint32_t)ERR_WAIT_TIMEOUT);
+    return false;
+}
+__device__ __forceinline__ void fence_barrier_init() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// 1-D bulk copy global -> shared, completion counted in bytes on an mbarrier.
+// dst/src 16-byte aligned, bytes a positive multiple of 16.
+__device__ __forceinline__ void bulk_g2s(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     dst_smem),
+                 "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+
+__device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
+__device__ __forceinline__ float lds_f32(uint32_t addr) {
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+#endif  // __CUDACC__
+
+// ---- host-side launch bookkeeping -------------------------------------------------------------
+void count_launch(int n = 1);
+void set_error(const char* fmt, ...);
+
+// ---- kernel launchers (one per .cu file) ------------------------------------------------------
+
+// coarse.cu
+cudaError_t launch_centroid_norms(const void* centroids, int bf16, int nlist, int d, float* cnorm, cudaStream_t s);
+cudaError_t launch_coarse_scores(const IndexImpl* ix, const float* queries, int nq, float* scores, cudaStream_t s);
+cudaError_t launch_select_probes(const IndexImpl* ix, const float* queries, const float* scores, int nq, int nprobe,
+                                 int32_t* probe_list, float* probe_term, cudaStream_t s);
+// scan.cu
+bool scan_supported(int M);
+cudaError_t scan_plan(const IndexImpl* ix, ScanPlan* plan);
+cudaError_t launch_transpose_codebook(const float* cb, int M, int dsub, float* cbT, cudaStream_t s);
+cudaError_t launch_plan_work(const IndexImpl* ix, const int32_t* probe_list, int npairs, int tile_vecs,
+                             int32_t* pair_tiles, int64_t* work_prefix, cudaStream_t s);
+cudaError_t launch_scan(const IndexImpl* ix, const ScanPlan& plan, const float* queries, const int32_t* probe_list,
+                        const float* probe_term, const int64_t* work_prefix, int nq, int nprobe, int k,
+                        unsigned long long* qthresh, int32_t* slot_cnt, unsigned long long* slot_keys,
+                        uint32_t* err_word, cudaStream_t s);
+// merge.cu
+cudaError_t launch_merge(const IndexImpl* ix, const int64_t* work_prefix, int nq, int nprobe, int k, int ctas,
+                         const int32_t* slot_cnt, const unsigned long long* slot_keys, int64_t* out_ids,
+                         float* out_dists, cudaStream_t s);
+cudaError_t launch_fill_u64(unsigned long long* p, size_t n, unsigned long long v, cudaStream_t s);
+// flat.cu
+size_t flat_workspace_bytes(int64_t N, int nq, int k);
+cudaError_t launch_flat_search(const void* db, int64_t N, int d, const void* queries, int nq, int k, int64_t* out_ids,
+                               float* out_scores, void* workspace, cudaStream_t s);
+
+}  // namespace rago

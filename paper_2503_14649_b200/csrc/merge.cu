@@ -1,0 +1,86 @@
+// Final top-k per query: merge the partial candidate lists the scan CTAs left behind, sort, map
+// storage positions to caller ids, and write results best-first.
+#include "topk.cuh"
+
+namespace rago {
+
+constexpr int MERGE_THREADS = 256;
+
+// Slot numbering: CTA b working on pair p writes slot p + b.  Along the CTAs' contiguous walk over the
+// pairs that number strictly increases, so the slots of one query form one range.
+__device__ __forceinline__ long long cta_of_unit(long long u, long long W, int ctas) {
+    // CTA b owns units [b*W/ctas, (b+1)*W/ctas): the largest b with floor(b*W/ctas) <= u
+    return ((u + 1) * ctas - 1) / W;
+}
+
+__global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(
+    const int64_t* __restrict__ work_prefix, const int64_t* __restrict__ ids, int npairs, int nprobe, int k, int ctas,
+    int metric, const int32_t* __restrict__ slot_cnt, const unsigned long long* __restrict__ slot_keys,
+    int64_t* __restrict__ out_ids, float* __restrict__ out_dists) {
+    __shared__ unsigned long long keys[TOPK_CAP];
+    __shared__ int cnt;
+    const int q = blockIdx.x, tid = threadIdx.x;
+    auto sync = [] { __syncthreads(); };
+    if (tid == 0) cnt = 0;
+    __syncthreads();
+    const long long W = work_prefix[npairs];
+    const long long u0 = work_prefix[(size_t)q * nprobe], u1 = work_prefix[(size_t)(q + 1) * nprobe];
+    unsigned long long tau = KEY_MAX;
+    if (u1 > u0) {
+        const long long s0 = (long long)q * nprobe + cta_of_unit(u0, W, ctas);
+        const long long s1 = (long long)(q + 1) * nprobe - 1 + cta_of_unit(u1 - 1, W, ctas);
+        for (long long s = s0; s <= s1; ++s) {
+            const int c = slot_cnt[s];  // <= k
+            if (c == 0) continue;       // uniform: every thread reads the same word
+            if (cnt + c > TOPK_CAP) {
+                const int kept = block_select(keys, &cnt, k, tid, MERGE_THREADS, sync);
+                if (kept == k) tau = keys[k - 1];
+                __syncthreads();
+            }
+            for (int i0 = 0; i0 < c; i0 += MERGE_THREADS) {
+                const int i = i0 + tid;
+                unsigned long long key = KEY_MAX;
+                if (i < c) key = slot_keys[(size_t)s * k + i];
+                warp_push(keys, &cnt, i < c && key < tau, key);
+            }
+            __syncthreads();
+        }
+    }
+    __syncthreads();
+    const int kept = block_select(keys, &cnt, k, tid, MERGE_THREADS, sync);
+    for (int i = tid; i < k; i += MERGE_THREADS) {
+        int64_t id = -1;
+        float dist = metric == RAGO_L2 ? __int_as_float(0x7f800000) : __int_as_float(0xff800000);
+        if (i < kept) {
+            const unsigned long long key = keys[i];
+            id = ids[(uint32_t)(key & 0xFFFFFFFFull)];
+            const float sc = orderable_f32((uint32_t)(key >> 32));
+            dist = metric == RAGO_L2 ? sc : -sc;
+        }
+        out_ids[(size_t)q * k + i] = id;
+        out_dists[(size_t)q * k + i] = dist;
+    }
+}
+
+cudaError_t launch_merge(const IndexImpl* ix, const int64_t* work_prefix, int nq, int nprobe, int k, int ctas,
+                         const int32_t* slot_cnt, const unsigned long long* slot_keys, int64_t* out_ids,
+                         float* out_dists, cudaStream_t s) {
+    merge_kernel<<<nq, MERGE_THREADS, 0, s>>>(work_prefix, ix->ids, nq * nprobe, nprobe, k, ctas, ix->metric,
+                                              slot_cnt, slot_keys, out_ids, out_dists);
+    count_launch();
+    return cudaGetLastError();
+}
+
+__global__ void fill_u64_kernel(unsigned long long* p, size_t n, unsigned long long v) {
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+        p[i] = v;
+}
+cudaError_t launch_fill_u64(unsigned long long* p, size_t n, unsigned long long v, cudaStream_t s) {
+    if (n == 0) return cudaSuccess;
+    const int blocks = (int)((n + 255) / 256 < 1024 ? (n + 255) / 256 : 1024);
+    fill_u64_kernel<<<blocks, 256, 0, s>>>(p, n, v);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace rago

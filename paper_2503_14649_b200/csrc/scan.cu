@@ -1,0 +1,484 @@
+// Lookup-table construction + asymmetric-distance scan of the probed inverted lists.
+//
+// One persistent CTA per SM walks a contiguous, equally sized share of the batch's code tiles
+// (pairs (query, probed list) in probe order, each list cut into tiles of TV vectors).  A producer
+// warp streams code tiles global -> shared with 1-D bulk copies (cp.async.bulk + mbarrier, a ring of
+// S tiles in flight); consumer warps build the fp32 lookup table of the current pair in shared
+// memory, then every lane owns one (virtual) code row of the tile and sums table entries.
+//
+// Shared-memory access pattern.  A code row is read as 32-bit words; at step (blk, il, t) lane L
+// reads word  blk*G + (il ^ a(L))  and uses byte  t ^ b(L)  of it, so that within any one
+// instruction the 32 lanes touch 32 different banks both for the code words (rows are M bytes
+// apart) and for the table (stored [codeword][sub-space], bank = sub-space mod 32).  Rows wider than
+// 32*odd bytes are split into R "virtual rows" handled by adjacent lanes and summed with a shuffle;
+// sub-space counts that are 16 mod 32 keep two table copies so lanes L and L^4 never collide.
+//
+// Candidates better than the running threshold go to a shared buffer (topk.cuh); the threshold of a
+// query is shared between CTAs through global memory, which only ever removes keys that cannot be
+// among the k best, so the result does not depend on timing.
+#include "topk.cuh"
+
+namespace rago {
+
+constexpr int NCW = 8;                          // consumer warps
+constexpr int NCT = NCW * 32;                   // consumer threads
+constexpr int SCAN_THREADS = NCT + 32;          // + one producer warp
+constexpr int MAX_STAGES = 4;
+constexpr int SMEM_LIMIT = 227 * 1024;
+constexpr int CTRL_BYTES = 1024;
+
+struct TileDesc {
+    int32_t pair;      // index into probe_list (query * nprobe + rank)
+    int32_t list;      // inverted list number
+    uint32_t pos0;     // storage position of the tile's first vector
+    int32_t nvec;      // vectors in this tile
+    int32_t newpair;   // first tile of this pair inside this CTA
+    int32_t pad[3];
+};
+
+struct ScanArgs {
+    const uint8_t* codes;
+    const int64_t* list_offsets;
+    const int32_t* probe_list;
+    const float* probe_term;
+    const float* queries;
+    const void* centroids;
+    const float* cbT;
+    const int64_t* work_prefix;
+    unsigned long long* qthresh;
+    int32_t* slot_cnt;
+    unsigned long long* slot_keys;
+    uint32_t* err;
+    int32_t coarse_bf16, npairs, nprobe, d, dsub, metric, k, stages;
+};
+
+template <int WV, int G, int R>
+struct Cfg {
+    static constexpr int MV = WV * 4;                   // bytes per virtual row
+    static constexpr int M = MV * R;                    // code bytes per vector
+    static constexpr int COPIES = G == 4 ? 2 : 1;
+    static constexpr int LSTRIDE = M * COPIES;          // table row stride (words)
+    static constexpr int LUT_BYTES = KSUB * LSTRIDE * 4;
+    static constexpr int RGW = MV >= 96 ? 1 : (96 / MV > 4 ? 4 : 96 / MV);  // 32-row groups per warp per tile
+    static constexpr int TILE_VROWS = NCW * 32 * RGW;
+    static constexpr int TV = TILE_VROWS / R;           // vectors per tile
+    static constexpr int TILE_BYTES = TILE_VROWS * MV;
+    static constexpr int KEYS_OFF = LUT_BYTES;
+    static constexpr int RT_OFF = KEYS_OFF + TOPK_CAP * 8;
+    static_assert(TILE_VROWS % R == 0, "tile must hold whole vectors");
+    static_assert(TV + MAX_K <= TOPK_CAP, "one tile of pushes plus k kept keys must fit the candidate buffer");
+    static_assert(LSTRIDE % 32 == 0, "table rows must keep bank = column mod 32");
+};
+
+// Control block at the end of dynamic shared memory.
+struct Ctrl {
+    unsigned long long full[MAX_STAGES];
+    unsigned long long empty[MAX_STAGES];
+    unsigned long long cbar;  // consumer barrier
+    TileDesc desc[MAX_STAGES];
+    int cnt;
+    uint32_t abort_flag;
+};
+static_assert(sizeof(Ctrl) <= CTRL_BYTES, "control block too large");
+
+template <int WV, int G, int R>
+__global__ void __launch_bounds__(SCAN_THREADS, 1) scan_kernel(const ScanArgs a) {
+    using C = Cfg<WV, G, R>;
+    extern __shared__ __align__(1024) uint8_t smem[];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int S = a.stages;
+    const uint32_t tiles_off = (uint32_t)align_up((size_t)C::RT_OFF + (size_t)a.d * 4, 128);
+    Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem + tiles_off + (size_t)S * C::TILE_BYTES);
+    float* lut = reinterpret_cast<float*>(smem);
+    unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem + C::KEYS_OFF);
+    float* rT = reinterpret_cast<float*>(smem + C::RT_OFF);
+    volatile uint32_t* abort_flag = &ctrl->abort_flag;
+
+    if (tid == 0) {
+        for (int s = 0; s < S; ++s) {
+            mbar_init(smem_u32(&ctrl->full[s]), 1);
+            mbar_init(smem_u32(&ctrl->empty[s]), NCW);
+        }
+        mbar_init(smem_u32(&ctrl->cbar), NCW);
+        ctrl->cnt = 0;
+        ctrl->abort_flag = 0;
+        fence_barrier_init();
+        fence_proxy_async();
+    }
+    __syncthreads();
+
+    // This CTA's share of the work units (tiles).
+    const long long W = a.work_prefix[a.npairs];
+    const long long u_begin = (long long)blockIdx.x * W / gridDim.x;
+    const long long u_end = (long long)(blockIdx.x + 1) * W / gridDim.x;
+    const int T = (int)(u_end - u_begin);
+    if (T <= 0) return;
+
+    if (warp == NCW) {
+        // ================= producer warp =================
+        // first pair whose range contains u_begin: largest p with work_prefix[p] <= u_begin
+        int lo = 0, hi = a.npairs;  // invariant: work_prefix[lo] <= u_begin < work_prefix[hi]
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (a.work_prefix[mid] <= u_begin) lo = mid; else hi = mid;
+        }
+        int cache_base = lo;  // lane i caches pair cache_base + i
+        int c_list = 0; long long c_off = 0, c_len = 0, c_ws = 0, c_we = 0;
+        auto fill = [&]() {
+            const int p = cache_base + lane;
+            if (p < a.npairs) {
+                c_list = a.probe_list[p];
+                c_off = a.list_offsets[c_list];
+                c_len = a.list_offsets[c_list + 1] - c_off;
+                c_ws = a.work_prefix[p];
+                c_we = a.work_prefix[p + 1];
+            } else {
+                c_list = 0; c_off = 0; c_len = 0; c_ws = c_we = W;
+            }
+        };
+        fill();
+        int cur = 0;
+        long long u = u_begin;
+        bool dead = false;
+        int issued = 0;
+        for (int n = 0; n < T && !dead; ++n, ++u) {
+            const int st = n % S;
+            if (n >= S) dead = !mbar_wait(smem_u32(&ctrl->empty[st]), ((n / S) - 1) & 1, abort_flag, a.err);
+            if (dead) break;
+            // advance to the pair that owns unit u (skips empty pairs)
+            for (;;) {
+                const long long we = __shfl_sync(0xffffffffu, c_we, cur);
+                if (u < we) break;
+                if (++cur == 32) { cache_base += 32; fill(); cur = 0; }
+            }
+            const long long ws = __shfl_sync(0xffffffffu, c_ws, cur);
+            const long long off = __shfl_sync(0xffffffffu, c_off, cur);
+            const long long len = __shfl_sync(0xffffffffu, c_len, cur);
+            const int list = __shfl_sync(0xffffffffu, c_list, cur);
+            if (lane == 0) {
+                const long long t_in_pair = u - ws;
+                const long long v0 = t_in_pair * C::TV;
+                long long nvec = len - v0;
+                if (nvec > C::TV) nvec = C::TV;
+                TileDesc& D = ctrl->desc[st];
+                D.pair = cache_base + cur;
+                D.list = list;
+                D.pos0 = (uint32_t)(off + v0);
+                D.nvec = (int32_t)nvec;
+                D.newpair = (n == 0 || t_in_pair == 0) ? 1 : 0;
+                const uint32_t bytes = (uint32_t)nvec * C::M;
+                const uint32_t bar = smem_u32(&ctrl->full[st]);
+                mbar_arrive_expect_tx(bar, bytes);
+                bulk_g2s(smem_u32(smem + tiles_off + (size_t)st * C::TILE_BYTES),
+                         a.codes + (size_t)(off + v0) * C::M, bytes, bar);
+            }
+            issued = n + 1;
+        }
+        if (dead && lane == 0) {
+            // let copies already in flight land before the CTA's shared memory goes away
+            for (int n = issued > S ? issued - S : 0; n < issued; ++n) {
+                const uint32_t bar = smem_u32(&ctrl->full[n % S]);
+                for (int it = 0; it < (1 << 16) && !mbar_try_wait(bar, (n / S) & 1); ++it) __nanosleep(64);
+            }
+        }
+        return;
+    }
+
+    // ================= consumer warps =================
+    const int ctid = tid;  // 0 .. NCT-1
+    uint32_t cphase = 0;
+    bool dead = false;
+    auto csync = [&]() {
+        if (dead) return;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&ctrl->cbar));
+        dead = !mbar_wait(smem_u32(&ctrl->cbar), cphase, abort_flag, a.err);
+        cphase ^= 1;
+    };
+
+    // lane constants of the access pattern
+    const int xa = G == 8 ? (lane >> 2) : (lane >> 3);  // word xor
+    const int xb = lane & 3;                            // byte xor
+    const int copy = G == 4 ? ((lane >> 2) & 1) : 0;
+    const int sr = lane % R;                            // which slice of the vector this lane sums
+    uint32_t lo[G][4], xo[G], sel[4];
+#pragma unroll
+    for (int il = 0; il < G; ++il) {
+        xo[il] = 4u * (uint32_t)(il ^ xa);
+#pragma unroll
+        for (int t = 0; t < 4; ++t)
+            lo[il][t] = 4u * (uint32_t)(copy * C::M + sr * C::MV + 4 * (il ^ xa) + (t ^ xb));
+    }
+#pragma unroll
+    for (int t = 0; t < 4; ++t) sel[t] = 0x4440u | (uint32_t)(t ^ xb);
+
+    int cur_pair = -1, cur_q = -1, lut_q = -1, lut_list = -1;
+    unsigned long long tau = KEY_MAX;
+    float bias = 0.f;
+    int ub = 0;
+    const int k = a.k;
+    const bool ip = a.metric == RAGO_IP;
+
+    auto finalize = [&]() {
+        csync();
+        if (dead) return;
+        int kept = ctrl->cnt;
+        if (kept > k) {
+            kept = block_select(keys, &ctrl->cnt, k, ctid, NCT, csync);
+            if (dead) return;
+            if (ctid == 0) atomicMin(&a.qthresh[cur_q], keys[k - 1]);
+        }
+        const size_t slot = (size_t)cur_pair + blockIdx.x;
+        for (int i = ctid; i < kept; i += NCT) a.slot_keys[slot * k + i] = keys[i];
+        if (ctid == 0) a.slot_cnt[slot] = kept;
+        csync();
+    };
+
+    auto begin_pair = [&](const TileDesc& D) {
+        cur_pair = D.pair;
+        cur_q = D.pair / a.nprobe;
+        const bool need = ip ? (lut_q != cur_q) : (lut_q != cur_q || lut_list != D.list);
+        if (need) {
+            const float* qrow = a.queries + (size_t)cur_q * a.d;
+            for (int j = ctid; j < a.d; j += NCT) {
+                float v = qrow[j];
+                if (!ip) {
+                    const float c = a.coarse_bf16
+                        ? __bfloat162float(static_cast<const __nv_bfloat16*>(a.centroids)[(size_t)D.list * a.d + j])
+                        : static_cast<const float*>(a.centroids)[(size_t)D.list * a.d + j];
+                    v -= c;
+                }
+                rT[(j % a.dsub) * C::M + j / a.dsub] = v;
+            }
+            csync();
+            if (dead) return;
+            const int dsub = a.dsub;
+            for (int e = ctid; e < KSUB * C::M; e += NCT) {
+                const int j = e / C::M, m = e - j * C::M;
+                const float* cw = a.cbT + (size_t)e * dsub;
+                float acc = 0.f;
+                if ((dsub & 3) == 0) {
+                    for (int t = 0; t < dsub; t += 4) {
+                        const float4 cv = __ldg(reinterpret_cast<const float4*>(cw + t));
+                        const float c4[4] = {cv.x, cv.y, cv.z, cv.w};
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const float r = rT[(t + i) * C::M + m];
+                            if (ip) acc = fmaf(r, c4[i], acc);
+                            else { const float df = r - c4[i]; acc = fmaf(df, df, acc); }
+                        }
+                    }
+                } else {
+                    for (int t = 0; t < dsub; ++t) {
+                        const float r = rT[t * C::M + m], cv = __ldg(cw + t);
+                        if (ip) acc = fmaf(r, cv, acc);
+                        else { const float df = r - cv; acc = fmaf(df, df, acc); }
+                    }
+                }
+                lut[j * C::LSTRIDE + m] = acc;
+                if (C::COPIES == 2) lut[j * C::LSTRIDE + C::M + m] = acc;
+            }
+            lut_q = cur_q;
+            lut_list = D.list;
+        }
+        bias = ip ? a.probe_term[D.pair] : 0.f;
+        if (ctid == 0) ctrl->cnt = 0;
+        tau = *reinterpret_cast<volatile unsigned long long*>(&a.qthresh[cur_q]);
+        ub = 0;
+        csync();
+    };
+
+    for (int n = 0; n < T; ++n) {
+        const int st = n % S;
+        dead = dead || !mbar_wait(smem_u32(&ctrl->full[st]), (n / S) & 1, abort_flag, a.err);
+        if (dead) break;
+        const TileDesc D = ctrl->desc[st];
+        if (D.newpair) {
+            if (cur_pair >= 0) finalize();
+            if (dead) break;
+            begin_pair(D);
+            if (dead) break;
+        } else if (ub + C::TV > TOPK_CAP) {
+            csync();
+            if (dead) break;
+            if (ctrl->cnt + C::TV > TOPK_CAP) {
+                const int kept = block_select(keys, &ctrl->cnt, k, ctid, NCT, csync);
+                if (dead) break;
+                if (kept == k) {
+                    if (keys[k - 1] < tau) tau = keys[k - 1];
+                    if (ctid == 0) atomicMin(&a.qthresh[cur_q], keys[k - 1]);
+                }
+            }
+            const unsigned long long g = *reinterpret_cast<volatile unsigned long long*>(&a.qthresh[cur_q]);
+            if (g < tau) tau = g;
+            ub = ctrl->cnt;
+            csync();
+            if (dead) break;
+        }
+
+        // ---- scan this tile: warp w owns row groups w*RGW .. w*RGW+RGW-1 ----
+        const int nvr = D.nvec * R;
+        const uint32_t tile_base = tiles_off + (uint32_t)st * C::TILE_BYTES;
+#pragma unroll 1
+        for (int rg = 0; rg < C::RGW; ++rg) {
+            const int vr0 = (warp * C::RGW + rg) * 32;
+            if (vr0 >= nvr) break;
+            const int vr = vr0 + lane;
+            const uint32_t rowoff = tile_base + (uint32_t)vr * C::MV;
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int blk = 0; blk < WV / G; ++blk) {
+#pragma unroll
+                for (int il = 0; il < G; ++il) {
+                    const uint32_t x = *reinterpret_cast<const uint32_t*>(smem + rowoff + xo[il] + blk * G * 4);
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+                        const uint32_t j = __byte_perm(x, 0u, sel[t]);
+                        acc[t] += *reinterpret_cast<const float*>(smem + j * (uint32_t)(C::LSTRIDE * 4) + lo[il][t] +
+                                                                  blk * G * 16);
+                    }
+                }
+            }
+            float s = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+            if (R >= 2) s += __shfl_xor_sync(0xffffffffu, s, 1);
+            if (R >= 4) s += __shfl_xor_sync(0xffffffffu, s, 2);
+            const float score = ip ? -(bias + s) : s;
+            const unsigned long long key = make_key(score, D.pos0 + (uint32_t)(vr / R));
+            warp_push(keys, &ctrl->cnt, vr < nvr && sr == 0 && key < tau, key);
+        }
+        ub += D.nvec;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&ctrl->empty[st]));
+    }
+    if (!dead && cur_pair >= 0) finalize();
+}
+
+// ---- host side ----------------------------------------------------------------------------------
+struct Variant {
+    int M;
+    void (*kernel)(const ScanArgs);
+    int lut_bytes, tile_bytes, tile_vecs;
+};
+#define RAGO_VARIANT(WV, G, R) \
+    { Cfg<WV, G, R>::M, scan_kernel<WV, G, R>, Cfg<WV, G, R>::LUT_BYTES, Cfg<WV, G, R>::TILE_BYTES, Cfg<WV, G, R>::TV }
+static const Variant kVariants[] = {
+    RAGO_VARIANT(4, 4, 1),   // M = 16
+    RAGO_VARIANT(8, 8, 1),   // M = 32
+    RAGO_VARIANT(12, 4, 1),  // M = 48
+    RAGO_VARIANT(8, 8, 2),   // M = 64
+    RAGO_VARIANT(20, 4, 1),  // M = 80
+    RAGO_VARIANT(24, 8, 1),  // M = 96
+    RAGO_VARIANT(8, 8, 4),   // M = 128
+};
+
+static const Variant* find_variant(int M) {
+    for (const Variant& v : kVariants)
+        if (v.M == M) return &v;
+    return nullptr;
+}
+
+bool scan_supported(int M) { return find_variant(M) != nullptr; }
+
+cudaError_t scan_plan(const IndexImpl* ix, ScanPlan* plan) {
+    const Variant* v = find_variant(ix->M);
+    if (!v) return cudaErrorInvalidValue;
+    const size_t fixed = align_up((size_t)v->lut_bytes + TOPK_CAP * 8 + (size_t)ix->d * 4, 128);
+    long long room = (long long)SMEM_LIMIT - (long long)fixed - CTRL_BYTES;
+    int stages = (int)(room / v->tile_bytes);
+    if (stages > MAX_STAGES) stages = MAX_STAGES;
+    if (stages < 2) return cudaErrorInvalidValue;
+    plan->tile_vecs = v->tile_vecs;
+    plan->stages = stages;
+    plan->ctas = ix->num_sms;
+    plan->smem_bytes = fixed + (size_t)stages * v->tile_bytes + CTRL_BYTES;
+    return cudaFuncSetAttribute(v->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan->smem_bytes);
+}
+
+cudaError_t launch_scan(const IndexImpl* ix, const ScanPlan& plan, const float* queries, const int32_t* probe_list,
+                        const float* probe_term, const int64_t* work_prefix, int nq, int nprobe, int k,
+                        unsigned long long* qthresh, int32_t* slot_cnt, unsigned long long* slot_keys,
+                        uint32_t* err_word, cudaStream_t s) {
+    const Variant* v = find_variant(ix->M);
+    if (!v) return cudaErrorInvalidValue;
+    ScanArgs a;
+    a.codes = ix->codes; a.list_offsets = ix->list_offsets; a.probe_list = probe_list; a.probe_term = probe_term;
+    a.queries = queries; a.centroids = ix->centroids; a.cbT = ix->cbT; a.work_prefix = work_prefix;
+    a.qthresh = qthresh; a.slot_cnt = slot_cnt; a.slot_keys = slot_keys; a.err = err_word;
+    a.coarse_bf16 = ix->coarse_bf16; a.npairs = nq * nprobe; a.nprobe = nprobe; a.d = ix->d; a.dsub = ix->dsub;
+    a.metric = ix->metric; a.k = k; a.stages = plan.stages;
+    v->kernel<<<plan.ctas, SCAN_THREADS, plan.smem_bytes, s>>>(a);
+    count_launch();
+    return cudaGetLastError();
+}
+
+// ---- codebook transpose: cb[m][j][t] -> cbT[j][m][t] -------------------------------------------
+__global__ void transpose_codebook_kernel(const float* __restrict__ cb, int M, int dsub, float* __restrict__ cbT) {
+    const int total = M * KSUB * dsub;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
+        const int t = i % dsub, jm = i / dsub, m = jm % M, j = jm / M;
+        cbT[i] = cb[((size_t)m * KSUB + j) * dsub + t];
+    }
+}
+cudaError_t launch_transpose_codebook(const float* cb, int M, int dsub, float* cbT, cudaStream_t s) {
+    transpose_codebook_kernel<<<256, 256, 0, s>>>(cb, M, dsub, cbT);
+    count_launch();
+    return cudaGetLastError();
+}
+
+// ---- work planning: tiles per pair and their exclusive prefix sum ------------------------------
+__global__ void pair_tiles_kernel(const int32_t* __restrict__ probe_list, const int64_t* __restrict__ offsets,
+                                  int npairs, int tile_vecs, int32_t* __restrict__ tiles) {
+    const int p = blockIdx.x * blockDim.x + threadIdx.x;
+    if (p >= npairs) return;
+    const int l = probe_list[p];
+    const long long len = offsets[l + 1] - offsets[l];
+    tiles[p] = (int32_t)((len + tile_vecs - 1) / tile_vecs);
+}
+
+constexpr int PFX_THREADS = 1024;
+__global__ void __launch_bounds__(PFX_THREADS) prefix_kernel(const int32_t* __restrict__ tiles, int npairs,
+                                                             int64_t* __restrict__ prefix) {
+    __shared__ long long warp_sums[32];
+    __shared__ long long carry_s;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) carry_s = 0;
+    __syncthreads();
+    for (int base = 0; base < npairs; base += PFX_THREADS) {
+        const int i = base + tid;
+        const long long v = i < npairs ? tiles[i] : 0;
+        long long incl = v;
+        for (int o = 1; o < 32; o <<= 1) {
+            const long long y = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += y;
+        }
+        if (lane == 31) warp_sums[warp] = incl;
+        __syncthreads();
+        if (warp == 0) {
+            long long w = warp_sums[lane];
+            for (int o = 1; o < 32; o <<= 1) {
+                const long long y = __shfl_up_sync(0xffffffffu, w, o);
+                if (lane >= o) w += y;
+            }
+            warp_sums[lane] = w;  // inclusive over warps
+        }
+        __syncthreads();
+        const long long carry = carry_s;
+        const long long before = carry + (warp ? warp_sums[warp - 1] : 0) + incl - v;
+        if (i < npairs) prefix[i] = before;
+        __syncthreads();
+        if (tid == PFX_THREADS - 1) carry_s = before + v;
+        __syncthreads();
+    }
+    if (tid == 0) prefix[npairs] = carry_s;
+}
+
+cudaError_t launch_plan_work(const IndexImpl* ix, const int32_t* probe_list, int npairs, int tile_vecs,
+                             int32_t* pair_tiles, int64_t* work_prefix, cudaStream_t s) {
+    pair_tiles_kernel<<<(npairs + 255) / 256, 256, 0, s>>>(probe_list, ix->list_offsets, npairs, tile_vecs,
+                                                          pair_tiles);
+    prefix_kernel<<<1, PFX_THREADS, 0, s>>>(pair_tiles, npairs, work_prefix);
+    count_launch(2);
+    return cudaGetLastError();
+}
+
+}  // namespace rago

@@ -1,0 +1,69 @@
+// Block-level streaming top-k on 64-bit keys in shared memory.
+//
+// A key is (order-preserving score bits << 32) | payload; smaller key = better result, and all keys
+// of one selection are distinct because payloads are.  Candidates that beat the current threshold
+// are appended to a buffer; when the buffer could overflow, the cooperating threads sort it and
+// keep the k smallest, which also tightens the threshold.  Rejecting a key only when it is larger
+// than the k-th smallest key of some subset of the candidates keeps the final top-k exact.
+#pragma once
+#include "common.cuh"
+
+namespace rago {
+
+// Ascending bitonic sort of n keys (n a power of two) by `nthreads` threads; sync() is the barrier
+// those threads share.  Ends with a barrier.
+template <class Sync>
+__device__ __forceinline__ void block_bitonic_sort(unsigned long long* keys, int n, int tid, int nthreads,
+                                                   Sync sync) {
+    for (int size = 2; size <= n; size <<= 1) {
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            for (int i = tid; i < (n >> 1); i += nthreads) {
+                const int lo = 2 * i - (i & (stride - 1));
+                const int hi = lo + stride;
+                const bool up = (lo & size) == 0;
+                const unsigned long long a = keys[lo], b = keys[hi];
+                if ((a > b) == up) {
+                    keys[lo] = b;
+                    keys[hi] = a;
+                }
+            }
+            sync();
+        }
+    }
+}
+
+// Sort the *cnt buffered keys ascending and cut the buffer to at most k entries.
+// Must be called by all cooperating threads, after a barrier that made *cnt and the keys visible.
+// Returns the new count; ends with a barrier.
+template <class Sync>
+__device__ __forceinline__ int block_select(unsigned long long* keys, int* cnt, int k, int tid, int nthreads,
+                                            Sync sync) {
+    int n = *cnt;
+    if (n > TOPK_CAP) n = TOPK_CAP;
+    int n2 = 2;
+    while (n2 < n) n2 <<= 1;
+    for (int i = n + tid; i < n2; i += nthreads) keys[i] = KEY_MAX;
+    sync();
+    block_bitonic_sort(keys, n2, tid, nthreads, sync);
+    const int kept = n < k ? n : k;
+    if (tid == 0) *cnt = kept;
+    sync();
+    return kept;
+}
+
+// Append `key` for the lanes with pred set; one shared atomic per warp.  Whole warp must call.
+__device__ __forceinline__ void warp_push(unsigned long long* keys, int* cnt, bool pred, unsigned long long key) {
+    const unsigned mask = __ballot_sync(0xffffffffu, pred);
+    if (mask == 0) return;
+    const int lane = threadIdx.x & 31;
+    const int leader = __ffs(mask) - 1;
+    int base = 0;
+    if (lane == leader) base = atomicAdd(cnt, __popc(mask));
+    base = __shfl_sync(0xffffffffu, base, leader);
+    if (pred) {
+        const int idx = base + __popc(mask & ((1u << lane) - 1u));
+        if (idx < TOPK_CAP) keys[idx] = key;
+    }
+}
+
+}  // namespace rago

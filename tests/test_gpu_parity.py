@@ -1,0 +1,186 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle, element by element,
+on the same seeded inputs.  ids must be equal except inside distance ties; distances within
+1e-4 relative (flat search: 1e-3)."""
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2503_14649_b200 import binding, synth
+from tests.helpers import host_index, match_results
+
+pytestmark = pytest.mark.gpu
+
+REL = 1e-4  # fp32 distances vs the double-precision oracle
+
+
+def _gpu_search(data, nprobe, k, queries=None):
+    ix = binding.load_index_from(data, "cuda")
+    q = (data.queries if queries is None else queries).cuda().contiguous()
+    ids, dists = ix.rago_search(q, nprobe, k)
+    lists, coarse = ix.rago_search_probes(q, nprobe)
+    torch.cuda.synchronize()
+    ix.rago_check()
+    out = ids.cpu().numpy(), dists.cpu().numpy(), lists.cpu().numpy(), coarse.cpu().numpy()
+    ix.close()
+    return out
+
+
+def _compare(data, nprobe, k, rel=REL, max_probe_mismatch=0):
+    hix = host_index(oracle, data)
+    q = data.queries.cpu().numpy()
+    oi, od, op = oracle.ivfpq_search(hix, q, nprobe, k, nthreads=oracle.default_threads(), want_probes=True)
+    _, oc = oracle.coarse(hix.centroids, q, nprobe, data.metric, coarse_bf16=data.coarse_bf16,
+                          nthreads=oracle.default_threads())
+    gi, gd, gl, gc = _gpu_search(data, nprobe, k)
+    bad_probe_queries = 0
+    for i in range(q.shape[0]):
+        # probe lists: same lists in the same order, except where coarse scores tie within tolerance
+        if not np.array_equal(gl[i], op[i]):
+            sgn = 1.0 if data.metric == "l2" else -1.0
+            assert not match_results(gl[i].astype(np.int64), sgn * gc[i], op[i].astype(np.int64), sgn * oc[i],
+                                     rel=rel), ("probe order", i, gl[i], op[i])
+            if set(gl[i].tolist()) != set(op[i].tolist()):
+                bad_probe_queries += 1
+                continue  # a different list was probed at a coarse tie: final results legitimately differ
+        assert np.allclose(gc[i], oc[i], rtol=rel, atol=rel * max(1.0, np.abs(oc[i]).max())), ("coarse", i)
+        sgn = 1.0 if data.metric == "l2" else -1.0
+        problems = match_results(gi[i], sgn * gd[i], oi[i], sgn * od[i], rel=rel)
+        assert not problems, ("query %d" % i, problems[:5])
+    assert bad_probe_queries <= max_probe_mismatch
+    return gi, gd
+
+
+CASES = [
+    # N, d, nlist, M, nq, nprobe, k, metric, bf16, zipf
+    (3000, 64, 16, 16, 9, 4, 10, "l2", False, None),
+    (3000, 64, 16, 32, 9, 4, 10, "ip", False, None),
+    (5000, 96, 12, 48, 5, 3, 17, "l2", False, None),
+    (5000, 128, 20, 64, 7, 20, 33, "l2", False, None),   # nprobe = nlist
+    (5000, 128, 20, 64, 7, 5, 8, "ip", True, None),
+    (4000, 160, 10, 80, 3, 2, 5, "l2", False, None),
+    (6000, 192, 24, 96, 11, 6, 100, "l2", False, 1.1),
+    (6000, 192, 24, 96, 11, 6, 100, "ip", True, 1.1),
+    (4000, 256, 8, 128, 4, 3, 12, "l2", True, None),
+    (2000, 32, 8, 16, 1, 8, 1, "l2", False, None),       # nq = 1, k = 1
+    (700, 48, 40, 16, 6, 40, 1024, "l2", False, None),   # k above the candidate count: padding
+]
+
+
+@pytest.mark.parametrize("case", CASES, ids=lambda c: "N%d_d%d_nl%d_M%d_%s%s" % (c[0], c[1], c[2], c[3], c[7],
+                                                                                   "_bf16" if c[8] else ""))
+def test_small_cases_match_oracle(case):
+    N, d, nlist, M, nq, nprobe, k, metric, bf16, zipf = case
+    data = synth.make_ivfpq(N, d, nlist, M, nq, metric=metric, seed=100 + N + M, zipf=zipf, coarse_bf16=bf16)
+    _compare(data, nprobe, k)
+
+
+def test_empty_lists_and_short_lists():
+    data = synth.make_ivfpq(900, 64, 16, 16, 8, metric="l2", seed=5)
+    # empty every other list by moving its vectors to the next one
+    L = (data.list_offsets[1:] - data.list_offsets[:-1]).clone()
+    for l in range(0, 16, 2):
+        L[l + 1] += L[l]
+        L[l] = 0
+    data.list_offsets = synth.offsets_from_lengths(L)
+    _compare(data, 16, 20)
+    # an entirely empty index
+    data0 = synth.make_ivfpq(0, 32, 4, 16, 3, metric="ip", seed=6)
+    gi, gd, _, _ = _gpu_search(data0, 2, 5)
+    assert (gi == -1).all() and np.isneginf(gd).all()
+
+
+def test_config1_full_size():
+    """Tiny IVF-PQ shape of the benchmark list, all 64 queries."""
+    c = synth.CONFIGS[1]
+    data = synth.make_config(1)
+    _compare(data, c["nprobe"], c["k"])
+
+
+def test_mid_shape_scaled_down_spans_many_tiles():
+    """Mid shape (d = 768, M = 96, Zipf lists) at 1/40 of the vectors: long lists are cut into many
+    tiles and split between CTAs, short ones have ragged tails."""
+    data = synth.make_ivfpq(250_000, 768, 256, 96, 48, metric="l2", seed=77, zipf=1.1)
+    _compare(data, 32, 100, max_probe_mismatch=1)
+
+
+def test_inner_product_bf16_coarse_hashed_index():
+    """Hyperscale shape in miniature: hash-coded M = 64 lists, bf16 centroids, inner product."""
+    data = synth.make_ivfpq_hashed(400_000, 768, 512, 64, 32, metric="ip", seed=31, coarse_bf16=True)
+    _compare(data, 64, 100, max_probe_mismatch=1)
+
+
+def test_iterative_small_batches_back_to_back():
+    """Latency shape in miniature: batches of 1, 4 and 16 queries issued on one stream reuse one
+    workspace; each must equal the oracle's answer for its own queries."""
+    data = synth.make_ivfpq_hashed(300_000, 512, 256, 32, 64, metric="l2", seed=41)
+    hix = host_index(oracle, data)
+    ix = binding.load_index_from(data, "cuda")
+    q = data.queries.cuda()
+    outs = []
+    pos = 0
+    for nb in synth.batch_size_stream(3, 12):
+        outs.append((pos, nb) + ix.rago_search(q[pos:pos + nb].contiguous(), 16, 20))
+        outs[-1] = (pos, nb, outs[-1][2].clone(), outs[-1][3].clone())
+        pos = (pos + nb) % 40
+    torch.cuda.synchronize()
+    ix.rago_check()
+    for pos, nb, gi, gd in outs:
+        oi, od = oracle.ivfpq_search(hix, data.queries[pos:pos + nb].numpy(), 16, 20)
+        for i in range(nb):
+            assert not match_results(gi[i].cpu().numpy(), gd[i].cpu().numpy(), oi[i], od[i], rel=REL)
+    ix.close()
+
+
+def test_results_do_not_depend_on_run():
+    """The shared per-query threshold makes scheduling vary between runs; results must not."""
+    data = synth.make_ivfpq(120_000, 192, 64, 96, 32, metric="l2", seed=8, zipf=1.1)
+    ix = binding.load_index_from(data, "cuda")
+    q = data.queries.cuda()
+    a = ix.rago_search(q, 16, 50)
+    a = (a[0].clone(), a[1].clone())
+    for _ in range(3):
+        b = ix.rago_search(q, 16, 50)
+        assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+    ix.close()
+
+
+@pytest.mark.parametrize("N,d,nq,k", [(5000, 64, 7, 10), (70_000, 128, 33, 100), (3, 64, 2, 5)])
+def test_flat_search_matches_oracle(N, d, nq, k):
+    db, q = synth.make_flat(N, d, nq, seed=N)
+    gi, gs = binding.rago_flat_search(db.cuda(), q.cuda(), k)
+    torch.cuda.synchronize()
+    oi, osc = oracle.flat_search(db.view(torch.uint16).numpy(), q.view(torch.uint16).numpy(), k,
+                                 nthreads=oracle.default_threads())
+    gi, gs = gi.cpu().numpy(), gs.cpu().numpy()
+    for i in range(nq):
+        assert not match_results(gi[i], -gs[i], oi[i], -osc[i], rel=1e-3), i
+
+
+def test_argument_errors_are_reported_before_any_launch():
+    data = synth.make_ivfpq(500, 32, 4, 16, 2, seed=1)
+    ix = binding.load_index_from(data, "cuda")
+    q = data.queries.cuda()
+    before = binding.rago_kernel_launches()
+    for kwargs in (dict(nprobe=5, k=3), dict(nprobe=0, k=3), dict(nprobe=2, k=0), dict(nprobe=2, k=2000)):
+        with pytest.raises(binding.RagoError):
+            ix.rago_search(q, **kwargs)
+    with pytest.raises(binding.RagoError) as e:
+        ix.rago_search(q, 2, 3, workspace=torch.empty(256, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == 4
+    with pytest.raises(binding.RagoError) as e:
+        ix.rago_search(torch.zeros(2 * 32 + 1, device="cuda")[1:].view(2, 32), 2, 3)  # 4-byte offset
+    assert e.value.status == 2
+    assert binding.rago_kernel_launches() == before
+    ix.close()
+    # unsupported sub-space count, non-monotone offsets
+    bad = synth.make_ivfpq(500, 48, 4, 24, 2, seed=1)
+    with pytest.raises(binding.RagoError) as e:
+        binding.load_index_from(bad, "cuda")
+    assert e.value.status == 3
+    data.list_offsets = data.list_offsets.clone()
+    data.list_offsets[2] = data.list_offsets[1] - 1
+    with pytest.raises(binding.RagoError) as e:
+        binding.load_index_from(data, "cuda")
+    assert e.value.status == 1
