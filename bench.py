@@ -1,0 +1,311 @@
+#!/usr/bin/env python
+"""Benchmark of the retrieval hot path on the Mid IVF-PQ workload.
+
+A step is one rago_search over a batch of 1024 queries (coarse distances + nprobe selection,
+table build, list scan, top-k merge) against a seeded synthetic index of 10 M vectors
+(d = 768, nlist = 4096 Zipf(1.1)-skewed lists, 96-byte PQ codes), nprobe = 32, k = 100.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+With N > 1 (under torchrun) every rank holds a replica of the index and searches its own batch:
+query batches are independent, so there is no data-path collective and scaling is weak.
+`--impl reference` times the CPU oracle, as it stands, on a bounded sample of the same workload.
+Prints one JSON line on rank 0.
+"""
+
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+WORKLOAD = 2  # index into synth.CONFIGS
+METRIC = "retrieval_qps"
+UNIT = "queries/s"
+
+
+def _peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons every 200 ms while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.rows = []
+        self.proc = None
+        self.index = index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
+                 "-lms", "200"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), [x.strip() for x in line.split(",")]))
+
+    def stop(self, t0, t1):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.25)
+        self.proc.terminate()
+        rows = [r for (t, r) in self.rows if t0 <= t <= t1 + 0.3] or [r for (_, r) in self.rows]
+        sm, mx, reasons = [], [], set()
+        for r in rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def _dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+def _oracle_sample(data, cfg, nsample, threads, repeat=1):
+    """Time the oracle on the first nsample queries; returns (seconds per pass, ids, dists)."""
+    import oracle
+    from tests.helpers import host_index
+    hix = host_index(oracle, data)
+    q = data.queries[:nsample].cpu().numpy()
+    best = None
+    for _ in range(repeat):
+        t0 = time.perf_counter()
+        ids, dists = oracle.ivfpq_search(hix, q, cfg["nprobe"], cfg["k"], nthreads=threads)
+        dt = time.perf_counter() - t0
+        best = dt if best is None else min(best, dt)
+    return best, ids, dists
+
+
+def run_reference(args):
+    """CPU oracle arm: each step searches a bounded sample of the workload's queries on the host cores."""
+    rank, world, _ = _dist_env()
+    if rank != 0:
+        return
+    import oracle
+    from paper_2503_14649_b200 import synth
+    from tests.helpers import host_index
+    cfg = synth.CONFIGS[WORKLOAD]
+    threads = oracle.default_threads()
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    data = synth.make_config(WORKLOAD, device=dev, scale=args.scale)
+    hix = host_index(oracle, data)
+    nsample = min(cfg["nq"], threads)  # one query per core per step
+    q = data.queries[:nsample].cpu().numpy()
+    for _ in range(args.warmup):
+        oracle.ivfpq_search(hix, q, cfg["nprobe"], cfg["k"], nthreads=threads)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.ivfpq_search(hix, q, cfg["nprobe"], cfg["k"], nthreads=threads)
+    dt = time.perf_counter() - t0
+    qps = nsample * args.steps / dt
+    sample = "%d of %d queries per step, full database, one query per thread" % (nsample, cfg["nq"])
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": qps, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": _config(cfg, data, args),
+        "cpu_baseline": {"value": qps, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": qps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def _config(cfg, data, args):
+    return {"workload": "Mid IVF-PQ (configs[1]): N=%d d=%d nlist=%d zipf=1.1 M=%d nq=%d nprobe=%d k=%d L2" % (
+        data.N, cfg["d"], cfg["nlist"], cfg["M"], cfg["nq"], cfg["nprobe"], cfg["k"]),
+        "global_batch": cfg["nq"] * max(1, args.gpus), "parallelism": "replicas x%d" % max(1, args.gpus),
+        "l2_policy": "inputs larger than L2 (0.96 GB of codes per replica)", "scale": args.scale}
+
+
+def run_ours(args):
+    from paper_2503_14649_b200 import binding, synth
+    rank, world, local = _dist_env()
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    else:
+        torch.cuda.set_device(0)
+        local = 0
+    dev = torch.device("cuda", local)
+    cfg = synth.CONFIGS[WORKLOAD]
+    nq, nprobe, k = cfg["nq"], cfg["nprobe"], cfg["k"]
+    data = synth.make_config(WORKLOAD, device=dev, scale=args.scale)
+    if world > 1:  # every rank searches its own batch against its replica
+        g = torch.Generator(device=dev)
+        g.manual_seed(1000 + rank)
+        comp = data.extra["query_component"].to(dev)
+        perm = torch.randperm(nq, generator=g, device=dev)
+        data.queries = data.queries[perm].contiguous()
+        data.extra["query_component"] = comp[perm].cpu()
+    ix = binding.rago_index_load(data.centroids, data.codebooks, data.codes, data.list_offsets.to(dev), data.ids,
+                                 data.metric)
+    q = data.queries.contiguous()
+    ws_bytes = ix.search_workspace_bytes(nq, nprobe, k)
+    ws = torch.empty(ws_bytes + ix.host_staging_bytes(nq, k), dtype=torch.uint8, device=dev)
+    out_ids = torch.empty((nq, k), dtype=torch.int64, device=dev)
+    out_d = torch.empty((nq, k), dtype=torch.float32, device=dev)
+
+    # bytes the scan logically reads: sum over queries of probed-list lengths x M
+    lists, _ = ix.rago_search_probes(q, nprobe, workspace=ws)
+    L = (data.list_offsets[1:] - data.list_offsets[:-1]).to(dev)
+    scanned_vectors = int(L[lists.long()].sum().item())
+    scan_bytes = scanned_vectors * cfg["M"]
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+
+    def step():
+        ix.rago_search(q, nprobe, k, out_ids, out_d, ws)
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    ix.rago_check(ws)
+    sampler = ClockSampler(local)
+    sampler.start()
+    ix.rago_profile_enable(True)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    stage_ms = []
+    barrier()
+    launches0 = binding.rago_kernel_launches()
+    t0 = time.time()
+    ev[0].record()
+    for i in range(args.steps):
+        step()
+        ev[i + 1].record()
+    barrier()
+    t1 = time.time()
+    launches = binding.rago_kernel_launches() - launches0
+    total_ms = ev[0].elapsed_time(ev[-1])
+    step_ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
+    stage_last = ix.rago_profile_read()  # stage split of the last timed step (events on the launching stream)
+    ix.rago_profile_enable(False)
+    clocks = sampler.stop(t0, t1)
+    ix.rago_check(ws)
+    # scan-kernel time over several steps, each read right after its step (outside the timed region)
+    ix.rago_profile_enable(True)
+    for _ in range(min(10, args.steps)):
+        step()
+        stage_ms.append(ix.rago_profile_read())
+    ix.rago_profile_enable(False)
+    scan_ms = float(np.mean([s["table_scan"] for s in stage_ms]))
+
+    if world > 1:
+        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        total_ms = float(t.item())
+    qps = nq * world * args.steps / (total_ms / 1e3)
+
+    # end to end through the host-buffer entry point: pinned queries in, pinned results out
+    hq = q.cpu().pin_memory()
+    hids = torch.empty((nq, k), dtype=torch.int64).pin_memory()
+    hd = torch.empty((nq, k), dtype=torch.float32).pin_memory()
+    for _ in range(2):
+        ix.rago_search_host(hq, nprobe, k, hids, hd, ws)
+    barrier()
+    e0 = torch.cuda.Event(enable_timing=True)
+    e1 = torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        ix.rago_search_host(hq, nprobe, k, hids, hd, ws)
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e_qps = nq * world * args.steps / (e2e_ms / 1e3)
+    assert torch.equal(hids, out_ids.cpu()), "host-buffer path disagrees with the device path"
+
+    if rank != 0:
+        if world > 1:
+            torch.distributed.destroy_process_group()
+        return
+
+    peak, peak_kind = _peaks()
+    achieved = scan_bytes / (scan_ms / 1e3) / 1e9
+    out = {
+        "metric": METRIC, "value": qps, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic", "config": _config(cfg, data, args),
+        "clocks": clocks,
+        "e2e": {"value": e2e_qps, "unit": UNIT, "h2d_bytes_per_step": nq * cfg["d"] * 4,
+                "d2h_bytes_per_step": nq * k * 12},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "hbm", "kernel": "scan_kernel (table build + ADC scan)", "achieved": achieved,
+                     "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+                     "algorithmic_bytes_per_launch": scan_bytes, "kernel_ms": scan_ms,
+                     "scanned_vectors_per_query": scanned_vectors / nq},
+        "stage_ms": {kk: float(np.mean([s[kk] for s in stage_ms])) for kk in stage_ms[0]},
+        "step_ms_p50": float(np.median(step_ms)), "step_ms_max": float(np.max(step_ms)),
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        import oracle
+        from tests.helpers import match_results
+        threads = oracle.default_threads()
+        nsample = min(nq, 4 * threads)
+        dt, oi, od = _oracle_sample(data, cfg, nsample, threads)
+        gi, gd = out_ids[:nsample].cpu().numpy(), out_d[:nsample].cpu().numpy()
+        mism = sum(1 for i in range(nsample) if match_results(gi[i], gd[i], oi[i], od[i], rel=1e-4))
+        out["cpu_baseline"] = {"value": nsample / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
+                               "sample": "first %d of %d queries, full database, one query per thread" % (nsample, nq),
+                               "seconds": dt, "queries_not_matching_gpu": mism}
+    print(json.dumps(out))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--scale", type=float, default=1.0, help="shrink N (development only; 1.0 = the named workload)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
