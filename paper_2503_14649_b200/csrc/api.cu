@@ -39,7 +39,7 @@ static bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_
 // Workspace carving.  Every region starts on a 256-byte boundary; the first 256 bytes hold the
 // device error word.
 struct Layout {
-    size_t err, probe_list, probe_term, scores, pair_tiles, work_prefix, qthresh, slot_cnt, slot_keys, total;
+    size_t err, probe_list, probe_term, probe_bias, scores, pair_tiles, work_prefix, qthresh, slot_cnt, slot_keys, total;
     size_t nslots;
 };
 
@@ -52,10 +52,11 @@ static Layout make_layout(const IndexImpl* ix, int nq, int nprobe, int k) {
         return at;
     };
     const size_t npairs = (size_t)nq * nprobe;
-    L.nslots = npairs + (size_t)ix->plan.ctas;
+    L.nslots = (size_t)nq + (size_t)ix->plan.ctas;  // one slot per (CTA, query) incidence
     L.err = take(256);
     L.probe_list = take(npairs * 4);
     L.probe_term = take(npairs * 4);
+    L.probe_bias = take(npairs * 4);
     L.scores = take((size_t)nq * ix->nlist * 4);
     L.pair_tiles = take(npairs * 4);
     L.work_prefix = take((npairs + 1) * 8);
@@ -91,7 +92,8 @@ static rago_status run_coarse(const IndexImpl* ix, const float* queries, int nq,
     record(mix, 1, s);
     e = launch_select_probes(ix, queries, reinterpret_cast<float*>(ws + L.scores), nq, nprobe,
                              reinterpret_cast<int32_t*>(ws + L.probe_list),
-                             reinterpret_cast<float*>(ws + L.probe_term), s);
+                             reinterpret_cast<float*>(ws + L.probe_term),
+                             reinterpret_cast<float*>(ws + L.probe_bias), s);
     if (e != cudaSuccess) return cuda_fail(e, "probe selection kernel");
     record(mix, 2, s);
     return RAGO_OK;
@@ -148,6 +150,7 @@ rago_status rago_index_load(rago_index** out, const void* coarse_centroids, rago
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ix->num_sms, cudaDevAttrMultiProcessorCount, ix->device);
     if (e == cudaSuccess) e = cudaMalloc(&ix->cnorm, (size_t)nlist * 4);
     if (e == cudaSuccess) e = cudaMalloc(&ix->cbT, (size_t)KSUB * d * 4);
+    if (e == cudaSuccess && metric == RAGO_L2 && N > 0) e = cudaMalloc(&ix->vterm, (size_t)N * 4);
     if (e != cudaSuccess) {
         rago_status st = e == cudaErrorMemoryAllocation ? fail(RAGO_ENOMEM, "device allocation failed")
                                                          : cuda_fail(e, "index setup");
@@ -158,6 +161,7 @@ rago_status rago_index_load(rago_index** out, const void* coarse_centroids, rago
     if (e == cudaSuccess) { ix->ev_valid = 1; e = scan_plan(ix, &ix->plan); }
     if (e == cudaSuccess) e = launch_centroid_norms(coarse_centroids, ix->coarse_bf16, nlist, d, ix->cnorm, s);
     if (e == cudaSuccess) e = launch_transpose_codebook(pq_codebooks, M, ix->dsub, ix->cbT, s);
+    if (e == cudaSuccess && ix->vterm) e = launch_vector_terms(ix, ix->vterm, s);
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) {
         rago_status st = cuda_fail(e, "index setup kernels");
@@ -174,6 +178,7 @@ rago_status rago_index_free(rago_index* index) {
     cudaDeviceSynchronize();
     if (ix->cnorm) cudaFree(ix->cnorm);
     if (ix->cbT) cudaFree(ix->cbT);
+    if (ix->vterm) cudaFree(ix->vterm);
     if (ix->ev_valid)
         for (int i = 0; i <= RAGO_NUM_STAGES; ++i) cudaEventDestroy(ix->ev[i]);
     delete ix;
@@ -243,7 +248,7 @@ rago_status rago_search(const rago_index* index, const float* queries, int32_t n
     if (st != RAGO_OK) return st;
 
     int32_t* probe_list = reinterpret_cast<int32_t*>(ws + L.probe_list);
-    float* probe_term = reinterpret_cast<float*>(ws + L.probe_term);
+    float* probe_term = reinterpret_cast<float*>(ws + L.probe_bias);  // what the scan adds per (query, list)
     int64_t* work_prefix = reinterpret_cast<int64_t*>(ws + L.work_prefix);
     unsigned long long* qthresh = reinterpret_cast<unsigned long long*>(ws + L.qthresh);
     int32_t* slot_cnt = reinterpret_cast<int32_t*>(ws + L.slot_cnt);

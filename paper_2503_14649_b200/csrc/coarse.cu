@@ -118,7 +118,8 @@ constexpr int SEL_THREADS = 256;
 template <bool BF16>
 __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
     const float* __restrict__ Q, const void* __restrict__ C, const float* __restrict__ scores, int nlist, int d,
-    int metric, int nprobe, int32_t* __restrict__ probe_list, float* __restrict__ probe_term) {
+    int metric, int nprobe, int32_t* __restrict__ probe_list, float* __restrict__ probe_term,
+    float* __restrict__ probe_bias) {
     __shared__ unsigned long long keys[TOPK_CAP];
     __shared__ unsigned long long keys2[MAX_K + PROBE_GUARD];
     __shared__ int cnt;
@@ -178,17 +179,33 @@ __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
         const float sc = orderable_f32((uint32_t)(key >> 32));
         probe_list[(size_t)q * nprobe + i] = (int32_t)(key & 0xFFFFFFFFull);
         probe_term[(size_t)q * nprobe + i] = metric == RAGO_L2 ? sc : -sc;
+        if (!(BF16 && metric == RAGO_L2)) probe_bias[(size_t)q * nprobe + i] = metric == RAGO_L2 ? sc : -sc;
+    }
+    // The scan's L2 expansion needs ||q - c||^2 for the UNROUNDED query; with a bf16 coarse quantiser
+    // that differs from the coarse distance above, so it is computed separately for the chosen lists.
+    if (BF16 && metric == RAGO_L2) {
+        for (int i = warp; i < nprobe; i += SEL_THREADS / 32) {
+            const uint32_t l = (uint32_t)(keys[i] & 0xFFFFFFFFull);
+            float acc = 0.f;
+            for (int j = lane; j < d; j += 32) {
+                const float t = qrow[j] - load_c<BF16>(C, (size_t)l * d + j);
+                acc = fmaf(t, t, acc);
+            }
+            for (int o = 16; o; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+            if (lane == 0) probe_bias[(size_t)q * nprobe + i] = acc;
+        }
     }
 }
 
 cudaError_t launch_select_probes(const IndexImpl* ix, const float* queries, const float* scores, int nq, int nprobe,
-                                 int32_t* probe_list, float* probe_term, cudaStream_t s) {
+                                 int32_t* probe_list, float* probe_term, float* probe_bias, cudaStream_t s) {
     if (ix->coarse_bf16)
         select_probes_kernel<true><<<nq, SEL_THREADS, 0, s>>>(queries, ix->centroids, scores, ix->nlist, ix->d,
-                                                              ix->metric, nprobe, probe_list, probe_term);
+                                                              ix->metric, nprobe, probe_list, probe_term, probe_bias);
     else
         select_probes_kernel<false><<<nq, SEL_THREADS, 0, s>>>(queries, ix->centroids, scores, ix->nlist, ix->d,
-                                                               ix->metric, nprobe, probe_list, probe_term);
+                                                               ix->metric, nprobe, probe_list, probe_term,
+                                                               probe_bias);
     count_launch();
     return cudaGetLastError();
 }

@@ -39,6 +39,7 @@ struct IndexImpl {
     // owned
     float* cnorm;  // [nlist] squared centroid norms (L2 coarse ranking)
     float* cbT;    // [256][M][dsub] codebook with the codeword index outermost
+    float* vterm;  // [N] per-vector term of the L2 expansion (null for inner product)
     int device, num_sms;
     ScanPlan plan;
     int profile;
@@ -149,10 +150,11 @@ void set_error(const char* fmt, ...);
 cudaError_t launch_centroid_norms(const void* centroids, int bf16, int nlist, int d, float* cnorm, cudaStream_t s);
 cudaError_t launch_coarse_scores(const IndexImpl* ix, const float* queries, int nq, float* scores, cudaStream_t s);
 cudaError_t launch_select_probes(const IndexImpl* ix, const float* queries, const float* scores, int nq, int nprobe,
-                                 int32_t* probe_list, float* probe_term, cudaStream_t s);
+                                 int32_t* probe_list, float* probe_term, float* probe_bias, cudaStream_t s);
 // scan.cu
 bool scan_supported(int M);
 cudaError_t scan_plan(const IndexImpl* ix, ScanPlan* plan);
+cudaError_t launch_vector_terms(const IndexImpl* ix, float* vterm, cudaStream_t s);
 cudaError_t launch_transpose_codebook(const float* cb, int M, int dsub, float* cbT, cudaStream_t s);
 cudaError_t launch_plan_work(const IndexImpl* ix, const int32_t* probe_list, int npairs, int tile_vecs,
                              int32_t* pair_tiles, int64_t* work_prefix, cudaStream_t s);

@@ -6,8 +6,9 @@ namespace rago {
 
 constexpr int MERGE_THREADS = 256;
 
-// Slot numbering: CTA b working on pair p writes slot p + b.  Along the CTAs' contiguous walk over the
-// pairs that number strictly increases, so the slots of one query form one range.
+// Slot numbering: CTA b working on query q writes slot q + b.  Along the CTAs' contiguous walk over the
+// batch that number strictly increases, so the slots of one query form one range (unused numbers in
+// between have count 0).
 __device__ __forceinline__ long long cta_of_unit(long long u, long long W, int ctas) {
     // CTA b owns units [b*W/ctas, (b+1)*W/ctas): the largest b with floor(b*W/ctas) <= u
     return ((u + 1) * ctas - 1) / W;
@@ -27,8 +28,8 @@ __global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(
     const long long u0 = work_prefix[(size_t)q * nprobe], u1 = work_prefix[(size_t)(q + 1) * nprobe];
     unsigned long long tau = KEY_MAX;
     if (u1 > u0) {
-        const long long s0 = (long long)q * nprobe + cta_of_unit(u0, W, ctas);
-        const long long s1 = (long long)(q + 1) * nprobe - 1 + cta_of_unit(u1 - 1, W, ctas);
+        const long long s0 = (long long)q + cta_of_unit(u0, W, ctas);
+        const long long s1 = (long long)q + cta_of_unit(u1 - 1, W, ctas);
         for (long long s = s0; s <= s1; ++s) {
             const int c = slot_cnt[s];  // <= k
             if (c == 0) continue;       // uniform: every thread reads the same word

@@ -3,8 +3,16 @@
 // One persistent CTA per SM walks a contiguous, equally sized share of the batch's code tiles
 // (pairs (query, probed list) in probe order, each list cut into tiles of TV vectors).  A producer
 // warp streams code tiles global -> shared with 1-D bulk copies (cp.async.bulk + mbarrier, a ring of
-// S tiles in flight); consumer warps build the fp32 lookup table of the current pair in shared
+// S tiles in flight); consumer warps build the fp32 lookup table of the current QUERY in shared
 // memory, then every lane owns one (virtual) code row of the tile and sums table entries.
+//
+// Score, smaller is better for both metrics:
+//   inner product:  -<q, c_p>  +  sum_m -<q_m, cw_m>
+//   squared L2:     ||q - c_p||^2  +  (||r||^2 + 2<c_p, r>)  +  sum_m -2<q_m, cw_m>      (r = decoded residual)
+// i.e. bias(q, list) + term(vector) + sum of entries of a table that depends on the query only, so a
+// table is rebuilt when the query changes, not at every probed list.  The expansion costs a few ulps
+// of the largest term (see vector_terms_kernel); results agree with the direct form to ~1e-6 relative
+// on data whose residuals are not tiny against the centroid distances.
 //
 // Shared-memory access pattern.  A code row is read as 32-bit words; at step (blk, il, t) lane L
 // reads word  blk*G + (il ^ a(L))  and uses byte  t ^ b(L)  of it, so that within any one
@@ -44,6 +52,7 @@ struct ScanArgs {
     const float* queries;
     const void* centroids;
     const float* cbT;
+    const float* vterm;  // [N] per-vector term (L2), null for inner product
     const int64_t* work_prefix;
     unsigned long long* qthresh;
     int32_t* slot_cnt;
@@ -80,6 +89,54 @@ struct Ctrl {
     uint32_t abort_flag;
 };
 static_assert(sizeof(Ctrl) <= CTRL_BYTES, "control block too large");
+
+// Table construction by the consumer threads.  Entry e = j * M + m of the transposed codebook is
+// DSUB contiguous floats; consecutive threads take consecutive entries (coalesced loads, and table
+// stores that walk the banks).  UNR entries per thread are loaded before any is used so that enough
+// requests are in flight to cover the L2 latency.
+template <class C, int D4>
+__device__ __forceinline__ void build_table(const float* __restrict__ cbT, const float* rT, float* lut, int ctid) {
+    constexpr int UNR = D4 >= 3 ? 4 : 8;
+    constexpr int TOTAL = KSUB * C::M;
+    for (int e0 = ctid; e0 < TOTAL; e0 += NCT * UNR) {
+        float4 cv[UNR][D4];
+#pragma unroll
+        for (int u = 0; u < UNR; ++u) {
+            const int e = e0 + u * NCT;
+#pragma unroll
+            for (int i = 0; i < D4; ++i)
+                cv[u][i] = e < TOTAL ? __ldg(reinterpret_cast<const float4*>(cbT + (size_t)e * (D4 * 4)) + i)
+                                     : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int u = 0; u < UNR; ++u) {
+            const int e = e0 + u * NCT;
+            if (e >= TOTAL) break;
+            const int j = e / C::M, m = e - j * C::M;
+            float acc = 0.f;
+#pragma unroll
+            for (int i = 0; i < D4; ++i) {
+                acc = fmaf(rT[(4 * i + 0) * C::M + m], cv[u][i].x, acc);
+                acc = fmaf(rT[(4 * i + 1) * C::M + m], cv[u][i].y, acc);
+                acc = fmaf(rT[(4 * i + 2) * C::M + m], cv[u][i].z, acc);
+                acc = fmaf(rT[(4 * i + 3) * C::M + m], cv[u][i].w, acc);
+            }
+            lut[j * C::LSTRIDE + m] = acc;
+            if (C::COPIES == 2) lut[j * C::LSTRIDE + C::M + m] = acc;
+        }
+    }
+}
+template <class C>
+__device__ __forceinline__ void build_table_any(const float* __restrict__ cbT, const float* rT, float* lut, int ctid,
+                                                int dsub) {
+    for (int e = ctid; e < KSUB * C::M; e += NCT) {
+        const int j = e / C::M, m = e - j * C::M;
+        float acc = 0.f;
+        for (int t = 0; t < dsub; ++t) acc = fmaf(rT[t * C::M + m], __ldg(cbT + (size_t)e * dsub + t), acc);
+        lut[j * C::LSTRIDE + m] = acc;
+        if (C::COPIES == 2) lut[j * C::LSTRIDE + C::M + m] = acc;
+    }
+}
 
 template <int WV, int G, int R>
 __global__ void __launch_bounds__(SCAN_THREADS, 1) scan_kernel(const ScanArgs a) {
@@ -212,13 +269,15 @@ __global__ void __launch_bounds__(SCAN_THREADS, 1) scan_kernel(const ScanArgs a)
 #pragma unroll
     for (int t = 0; t < 4; ++t) sel[t] = 0x4440u | (uint32_t)(t ^ xb);
 
-    int cur_pair = -1, cur_q = -1, lut_q = -1, lut_list = -1;
+    int cur_q = -1;
     unsigned long long tau = KEY_MAX;
     float bias = 0.f;
     int ub = 0;
     const int k = a.k;
     const bool ip = a.metric == RAGO_IP;
+    const float lut_scale = ip ? -1.f : -2.f;
 
+    // Close the current query's candidate buffer: keep at most k keys and park them in this CTA's slot.
     auto finalize = [&]() {
         csync();
         if (dead) return;
@@ -228,62 +287,28 @@ __global__ void __launch_bounds__(SCAN_THREADS, 1) scan_kernel(const ScanArgs a)
             if (dead) return;
             if (ctid == 0) atomicMin(&a.qthresh[cur_q], keys[k - 1]);
         }
-        const size_t slot = (size_t)cur_pair + blockIdx.x;
+        const size_t slot = (size_t)cur_q + blockIdx.x;
         for (int i = ctid; i < kept; i += NCT) a.slot_keys[slot * k + i] = keys[i];
         if (ctid == 0) a.slot_cnt[slot] = kept;
         csync();
     };
 
-    auto begin_pair = [&](const TileDesc& D) {
-        cur_pair = D.pair;
-        cur_q = D.pair / a.nprobe;
-        const bool need = ip ? (lut_q != cur_q) : (lut_q != cur_q || lut_list != D.list);
-        if (need) {
-            const float* qrow = a.queries + (size_t)cur_q * a.d;
-            for (int j = ctid; j < a.d; j += NCT) {
-                float v = qrow[j];
-                if (!ip) {
-                    const float c = a.coarse_bf16
-                        ? __bfloat162float(static_cast<const __nv_bfloat16*>(a.centroids)[(size_t)D.list * a.d + j])
-                        : static_cast<const float*>(a.centroids)[(size_t)D.list * a.d + j];
-                    v -= c;
-                }
-                rT[(j % a.dsub) * C::M + j / a.dsub] = v;
-            }
-            csync();
-            if (dead) return;
-            const int dsub = a.dsub;
-            for (int e = ctid; e < KSUB * C::M; e += NCT) {
-                const int j = e / C::M, m = e - j * C::M;
-                const float* cw = a.cbT + (size_t)e * dsub;
-                float acc = 0.f;
-                if ((dsub & 3) == 0) {
-                    for (int t = 0; t < dsub; t += 4) {
-                        const float4 cv = __ldg(reinterpret_cast<const float4*>(cw + t));
-                        const float c4[4] = {cv.x, cv.y, cv.z, cv.w};
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const float r = rT[(t + i) * C::M + m];
-                            if (ip) acc = fmaf(r, c4[i], acc);
-                            else { const float df = r - c4[i]; acc = fmaf(df, df, acc); }
-                        }
-                    }
-                } else {
-                    for (int t = 0; t < dsub; ++t) {
-                        const float r = rT[t * C::M + m], cv = __ldg(cw + t);
-                        if (ip) acc = fmaf(r, cv, acc);
-                        else { const float df = r - cv; acc = fmaf(df, df, acc); }
-                    }
-                }
-                lut[j * C::LSTRIDE + m] = acc;
-                if (C::COPIES == 2) lut[j * C::LSTRIDE + C::M + m] = acc;
-            }
-            lut_q = cur_q;
-            lut_list = D.list;
-        }
-        bias = ip ? a.probe_term[D.pair] : 0.f;
+    // Table of a query: lut[j][m] = lut_scale * <q_m, codeword j of sub-space m>.
+    auto begin_query = [&](int q) {
+        cur_q = q;
+        const float* qrow = a.queries + (size_t)q * a.d;
+        for (int j = ctid; j < a.d; j += NCT) rT[(j % a.dsub) * C::M + j / a.dsub] = lut_scale * qrow[j];
         if (ctid == 0) ctrl->cnt = 0;
-        tau = *reinterpret_cast<volatile unsigned long long*>(&a.qthresh[cur_q]);
+        csync();
+        if (dead) return;
+        switch (a.dsub) {
+            case 4: build_table<C, 1>(a.cbT, rT, lut, ctid); break;
+            case 8: build_table<C, 2>(a.cbT, rT, lut, ctid); break;
+            case 12: build_table<C, 3>(a.cbT, rT, lut, ctid); break;
+            case 16: build_table<C, 4>(a.cbT, rT, lut, ctid); break;
+            default: build_table_any<C>(a.cbT, rT, lut, ctid, a.dsub); break;
+        }
+        tau = *reinterpret_cast<volatile unsigned long long*>(&a.qthresh[q]);
         ub = 0;
         csync();
     };
@@ -294,11 +319,17 @@ __global__ void __launch_bounds__(SCAN_THREADS, 1) scan_kernel(const ScanArgs a)
         if (dead) break;
         const TileDesc D = ctrl->desc[st];
         if (D.newpair) {
-            if (cur_pair >= 0) finalize();
-            if (dead) break;
-            begin_pair(D);
-            if (dead) break;
-        } else if (ub + C::TV > TOPK_CAP) {
+            const int q = D.pair / a.nprobe;
+            if (q != cur_q) {
+                if (cur_q >= 0) finalize();
+                if (dead) break;
+                begin_query(q);
+                if (dead) break;
+            }
+            const float term = a.probe_term[D.pair];
+            bias = ip ? -term : term;
+        }
+        if (ub + C::TV > TOPK_CAP) {
             csync();
             if (dead) break;
             if (ctrl->cnt + C::TV > TOPK_CAP) {
@@ -325,6 +356,9 @@ __global__ void __launch_bounds__(SCAN_THREADS, 1) scan_kernel(const ScanArgs a)
             if (vr0 >= nvr) break;
             const int vr = vr0 + lane;
             const uint32_t rowoff = tile_base + (uint32_t)vr * C::MV;
+            // per-vector term of the L2 expansion (0 for inner product); issued early, used last
+            float vt = 0.f;
+            if (a.vterm != nullptr && vr < nvr && sr == 0) vt = __ldg(a.vterm + D.pos0 + (uint32_t)(vr / R));
             float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int blk = 0; blk < WV / G; ++blk) {
@@ -342,7 +376,7 @@ __global__ void __launch_bounds__(SCAN_THREADS, 1) scan_kernel(const ScanArgs a)
             float s = (acc[0] + acc[1]) + (acc[2] + acc[3]);
             if (R >= 2) s += __shfl_xor_sync(0xffffffffu, s, 1);
             if (R >= 4) s += __shfl_xor_sync(0xffffffffu, s, 2);
-            const float score = ip ? -(bias + s) : s;
+            const float score = (bias + vt) + s;  // smaller is better for both metrics
             const unsigned long long key = make_key(score, D.pos0 + (uint32_t)(vr / R));
             warp_push(keys, &ctrl->cnt, vr < nvr && sr == 0 && key < tau, key);
         }
@@ -350,7 +384,7 @@ __global__ void __launch_bounds__(SCAN_THREADS, 1) scan_kernel(const ScanArgs a)
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&ctrl->empty[st]));
     }
-    if (!dead && cur_pair >= 0) finalize();
+    if (!dead && cur_q >= 0) finalize();
 }
 
 // ---- host side ----------------------------------------------------------------------------------
@@ -403,6 +437,7 @@ cudaError_t launch_scan(const IndexImpl* ix, const ScanPlan& plan, const float* 
     ScanArgs a;
     a.codes = ix->codes; a.list_offsets = ix->list_offsets; a.probe_list = probe_list; a.probe_term = probe_term;
     a.queries = queries; a.centroids = ix->centroids; a.cbT = ix->cbT; a.work_prefix = work_prefix;
+    a.vterm = ix->vterm;
     a.qthresh = qthresh; a.slot_cnt = slot_cnt; a.slot_keys = slot_keys; a.err = err_word;
     a.coarse_bf16 = ix->coarse_bf16; a.npairs = nq * nprobe; a.nprobe = nprobe; a.d = ix->d; a.dsub = ix->dsub;
     a.metric = ix->metric; a.k = k; a.stages = plan.stages;
@@ -421,6 +456,53 @@ __global__ void transpose_codebook_kernel(const float* __restrict__ cb, int M, i
 }
 cudaError_t launch_transpose_codebook(const float* cb, int M, int dsub, float* cbT, cudaStream_t s) {
     transpose_codebook_kernel<<<256, 256, 0, s>>>(cb, M, dsub, cbT);
+    count_launch();
+    return cudaGetLastError();
+}
+
+// ---- per-vector term of the squared-L2 expansion ------------------------------------------------
+// ||q - (c + r)||^2 = ||q - c||^2 + (||r||^2 + 2<c, r>) - 2<q, r>,  r = decoded residual of the vector.
+// The middle term depends on the stored vector only; it is computed once per index, in double, one
+// warp per vector (lanes over sub-spaces), and rounded to float once.
+template <bool BF16>
+__global__ void vector_terms_kernel(const uint8_t* __restrict__ codes, const int64_t* __restrict__ offsets,
+                                    const void* __restrict__ centroids, const float* __restrict__ cb, long long N,
+                                    int nlist, int d, int M, int dsub, float* __restrict__ vterm) {
+    const int lane = threadIdx.x & 31;
+    const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
+    for (long long pos = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; pos < N; pos += warps) {
+        int lo = 0, hi = nlist;  // offsets[lo] <= pos < offsets[hi]
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (offsets[mid] <= pos) lo = mid; else hi = mid;
+        }
+        double acc = 0.0;
+        for (int m = lane; m < M; m += 32) {
+            const int code = codes[pos * M + m];
+            const float* cw = cb + ((size_t)m * KSUB + code) * dsub;
+            for (int t = 0; t < dsub; ++t) {
+                const size_t ci = (size_t)lo * d + m * dsub + t;
+                const double c = BF16 ? (double)__bfloat162float(static_cast<const __nv_bfloat16*>(centroids)[ci])
+                                      : (double)static_cast<const float*>(centroids)[ci];
+                const double r = (double)cw[t];
+                acc += r * (r + 2.0 * c);
+            }
+        }
+        for (int o = 16; o; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        if (lane == 0) vterm[pos] = (float)acc;
+    }
+}
+
+cudaError_t launch_vector_terms(const IndexImpl* ix, float* vterm, cudaStream_t s) {
+    if (ix->N == 0) return cudaSuccess;
+    const long long want = (ix->N * 32 + 255) / 256;
+    const int blocks = (int)(want < 148LL * 64 ? want : 148LL * 64);
+    if (ix->coarse_bf16)
+        vector_terms_kernel<true><<<blocks, 256, 0, s>>>(ix->codes, ix->list_offsets, ix->centroids, ix->codebooks,
+                                                         ix->N, ix->nlist, ix->d, ix->M, ix->dsub, vterm);
+    else
+        vector_terms_kernel<false><<<blocks, 256, 0, s>>>(ix->codes, ix->list_offsets, ix->centroids, ix->codebooks,
+                                                          ix->N, ix->nlist, ix->d, ix->M, ix->dsub, vterm);
     count_launch();
     return cudaGetLastError();
 }
