@@ -150,7 +150,7 @@ rago_status rago_index_load(rago_index** out, const void* coarse_centroids, rago
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ix->num_sms, cudaDevAttrMultiProcessorCount, ix->device);
     if (e == cudaSuccess) e = cudaMalloc(&ix->cnorm, (size_t)nlist * 4);
     if (e == cudaSuccess) e = cudaMalloc(&ix->cbT, (size_t)KSUB * d * 4);
-    if (e == cudaSuccess && metric == RAGO_L2 && N > 0) e = cudaMalloc(&ix->vterm, (size_t)N * 4);
+    if (e == cudaSuccess && metric == RAGO_L2 && N > 0) e = cudaMalloc(&ix->vterm, ((size_t)N + 4) * 4);  // + slack: tiles copy whole 16-byte groups
     if (e != cudaSuccess) {
         rago_status st = e == cudaErrorMemoryAllocation ? fail(RAGO_ENOMEM, "device allocation failed")
                                                          : cuda_fail(e, "index setup");
@@ -338,6 +338,7 @@ rago_status rago_check(void* workspace, void* cuda_stream) {
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) return cuda_fail(e, "reading the error word");
     if (w == ERR_WAIT_TIMEOUT) return fail(RAGO_ETIMEOUT, "a bounded device-side wait expired");
+    if (w == ERR_SMEM_LAYOUT) return fail(RAGO_ECUDA, "the scan kernel's shared-memory plan does not fit this device");
     if (w != ERR_NONE) return fail(RAGO_ECUDA, "device error word = %u", w);
     return RAGO_OK;
 }

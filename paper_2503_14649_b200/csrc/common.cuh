@@ -16,7 +16,7 @@ constexpr int PROBE_GUARD = 8;       // extra coarse candidates re-scored exactl
 constexpr unsigned long long KEY_MAX = 0xFFFFFFFFFFFFFFFFull;
 
 // Device-side error word (first word of every workspace).
-enum : uint32_t { ERR_NONE = 0, ERR_WAIT_TIMEOUT = 1 };
+enum : uint32_t { ERR_NONE = 0, ERR_WAIT_TIMEOUT = 1, ERR_SMEM_LAYOUT = 2 };
 
 // Launch shape of the table-build + scan kernel for one index (fixed at index load).
 struct ScanPlan {

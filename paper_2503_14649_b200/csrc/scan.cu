@@ -12,14 +12,21 @@
 // i.e. bias(q, list) + term(vector) + sum of entries of a table that depends on the query only, so a
 // table is rebuilt when the query changes, not at every probed list.  The expansion costs a few ulps
 // of the largest term (see vector_terms_kernel); results agree with the direct form to ~1e-6 relative
-// on data whose residuals are not tiny against the centroid distances.
+// on data whose residuals are not tiny against the centroid distances.  The per-vector terms of a tile
+// travel with it (a second bulk copy on the same barrier).
 //
 // Shared-memory access pattern.  A code row is read as 32-bit words; at step (blk, il, t) lane L
 // reads word  blk*G + (il ^ a(L))  and uses byte  t ^ b(L)  of it, so that within any one
 // instruction the 32 lanes touch 32 different banks both for the code words (rows are M bytes
-// apart) and for the table (stored [codeword][sub-space], bank = sub-space mod 32).  Rows wider than
-// 32*odd bytes are split into R "virtual rows" handled by adjacent lanes and summed with a shuffle;
-// sub-space counts that are 16 mod 32 keep two table copies so lanes L and L^4 never collide.
+// apart) and for the table (bank = table column mod 32).  Rows wider than 32*odd bytes are split
+// into R "virtual rows" handled by adjacent lanes and summed with a shuffle; sub-space counts that
+// are 16 mod 32 keep two table copies so lanes L and L^4 never collide.
+//
+// Table addressing.  Per code byte the inner loop spends one byte-permute, one shared load and one
+// add: the table is stored as 64-column banks of 256 rows x 256 bytes that start at a shared-memory
+// address which is a multiple of 64 KB, so the load address  (bank << 16) | (code << 8) | column*4
+// is assembled by a single PRMT from the code word and a per-lane constant.  Tables wider than two
+// banks (M = 80 with its two copies) fall back to a multiply-add address.
 //
 // Candidates better than the running threshold go to a shared buffer (topk.cuh); the threshold of a
 // query is shared between CTAs through global memory, which only ever removes keys that cannot be
@@ -28,12 +35,11 @@
 
 namespace rago {
 
-constexpr int NCW = 8;                          // consumer warps
-constexpr int NCT = NCW * 32;                   // consumer threads
-constexpr int SCAN_THREADS = NCT + 32;          // + one producer warp
 constexpr int MAX_STAGES = 4;
-constexpr int SMEM_LIMIT = 227 * 1024;
+constexpr int SMEM_OPTIN = 227 * 1024;          // dynamic shared memory asked for (the sm_100 per-block limit)
+constexpr uint32_t SMEM_BASE_EXPECTED = 1024;   // shared-window address of dynamic shared memory when the kernel has no static part
 constexpr int CTRL_BYTES = 1024;
+constexpr uint32_t LUT_WINDOW = 0x10000;        // banked tables start here (absolute shared address)
 
 struct TileDesc {
     int32_t pair;      // index into probe_list (query * nprobe + rank)
@@ -41,7 +47,9 @@ struct TileDesc {
     uint32_t pos0;     // storage position of the tile's first vector
     int32_t nvec;      // vectors in this tile
     int32_t newpair;   // first tile of this pair inside this CTA
-    int32_t pad[3];
+    int32_t vrem;      // index of the first vector's term inside the staged term block (0..3)
+    uint32_t tile_addr;  // shared address of the stage's code tile
+    uint32_t vt_addr;    // shared address of the stage's per-vector terms
 };
 
 struct ScanArgs {
@@ -50,36 +58,105 @@ struct ScanArgs {
     const int32_t* probe_list;
     const float* probe_term;
     const float* queries;
-    const void* centroids;
     const float* cbT;
-    const float* vterm;  // [N] per-vector term (L2), null for inner product
+    const float* vterm;  // [N + 4] per-vector term (L2), null for inner product
     const int64_t* work_prefix;
     unsigned long long* qthresh;
     int32_t* slot_cnt;
     unsigned long long* slot_keys;
     uint32_t* err;
-    int32_t coarse_bf16, npairs, nprobe, d, dsub, metric, k, stages;
+    int32_t npairs, nprobe, d, dsub, metric, k, stages;
+    uint32_t dyn_bytes;
 };
 
-template <int WV, int G, int R>
+template <int WV, int G, int R, int NCW_>
 struct Cfg {
+    static constexpr int NCW = NCW_;                    // consumer warps
+    static constexpr int NCT = NCW * 32;                // consumer threads
+    static constexpr int THREADS = NCT + 32;            // + one producer warp
     static constexpr int MV = WV * 4;                   // bytes per virtual row
     static constexpr int M = MV * R;                    // code bytes per vector
+    static constexpr int NBLK = WV / G;                 // blocks of G words per virtual row
     static constexpr int COPIES = G == 4 ? 2 : 1;
-    static constexpr int LSTRIDE = M * COPIES;          // table row stride (words)
-    static constexpr int LUT_BYTES = KSUB * LSTRIDE * 4;
-    static constexpr int RGW = MV >= 96 ? 1 : (96 / MV > 4 ? 4 : 96 / MV);  // 32-row groups per warp per tile
+    static constexpr int COPY_OFF = COPIES == 1 ? 0 : (M == 16 ? 16 : (M == 48 ? 80 : M));  // 16 mod 32
+    static constexpr int NCOLS = COPIES == 1 ? M : COPY_OFF + M;
+    static constexpr bool BANKED = NCOLS <= 128;        // PRMT addressing
+    static constexpr int NBANK = (NCOLS + 63) / 64;
+    static constexpr int LSTRIDE = NCOLS;               // words per table row (multiply-add addressing)
+    static constexpr int LUT_BYTES = BANKED ? NBANK * 65536 : KSUB * LSTRIDE * 4;
+    static constexpr int RGW = MV >= 80 ? 1 : 2;        // 32-row groups per warp per tile
     static constexpr int TILE_VROWS = NCW * 32 * RGW;
     static constexpr int TV = TILE_VROWS / R;           // vectors per tile
     static constexpr int TILE_BYTES = TILE_VROWS * MV;
-    static constexpr int KEYS_OFF = LUT_BYTES;
-    static constexpr int RT_OFF = KEYS_OFF + TOPK_CAP * 8;
+    static constexpr int VT_BYTES = (TV + 4) * 4;       // staged per-vector terms (start rounded down to 16 bytes)
+    static_assert(WV % G == 0, "virtual rows are whole blocks");
     static_assert(TILE_VROWS % R == 0, "tile must hold whole vectors");
     static_assert(TV + MAX_K <= TOPK_CAP, "one tile of pushes plus k kept keys must fit the candidate buffer");
-    static_assert(LSTRIDE % 32 == 0, "table rows must keep bank = column mod 32");
+    static_assert(COPY_OFF % 32 == (COPIES == 2 ? 16 : 0), "second copy must sit 16 banks away");
+    static_assert(LSTRIDE % 32 == 0 || BANKED, "table rows must keep bank = column mod 32");
+    static_assert(VT_BYTES % 16 == 0 && TILE_BYTES % 16 == 0, "bulk-copy destinations are 16-byte granular");
+    // banked addressing: the columns one lane touches in one block stay inside one 64-column bank
+    __host__ __device__ static constexpr bool banked_ok() {
+        for (int copy = 0; copy < COPIES; ++copy)
+            for (int sr = 0; sr < R; ++sr)
+                for (int blk = 0; blk < NBLK; ++blk) {
+                    const int cb = copy * COPY_OFF + sr * MV;
+                    if ((cb % 64) + ((blk * 4 * G) % 64) + 4 * G > 64) return false;
+                }
+        return true;
+    }
+    static_assert(!BANKED || banked_ok(), "a lane's columns of one block straddle two banks");
+    // address of table entry (code j, column col) relative to the table's start
+    __host__ __device__ static constexpr uint32_t lut_off(int j, int col) {
+        return BANKED ? (uint32_t)(col / 64) * 65536u + (uint32_t)j * 256u + (uint32_t)(col % 64) * 4u
+                      : ((uint32_t)j * LSTRIDE + (uint32_t)col) * 4u;
+    }
+    // immediate added for block blk (banked addressing)
+    __host__ __device__ static constexpr uint32_t blk_imm(int blk) {
+        return (uint32_t)((blk * 4 * G) / 64) * 65536u + (uint32_t)((blk * 4 * G) % 64) * 4u;
+    }
 };
 
-// Control block at the end of dynamic shared memory.
+// Absolute shared-memory addresses of everything the kernel keeps there.  The same function runs on
+// the host (to choose the number of stages, with the expected window base) and in the kernel (with
+// the real base); a plan that does not fit makes the kernel report an error and return.
+struct SmemPlan {
+    uint32_t lut, ctrl, keys, rT, vt[MAX_STAGES], tile[MAX_STAGES];
+    int ok;
+};
+
+template <class C>
+__host__ __device__ inline SmemPlan plan_smem(uint32_t base, uint32_t dyn_bytes, int d, int stages) {
+    SmemPlan p;
+    p.ok = 1;
+    const uint32_t end = base + dyn_bytes;
+    uint32_t lo_cur, lo_end, hi_cur;
+    if (C::BANKED) {
+        p.lut = LUT_WINDOW;
+        if (base > LUT_WINDOW) p.ok = 0;
+        lo_cur = base; lo_end = LUT_WINDOW; hi_cur = LUT_WINDOW + C::LUT_BYTES;
+    } else {
+        p.lut = (base + 127u) & ~127u;
+        lo_cur = lo_end = 0; hi_cur = p.lut + C::LUT_BYTES;
+    }
+    if (hi_cur > end) p.ok = 0;
+    auto take = [&](uint32_t bytes, uint32_t align) -> uint32_t {
+        uint32_t a = (lo_cur + align - 1) & ~(align - 1);
+        if (a + bytes <= lo_end) { lo_cur = a + bytes; return a; }
+        a = (hi_cur + align - 1) & ~(align - 1);
+        if (a + bytes <= end) { hi_cur = a + bytes; return a; }
+        p.ok = 0;
+        return base;
+    };
+    p.ctrl = take(CTRL_BYTES, 16);
+    p.keys = take(TOPK_CAP * 8, 16);
+    p.rT = take((uint32_t)d * 4, 16);
+    for (int s = 0; s < MAX_STAGES; ++s) p.vt[s] = s < stages ? take(C::VT_BYTES, 16) : base;
+    for (int s = 0; s < MAX_STAGES; ++s) p.tile[s] = s < stages ? take(C::TILE_BYTES, 128) : base;
+    return p;
+}
+
+// Control block.
 struct Ctrl {
     unsigned long long full[MAX_STAGES];
     unsigned long long empty[MAX_STAGES];
@@ -90,19 +167,35 @@ struct Ctrl {
 };
 static_assert(sizeof(Ctrl) <= CTRL_BYTES, "control block too large");
 
+template <int IMM>
+__device__ __forceinline__ float lds_f32_imm(uint32_t addr) {
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1+%2];" : "=f"(v) : "r"(addr), "n"(IMM));
+    return v;
+}
+template <int IMM>
+__device__ __forceinline__ uint32_t lds_u32_imm(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1+%2];" : "=r"(v) : "r"(addr), "n"(IMM));
+    return v;
+}
+__device__ __forceinline__ void sts_f32(uint32_t addr, float v) {
+    asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+}
+
 // Table construction by the consumer threads.  Entry e = j * M + m of the transposed codebook is
 // DSUB contiguous floats; consecutive threads take consecutive entries (coalesced loads, and table
 // stores that walk the banks).  UNR entries per thread are loaded before any is used so that enough
 // requests are in flight to cover the L2 latency.
 template <class C, int D4>
-__device__ __forceinline__ void build_table(const float* __restrict__ cbT, const float* rT, float* lut, int ctid) {
+__device__ __forceinline__ void build_table(const float* __restrict__ cbT, const float* rT, uint32_t lut, int ctid) {
     constexpr int UNR = D4 >= 3 ? 4 : 8;
     constexpr int TOTAL = KSUB * C::M;
-    for (int e0 = ctid; e0 < TOTAL; e0 += NCT * UNR) {
+    for (int e0 = ctid; e0 < TOTAL; e0 += C::NCT * UNR) {
         float4 cv[UNR][D4];
 #pragma unroll
         for (int u = 0; u < UNR; ++u) {
-            const int e = e0 + u * NCT;
+            const int e = e0 + u * C::NCT;
 #pragma unroll
             for (int i = 0; i < D4; ++i)
                 cv[u][i] = e < TOTAL ? __ldg(reinterpret_cast<const float4*>(cbT + (size_t)e * (D4 * 4)) + i)
@@ -110,7 +203,7 @@ __device__ __forceinline__ void build_table(const float* __restrict__ cbT, const
         }
 #pragma unroll
         for (int u = 0; u < UNR; ++u) {
-            const int e = e0 + u * NCT;
+            const int e = e0 + u * C::NCT;
             if (e >= TOTAL) break;
             const int j = e / C::M, m = e - j * C::M;
             float acc = 0.f;
@@ -121,34 +214,71 @@ __device__ __forceinline__ void build_table(const float* __restrict__ cbT, const
                 acc = fmaf(rT[(4 * i + 2) * C::M + m], cv[u][i].z, acc);
                 acc = fmaf(rT[(4 * i + 3) * C::M + m], cv[u][i].w, acc);
             }
-            lut[j * C::LSTRIDE + m] = acc;
-            if (C::COPIES == 2) lut[j * C::LSTRIDE + C::M + m] = acc;
+            sts_f32(lut + C::lut_off(j, m), acc);
+            if (C::COPIES == 2) sts_f32(lut + C::lut_off(j, C::COPY_OFF + m), acc);
         }
     }
 }
 template <class C>
-__device__ __forceinline__ void build_table_any(const float* __restrict__ cbT, const float* rT, float* lut, int ctid,
-                                                int dsub) {
-    for (int e = ctid; e < KSUB * C::M; e += NCT) {
+__device__ __forceinline__ void build_table_any(const float* __restrict__ cbT, const float* rT, uint32_t lut,
+                                                int ctid, int dsub) {
+    for (int e = ctid; e < KSUB * C::M; e += C::NCT) {
         const int j = e / C::M, m = e - j * C::M;
         float acc = 0.f;
         for (int t = 0; t < dsub; ++t) acc = fmaf(rT[t * C::M + m], __ldg(cbT + (size_t)e * dsub + t), acc);
-        lut[j * C::LSTRIDE + m] = acc;
-        if (C::COPIES == 2) lut[j * C::LSTRIDE + C::M + m] = acc;
+        sts_f32(lut + C::lut_off(j, m), acc);
+        if (C::COPIES == 2) sts_f32(lut + C::lut_off(j, C::COPY_OFF + m), acc);
     }
 }
 
-template <int WV, int G, int R>
-__global__ void __launch_bounds__(SCAN_THREADS, 1) scan_kernel(const ScanArgs a) {
-    using C = Cfg<WV, G, R>;
+// One block (G code words = 4G sub-spaces) of one virtual row: load the words, then 4G lookups.
+template <class C, int G, int BLK>
+__device__ __forceinline__ void scan_block(uint32_t rowaddr, const uint32_t (&xo)[G], const uint32_t (&cc)[G][2],
+                                           const uint32_t (&sel)[4], const uint32_t (&lo)[G][4], uint32_t lut,
+                                           float (&acc)[4]) {
+    uint32_t x[G];
+#pragma unroll
+    for (int il = 0; il < G; ++il) x[il] = lds_u32_imm<BLK * G * 4>(rowaddr + xo[il]);
+#pragma unroll
+    for (int il = 0; il < G; ++il) {
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            if (C::BANKED) {
+                const uint32_t a = __byte_perm(x[il], cc[il][t >> 1], sel[t]);
+                acc[t] += lds_f32_imm<(int)C::blk_imm(BLK)>(a);
+            } else {
+                const uint32_t j = __byte_perm(x[il], 0u, sel[t]);
+                acc[t] += lds_f32_imm<BLK * G * 16>(lut + j * (uint32_t)(C::LSTRIDE * 4) + lo[il][t]);
+            }
+        }
+    }
+}
+template <class C, int G, int BLK>
+struct ScanBlocks {
+    __device__ __forceinline__ static void run(uint32_t rowaddr, const uint32_t (&xo)[G], const uint32_t (&cc)[G][2],
+                                               const uint32_t (&sel)[4], const uint32_t (&lo)[G][4], uint32_t lut,
+                                               float (&acc)[4]) {
+        scan_block<C, G, BLK>(rowaddr, xo, cc, sel, lo, lut, acc);
+        if constexpr (BLK + 1 < C::NBLK) ScanBlocks<C, G, BLK + 1>::run(rowaddr, xo, cc, sel, lo, lut, acc);
+    }
+};
+
+template <int WV, int G, int R, int NCW_>
+__global__ void __launch_bounds__(Cfg<WV, G, R, NCW_>::THREADS, 1) scan_kernel(const ScanArgs a) {
+    using C = Cfg<WV, G, R, NCW_>;
+    constexpr int NCW = C::NCW, NCT = C::NCT;
     extern __shared__ __align__(1024) uint8_t smem[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int S = a.stages;
-    const uint32_t tiles_off = (uint32_t)align_up((size_t)C::RT_OFF + (size_t)a.d * 4, 128);
-    Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem + tiles_off + (size_t)S * C::TILE_BYTES);
-    float* lut = reinterpret_cast<float*>(smem);
-    unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem + C::KEYS_OFF);
-    float* rT = reinterpret_cast<float*>(smem + C::RT_OFF);
+    const uint32_t base = smem_u32(smem);
+    const SmemPlan P = plan_smem<C>(base, a.dyn_bytes, a.d, S);
+    if (!P.ok) {  // uniform: every thread sees the same plan
+        if (tid == 0) atomicExch(a.err, (uint32_t)ERR_SMEM_LAYOUT);
+        return;
+    }
+    Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem + (P.ctrl - base));
+    unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem + (P.keys - base));
+    float* rT = reinterpret_cast<float*>(smem + (P.rT - base));
     volatile uint32_t* abort_flag = &ctrl->abort_flag;
 
     if (tid == 0) {
@@ -217,17 +347,23 @@ __global__ void __launch_bounds__(SCAN_THREADS, 1) scan_kernel(const ScanArgs a)
                 const long long v0 = t_in_pair * C::TV;
                 long long nvec = len - v0;
                 if (nvec > C::TV) nvec = C::TV;
+                const uint32_t pos0 = (uint32_t)(off + v0);
                 TileDesc& D = ctrl->desc[st];
                 D.pair = cache_base + cur;
                 D.list = list;
-                D.pos0 = (uint32_t)(off + v0);
+                D.pos0 = pos0;
                 D.nvec = (int32_t)nvec;
                 D.newpair = (n == 0 || t_in_pair == 0) ? 1 : 0;
+                D.vrem = (int32_t)(pos0 & 3u);
+                D.tile_addr = P.tile[st];
+                D.vt_addr = P.vt[st];
                 const uint32_t bytes = (uint32_t)nvec * C::M;
+                // per-vector terms: start rounded down to a 16-byte boundary, length rounded up
+                const uint32_t vbytes = a.vterm ? (((pos0 & 3u) + (uint32_t)nvec) * 4u + 15u) & ~15u : 0u;
                 const uint32_t bar = smem_u32(&ctrl->full[st]);
-                mbar_arrive_expect_tx(bar, bytes);
-                bulk_g2s(smem_u32(smem + tiles_off + (size_t)st * C::TILE_BYTES),
-                         a.codes + (size_t)(off + v0) * C::M, bytes, bar);
+                mbar_arrive_expect_tx(bar, bytes + vbytes);
+                bulk_g2s(P.tile[st], a.codes + (size_t)pos0 * C::M, bytes, bar);
+                if (vbytes) bulk_g2s(P.vt[st], a.vterm + (pos0 & ~3u), vbytes, bar);
             }
             issued = n + 1;
         }
@@ -258,16 +394,26 @@ __global__ void __launch_bounds__(SCAN_THREADS, 1) scan_kernel(const ScanArgs a)
     const int xb = lane & 3;                            // byte xor
     const int copy = G == 4 ? ((lane >> 2) & 1) : 0;
     const int sr = lane % R;                            // which slice of the vector this lane sums
-    uint32_t lo[G][4], xo[G], sel[4];
+    const int colbase = copy * C::COPY_OFF + sr * C::MV;
+    uint32_t xo[G], cc[G][2], lo[G][4], sel[4];
 #pragma unroll
     for (int il = 0; il < G; ++il) {
         xo[il] = 4u * (uint32_t)(il ^ xa);
 #pragma unroll
         for (int t = 0; t < 4; ++t)
-            lo[il][t] = 4u * (uint32_t)(copy * C::M + sr * C::MV + 4 * (il ^ xa) + (t ^ xb));
+            lo[il][t] = C::BANKED ? 0u : 4u * (uint32_t)(colbase + 4 * (il ^ xa) + (t ^ xb));
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            // bytes: column*4 for t = 2h, column*4 for t = 2h+1, table bank, 0
+            const uint32_t c0 = 4u * (uint32_t)((colbase % 64) + 4 * (il ^ xa) + ((2 * h) ^ xb));
+            const uint32_t c1 = 4u * (uint32_t)((colbase % 64) + 4 * (il ^ xa) + ((2 * h + 1) ^ xb));
+            cc[il][h] = c0 | (c1 << 8) | (((P.lut >> 16) + (uint32_t)(colbase / 64)) << 16);
+        }
     }
 #pragma unroll
-    for (int t = 0; t < 4; ++t) sel[t] = 0x4440u | (uint32_t)(t ^ xb);
+    for (int t = 0; t < 4; ++t)
+        sel[t] = C::BANKED ? ((uint32_t)(4 + (t & 1)) | ((uint32_t)(t ^ xb) << 4) | 0x7600u)
+                           : (0x4440u | (uint32_t)(t ^ xb));
 
     int cur_q = -1;
     unsigned long long tau = KEY_MAX;
@@ -293,7 +439,7 @@ __global__ void __launch_bounds__(SCAN_THREADS, 1) scan_kernel(const ScanArgs a)
         csync();
     };
 
-    // Table of a query: lut[j][m] = lut_scale * <q_m, codeword j of sub-space m>.
+    // Table of a query: entry (j, m) = lut_scale * <q_m, codeword j of sub-space m>.
     auto begin_query = [&](int q) {
         cur_q = q;
         const float* qrow = a.queries + (size_t)q * a.d;
@@ -302,11 +448,11 @@ __global__ void __launch_bounds__(SCAN_THREADS, 1) scan_kernel(const ScanArgs a)
         csync();
         if (dead) return;
         switch (a.dsub) {
-            case 4: build_table<C, 1>(a.cbT, rT, lut, ctid); break;
-            case 8: build_table<C, 2>(a.cbT, rT, lut, ctid); break;
-            case 12: build_table<C, 3>(a.cbT, rT, lut, ctid); break;
-            case 16: build_table<C, 4>(a.cbT, rT, lut, ctid); break;
-            default: build_table_any<C>(a.cbT, rT, lut, ctid, a.dsub); break;
+            case 4: build_table<C, 1>(a.cbT, rT, P.lut, ctid); break;
+            case 8: build_table<C, 2>(a.cbT, rT, P.lut, ctid); break;
+            case 12: build_table<C, 3>(a.cbT, rT, P.lut, ctid); break;
+            case 16: build_table<C, 4>(a.cbT, rT, P.lut, ctid); break;
+            default: build_table_any<C>(a.cbT, rT, P.lut, ctid, a.dsub); break;
         }
         tau = *reinterpret_cast<volatile unsigned long long*>(&a.qthresh[q]);
         ub = 0;
@@ -349,33 +495,22 @@ __global__ void __launch_bounds__(SCAN_THREADS, 1) scan_kernel(const ScanArgs a)
 
         // ---- scan this tile: warp w owns row groups w*RGW .. w*RGW+RGW-1 ----
         const int nvr = D.nvec * R;
-        const uint32_t tile_base = tiles_off + (uint32_t)st * C::TILE_BYTES;
+        const uint32_t tile_base = D.tile_addr;
+        const uint32_t vt_base = D.vt_addr + (uint32_t)D.vrem * 4u;
 #pragma unroll 1
         for (int rg = 0; rg < C::RGW; ++rg) {
             const int vr0 = (warp * C::RGW + rg) * 32;
             if (vr0 >= nvr) break;
             const int vr = vr0 + lane;
-            const uint32_t rowoff = tile_base + (uint32_t)vr * C::MV;
-            // per-vector term of the L2 expansion (0 for inner product); issued early, used last
-            float vt = 0.f;
-            if (a.vterm != nullptr && vr < nvr && sr == 0) vt = __ldg(a.vterm + D.pos0 + (uint32_t)(vr / R));
+            const uint32_t rowaddr = tile_base + (uint32_t)vr * C::MV;
             float acc[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-            for (int blk = 0; blk < WV / G; ++blk) {
-#pragma unroll
-                for (int il = 0; il < G; ++il) {
-                    const uint32_t x = *reinterpret_cast<const uint32_t*>(smem + rowoff + xo[il] + blk * G * 4);
-#pragma unroll
-                    for (int t = 0; t < 4; ++t) {
-                        const uint32_t j = __byte_perm(x, 0u, sel[t]);
-                        acc[t] += *reinterpret_cast<const float*>(smem + j * (uint32_t)(C::LSTRIDE * 4) + lo[il][t] +
-                                                                  blk * G * 16);
-                    }
-                }
-            }
+            ScanBlocks<C, G, 0>::run(rowaddr, xo, cc, sel, lo, P.lut, acc);
             float s = (acc[0] + acc[1]) + (acc[2] + acc[3]);
             if (R >= 2) s += __shfl_xor_sync(0xffffffffu, s, 1);
             if (R >= 4) s += __shfl_xor_sync(0xffffffffu, s, 2);
+            // per-vector term of the L2 expansion (0 for inner product); rows past the tile's end read
+            // stale but in-bounds shared memory and are never pushed
+            const float vt = a.vterm != nullptr ? lds_f32(vt_base + (uint32_t)(vr / R) * 4u) : 0.f;
             const float score = (bias + vt) + s;  // smaller is better for both metrics
             const unsigned long long key = make_key(score, D.pos0 + (uint32_t)(vr / R));
             warp_push(keys, &ctrl->cnt, vr < nvr && sr == 0 && key < tau, key);
@@ -391,18 +526,26 @@ __global__ void __launch_bounds__(SCAN_THREADS, 1) scan_kernel(const ScanArgs a)
 struct Variant {
     int M;
     void (*kernel)(const ScanArgs);
-    int lut_bytes, tile_bytes, tile_vecs;
+    int threads, tile_vecs;
+    int (*stages_for)(int d);
 };
-#define RAGO_VARIANT(WV, G, R) \
-    { Cfg<WV, G, R>::M, scan_kernel<WV, G, R>, Cfg<WV, G, R>::LUT_BYTES, Cfg<WV, G, R>::TILE_BYTES, Cfg<WV, G, R>::TV }
+template <class C>
+static int stages_for(int d) {
+    for (int s = MAX_STAGES; s >= 2; --s)
+        if (plan_smem<C>(SMEM_BASE_EXPECTED, SMEM_OPTIN, d, s).ok) return s;
+    return 0;
+}
+#define RAGO_VARIANT(WV, G, R, NCW) \
+    { Cfg<WV, G, R, NCW>::M, scan_kernel<WV, G, R, NCW>, Cfg<WV, G, R, NCW>::THREADS, Cfg<WV, G, R, NCW>::TV, \
+      stages_for<Cfg<WV, G, R, NCW>> }
 static const Variant kVariants[] = {
-    RAGO_VARIANT(4, 4, 1),   // M = 16
-    RAGO_VARIANT(8, 8, 1),   // M = 32
-    RAGO_VARIANT(12, 4, 1),  // M = 48
-    RAGO_VARIANT(8, 8, 2),   // M = 64
-    RAGO_VARIANT(20, 4, 1),  // M = 80
-    RAGO_VARIANT(24, 8, 1),  // M = 96
-    RAGO_VARIANT(8, 8, 4),   // M = 128
+    RAGO_VARIANT(4, 4, 1, 16),   // M = 16
+    RAGO_VARIANT(8, 8, 1, 16),   // M = 32
+    RAGO_VARIANT(12, 4, 1, 12),  // M = 48
+    RAGO_VARIANT(8, 8, 2, 16),   // M = 64
+    RAGO_VARIANT(20, 4, 1, 8),   // M = 80
+    RAGO_VARIANT(24, 8, 1, 12),  // M = 96
+    RAGO_VARIANT(8, 8, 4, 12),   // M = 128
 };
 
 static const Variant* find_variant(int M) {
@@ -416,16 +559,13 @@ bool scan_supported(int M) { return find_variant(M) != nullptr; }
 cudaError_t scan_plan(const IndexImpl* ix, ScanPlan* plan) {
     const Variant* v = find_variant(ix->M);
     if (!v) return cudaErrorInvalidValue;
-    const size_t fixed = align_up((size_t)v->lut_bytes + TOPK_CAP * 8 + (size_t)ix->d * 4, 128);
-    long long room = (long long)SMEM_LIMIT - (long long)fixed - CTRL_BYTES;
-    int stages = (int)(room / v->tile_bytes);
-    if (stages > MAX_STAGES) stages = MAX_STAGES;
+    const int stages = v->stages_for(ix->d);
     if (stages < 2) return cudaErrorInvalidValue;
     plan->tile_vecs = v->tile_vecs;
     plan->stages = stages;
     plan->ctas = ix->num_sms;
-    plan->smem_bytes = fixed + (size_t)stages * v->tile_bytes + CTRL_BYTES;
-    return cudaFuncSetAttribute(v->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan->smem_bytes);
+    plan->smem_bytes = SMEM_OPTIN;
+    return cudaFuncSetAttribute(v->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_OPTIN);
 }
 
 cudaError_t launch_scan(const IndexImpl* ix, const ScanPlan& plan, const float* queries, const int32_t* probe_list,
@@ -436,12 +576,12 @@ cudaError_t launch_scan(const IndexImpl* ix, const ScanPlan& plan, const float* 
     if (!v) return cudaErrorInvalidValue;
     ScanArgs a;
     a.codes = ix->codes; a.list_offsets = ix->list_offsets; a.probe_list = probe_list; a.probe_term = probe_term;
-    a.queries = queries; a.centroids = ix->centroids; a.cbT = ix->cbT; a.work_prefix = work_prefix;
+    a.queries = queries; a.cbT = ix->cbT; a.work_prefix = work_prefix;
     a.vterm = ix->vterm;
     a.qthresh = qthresh; a.slot_cnt = slot_cnt; a.slot_keys = slot_keys; a.err = err_word;
-    a.coarse_bf16 = ix->coarse_bf16; a.npairs = nq * nprobe; a.nprobe = nprobe; a.d = ix->d; a.dsub = ix->dsub;
-    a.metric = ix->metric; a.k = k; a.stages = plan.stages;
-    v->kernel<<<plan.ctas, SCAN_THREADS, plan.smem_bytes, s>>>(a);
+    a.npairs = nq * nprobe; a.nprobe = nprobe; a.d = ix->d; a.dsub = ix->dsub;
+    a.metric = ix->metric; a.k = k; a.stages = plan.stages; a.dyn_bytes = (uint32_t)plan.smem_bytes;
+    v->kernel<<<plan.ctas, v->threads, plan.smem_bytes, s>>>(a);
     count_launch();
     return cudaGetLastError();
 }
