@@ -118,6 +118,36 @@ rago_status rago_search_probes(const rago_index* index, const float* queries, in
                                void* cuda_stream);
 
 /*
+ * The coarse step for callers that cannot allocate device memory.  (The paper has no counterpart
+ * to this call; it exists for deployment reasons only.)
+ *
+ * Who needs it: a retrieval worker that shares its GPU with an LLM server whose memory pool has
+ * already claimed the free HBM, so that a cudaMalloc for a workspace would fail or stall the
+ * other tenant; code that runs where an allocation is not allowed because it synchronises the
+ * device (inside a latency-critical serving loop, or between the steps of another stream's
+ * pipeline); and embedders that hand the library nothing but input and output buffers.
+ *
+ * Same inputs, outputs and results as rago_search_probes, but there is no workspace argument:
+ * the query-by-list score matrix is kept in an array of RAGO_NOALLOC_SCRATCH_BYTES that is part
+ * of the library image (each GPU that loads the library gives up that much memory until the
+ * process ends).  The call itself allocates and frees nothing.
+ *
+ *   limit     align256(nq * nlist * 4) + align256(nq * nprobe * 4) <= RAGO_NOALLOC_SCRATCH_BYTES;
+ *             a larger batch is refused with RAGO_ENOMEM and a message that names the limit
+ *             (split the batch, or use rago_search_probes).
+ *   set-up    the first call on each device looks up the array's device address
+ *             (cudaGetSymbolAddress) with that device current; make that first call before
+ *             starting any stream capture.
+ *   sharing   all calls on a device use the same array and find the previous call's contents in
+ *             it.  Nothing needs clearing (every word read is written first by the same call),
+ *             but two calls that overlap on the GPU - different streams, or different host
+ *             threads - race on it and return garbage.  Serialise them on one stream.
+ */
+#define RAGO_NOALLOC_SCRATCH_BYTES (4 * 1024 * 1024)
+rago_status rago_search_probes_noalloc(const rago_index* index, const float* queries, int32_t nq, int32_t nprobe,
+                                       int32_t* out_lists, float* out_coarse, void* cuda_stream);
+
+/*
  * rago_search for callers whose queries and results live in HOST memory: copies the queries to
  * the device, searches, copies ids and distances back, all on `cuda_stream`, then synchronises
  * that stream.  `workspace` must be 256-byte aligned and hold

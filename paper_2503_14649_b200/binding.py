@@ -25,7 +25,7 @@ NUM_STAGES = 5
 STAGE_NAMES = ("coarse_scores", "probe_select", "plan", "table_scan", "merge")
 
 EXPORTS = ("rago_index_load", "rago_index_free", "rago_search_workspace_bytes", "rago_search",
-           "rago_search_probes", "rago_search_host", "rago_host_staging_bytes", "rago_flat_search",
+           "rago_search_probes", "rago_search_probes_noalloc", "rago_search_host", "rago_host_staging_bytes", "rago_flat_search",
            "rago_flat_workspace_bytes", "rago_check", "rago_profile_enable", "rago_profile_read",
            "rago_kernel_launches", "rago_last_error")
 
@@ -52,6 +52,7 @@ def lib() -> ctypes.CDLL:
         L.rago_host_staging_bytes.argtypes = [vp, i32, i32, ctypes.POINTER(sz)]
         L.rago_search.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, sz, vp]
         L.rago_search_probes.argtypes = [vp, vp, i32, i32, vp, vp, vp, sz, vp]
+        L.rago_search_probes_noalloc.argtypes = [vp, vp, i32, i32, vp, vp, vp]
         L.rago_search_host.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, sz, vp]
         L.rago_flat_search.argtypes = [vp, i64, i32, vp, i32, i32, vp, vp, vp, sz, vp]
         L.rago_flat_workspace_bytes.argtypes = [i64, i32, i32, i32, ctypes.POINTER(sz)]
@@ -152,6 +153,13 @@ class Index:
         _check(lib().rago_search_probes(self._h, _ptr(queries), nq, nprobe, _ptr(lists), _ptr(coarse),
                                         _ptr(workspace), workspace.numel(), _stream()))
         return lists, coarse
+
+    def rago_search_probes_noalloc(self, queries: torch.Tensor, nprobe: int, out_lists: torch.Tensor,
+                                   out_coarse: torch.Tensor):
+        """rago_search_probes without a workspace: scratch is the library's built-in array, so the
+        call allocates nothing (the outputs are the caller's).  Calls must not overlap on the GPU."""
+        _check(lib().rago_search_probes_noalloc(self._h, _ptr(queries), queries.shape[0], nprobe, _ptr(out_lists),
+                                                _ptr(out_coarse), _stream()))
 
     def rago_search_host(self, host_queries: torch.Tensor, nprobe: int, k: int, host_out_ids: torch.Tensor,
                          host_out_dists: torch.Tensor, workspace: torch.Tensor):
