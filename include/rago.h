@@ -182,6 +182,17 @@ rago_status rago_flat_workspace_bytes(int64_t N, int32_t d, int32_t nq, int32_t 
  */
 rago_status rago_check(void* workspace, void* cuda_stream);
 
+/*
+ * Which kernel computes the coarse scores: 0 = automatic (tensor cores for batches of more than 16
+ * queries, the fp32 kernel for smaller ones), 1 = always the fp32 kernel, 2 = always tensor cores.
+ * The tensor-core kernel multiplies bf16 operands; fp32 queries and centroids are split into three
+ * bf16 parts each and the six leading part products are accumulated in fp32, so both kernels rank
+ * the lists alike up to fp32 rounding, and either way the best nprobe + 8 lists are re-scored
+ * exactly before the final cut.  Workspace sizes depend on the mode: set it before asking for
+ * them.  Mode 2 on an index whose d is not a multiple of 8 returns RAGO_EUNSUPPORTED.
+ */
+rago_status rago_set_coarse_mode(rago_index* index, int32_t mode);
+
 /* Per-stage device timings of rago_search.  When enabled, rago_search records CUDA events on the
  * caller's stream around each stage; rago_profile_read synchronises and returns the last call's
  * stage times in milliseconds (out_ms[RAGO_NUM_STAGES]). */

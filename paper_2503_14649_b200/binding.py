@@ -26,7 +26,7 @@ STAGE_NAMES = ("coarse_scores", "probe_select", "plan", "table_scan", "merge")
 
 EXPORTS = ("rago_index_load", "rago_index_free", "rago_search_workspace_bytes", "rago_search",
            "rago_search_probes", "rago_search_probes_noalloc", "rago_search_host", "rago_host_staging_bytes", "rago_flat_search",
-           "rago_flat_workspace_bytes", "rago_check", "rago_profile_enable", "rago_profile_read",
+           "rago_flat_workspace_bytes", "rago_check", "rago_set_coarse_mode", "rago_profile_enable", "rago_profile_read",
            "rago_kernel_launches", "rago_last_error")
 
 
@@ -57,6 +57,7 @@ def lib() -> ctypes.CDLL:
         L.rago_flat_search.argtypes = [vp, i64, i32, vp, i32, i32, vp, vp, vp, sz, vp]
         L.rago_flat_workspace_bytes.argtypes = [i64, i32, i32, i32, ctypes.POINTER(sz)]
         L.rago_check.argtypes = [vp, vp]
+        L.rago_set_coarse_mode.argtypes = [vp, i32]
         L.rago_profile_enable.argtypes = [vp, i32]
         L.rago_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
         L.rago_kernel_launches.restype = i64
@@ -170,6 +171,10 @@ class Index:
     def rago_check(self, workspace: Optional[torch.Tensor] = None):
         ws = workspace if workspace is not None else self._ws
         _check(lib().rago_check(_ptr(ws), _stream()))
+
+    def rago_set_coarse_mode(self, mode: int):
+        _check(lib().rago_set_coarse_mode(self._h, int(mode)))
+        self._ws = None  # workspace sizes depend on the mode
 
     def rago_profile_enable(self, enable: bool = True):
         _check(lib().rago_profile_enable(self._h, int(enable)))

@@ -40,8 +40,18 @@ static bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_
 // device error word.
 struct Layout {
     size_t err, probe_list, probe_term, probe_bias, scores, pair_tiles, work_prefix, qthresh, slot_cnt, slot_keys, total;
+    size_t qparts, cand, cand_cnt;  // tensor-core coarse step: query parts, candidate lists and their counts
     size_t nslots;
+    int tc, tc_mode, tc_cap, tc_mg, tc_nsplit;  // coarse plan for this (nq, nprobe)
 };
+
+// Which coarse kernel a batch takes.  The tensor-core kernel pays off once a batch fills a good part of
+// a 128-row tile; tiny batches (the latency-bound iterative-retrieval shape) stay on the fp32 pipes.
+constexpr int TC_MIN_NQ = 17;
+static bool use_tensor_cores(const IndexImpl* ix, int nq) {
+    if (!ix->tc_ok || ix->coarse_mode == 1) return false;
+    return ix->coarse_mode == 2 || nq >= TC_MIN_NQ;
+}
 
 static Layout make_layout(const IndexImpl* ix, int nq, int nprobe, int k) {
     Layout L;
@@ -57,7 +67,23 @@ static Layout make_layout(const IndexImpl* ix, int nq, int nprobe, int k) {
     L.probe_list = take(npairs * 4);
     L.probe_term = take(npairs * 4);
     L.probe_bias = take(npairs * 4);
-    L.scores = take((size_t)nq * ix->nlist * 4);
+    L.tc = use_tensor_cores(ix, nq) ? 1 : 0;
+    L.tc_mode = 1; L.tc_cap = 0; L.tc_mg = 1; L.tc_nsplit = 1;
+    L.qparts = L.cand = L.cand_cnt = 0;
+    if (L.tc) {
+        int nsel = nprobe + PROBE_GUARD;
+        if (nsel > ix->nlist) nsel = ix->nlist;
+        int mgroups = 1;
+        gemm_grid(nq, ix->nlist, ix->num_sms, &L.tc_mg, &L.tc_nsplit, &mgroups);
+        L.tc_cap = gemm_cand_cap(nsel);
+        L.tc_mode = L.tc_cap ? 0 : 1;
+        L.qparts = take((size_t)ix->cparts_n * nq * ix->d * 2);
+        if (L.tc_mode == 0) {
+            L.cand = take((size_t)nq * L.tc_nsplit * L.tc_cap * 8);
+            L.cand_cnt = take((size_t)nq * L.tc_nsplit * 4);
+        }
+    }
+    L.scores = take((!L.tc || L.tc_mode == 1) ? (size_t)nq * ix->nlist * 4 : 0);
     L.pair_tiles = take(npairs * 4);
     L.work_prefix = take((npairs + 1) * 8);
     L.qthresh = take((size_t)nq * 8);
@@ -86,14 +112,54 @@ static rago_status run_coarse(const IndexImpl* ix, const float* queries, int nq,
                               const Layout& L, cudaStream_t s) {
     IndexImpl* mix = const_cast<IndexImpl*>(ix);
     cudaError_t e;
+    int32_t* probe_list = reinterpret_cast<int32_t*>(ws + L.probe_list);
+    float* probe_term = reinterpret_cast<float*>(ws + L.probe_term);
+    float* probe_bias = reinterpret_cast<float*>(ws + L.probe_bias);
+    float* scores = reinterpret_cast<float*>(ws + L.scores);
     record(mix, 0, s);
-    e = launch_coarse_scores(ix, queries, nq, reinterpret_cast<float*>(ws + L.scores), s);
-    if (e != cudaSuccess) return cuda_fail(e, "coarse score kernel");
-    record(mix, 1, s);
-    e = launch_select_probes(ix, queries, reinterpret_cast<float*>(ws + L.scores), nq, nprobe,
-                             reinterpret_cast<int32_t*>(ws + L.probe_list),
-                             reinterpret_cast<float*>(ws + L.probe_term),
-                             reinterpret_cast<float*>(ws + L.probe_bias), s);
+    if (L.tc) {
+        // queries -> stacked bf16 parts, then the tensor-core kernel with the selection fused in
+        const int parts = ix->cparts_n;
+        e = launch_split_bf16(queries, (size_t)nq * ix->d, parts, ws + L.qparts, s);
+        if (e != cudaSuccess) return cuda_fail(e, "query split kernel");
+        alignas(64) unsigned char tmap_a[128];
+        e = make_tmap_bf16(tmap_a, ws + L.qparts, (uint64_t)parts * nq, (uint64_t)ix->d, 128);
+        if (e != cudaSuccess) return cuda_fail(e, "encoding the query tensor map");
+        GemmLaunch G;
+        G.tmap_a = tmap_a; G.tmap_b = ix->tmap_b;
+        G.nrows = nq; G.ncols = ix->nlist; G.d = ix->d;
+        G.a_part_rows = nq; G.b_part_rows = ix->nlist;
+        if (parts == 1) {
+            G.nterms = 1; G.term_a[0] = 0; G.term_b[0] = 0;
+            for (int t = 1; t < 6; ++t) G.term_a[t] = G.term_b[t] = 0;
+        } else {  // smallest products first: (2,0) (1,1) (0,2) (1,0) (0,1) (0,0)
+            const int ta[6] = {2, 1, 0, 1, 0, 0}, tb[6] = {0, 1, 2, 0, 1, 0};
+            G.nterms = 6;
+            for (int t = 0; t < 6; ++t) { G.term_a[t] = ta[t]; G.term_b[t] = tb[t]; }
+        }
+        G.mg = L.tc_mg; G.nsplit = L.tc_nsplit;
+        G.alpha = ix->metric == RAGO_L2 ? -2.f : -1.f;
+        G.colterm = ix->metric == RAGO_L2 ? ix->cnorm : nullptr;
+        G.mode = L.tc_mode; G.cap = L.tc_cap;
+        G.nsel = nprobe + PROBE_GUARD < ix->nlist ? nprobe + PROBE_GUARD : ix->nlist;
+        G.cand = reinterpret_cast<unsigned long long*>(ws + L.cand);
+        G.cand_cnt = reinterpret_cast<int32_t*>(ws + L.cand_cnt);
+        G.scores = scores;
+        G.err = reinterpret_cast<uint32_t*>(ws + L.err);
+        e = launch_gemm_select(G, s);
+        if (e != cudaSuccess) return cuda_fail(e, "tensor-core coarse kernel");
+        record(mix, 1, s);
+        if (L.tc_mode == 0)
+            e = launch_select_probes_cand(ix, queries, G.cand, G.cand_cnt, L.tc_nsplit, L.tc_cap, nq, nprobe, probe_list,
+                                          probe_term, probe_bias, s);
+        else
+            e = launch_select_probes(ix, queries, scores, nq, nprobe, probe_list, probe_term, probe_bias, s);
+    } else {
+        e = launch_coarse_scores(ix, queries, nq, scores, s);
+        if (e != cudaSuccess) return cuda_fail(e, "coarse score kernel");
+        record(mix, 1, s);
+        e = launch_select_probes(ix, queries, scores, nq, nprobe, probe_list, probe_term, probe_bias, s);
+    }
     if (e != cudaSuccess) return cuda_fail(e, "probe selection kernel");
     record(mix, 2, s);
     return RAGO_OK;
@@ -162,6 +228,21 @@ rago_status rago_index_load(rago_index** out, const void* coarse_centroids, rago
     if (e == cudaSuccess) e = launch_centroid_norms(coarse_centroids, ix->coarse_bf16, nlist, d, ix->cnorm, s);
     if (e == cudaSuccess) e = launch_transpose_codebook(pq_codebooks, M, ix->dsub, ix->cbT, s);
     if (e == cudaSuccess && ix->vterm) e = launch_vector_terms(ix, ix->vterm, s);
+    // tensor-core coarse operand: the centroids as stacked bf16 parts, and their tensor map
+    if (e == cudaSuccess && d % 8 == 0) {
+        const void* bsrc = coarse_centroids;
+        ix->cparts_n = 1;
+        if (!ix->coarse_bf16) {
+            ix->cparts_n = 3;
+            e = cudaMalloc(&ix->cparts, (size_t)3 * nlist * d * 2);
+            if (e == cudaSuccess) e = launch_split_bf16(static_cast<const float*>(coarse_centroids), (size_t)nlist * d, 3, ix->cparts, s);
+            bsrc = ix->cparts;
+        }
+        if (e == cudaSuccess && gemm_select_init() == cudaSuccess &&
+            make_tmap_bf16(ix->tmap_b, bsrc, (uint64_t)ix->cparts_n * nlist, (uint64_t)d, 256) == cudaSuccess)
+            ix->tc_ok = 1;
+        cudaGetLastError();  // a missing tensor-core path is not an error: the fp32 kernel serves every batch
+    }
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) {
         rago_status st = cuda_fail(e, "index setup kernels");
@@ -179,6 +260,7 @@ rago_status rago_index_free(rago_index* index) {
     if (ix->cnorm) cudaFree(ix->cnorm);
     if (ix->cbT) cudaFree(ix->cbT);
     if (ix->vterm) cudaFree(ix->vterm);
+    if (ix->cparts) cudaFree(ix->cparts);
     if (ix->ev_valid)
         for (int i = 0; i <= RAGO_NUM_STAGES; ++i) cudaEventDestroy(ix->ev[i]);
     delete ix;
@@ -216,10 +298,12 @@ rago_status rago_search_probes(const rago_index* index, const float* queries, in
     if (workspace_bytes < L.total) return fail(RAGO_ENOMEM, "workspace holds %zu bytes, %zu needed", workspace_bytes, L.total);
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     uint8_t* ws = static_cast<uint8_t*>(workspace);
+    cudaError_t e = cudaMemsetAsync(ws + L.err, 0, 256, s);
+    if (e != cudaSuccess) return cuda_fail(e, "clearing the error word");
     st = run_coarse(ix, queries, nq, nprobe, ws, L, s);
     if (st != RAGO_OK) return st;
     const size_t bytes = (size_t)nq * nprobe * 4;
-    cudaError_t e = cudaMemcpyAsync(out_lists, ws + L.probe_list, bytes, cudaMemcpyDeviceToDevice, s);
+    e = cudaMemcpyAsync(out_lists, ws + L.probe_list, bytes, cudaMemcpyDeviceToDevice, s);
     if (e == cudaSuccess) e = cudaMemcpyAsync(out_coarse, ws + L.probe_term, bytes, cudaMemcpyDeviceToDevice, s);
     if (e != cudaSuccess) return cuda_fail(e, "copying probe table");
     return RAGO_OK;
@@ -340,6 +424,15 @@ rago_status rago_check(void* workspace, void* cuda_stream) {
     if (w == ERR_WAIT_TIMEOUT) return fail(RAGO_ETIMEOUT, "a bounded device-side wait expired");
     if (w == ERR_SMEM_LAYOUT) return fail(RAGO_ECUDA, "the scan kernel's shared-memory plan does not fit this device");
     if (w != ERR_NONE) return fail(RAGO_ECUDA, "device error word = %u", w);
+    return RAGO_OK;
+}
+
+rago_status rago_set_coarse_mode(rago_index* index, int32_t mode) {
+    if (!index) return fail(RAGO_EINVAL, "index is null");
+    if (mode < 0 || mode > 2) return fail(RAGO_EINVAL, "mode = %d: 0 auto, 1 fp32 pipes, 2 tensor cores", mode);
+    IndexImpl* ix = reinterpret_cast<IndexImpl*>(index);
+    if (mode == 2 && !ix->tc_ok) return fail(RAGO_EUNSUPPORTED, "the tensor-core coarse path is not available for this index");
+    ix->coarse_mode = mode;
     return RAGO_OK;
 }
 

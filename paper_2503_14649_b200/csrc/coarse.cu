@@ -115,10 +115,13 @@ cudaError_t launch_coarse_scores(const IndexImpl* ix, const float* queries, int 
 // ---- per-query selection of the nprobe best lists ----------------------------------------------
 constexpr int SEL_THREADS = 256;
 
+// Candidates come either from a score row (scores != null: all nlist lists) or from the candidate
+// lists the tensor-core kernel left behind (cand[q][split][cap] keys with counts cand_cnt[q][split]).
 template <bool BF16>
 __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
-    const float* __restrict__ Q, const void* __restrict__ C, const float* __restrict__ scores, int nlist, int d,
-    int metric, int nprobe, int32_t* __restrict__ probe_list, float* __restrict__ probe_term,
+    const float* __restrict__ Q, const void* __restrict__ C, const float* __restrict__ scores,
+    const unsigned long long* __restrict__ cand, const int32_t* __restrict__ cand_cnt, int nsplit, int cap, int nlist,
+    int d, int metric, int nprobe, int32_t* __restrict__ probe_list, float* __restrict__ probe_term,
     float* __restrict__ probe_bias) {
     __shared__ unsigned long long keys[TOPK_CAP];
     __shared__ unsigned long long keys2[MAX_K + PROBE_GUARD];
@@ -131,12 +134,20 @@ __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
     __syncthreads();
     unsigned long long tau = KEY_MAX;
     int ub = 0;  // upper bound of cnt, identical in every thread
-    const float* srow = scores + (size_t)q * nlist;
-    for (int l0 = 0; l0 < nlist; l0 += SEL_THREADS) {
+    const float* srow = scores ? scores + (size_t)q * nlist : nullptr;
+    const int nitems = scores ? nlist : nsplit * cap;
+    for (int l0 = 0; l0 < nitems; l0 += SEL_THREADS) {
         const int l = l0 + tid;
         unsigned long long key = KEY_MAX;
-        if (l < nlist) key = make_key(srow[l], (uint32_t)l);
-        warp_push(keys, &cnt, l < nlist && key < tau, key);
+        if (l < nitems) {
+            if (scores) {
+                key = make_key(srow[l], (uint32_t)l);
+            } else {
+                const int sp = l / cap, i = l - sp * cap;
+                if (i < cand_cnt[(size_t)q * nsplit + sp]) key = cand[((size_t)q * nsplit + sp) * cap + i];
+            }
+        }
+        warp_push(keys, &cnt, key < tau, key);
         ub += SEL_THREADS;
         if (ub + SEL_THREADS > TOPK_CAP) {
             __syncthreads();
@@ -197,17 +208,33 @@ __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
     }
 }
 
-cudaError_t launch_select_probes(const IndexImpl* ix, const float* queries, const float* scores, int nq, int nprobe,
-                                 int32_t* probe_list, float* probe_term, float* probe_bias, cudaStream_t s) {
+static cudaError_t launch_select_any(const IndexImpl* ix, const float* queries, const float* scores,
+                                     const unsigned long long* cand, const int32_t* cand_cnt, int nsplit, int cap, int nq,
+                                     int nprobe, int32_t* probe_list, float* probe_term, float* probe_bias,
+                                     cudaStream_t s) {
     if (ix->coarse_bf16)
-        select_probes_kernel<true><<<nq, SEL_THREADS, 0, s>>>(queries, ix->centroids, scores, ix->nlist, ix->d,
-                                                              ix->metric, nprobe, probe_list, probe_term, probe_bias);
+        select_probes_kernel<true><<<nq, SEL_THREADS, 0, s>>>(queries, ix->centroids, scores, cand, cand_cnt, nsplit, cap,
+                                                              ix->nlist, ix->d, ix->metric, nprobe, probe_list,
+                                                              probe_term, probe_bias);
     else
-        select_probes_kernel<false><<<nq, SEL_THREADS, 0, s>>>(queries, ix->centroids, scores, ix->nlist, ix->d,
-                                                               ix->metric, nprobe, probe_list, probe_term,
-                                                               probe_bias);
+        select_probes_kernel<false><<<nq, SEL_THREADS, 0, s>>>(queries, ix->centroids, scores, cand, cand_cnt, nsplit,
+                                                               cap, ix->nlist, ix->d, ix->metric, nprobe, probe_list,
+                                                               probe_term, probe_bias);
     count_launch();
     return cudaGetLastError();
+}
+
+cudaError_t launch_select_probes(const IndexImpl* ix, const float* queries, const float* scores, int nq, int nprobe,
+                                 int32_t* probe_list, float* probe_term, float* probe_bias, cudaStream_t s) {
+    return launch_select_any(ix, queries, scores, nullptr, nullptr, 0, 0, nq, nprobe, probe_list, probe_term,
+                             probe_bias, s);
+}
+
+cudaError_t launch_select_probes_cand(const IndexImpl* ix, const float* queries, const unsigned long long* cand,
+                                      const int32_t* cand_cnt, int nsplit, int cap, int nq, int nprobe,
+                                      int32_t* probe_list, float* probe_term, float* probe_bias, cudaStream_t s) {
+    return launch_select_any(ix, queries, nullptr, cand, cand_cnt, nsplit, cap, nq, nprobe, probe_list, probe_term,
+                             probe_bias, s);
 }
 
 }  // namespace rago

@@ -40,6 +40,11 @@ struct IndexImpl {
     float* cnorm;  // [nlist] squared centroid norms (L2 coarse ranking)
     float* cbT;    // [256][M][dsub] codebook with the codeword index outermost
     float* vterm;  // [N] per-vector term of the L2 expansion (null for inner product)
+    void* cparts;  // bf16 [parts][nlist][d]: the centroids as a sum of bf16 parts (fp32 index); null for a bf16 index
+    int cparts_n;  // parts of the tensor-core coarse operand: 3 (fp32 index) or 1 (bf16 index, borrowed array)
+    int tc_ok;     // tensor-core coarse path available (tensor map encoded)
+    int coarse_mode;  // 0 auto, 1 fp32 pipes, 2 tensor cores
+    alignas(64) unsigned char tmap_b[128];  // CUtensorMap of the stacked centroid parts
     int device, num_sms;
     ScanPlan plan;
     int profile;
@@ -151,6 +156,28 @@ cudaError_t launch_centroid_norms(const void* centroids, int bf16, int nlist, in
 cudaError_t launch_coarse_scores(const IndexImpl* ix, const float* queries, int nq, float* scores, cudaStream_t s);
 cudaError_t launch_select_probes(const IndexImpl* ix, const float* queries, const float* scores, int nq, int nprobe,
                                  int32_t* probe_list, float* probe_term, float* probe_bias, cudaStream_t s);
+cudaError_t launch_select_probes_cand(const IndexImpl* ix, const float* queries, const unsigned long long* cand,
+                                      const int32_t* cand_cnt, int nsplit, int cap, int nq, int nprobe,
+                                      int32_t* probe_list, float* probe_term, float* probe_bias, cudaStream_t s);
+// gemm_select.cu
+constexpr int GEMM_CAP_SMALL = 256, GEMM_CAP_LARGE = 1024;  // candidate-list capacities (keys per row and column range)
+struct GemmLaunch {
+    const void* tmap_a;          // CUtensorMap of A: bf16 [a parts * a_part_rows][d]
+    const void* tmap_b;          // CUtensorMap of B: bf16 [b parts * b_part_rows][d]
+    int nrows; int64_t ncols; int d;
+    int a_part_rows; int64_t b_part_rows;
+    int nterms; int term_a[6], term_b[6];
+    int mg, nsplit;              // from gemm_grid
+    float alpha; const float* colterm;
+    int mode, nsel, cap;
+    unsigned long long* cand; int32_t* cand_cnt; float* scores; uint32_t* err;
+};
+cudaError_t gemm_select_init();
+cudaError_t make_tmap_bf16(void* out_map, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows);
+int gemm_cand_cap(int nsel);  // 0: nsel too large for the fused selection
+void gemm_grid(int nrows, int64_t ncols, int num_sms, int* mg, int* nsplit, int* mgroups);
+cudaError_t launch_gemm_select(const GemmLaunch& L, cudaStream_t s);
+cudaError_t launch_split_bf16(const float* x, size_t n, int parts, void* out, cudaStream_t s);
 // scan.cu
 bool scan_supported(int M);
 cudaError_t scan_plan(const IndexImpl* ix, ScanPlan* plan);

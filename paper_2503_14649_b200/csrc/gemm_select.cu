@@ -1,0 +1,448 @@
+// Dense scores on the 5th-generation tensor cores with the per-row selection fused into the epilogue.
+//
+//   S[r][c] = alpha * sum_t <A_{ta(t)}[r], B_{tb(t)}[c]>  +  colterm[c]          smaller = better
+//
+// A (queries) and B (coarse centroids, or the flat database) are bf16, row-major with the
+// contraction dimension innermost.  fp32 operands are represented as sums of bf16 "parts"
+// (x = x0 + x1 + x2 exactly up to 24 bits) and the product as the six part pairs whose weight is at
+// least 2^-16 relative; each pair is simply more K-blocks accumulated into the same TMEM tile.
+//
+// One CTA = 128 x 256 output tile, K-blocks of 64 bf16 (one 128-byte swizzle span):
+//   warp 0   TMA producer: cp.async.bulk.tensor (tiled, 128B swizzle) into a 4-stage ring, mbarrier tx counts
+//   warp 1   one lane issues tcgen05.mma (M128 N256 K16, bf16 -> fp32 in TMEM), tcgen05.commit frees stages
+//   warps 2-5 epilogue: tcgen05.ld 32 columns at a time, thread = output row; two TMEM accumulators
+//            (2 x 256 columns) let the epilogue of one tile overlap the MMAs of the next; the warps never
+//            wait for each other
+// A CTA owns a contiguous range of column tiles for one or two row tiles, so a row's running state
+// (threshold, candidate count) lives in the registers of the thread that owns the row.
+//
+// Fused selection (mode 0).  A value below the row's threshold is appended to the row's candidate
+// list in global memory (capacity CAP = 32*NK keys, 64-bit key = ordered score bits << 32 | column).
+// When a list could overflow, its warp loads it into registers (NK keys per lane), finds the nsel-th
+// smallest score by a 32-step bit-wise search with warp-wide counts, keeps exactly nsel keys and
+// lowers the threshold.  The threshold is always the nsel-th smallest of a subset of the row, so no
+// key that belongs to the row's nsel best is ever dropped; the lists of all column ranges are merged
+// by the caller.  Mode 1 writes the score matrix instead.
+//
+// Every wait is bounded (common.cuh); on a timeout the roles leave their loops, the error word is
+// set, TMEM is still released.
+#include <cuda.h>
+
+#include "topk.cuh"
+
+namespace rago {
+
+constexpr int GBM = 128, GBN = 256, GBK = 64;
+constexpr int G_STAGES = 4;
+constexpr int G_A_BYTES = GBM * GBK * 2;
+constexpr int G_B_BYTES = GBN * GBK * 2;
+constexpr int G_STAGE_BYTES = G_A_BYTES + G_B_BYTES;
+constexpr int G_THREADS = 192;
+constexpr int G_TMEM_COLS = 512;
+constexpr int G_CN_BYTES = 4 * 2 * GBN * 4;  // column terms: one copy per epilogue warp and accumulator
+constexpr int G_SMEM_BYTES = G_STAGES * G_STAGE_BYTES + G_CN_BYTES + 256 + 1024;  // + barriers + alignment slack
+
+// tcgen05 instruction descriptor, kind::f16: D = f32 (bits 4-5 = 1), A = B = bf16 (bits 7-9, 10-12 = 1),
+// both operands K-major (bits 15, 16 = 0), N >> 3 in bits 17-22, M >> 4 in bits 24-28.
+constexpr uint32_t G_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(GBN >> 3) << 17) | ((uint32_t)(GBM >> 4) << 24);
+
+// ---- PTX wrappers ---------------------------------------------------------------------------
+__device__ __forceinline__ void tma_load_2d(const CUtensorMap* map, uint32_t bar, uint32_t dst, int x, int y) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t slot_smem, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(ncols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+        : "memory");
+}
+// 32 lanes x 32 consecutive fp32 columns: thread i of the warp gets TMEM lane (base lane + i).
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+// Shared-memory matrix descriptor of a K-major bf16 tile whose rows are 128 bytes (one swizzle span):
+// start address >> 4 in bits 0-13, leading-dimension offset (unused for this layout) 1 in bits 16-29,
+// stride between 8-row groups (1024 bytes) >> 4 in bits 32-45, descriptor version 1 in bits 46-47,
+// layout type 2 (128-byte swizzle) in bits 61-63.  The tile base is 1024-byte aligned; a K step of 16
+// elements (32 bytes) inside the span advances the start-address field by 2.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) |
+           ((uint64_t)2 << 61);
+}
+
+struct GemmArgs {
+    int nrows, ncols;            // valid rows of A (queries) and of B (lists / database rows)
+    int a_part_rows, b_part_rows;  // row distance between consecutive parts in the stacked operands
+    int kblocks;                 // ceil(d / 64)
+    int nterms;
+    int term_a[6], term_b[6];    // part pair of each term
+    int mtiles, ntiles, mg;      // row tiles, column tiles, row tiles per CTA (1 or 2)
+    float alpha;
+    const float* colterm;        // [ncols] or null
+    int mode;                    // 0: candidate lists, 1: score matrix
+    int nsel;                    // keys a row must keep (mode 0)
+    unsigned long long* cand;    // [nrows][nsplit][CAP]
+    int32_t* cand_cnt;           // [nrows][nsplit]
+    float* scores;               // [nrows][ncols] (mode 1)
+    uint32_t* err;
+};
+
+// Keep the nsel smallest of the n (> nsel) keys of one list; returns the new threshold score.
+template <int NK>
+__device__ __forceinline__ float compact_list(unsigned long long* list, int n, int nsel, int lane) {
+    unsigned long long k[NK];
+#pragma unroll
+    for (int j = 0; j < NK; ++j) {
+        const int idx = lane + 32 * j;
+        k[j] = idx < n ? list[idx] : KEY_MAX;
+    }
+    uint32_t v = 0;  // becomes the nsel-th smallest score (ordered bits)
+#pragma unroll 1
+    for (int b = 31; b >= 0; --b) {
+        const uint32_t trial = v | (1u << b);
+        uint32_t c = 0;
+#pragma unroll
+        for (int j = 0; j < NK; ++j) c += ((uint32_t)(k[j] >> 32) < trial) ? 1u : 0u;
+        c = __reduce_add_sync(0xffffffffu, c);
+        if (c < (uint32_t)nsel) v = trial;
+    }
+    uint32_t less = 0;
+#pragma unroll
+    for (int j = 0; j < NK; ++j) less += ((uint32_t)(k[j] >> 32) < v) ? 1u : 0u;
+    less = __reduce_add_sync(0xffffffffu, less);
+    int need = nsel - (int)less;  // keys equal to v that still have to be kept (>= 1)
+    __syncwarp();
+    const uint32_t lt_mask = (1u << lane) - 1u;
+    int base = 0;
+#pragma unroll
+    for (int j = 0; j < NK; ++j) {
+        const uint32_t s = (uint32_t)(k[j] >> 32);
+        const bool eq = s == v && k[j] != KEY_MAX;
+        const uint32_t meq = __ballot_sync(0xffffffffu, eq);
+        const bool keep = s < v || (eq && __popc(meq & lt_mask) < need);
+        const uint32_t mk = __ballot_sync(0xffffffffu, keep);
+        if (keep) list[base + __popc(mk & lt_mask)] = k[j];
+        base += __popc(mk);
+        const int eq_kept = __popc(meq) < need ? __popc(meq) : need;
+        need -= eq_kept;
+    }
+    __syncwarp();
+    return orderable_f32(v);
+}
+
+template <int NK>
+__global__ void __launch_bounds__(G_THREADS, 1)
+gemm_select_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmArgs a) {
+    constexpr int CAP = NK * 32;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;  // swizzled tiles need 1024-byte alignment
+    uint8_t* smem = smem_raw + (base - raw);
+    float* cn_all = reinterpret_cast<float*>(smem + G_STAGES * G_STAGE_BYTES);  // [4 warps][2][GBN] column terms
+    unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + G_STAGES * G_STAGE_BYTES + G_CN_BYTES);
+    const uint32_t bar0 = base + G_STAGES * G_STAGE_BYTES + G_CN_BYTES;
+    auto full_bar = [&](int s) { return bar0 + 8u * s; };
+    auto empty_bar = [&](int s) { return bar0 + 8u * (G_STAGES + s); };
+    auto tfull_bar = [&](int b) { return bar0 + 8u * (2 * G_STAGES + b); };
+    auto tempty_bar = [&](int b) { return bar0 + 8u * (2 * G_STAGES + 2 + b); };
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * G_STAGES + 4);
+    volatile uint32_t* abort_flag = tmem_slot + 1;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) {
+        for (int s = 0; s < G_STAGES; ++s) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(empty_bar(s), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(tfull_bar(b), 1);
+            mbar_init(tempty_bar(b), 4);
+        }
+        *abort_flag = 0;
+        fence_barrier_init();
+        fence_proxy_async();
+    }
+    if (warp == 0) tmem_alloc(smem_u32(tmem_slot), G_TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int split = blockIdx.x, nsplit = gridDim.x;
+    const int m0 = blockIdx.y * a.mg;
+    const int mcount = (a.mtiles - m0) < a.mg ? (a.mtiles - m0) : a.mg;
+    const int nt_begin = (int)((long long)split * a.ntiles / nsplit);
+    const int nt_end = (int)((long long)(split + 1) * a.ntiles / nsplit);
+    const int nunits = (nt_end - nt_begin) * mcount;
+    const int kiters = a.nterms * a.kblocks;
+
+    if (warp == 0) {
+        // ================= TMA producer =================
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool dead = false;
+            for (int u = 0; u < nunits && !dead; ++u) {
+                const int nt = nt_begin + u / mcount, m = m0 + u % mcount;
+                for (int t = 0; t < a.nterms && !dead; ++t) {
+                    const int ya = a.term_a[t] * a.a_part_rows + m * GBM;
+                    const int yb = a.term_b[t] * a.b_part_rows + nt * GBN;
+                    for (int kb = 0; kb < a.kblocks; ++kb, ++it) {
+                        const int s = it % G_STAGES;
+                        const uint32_t ph = (it / G_STAGES) & 1u;
+                        if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, a.err)) { dead = true; break; }
+                        mbar_arrive_expect_tx(full_bar(s), G_STAGE_BYTES);
+                        tma_load_2d(&tmA, full_bar(s), base + s * G_STAGE_BYTES, kb * GBK, ya);
+                        tma_load_2d(&tmB, full_bar(s), base + s * G_STAGE_BYTES + G_A_BYTES, kb * GBK, yb);
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ================= MMA issuer =================
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool dead = false;
+            for (int u = 0; u < nunits && !dead; ++u) {
+                const int buf = u & 1;
+                const uint32_t uph = (u >> 1) & 1u;
+                if (!mbar_wait(tempty_bar(buf), uph ^ 1u, abort_flag, a.err)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * GBN);
+                for (int ki = 0; ki < kiters; ++ki, ++it) {
+                    const int s = it % G_STAGES;
+                    const uint32_t ph = (it / G_STAGES) & 1u;
+                    if (!mbar_wait(full_bar(s), ph, abort_flag, a.err)) { dead = true; break; }
+                    tc_fence_after();
+                    const uint64_t da = smem_desc_sw128(base + s * G_STAGE_BYTES);
+                    const uint64_t db = smem_desc_sw128(base + s * G_STAGE_BYTES + G_A_BYTES);
+#pragma unroll
+                    for (int k = 0; k < GBK / 16; ++k)
+                        tc_mma_bf16(d_tmem, da + 2u * k, db + 2u * k, G_IDESC, (ki | k) != 0 ? 1u : 0u);
+                    tc_commit(empty_bar(s));  // frees the stage once these MMAs have read it
+                }
+                if (!dead) tc_commit(tfull_bar(buf));  // accumulator complete
+            }
+        }
+    } else {
+        // ================= epilogue warps =================
+        const int q4 = warp & 3;  // TMEM lane quarter this warp may read
+        float* cn = cn_all + (warp - 2) * 2 * GBN;  // this warp's own copy: no cross-warp barrier needed
+        const float inf = __int_as_float(0x7f800000);
+        float tau0 = inf, tau1 = inf;
+        int cnt0 = 0, cnt1 = 0;
+        {
+            const int r0 = m0 * GBM + q4 * 32 + lane, r1 = r0 + GBM;
+            if (r0 >= a.nrows) tau0 = -inf;
+            if (r1 >= a.nrows || mcount < 2) tau1 = -inf;
+        }
+        bool dead = false;
+        for (int u = 0; u < nunits && !dead; ++u) {
+            const int nt = nt_begin + u / mcount, g = u % mcount;
+            const int buf = u & 1;
+            const uint32_t uph = (u >> 1) & 1u;
+            for (int i = lane; i < GBN; i += 32) {
+                const int col = nt * GBN + i;
+                cn[buf * GBN + i] = col < a.ncols ? (a.colterm ? __ldg(a.colterm + col) : 0.f) : inf;
+            }
+            __syncwarp();
+            if (!mbar_wait(tfull_bar(buf), uph, abort_flag, a.err)) { dead = true; break; }
+            tc_fence_after();
+            const int row = (m0 + g) * GBM + q4 * 32 + lane;
+            const uint32_t taddr = tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(buf * GBN);
+            if (a.mode == 0) {
+                float tau = g ? tau1 : tau0;
+                int cnt = g ? cnt1 : cnt0;
+                unsigned long long* list =
+                    a.cand + ((size_t)(row < a.nrows ? row : 0) * nsplit + split) * CAP;  // never written for padding rows
+#pragma unroll 1
+                for (int c0 = 0; c0 < GBN; c0 += 32) {
+                    float v[32];
+                    tmem_ld32(taddr + c0, v);
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const float s = fmaf(a.alpha, v[j], cn[buf * GBN + c0 + j]);
+                        if (s < tau) {
+                            list[cnt] = make_key(s, (uint32_t)(nt * GBN + c0 + j));
+                            ++cnt;
+                        }
+                    }
+                    uint32_t todo = __ballot_sync(0xffffffffu, cnt > CAP - 32);
+                    while (todo) {  // warp-uniform
+                        const int r = __ffs(todo) - 1;
+                        todo &= todo - 1;
+                        const int n = __shfl_sync(0xffffffffu, cnt, r);
+                        const unsigned long long lp = __shfl_sync(0xffffffffu, (unsigned long long)list, r);
+                        __syncwarp();
+                        const float nt_tau = compact_list<NK>(reinterpret_cast<unsigned long long*>(lp), n, a.nsel, lane);
+                        if (lane == r) { cnt = a.nsel; tau = nt_tau; }
+                    }
+                }
+                if (g) { tau1 = tau; cnt1 = cnt; } else { tau0 = tau; cnt0 = cnt; }
+            } else {
+#pragma unroll 1
+                for (int c0 = 0; c0 < GBN; c0 += 32) {
+                    float v[32];
+                    tmem_ld32(taddr + c0, v);
+                    if (row < a.nrows) {
+                        float* out = a.scores + (size_t)row * a.ncols + nt * GBN + c0;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (nt * GBN + c0 + j < a.ncols) out[j] = fmaf(a.alpha, v[j], cn[buf * GBN + c0 + j]);
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar(buf));
+        }
+        if (a.mode == 0 && !dead) {
+            const int r0 = m0 * GBM + q4 * 32 + lane, r1 = r0 + GBM;
+            if (r0 < a.nrows) a.cand_cnt[(size_t)r0 * nsplit + split] = cnt0;
+            if (mcount == 2 && r1 < a.nrows) a.cand_cnt[(size_t)r1 * nsplit + split] = cnt1;
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after();
+        if (*abort_flag) __nanosleep(100000);  // let copies / MMAs in flight drain after a timed-out wait
+        tmem_dealloc(tmem_base, G_TMEM_COLS);
+    }
+}
+
+// ---- host side ----------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// Tensor map of a row-major bf16 matrix [rows][cols] read in boxes of box_rows x 64 columns, 128-byte swizzle.
+cudaError_t make_tmap_bf16(void* out_map, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return cudaErrorNotSupported;
+    if (rows == 0 || cols == 0 || (cols * 2) % 16 != 0 || reinterpret_cast<uintptr_t>(ptr) % 16 != 0)
+        return cudaErrorInvalidValue;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * 2};
+    const cuuint32_t box[2] = {GBK, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(static_cast<CUtensorMap*>(out_map), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr),
+                    dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+int gemm_cand_cap(int nsel) { return nsel <= GEMM_CAP_SMALL - 64 ? GEMM_CAP_SMALL : (nsel <= GEMM_CAP_LARGE - 64 ? GEMM_CAP_LARGE : 0); }
+
+void gemm_grid(int nrows, int64_t ncols, int num_sms, int* mg, int* nsplit, int* mgroups) {
+    const int mtiles = (nrows + GBM - 1) / GBM;
+    const int64_t ntiles = (ncols + GBN - 1) / GBN;
+    int best_mg = 1, best_split = 1;
+    int64_t best_units = -1;
+    for (int g = 1; g <= 2; ++g) {
+        if (g > mtiles) break;
+        const int groups = (mtiles + g - 1) / g;
+        int64_t split = num_sms / groups;
+        if (split < 1) split = 1;
+        if (split > ntiles) split = ntiles;
+        const int64_t units = ((ntiles + split - 1) / split) * g;
+        if (best_units < 0 || units <= best_units) { best_units = units; best_mg = g; best_split = (int)split; }
+    }
+    *mg = best_mg;
+    *nsplit = best_split;
+    *mgroups = (mtiles + best_mg - 1) / best_mg;
+}
+
+cudaError_t gemm_select_init() {
+    cudaError_t e = cudaFuncSetAttribute(gemm_select_kernel<GEMM_CAP_SMALL / 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_SMEM_BYTES);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(gemm_select_kernel<GEMM_CAP_LARGE / 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_SMEM_BYTES);
+    return e;
+}
+
+cudaError_t launch_gemm_select(const GemmLaunch& L, cudaStream_t s) {
+    GemmArgs a;
+    a.nrows = L.nrows; a.ncols = (int)L.ncols;
+    a.a_part_rows = L.a_part_rows; a.b_part_rows = (int)L.b_part_rows;
+    a.kblocks = (L.d + GBK - 1) / GBK;
+    a.nterms = L.nterms;
+    for (int t = 0; t < 6; ++t) { a.term_a[t] = L.term_a[t]; a.term_b[t] = L.term_b[t]; }
+    a.mtiles = (L.nrows + GBM - 1) / GBM;
+    a.ntiles = (int)((L.ncols + GBN - 1) / GBN);
+    a.mg = L.mg;
+    a.alpha = L.alpha; a.colterm = L.colterm;
+    a.mode = L.mode; a.nsel = L.nsel;
+    a.cand = L.cand; a.cand_cnt = L.cand_cnt; a.scores = L.scores; a.err = L.err;
+    const dim3 grid(L.nsplit, (a.mtiles + L.mg - 1) / L.mg);
+    const CUtensorMap* ma = reinterpret_cast<const CUtensorMap*>(L.tmap_a);
+    const CUtensorMap* mb = reinterpret_cast<const CUtensorMap*>(L.tmap_b);
+    if (L.mode == 0 && L.cap == GEMM_CAP_LARGE)
+        gemm_select_kernel<GEMM_CAP_LARGE / 32><<<grid, G_THREADS, G_SMEM_BYTES, s>>>(*ma, *mb, a);
+    else
+        gemm_select_kernel<GEMM_CAP_SMALL / 32><<<grid, G_THREADS, G_SMEM_BYTES, s>>>(*ma, *mb, a);
+    count_launch();
+    return cudaGetLastError();
+}
+
+// ---- fp32 -> stacked bf16 parts: out[p][i] = bf16 part p of x[i] ---------------------------------
+__global__ void split_bf16_kernel(const float* __restrict__ x, size_t n, int parts, __nv_bfloat16* __restrict__ out) {
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        float r = x[i];
+        for (int p = 0; p < parts; ++p) {
+            const __nv_bfloat16 h = __float2bfloat16_rn(r);
+            out[(size_t)p * n + i] = h;
+            r -= __bfloat162float(h);
+        }
+    }
+}
+cudaError_t launch_split_bf16(const float* x, size_t n, int parts, void* out, cudaStream_t s) {
+    if (n == 0) return cudaSuccess;
+    const size_t want = (n + 255) / 256;
+    const int blocks = (int)(want < 148 * 8 ? want : 148 * 8);
+    split_bf16_kernel<<<blocks, 256, 0, s>>>(x, n, parts, static_cast<__nv_bfloat16*>(out));
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace rago
