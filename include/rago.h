@@ -167,7 +167,7 @@ rago_status rago_host_staging_bytes(const rago_index* index, int32_t nq, int32_t
  *   queries     dev [nq][d] bf16, 16-byte aligned
  *   out_ids     dev [nq][k] int64 row numbers; out_scores dev [nq][k] fp32
  *   workspace   dev, 256-byte aligned, rago_flat_workspace_bytes(...) bytes
- *   1 <= k <= 1024, N < 2^32.
+ *   1 <= k <= 1024, N < 2^31.
  */
 rago_status rago_flat_search(const void* db, int64_t N, int32_t d, const void* queries, int32_t nq, int32_t k,
                              int64_t* out_ids, float* out_scores, void* workspace, size_t workspace_bytes,

@@ -389,7 +389,7 @@ rago_status rago_flat_workspace_bytes(int64_t N, int32_t d, int32_t nq, int32_t 
     if (!out_bytes) return fail(RAGO_EINVAL, "out_bytes is null");
     if (N < 0 || d <= 0 || nq < 0 || k < 1) return fail(RAGO_EINVAL, "bad sizes");
     if (k > MAX_K) return fail(RAGO_EUNSUPPORTED, "k = %d exceeds %d", k, MAX_K);
-    *out_bytes = flat_workspace_bytes(N, nq, k);
+    *out_bytes = flat_workspace_bytes(N, d, nq, k);
     return RAGO_OK;
 }
 
@@ -400,12 +400,12 @@ rago_status rago_flat_search(const void* db, int64_t N, int32_t d, const void* q
     if (k < 1) return fail(RAGO_EINVAL, "k = %d must be at least 1", k);
     if (k > MAX_K) return fail(RAGO_EUNSUPPORTED, "k = %d exceeds %d", k, MAX_K);
     if (d % 64 != 0 || d > 4096) return fail(RAGO_EUNSUPPORTED, "d = %d must be a multiple of 64, at most 4096", d);
-    if (N >= (1LL << 32)) return fail(RAGO_EUNSUPPORTED, "N needs more than 32-bit row numbers");
+    if (N >= (1LL << 31)) return fail(RAGO_EUNSUPPORTED, "N needs more than 31-bit row numbers");
     if (nq == 0) return RAGO_OK;
     if ((N > 0 && !db) || !queries || !out_ids || !out_scores || !workspace) return fail(RAGO_EINVAL, "null pointer");
     if (!aligned(db, 16) || !aligned(queries, 16) || !aligned(workspace, 256))
         return fail(RAGO_EALIGN, "db and queries need 16-byte, workspace 256-byte alignment");
-    const size_t need = flat_workspace_bytes(N, nq, k);
+    const size_t need = flat_workspace_bytes(N, d, nq, k);
     if (workspace_bytes < need) return fail(RAGO_ENOMEM, "workspace holds %zu bytes, %zu needed", workspace_bytes, need);
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     cudaError_t e = cudaMemsetAsync(workspace, 0, 256, s);

@@ -195,7 +195,7 @@ cudaError_t launch_merge(const IndexImpl* ix, const int64_t* work_prefix, int nq
                          float* out_dists, cudaStream_t s);
 cudaError_t launch_fill_u64(unsigned long long* p, size_t n, unsigned long long v, cudaStream_t s);
 // flat.cu
-size_t flat_workspace_bytes(int64_t N, int nq, int k);
+size_t flat_workspace_bytes(int64_t N, int d, int nq, int k);
 cudaError_t launch_flat_search(const void* db, int64_t N, int d, const void* queries, int nq, int k, int64_t* out_ids,
                                float* out_scores, void* workspace, cudaStream_t s);
 

@@ -1,7 +1,11 @@
 // Exact flat search: score = <q, y_i> over bf16 inputs, fp32 accumulation, k largest per query.
 //
-// The database is processed in panels of PANEL rows: scores of a panel go to scratch, each
-// (query, 64K-row chunk) keeps its k best as 64-bit keys, and a final pass merges the chunks.
+// Main path (k <= 960): the tensor-core kernel of gemm_select.cu with rows = queries and columns =
+// database rows; every CTA streams its own range of the database once (both 128-query row tiles are
+// multiplied against a database tile while it is hot) and keeps each query's k best of that range;
+// flat_merge_kernel merges the ranges.  No score is ever written to memory.
+// Fallback (larger k): the database is processed in panels of PANEL rows on the fp32 pipes: scores of
+// a panel go to scratch, each (query, 64K-row chunk) keeps its k best, and the same merge finishes.
 #include "topk.cuh"
 
 namespace rago {
@@ -103,7 +107,8 @@ __global__ void __launch_bounds__(FSEL_THREADS) flat_select_kernel(const float* 
     if (tid == 0) slot_cnt[slot] = kept;
 }
 
-__global__ void __launch_bounds__(FSEL_THREADS) flat_merge_kernel(int nchunks, int k,
+// slot (q, ch) holds slot_cnt keys at slot_keys[(q * nchunks + ch) * stride ...].
+__global__ void __launch_bounds__(FSEL_THREADS) flat_merge_kernel(int nchunks, int k, int stride,
                                                                   const int32_t* __restrict__ slot_cnt,
                                                                   const unsigned long long* __restrict__ slot_keys,
                                                                   int64_t* __restrict__ out_ids,
@@ -126,7 +131,7 @@ __global__ void __launch_bounds__(FSEL_THREADS) flat_merge_kernel(int nchunks, i
         for (int i0 = 0; i0 < c; i0 += FSEL_THREADS) {
             const int i = i0 + tid;
             unsigned long long key = KEY_MAX;
-            if (i < c) key = slot_keys[slot * k + i];
+            if (i < c) key = slot_keys[slot * stride + i];
             warp_push(keys, &cnt, i < c && key < tau, key);
         }
         __syncthreads();
@@ -144,8 +149,31 @@ __global__ void __launch_bounds__(FSEL_THREADS) flat_merge_kernel(int nchunks, i
     }
 }
 
-// Workspace: [err 256 B][scores nq*PANEL f32][slot_cnt nq*nchunks i32][slot_keys nq*nchunks*k u64]
-size_t flat_workspace_bytes(int64_t N, int nq, int k) {
+static int sm_count() {
+    static int sms = 0;
+    if (!sms) {
+        int dev = 0, n = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
+            sms = n;
+        else {
+            cudaGetLastError();
+            return 148;  // no device yet (size queries on a host without one): the B200 count
+        }
+    }
+    return sms;
+}
+
+static bool flat_on_tensor_cores(int d, int k) { return gemm_cand_cap(k) != 0 && d % 8 == 0; }
+
+// Workspace, tensor-core path: [err 256 B][cand nq*nsplit*cap u64][cand_cnt nq*nsplit i32]
+//            fallback:         [err 256 B][scores nq*PANEL f32][slot_cnt nq*nchunks i32][slot_keys nq*nchunks*k u64]
+size_t flat_workspace_bytes(int64_t N, int d, int nq, int k) {
+    if (flat_on_tensor_cores(d, k)) {
+        int mg, nsplit, mgroups;
+        gemm_grid(nq > 0 ? nq : 1, N > 0 ? N : 1, sm_count(), &mg, &nsplit, &mgroups);
+        return 256 + align_up((size_t)nq * nsplit * gemm_cand_cap(k) * 8, 256) + align_up((size_t)nq * nsplit * 4, 256);
+    }
     const size_t nchunks = (size_t)((N + FLAT_CHUNK - 1) / FLAT_CHUNK);
     size_t b = 256;
     b += align_up((size_t)nq * FLAT_PANEL * 4, 256);
@@ -156,6 +184,38 @@ size_t flat_workspace_bytes(int64_t N, int nq, int k) {
 
 cudaError_t launch_flat_search(const void* db, int64_t N, int d, const void* queries, int nq, int k, int64_t* out_ids,
                                float* out_scores, void* workspace, cudaStream_t s) {
+    if (flat_on_tensor_cores(d, k) && N > 0) {
+        cudaError_t e = gemm_select_init();
+        if (e != cudaSuccess) return e;
+        int mg, nsplit, mgroups;
+        gemm_grid(nq, N, sm_count(), &mg, &nsplit, &mgroups);
+        const int cap = gemm_cand_cap(k);
+        uint8_t* w = static_cast<uint8_t*>(workspace) + 256;
+        unsigned long long* cand = reinterpret_cast<unsigned long long*>(w);
+        w += align_up((size_t)nq * nsplit * cap * 8, 256);
+        int32_t* cand_cnt = reinterpret_cast<int32_t*>(w);
+        alignas(64) unsigned char tmap_a[128], tmap_b[128];
+        e = make_tmap_bf16(tmap_a, queries, (uint64_t)nq, (uint64_t)d, 128);
+        if (e == cudaSuccess) e = make_tmap_bf16(tmap_b, db, (uint64_t)N, (uint64_t)d, 256);
+        if (e != cudaSuccess) return e;
+        GemmLaunch G;
+        G.tmap_a = tmap_a; G.tmap_b = tmap_b;
+        G.nrows = nq; G.ncols = N; G.d = d;
+        G.a_part_rows = nq; G.b_part_rows = N;
+        G.nterms = 1;
+        for (int t = 0; t < 6; ++t) G.term_a[t] = G.term_b[t] = 0;
+        G.mg = mg; G.nsplit = nsplit;
+        G.alpha = -1.f;  // smaller = better
+        G.colterm = nullptr;
+        G.mode = 0; G.nsel = k < N ? k : (int)N; G.cap = cap;
+        G.cand = cand; G.cand_cnt = cand_cnt; G.scores = nullptr;
+        G.err = static_cast<uint32_t*>(workspace);
+        e = launch_gemm_select(G, s);
+        if (e != cudaSuccess) return e;
+        flat_merge_kernel<<<nq, FSEL_THREADS, 0, s>>>(nsplit, k, cap, cand_cnt, cand, out_ids, out_scores);
+        count_launch();
+        return cudaGetLastError();
+    }
     const int nchunks = (int)((N + FLAT_CHUNK - 1) / FLAT_CHUNK);
     uint8_t* w = static_cast<uint8_t*>(workspace) + 256;
     float* scores = reinterpret_cast<float*>(w);
@@ -175,7 +235,7 @@ cudaError_t launch_flat_search(const void* db, int64_t N, int d, const void* que
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
-    flat_merge_kernel<<<nq, FSEL_THREADS, 0, s>>>(nchunks, k, slot_cnt, slot_keys, out_ids, out_scores);
+    flat_merge_kernel<<<nq, FSEL_THREADS, 0, s>>>(nchunks, k, k, slot_cnt, slot_keys, out_ids, out_scores);
     count_launch();
     return cudaGetLastError();
 }

@@ -146,7 +146,10 @@ def test_results_do_not_depend_on_run():
     ix.close()
 
 
-@pytest.mark.parametrize("N,d,nq,k", [(5000, 64, 7, 10), (70_000, 128, 33, 100), (3, 64, 2, 5)])
+@pytest.mark.parametrize("N,d,nq,k", [(5000, 64, 7, 10), (70_000, 128, 33, 100), (3, 64, 2, 5),
+                                      (200_000, 64, 200, 100),   # two row tiles, lists compacted while streaming
+                                      (40_000, 64, 9, 300),      # wide candidate lists
+                                      (30_000, 64, 5, 1000)])    # k above the fused selection: fp32-pipe fallback
 def test_flat_search_matches_oracle(N, d, nq, k):
     db, q = synth.make_flat(N, d, nq, seed=N)
     gi, gs = binding.rago_flat_search(db.cuda(), q.cuda(), k)

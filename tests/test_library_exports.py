@@ -35,7 +35,7 @@ def test_host_only_calls_work_without_a_device():
     assert lib.rago_flat_workspace_bytes(10, 64, 2, 0, ctypes.byref(out)) == 1
     assert b"sizes" in lib.rago_last_error()
     assert lib.rago_flat_workspace_bytes(10_000_000, 1024, 256, 100, ctypes.byref(out)) == 0
-    assert out.value > 256 * (1 << 20) * 4
+    assert out.value >= 256 * 148 * 256 * 8  # 256 queries x 148 database ranges x 256 keys
     assert lib.rago_search_workspace_bytes(None, 1, 1, 1, ctypes.byref(out)) == 1
     assert lib.rago_index_free(None) == 0
 
