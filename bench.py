@@ -292,6 +292,116 @@ def run_ours(args):
         torch.distributed.destroy_process_group()
 
 
+def _tensor_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return float(d["bf16_tflops"]), float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), float(d["hbm_gbs"]), "measured"
+    return 1590.0, 1400.0, 6650.0, "fallback"
+
+
+def _time_steps(fn, steps, warmup):
+    """CUDA-event time of `steps` calls of fn on the current stream, after warm-up; returns (total ms, per-step ms)."""
+    for _ in range(max(3, warmup)):
+        fn()
+    torch.cuda.synchronize()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    ev[0].record()
+    for i in range(steps):
+        fn()
+        ev[i + 1].record()
+    torch.cuda.synchronize()
+    return ev[0].elapsed_time(ev[-1]), [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
+
+
+def run_flat(args):
+    """Secondary workload: exact flat search, N = 10 M x 1024 bf16 rows, 256 queries, k = 100 (cosine on unit rows)."""
+    from paper_2503_14649_b200 import binding, synth
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    c = synth.CONFIGS[5]
+    N = max(1, int(round(c["N"] * args.scale)))
+    d, nq, k = c["d"], c["nq"], c["k"]
+    db, q = synth.make_flat(N, d, nq, device=dev)
+    ws = torch.empty(binding.rago_flat_workspace_bytes(N, d, nq, k), dtype=torch.uint8, device=dev)
+    sampler = ClockSampler(0)
+    out = {}
+
+    def step():
+        out["r"] = binding.rago_flat_search(db, q, k, workspace=ws)
+
+    launches0 = binding.rago_kernel_launches()
+    sampler.start()
+    t0 = time.time()
+    total_ms, step_ms = _time_steps(step, args.steps, args.warmup)
+    t1 = time.time()
+    clocks = sampler.stop(t0, t1)
+    launches = (binding.rago_kernel_launches() - launches0) * args.steps // (args.steps + max(3, args.warmup))
+    ms = total_ms / args.steps
+    burst, sustained, hbm, kind = _tensor_peaks()
+    tflops = 2.0 * nq * N * d / (ms / 1e3) / 1e12
+    gbs = N * d * 2 / (ms / 1e3) / 1e9
+    print(json.dumps({
+        "metric": METRIC, "value": nq / (ms / 1e3), "unit": UNIT, "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": "Exact flat search (configs[4]): N=%d d=%d bf16 unit rows, nq=%d k=%d" % (N, d, nq, k),
+                   "l2_policy": "database (%.1f GB) larger than L2" % (N * d * 2 / 1e9), "scale": args.scale},
+        "clocks": clocks, "gpu_launches": int(launches),
+        "roofline": {"bound": "tensor", "kernel": "gemm_select_kernel + flat_merge_kernel (whole call)", "achieved": tflops,
+                     "peak": sustained, "peak_kind": kind + " (sustained bf16)", "unit": "TFLOP/s", "frac": tflops / sustained,
+                     "frac_of_burst": tflops / burst, "traffic": None,
+                     "hbm": {"achieved": gbs, "peak": hbm, "frac": gbs / hbm, "unit": "GB/s"}},
+        "step_ms_p50": float(np.median(step_ms)), "step_ms_max": float(np.max(step_ms))}))
+
+
+def run_coarse_hyper(args):
+    """Secondary workload: the coarse step of the Hyperscale shape alone: 4096 queries x 65 536 bf16 centroids,
+    d = 768, inner product, nprobe = 64 (a 4096 x 768 x 65 536 contraction with the selection fused in)."""
+    from paper_2503_14649_b200 import binding, synth
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    c = synth.CONFIGS[3]
+    nq, nprobe, nlist, d = c["nq"], c["nprobe"], c["nlist"], c["d"]
+    data = synth.make_ivfpq_hashed(nlist * 4, d, nlist, c["M"], nq, metric=c["metric"], coarse_bf16=True, device=dev)
+    ix = binding.rago_index_load(data.centroids, data.codebooks, data.codes, data.list_offsets.to(dev), data.ids, data.metric)
+    q = data.queries.contiguous()
+    ws = torch.empty(ix.search_workspace_bytes(nq, nprobe, 1), dtype=torch.uint8, device=dev)
+    sampler = ClockSampler(0)
+    sampler.start()
+    t0 = time.time()
+    total_ms, step_ms = _time_steps(lambda: ix.rago_search_probes(q, nprobe, workspace=ws), args.steps, args.warmup)
+    t1 = time.time()
+    clocks = sampler.stop(t0, t1)
+    ix.rago_check(ws)
+    ix.rago_profile_enable(True)
+    out_i = torch.empty((nq, 1), dtype=torch.int64, device=dev)
+    out_d = torch.empty((nq, 1), dtype=torch.float32, device=dev)
+    ws2 = torch.empty(ix.search_workspace_bytes(nq, nprobe, 1), dtype=torch.uint8, device=dev)
+    stage = []
+    for _ in range(5):
+        ix.rago_search(q, nprobe, 1, out_i, out_d, ws2)
+        stage.append(ix.rago_profile_read())
+    gemm_ms = float(np.median([s["coarse_scores"] for s in stage]))
+    sel_ms = float(np.median([s["probe_select"] for s in stage]))
+    ms = total_ms / args.steps
+    burst, sustained, hbm, kind = _tensor_peaks()
+    tflops = 2.0 * nq * nlist * d / (gemm_ms / 1e3) / 1e12
+    print(json.dumps({
+        "metric": "coarse_qps", "value": nq / (ms / 1e3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "Hyperscale coarse step (configs[2], coarse only): nq=%d nlist=%d d=%d bf16 nprobe=%d IP"
+                   % (nq, nlist, d, nprobe), "l2_policy": "centroids 100 MB, L2 flushed by the candidate lists"},
+        "clocks": clocks,
+        "roofline": {"bound": "tensor", "kernel": "split_bf16_kernel + gemm_select_kernel", "achieved": tflops, "peak": burst,
+                     "peak_kind": kind + " (burst bf16)", "unit": "TFLOP/s", "frac": tflops / burst,
+                     "frac_of_sustained": tflops / sustained, "traffic": None, "kernel_ms": gemm_ms},
+        "stage_ms": {"coarse_scores": gemm_ms, "probe_select": sel_ms},
+        "step_ms_p50": float(np.median(step_ms))}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -300,9 +410,15 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--scale", type=float, default=1.0, help="shrink N (development only; 1.0 = the named workload)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", default="mid", choices=["mid", "flat", "coarse_hyper"],
+                    help="mid = the headline Mid IVF-PQ workload (default); the others are secondary measurements")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload == "flat":
+        run_flat(args)
+    elif args.workload == "coarse_hyper":
+        run_coarse_hyper(args)
     else:
         run_ours(args)
 
