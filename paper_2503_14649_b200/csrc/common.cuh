@@ -100,16 +100,28 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait: gives up after ~2^22 polls (with back-off) or as soon as *abort_flag is set by
-// another warp.  On give-up it raises the CTA abort flag and the global error word; callers keep
-// their control flow (so CTA-wide barriers still match) but the data is garbage.
+// try_wait that lets the hardware park the thread for up to `ns` nanoseconds before it answers.
+__device__ __forceinline__ bool mbar_try_wait_hint(uint32_t bar, uint32_t parity, uint32_t ns) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(ns)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: each poll may park the thread for up to 4 us, and the wait gives up after 2^18
+// polls (about a second) or as soon as *abort_flag is set by another warp.  On give-up it raises the
+// CTA abort flag and the global error word; callers keep their control flow (so CTA-wide barriers
+// still match) but the data is garbage.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
                                           uint32_t* err_word) {
     if (mbar_try_wait(bar, parity)) return true;
-    for (uint32_t it = 0; it < (1u << 22); ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (it > 64) __nanosleep(it > 4096 ? 256 : 32);
-        if ((it & 63) == 63 && *abort_flag) return false;
+    for (uint32_t it = 0; it < (1u << 18); ++it) {
+        if (mbar_try_wait_hint(bar, parity, 4000u)) return true;
+        if ((it & 15) == 15 && *abort_flag) return false;
     }
     *abort_flag = 1;
     atomicExch(err_word, (uint32_t)ERR_WAIT_TIMEOUT);
@@ -160,7 +172,7 @@ cudaError_t launch_select_probes_cand(const IndexImpl* ix, const float* queries,
                                       const int32_t* cand_cnt, int nsplit, int cap, int nq, int nprobe,
                                       int32_t* probe_list, float* probe_term, float* probe_bias, cudaStream_t s);
 // gemm_select.cu
-constexpr int GEMM_CAP_SMALL = 256, GEMM_CAP_LARGE = 1024;  // candidate-list capacities (keys per row and column range)
+constexpr int GEMM_CAP_SMALL = 512, GEMM_CAP_LARGE = 1024;  // candidate-list capacities (keys per row and column range)
 struct GemmLaunch {
     const void* tmap_a;          // CUtensorMap of A: bf16 [a parts * a_part_rows][d]
     const void* tmap_b;          // CUtensorMap of B: bf16 [b parts * b_part_rows][d]

@@ -18,10 +18,10 @@
 //
 // Fused selection (mode 0).  A value below the row's threshold is appended to the row's candidate
 // list in global memory (capacity CAP = 32*NK keys, 64-bit key = ordered score bits << 32 | column).
-// When a list could overflow, its warp loads it into registers (NK keys per lane), finds the nsel-th
-// smallest score by a 32-step bit-wise search with warp-wide counts, keeps exactly nsel keys and
-// lowers the threshold.  The threshold is always the nsel-th smallest of a subset of the row, so no
-// key that belongs to the row's nsel best is ever dropped; the lists of all column ranges are merged
+// When a list could overflow, its warp loads it into registers (NK keys per lane), bisects for a cut
+// value that keeps between nsel and nsel + slack keys (a few warp-wide counts), writes the kept keys
+// back and lowers the threshold.  The threshold is always at least the nsel-th smallest of a subset of
+// the row, so no key that belongs to the row's nsel best is ever dropped; the lists of all column ranges are merged
 // by the caller.  Mode 1 writes the score matrix instead.
 //
 // Every wait is bounded (common.cuh); on a timeout the roles leave their loops, the error word is
@@ -116,47 +116,67 @@ struct GemmArgs {
     uint32_t* err;
 };
 
-// Keep the nsel smallest of the n (> nsel) keys of one list; returns the new threshold score.
+// Cut one list of n (> nsel) keys down to between nsel and nkeep keys and return the new threshold.
+// The cut value T is found by bisection on the ordered score bits between the list's minimum and
+// maximum: it stops as soon as nsel <= #(score <= T) <= nkeep, which takes a handful of warp-wide
+// counts instead of one per bit; if it runs down to a single value (a tie group larger than the slack)
+// only as many of the tied keys are kept as are needed to reach nsel.  Every kept set contains the
+// nsel smallest keys of the list, and the threshold is the largest kept score.
 template <int NK>
-__device__ __forceinline__ float compact_list(unsigned long long* list, int n, int nsel, int lane) {
-    unsigned long long k[NK];
+__device__ __forceinline__ float compact_list(unsigned long long* list, int n, int nsel, int nkeep, int lane, int* kept) {
+    uint32_t s[NK];
+    uint32_t pl[NK];
+    uint32_t mn = 0xFFFFFFFFu, mx = 0u;
 #pragma unroll
     for (int j = 0; j < NK; ++j) {
         const int idx = lane + 32 * j;
-        k[j] = idx < n ? list[idx] : KEY_MAX;
+        const unsigned long long k = idx < n ? list[idx] : KEY_MAX;
+        s[j] = (uint32_t)(k >> 32);
+        pl[j] = (uint32_t)k;
+        if (idx < n) {
+            mn = s[j] < mn ? s[j] : mn;
+            mx = s[j] > mx ? s[j] : mx;
+        }
     }
-    uint32_t v = 0;  // becomes the nsel-th smallest score (ordered bits)
+    mn = __reduce_min_sync(0xffffffffu, mn);
+    mx = __reduce_max_sync(0xffffffffu, mx);
+    // invariant: #(score <= lo) < nsel <= #(score <= hi)   (lo = mn - 1 as a 64-bit value to allow mn = 0)
+    long long lo = (long long)mn - 1, hi = mx;
+    uint32_t c_hi = (uint32_t)n;
 #pragma unroll 1
-    for (int b = 31; b >= 0; --b) {
-        const uint32_t trial = v | (1u << b);
+    while (hi - lo > 1 && c_hi > (uint32_t)nkeep) {
+        const uint32_t mid = (uint32_t)(lo + (hi - lo) / 2);
         uint32_t c = 0;
 #pragma unroll
-        for (int j = 0; j < NK; ++j) c += ((uint32_t)(k[j] >> 32) < trial) ? 1u : 0u;
+        for (int j = 0; j < NK; ++j) c += (s[j] <= mid) ? 1u : 0u;  // padding keys carry the largest score pattern
         c = __reduce_add_sync(0xffffffffu, c);
-        if (c < (uint32_t)nsel) v = trial;
+        if (c < (uint32_t)nsel) lo = mid; else { hi = mid; c_hi = c; }
     }
+    const uint32_t T = (uint32_t)hi;
+    // keys below T are all kept; keys equal to T only as far as needed when the tie group is too large
     uint32_t less = 0;
 #pragma unroll
-    for (int j = 0; j < NK; ++j) less += ((uint32_t)(k[j] >> 32) < v) ? 1u : 0u;
+    for (int j = 0; j < NK; ++j) less += (s[j] < T) ? 1u : 0u;
     less = __reduce_add_sync(0xffffffffu, less);
-    int need = nsel - (int)less;  // keys equal to v that still have to be kept (>= 1)
+    int need = c_hi <= (uint32_t)nkeep ? (int)(c_hi - less) : nsel - (int)less;  // keys equal to T to keep
     __syncwarp();
     const uint32_t lt_mask = (1u << lane) - 1u;
     int base = 0;
 #pragma unroll
     for (int j = 0; j < NK; ++j) {
-        const uint32_t s = (uint32_t)(k[j] >> 32);
-        const bool eq = s == v && k[j] != KEY_MAX;
+        const bool valid = lane + 32 * j < n;
+        const bool eq = valid && s[j] == T;
         const uint32_t meq = __ballot_sync(0xffffffffu, eq);
-        const bool keep = s < v || (eq && __popc(meq & lt_mask) < need);
+        const bool keep = valid && (s[j] < T || (eq && __popc(meq & lt_mask) < need));
         const uint32_t mk = __ballot_sync(0xffffffffu, keep);
-        if (keep) list[base + __popc(mk & lt_mask)] = k[j];
+        if (keep) list[base + __popc(mk & lt_mask)] = ((unsigned long long)s[j] << 32) | pl[j];
         base += __popc(mk);
         const int eq_kept = __popc(meq) < need ? __popc(meq) : need;
         need -= eq_kept;
     }
     __syncwarp();
-    return orderable_f32(v);
+    *kept = base;
+    return orderable_f32(T);
 }
 
 template <int NK>
@@ -283,16 +303,28 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                 int cnt = g ? cnt1 : cnt0;
                 unsigned long long* list =
                     a.cand + ((size_t)(row < a.nrows ? row : 0) * nsplit + split) * CAP;  // never written for padding rows
+                const int nkeep = a.nsel + (CAP - 64 - a.nsel) / 2;  // slack the bisection may leave in a list
 #pragma unroll 1
                 for (int c0 = 0; c0 < GBN; c0 += 32) {
                     float v[32];
                     tmem_ld32(taddr + c0, v);
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const float s = fmaf(a.alpha, v[j], cn[buf * GBN + c0 + j]);
-                        if (s < tau) {
-                            list[cnt] = make_key(s, (uint32_t)(nt * GBN + c0 + j));
-                            ++cnt;
+                    for (int j0 = 0; j0 < 32; j0 += 8) {
+                        float sc[8];
+                        float m = inf;
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            sc[j] = fmaf(a.alpha, v[j0 + j], cn[buf * GBN + c0 + j0 + j]);
+                            m = fminf(m, sc[j]);
+                        }
+                        if (__any_sync(0xffffffffu, m < tau)) {  // rare once the thresholds have settled
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                if (sc[j] < tau) {
+                                    list[cnt] = make_key(sc[j], (uint32_t)(nt * GBN + c0 + j0 + j));
+                                    ++cnt;
+                                }
+                            }
                         }
                     }
                     uint32_t todo = __ballot_sync(0xffffffffu, cnt > CAP - 32);
@@ -302,8 +334,10 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                         const int n = __shfl_sync(0xffffffffu, cnt, r);
                         const unsigned long long lp = __shfl_sync(0xffffffffu, (unsigned long long)list, r);
                         __syncwarp();
-                        const float nt_tau = compact_list<NK>(reinterpret_cast<unsigned long long*>(lp), n, a.nsel, lane);
-                        if (lane == r) { cnt = a.nsel; tau = nt_tau; }
+                        int kept = 0;
+                        const float nt_tau =
+                            compact_list<NK>(reinterpret_cast<unsigned long long*>(lp), n, a.nsel, nkeep, lane, &kept);
+                        if (lane == r) { cnt = kept; tau = nt_tau; }
                     }
                 }
                 if (g) { tau1 = tau; cnt1 = cnt; } else { tau0 = tau; cnt0 = cnt; }
@@ -373,7 +407,7 @@ cudaError_t make_tmap_bf16(void* out_map, const void* ptr, uint64_t rows, uint64
     return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
-int gemm_cand_cap(int nsel) { return nsel <= GEMM_CAP_SMALL - 64 ? GEMM_CAP_SMALL : (nsel <= GEMM_CAP_LARGE - 64 ? GEMM_CAP_LARGE : 0); }
+int gemm_cand_cap(int nsel) { return nsel <= GEMM_CAP_SMALL - 128 ? GEMM_CAP_SMALL : (nsel <= GEMM_CAP_LARGE - 64 ? GEMM_CAP_LARGE : 0); }
 
 void gemm_grid(int nrows, int64_t ncols, int num_sms, int* mg, int* nsplit, int* mgroups) {
     const int mtiles = (nrows + GBM - 1) / GBM;
