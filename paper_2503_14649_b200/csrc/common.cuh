@@ -117,10 +117,11 @@ __device__ __forceinline__ bool mbar_try_wait_hint(uint32_t bar, uint32_t parity
 // CTA abort flag and the global error word; callers keep their control flow (so CTA-wide barriers
 // still match) but the data is garbage.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                          uint32_t* err_word) {
+                                          uint32_t* err_word, uint32_t backoff_ns = 0) {
     if (mbar_try_wait(bar, parity)) return true;
     for (uint32_t it = 0; it < (1u << 18); ++it) {
         if (mbar_try_wait_hint(bar, parity, 4000u)) return true;
+        if (backoff_ns) __nanosleep(backoff_ns);  // single-lane roles: leave the issue slots to the working warps
         if ((it & 15) == 15 && *abort_flag) return false;
     }
     *abort_flag = 1;

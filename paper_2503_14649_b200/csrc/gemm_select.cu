@@ -53,6 +53,12 @@ __device__ __forceinline__ void tma_load_2d(const CUtensorMap* map, uint32_t bar
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
         : "memory");
 }
+// Pull a tile into L2 ahead of its load (no shared memory, no completion to wait for).
+__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* map, int x, int y) {
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(reinterpret_cast<uint64_t>(map)),
+                 "r"(x), "r"(y)
+                 : "memory");
+}
 __device__ __forceinline__ void tmem_alloc(uint32_t slot_smem, uint32_t ncols) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(ncols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -97,6 +103,20 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
 __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
     return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) |
            ((uint64_t)2 << 61);
+}
+
+// if (score < tau) { *slot = key(score, col); ++cnt; }  without a branch
+__device__ __forceinline__ void push_if_below(unsigned long long* slot, float score, float tau, uint32_t col, int& cnt) {
+    const uint32_t u = __float_as_uint(score);
+    const uint32_t ord = u ^ ((uint32_t)((int32_t)u >> 31) | 0x80000000u);  // order-preserving bits (f32_orderable)
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.lt.f32 p, %1, %2;\n\t"
+        "@p st.global.v2.u32 [%3], {%4, %5};\n\t"
+        "@p add.s32 %0, %0, 1;\n\t}"
+        : "+r"(cnt)
+        : "f"(score), "f"(tau), "l"(slot), "r"(col), "r"(ord)
+        : "memory");
 }
 
 struct GemmArgs {
@@ -228,22 +248,33 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
     if (warp == 0) {
         // ================= TMA producer =================
         if (lane == 0) {
-            uint32_t it = 0;
-            bool dead = false;
-            for (int u = 0; u < nunits && !dead; ++u) {
+            constexpr int PF = 2 * G_STAGES;  // B tiles are pulled into L2 this many k-blocks ahead of their load
+            const int total = nunits * kiters;
+            auto coords = [&](int gi, int& kx, int& ya, int& yb) {
+                const int u = gi / kiters, r = gi - u * kiters;
+                const int t = r / a.kblocks, kb = r - t * a.kblocks;
                 const int nt = nt_begin + u / mcount, m = m0 + u % mcount;
-                for (int t = 0; t < a.nterms && !dead; ++t) {
-                    const int ya = a.term_a[t] * a.a_part_rows + m * GBM;
-                    const int yb = a.term_b[t] * a.b_part_rows + nt * GBN;
-                    for (int kb = 0; kb < a.kblocks; ++kb, ++it) {
-                        const int s = it % G_STAGES;
-                        const uint32_t ph = (it / G_STAGES) & 1u;
-                        if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, a.err)) { dead = true; break; }
-                        mbar_arrive_expect_tx(full_bar(s), G_STAGE_BYTES);
-                        tma_load_2d(&tmA, full_bar(s), base + s * G_STAGE_BYTES, kb * GBK, ya);
-                        tma_load_2d(&tmB, full_bar(s), base + s * G_STAGE_BYTES + G_A_BYTES, kb * GBK, yb);
-                    }
+                kx = kb * GBK;
+                ya = a.term_a[t] * a.a_part_rows + m * GBM;
+                yb = a.term_b[t] * a.b_part_rows + nt * GBN;
+            };
+            int kx, ya, yb;
+            for (int gi = 0; gi < PF && gi < total; ++gi) {
+                coords(gi, kx, ya, yb);
+                tma_prefetch_2d(&tmB, kx, yb);
+            }
+            for (int gi = 0; gi < total; ++gi) {
+                const int s = gi % G_STAGES;
+                const uint32_t ph = (uint32_t)(gi / G_STAGES) & 1u;
+                if (gi + PF < total) {
+                    coords(gi + PF, kx, ya, yb);
+                    tma_prefetch_2d(&tmB, kx, yb);
                 }
+                coords(gi, kx, ya, yb);
+                if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, a.err, 64)) break;
+                mbar_arrive_expect_tx(full_bar(s), G_STAGE_BYTES);
+                tma_load_2d(&tmA, full_bar(s), base + s * G_STAGE_BYTES, kx, ya);
+                tma_load_2d(&tmB, full_bar(s), base + s * G_STAGE_BYTES + G_A_BYTES, kx, yb);
             }
         }
     } else if (warp == 1) {
@@ -254,13 +285,13 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             for (int u = 0; u < nunits && !dead; ++u) {
                 const int buf = u & 1;
                 const uint32_t uph = (u >> 1) & 1u;
-                if (!mbar_wait(tempty_bar(buf), uph ^ 1u, abort_flag, a.err)) break;
+                if (!mbar_wait(tempty_bar(buf), uph ^ 1u, abort_flag, a.err, 64)) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * GBN);
                 for (int ki = 0; ki < kiters; ++ki, ++it) {
                     const int s = it % G_STAGES;
                     const uint32_t ph = (it / G_STAGES) & 1u;
-                    if (!mbar_wait(full_bar(s), ph, abort_flag, a.err)) { dead = true; break; }
+                    if (!mbar_wait(full_bar(s), ph, abort_flag, a.err, 32)) { dead = true; break; }
                     tc_fence_after();
                     const uint64_t da = smem_desc_sw128(base + s * G_STAGE_BYTES);
                     const uint64_t db = smem_desc_sw128(base + s * G_STAGE_BYTES + G_A_BYTES);
@@ -303,29 +334,18 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                 int cnt = g ? cnt1 : cnt0;
                 unsigned long long* list =
                     a.cand + ((size_t)(row < a.nrows ? row : 0) * nsplit + split) * CAP;  // never written for padding rows
-                const int nkeep = a.nsel + (CAP - 64 - a.nsel) / 2;  // slack the bisection may leave in a list
+                const int slack = a.nsel / 4 > 8 ? a.nsel / 4 : 8;
+                const int nkeep = a.nsel + slack < CAP - 64 ? a.nsel + slack : CAP - 64;  // what the bisection may leave in a list
 #pragma unroll 1
                 for (int c0 = 0; c0 < GBN; c0 += 32) {
                     float v[32];
                     tmem_ld32(taddr + c0, v);
+                    // straight-line, branch-free: a passing value is stored by a predicated instruction
+                    const uint32_t col0 = (uint32_t)(nt * GBN + c0);
 #pragma unroll
-                    for (int j0 = 0; j0 < 32; j0 += 8) {
-                        float sc[8];
-                        float m = inf;
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            sc[j] = fmaf(a.alpha, v[j0 + j], cn[buf * GBN + c0 + j0 + j]);
-                            m = fminf(m, sc[j]);
-                        }
-                        if (__any_sync(0xffffffffu, m < tau)) {  // rare once the thresholds have settled
-#pragma unroll
-                            for (int j = 0; j < 8; ++j) {
-                                if (sc[j] < tau) {
-                                    list[cnt] = make_key(sc[j], (uint32_t)(nt * GBN + c0 + j0 + j));
-                                    ++cnt;
-                                }
-                            }
-                        }
+                    for (int j = 0; j < 32; ++j) {
+                        const float sc = fmaf(a.alpha, v[j], cn[buf * GBN + c0 + j]);
+                        push_if_below(list + cnt, sc, tau, col0 + j, cnt);
                     }
                     uint32_t todo = __ballot_sync(0xffffffffu, cnt > CAP - 32);
                     while (todo) {  // warp-uniform
