@@ -41,6 +41,8 @@ static bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_
 struct Layout {
     size_t err, probe_list, probe_term, probe_bias, scores, pair_tiles, work_prefix, qthresh, slot_cnt, slot_keys, total;
     size_t qparts, cand, cand_cnt;  // tensor-core coarse step: query parts, candidate lists and their counts
+    size_t pilot_scores, row_tau;   // pilot pass: scores of the sampled lists, per-query starting thresholds
+    int pilot_cols;                 // 0: no pilot pass
     size_t nslots;
     int tc, tc_mode, tc_cap, tc_mg, tc_nsplit;  // coarse plan for this (nq, nprobe)
 };
@@ -69,7 +71,8 @@ static Layout make_layout(const IndexImpl* ix, int nq, int nprobe, int k) {
     L.probe_bias = take(npairs * 4);
     L.tc = use_tensor_cores(ix, nq) ? 1 : 0;
     L.tc_mode = 1; L.tc_cap = 0; L.tc_mg = 1; L.tc_nsplit = 1;
-    L.qparts = L.cand = L.cand_cnt = 0;
+    L.qparts = L.cand = L.cand_cnt = L.pilot_scores = L.row_tau = 0;
+    L.pilot_cols = 0;
     if (L.tc) {
         int nsel = nprobe + PROBE_GUARD;
         if (nsel > ix->nlist) nsel = ix->nlist;
@@ -81,6 +84,13 @@ static Layout make_layout(const IndexImpl* ix, int nq, int nprobe, int k) {
         if (L.tc_mode == 0) {
             L.cand = take((size_t)nq * L.tc_nsplit * L.tc_cap * 8);
             L.cand_cnt = take((size_t)nq * L.tc_nsplit * 4);
+            // a pilot pass pays off when a CTA sees many column tiles per row and the sample can hold nsel values
+            const int np = ix->pilot_stride ? ix->nlist / ix->pilot_stride : 0;
+            if (np >= 4 * nsel && ix->nlist >= 8192) {
+                L.pilot_cols = np;
+                L.pilot_scores = take((size_t)nq * np * 4);
+                L.row_tau = take((size_t)nq * 4);
+            }
         }
     }
     L.scores = take((!L.tc || L.tc_mode == 1) ? (size_t)nq * ix->nlist * 4 : 0);
@@ -140,12 +150,30 @@ static rago_status run_coarse(const IndexImpl* ix, const float* queries, int nq,
         G.mg = L.tc_mg; G.nsplit = L.tc_nsplit;
         G.alpha = ix->metric == RAGO_L2 ? -2.f : -1.f;
         G.colterm = ix->metric == RAGO_L2 ? ix->cnorm : nullptr;
+        G.colterm_stride = 1;
+        G.row_tau = nullptr;
         G.mode = L.tc_mode; G.cap = L.tc_cap;
         G.nsel = nprobe + PROBE_GUARD < ix->nlist ? nprobe + PROBE_GUARD : ix->nlist;
         G.cand = reinterpret_cast<unsigned long long*>(ws + L.cand);
         G.cand_cnt = reinterpret_cast<int32_t*>(ws + L.cand_cnt);
         G.scores = scores;
         G.err = reinterpret_cast<uint32_t*>(ws + L.err);
+        if (L.pilot_cols) {
+            // pilot pass: score every pilot_stride-th list, take each query's nsel-th smallest as its starting threshold
+            GemmLaunch P = G;
+            int mgroups = 1;
+            P.tmap_b = ix->tmap_b_pilot;
+            P.ncols = L.pilot_cols; P.b_part_rows = L.pilot_cols;
+            gemm_grid(nq, L.pilot_cols, ix->num_sms, &P.mg, &P.nsplit, &mgroups);
+            P.colterm_stride = ix->pilot_stride;
+            P.mode = 1;
+            P.scores = reinterpret_cast<float*>(ws + L.pilot_scores);
+            e = launch_gemm_select(P, s);
+            if (e == cudaSuccess)
+                e = launch_row_tau(P.scores, nq, L.pilot_cols, G.nsel, reinterpret_cast<float*>(ws + L.row_tau), s);
+            if (e != cudaSuccess) return cuda_fail(e, "pilot pass of the coarse step");
+            G.row_tau = reinterpret_cast<float*>(ws + L.row_tau);
+        }
         e = launch_gemm_select(G, s);
         if (e != cudaSuccess) return cuda_fail(e, "tensor-core coarse kernel");
         record(mix, 1, s);
@@ -241,6 +269,11 @@ rago_status rago_index_load(rago_index** out, const void* coarse_centroids, rago
         if (e == cudaSuccess && gemm_select_init() == cudaSuccess &&
             make_tmap_bf16(ix->tmap_b, bsrc, (uint64_t)ix->cparts_n * nlist, (uint64_t)d, 256) == cudaSuccess)
             ix->tc_ok = 1;
+        const int ps = gemm_pilot_stride(nlist);
+        if (ix->tc_ok && nlist % ps == 0 &&
+            make_tmap_bf16(ix->tmap_b_pilot, bsrc, (uint64_t)ix->cparts_n * (nlist / ps), (uint64_t)d, 256,
+                           (uint64_t)ps * d) == cudaSuccess)
+            ix->pilot_stride = ps;
         cudaGetLastError();  // a missing tensor-core path is not an error: the fp32 kernel serves every batch
     }
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);

@@ -45,6 +45,8 @@ struct IndexImpl {
     int tc_ok;     // tensor-core coarse path available (tensor map encoded)
     int coarse_mode;  // 0 auto, 1 fp32 pipes, 2 tensor cores
     alignas(64) unsigned char tmap_b[128];  // CUtensorMap of the stacked centroid parts
+    alignas(64) unsigned char tmap_b_pilot[128];  // the same, every pilot_stride-th centroid
+    int pilot_stride;  // 0: no pilot pass for this index
     int device, num_sms;
     ScanPlan plan;
     int profile;
@@ -181,12 +183,17 @@ struct GemmLaunch {
     int a_part_rows; int64_t b_part_rows;
     int nterms; int term_a[6], term_b[6];
     int mg, nsplit;              // from gemm_grid
-    float alpha; const float* colterm;
+    float alpha; const float* colterm; int colterm_stride;
+    const float* row_tau;        // initial per-row thresholds (mode 0) or null
     int mode, nsel, cap;
     unsigned long long* cand; int32_t* cand_cnt; float* scores; uint32_t* err;
 };
 cudaError_t gemm_select_init();
-cudaError_t make_tmap_bf16(void* out_map, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows);
+cudaError_t make_tmap_bf16(void* out_map, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows,
+                           uint64_t row_stride = 0);
+// The pilot pass scores every stride-th column: 16, or more when that would still leave over 32 768 columns.
+inline int gemm_pilot_stride(int64_t ncols) { const int64_t s = (ncols + 32767) / 32768; return s > 16 ? (int)s : 16; }
+cudaError_t launch_row_tau(const float* scores, int nrows, int n, int nsel, float* row_tau, cudaStream_t s);
 int gemm_cand_cap(int nsel);  // 0: nsel too large for the fused selection
 void gemm_grid(int nrows, int64_t ncols, int num_sms, int* mg, int* nsplit, int* mgroups);
 cudaError_t launch_gemm_select(const GemmLaunch& L, cudaStream_t s);

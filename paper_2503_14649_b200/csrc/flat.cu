@@ -166,13 +166,21 @@ static int sm_count() {
 
 static bool flat_on_tensor_cores(int d, int k) { return gemm_cand_cap(k) != 0 && d % 8 == 0; }
 
-// Workspace, tensor-core path: [err 256 B][cand nq*nsplit*cap u64][cand_cnt nq*nsplit i32]
+// Pilot pass of the flat search: worth it for large databases; the sample must hold 4 k rows.
+static int flat_pilot_cols(int64_t N, int k) {
+    if (N < (1 << 18)) return 0;
+    const int64_t np = N / gemm_pilot_stride(N);
+    return np >= 4LL * k ? (int)np : 0;
+}
+
+// Workspace, tensor-core path: [err 256 B][cand nq*nsplit*cap u64][cand_cnt nq*nsplit i32][pilot scores nq*np f32][row_tau nq f32]
 //            fallback:         [err 256 B][scores nq*PANEL f32][slot_cnt nq*nchunks i32][slot_keys nq*nchunks*k u64]
 size_t flat_workspace_bytes(int64_t N, int d, int nq, int k) {
     if (flat_on_tensor_cores(d, k)) {
         int mg, nsplit, mgroups;
         gemm_grid(nq > 0 ? nq : 1, N > 0 ? N : 1, sm_count(), &mg, &nsplit, &mgroups);
-        return 256 + align_up((size_t)nq * nsplit * gemm_cand_cap(k) * 8, 256) + align_up((size_t)nq * nsplit * 4, 256);
+        return 256 + align_up((size_t)nq * nsplit * gemm_cand_cap(k) * 8, 256) + align_up((size_t)nq * nsplit * 4, 256) +
+               align_up((size_t)nq * flat_pilot_cols(N, k) * 4, 256) + align_up((size_t)nq * 4, 256);
     }
     const size_t nchunks = (size_t)((N + FLAT_CHUNK - 1) / FLAT_CHUNK);
     size_t b = 256;
@@ -194,6 +202,11 @@ cudaError_t launch_flat_search(const void* db, int64_t N, int d, const void* que
         unsigned long long* cand = reinterpret_cast<unsigned long long*>(w);
         w += align_up((size_t)nq * nsplit * cap * 8, 256);
         int32_t* cand_cnt = reinterpret_cast<int32_t*>(w);
+        w += align_up((size_t)nq * nsplit * 4, 256);
+        const int np = flat_pilot_cols(N, k);
+        float* pilot_scores = reinterpret_cast<float*>(w);
+        w += align_up((size_t)nq * np * 4, 256);
+        float* row_tau = reinterpret_cast<float*>(w);
         alignas(64) unsigned char tmap_a[128], tmap_b[128];
         e = make_tmap_bf16(tmap_a, queries, (uint64_t)nq, (uint64_t)d, 128);
         if (e == cudaSuccess) e = make_tmap_bf16(tmap_b, db, (uint64_t)N, (uint64_t)d, 256);
@@ -206,10 +219,28 @@ cudaError_t launch_flat_search(const void* db, int64_t N, int d, const void* que
         for (int t = 0; t < 6; ++t) G.term_a[t] = G.term_b[t] = 0;
         G.mg = mg; G.nsplit = nsplit;
         G.alpha = -1.f;  // smaller = better
-        G.colterm = nullptr;
+        G.colterm = nullptr; G.colterm_stride = 1;
+        G.row_tau = nullptr;
         G.mode = 0; G.nsel = k < N ? k : (int)N; G.cap = cap;
         G.cand = cand; G.cand_cnt = cand_cnt; G.scores = nullptr;
         G.err = static_cast<uint32_t*>(workspace);
+        if (np) {
+            // pilot pass over every stride-th row: each query starts from the k-th best score of that sample
+            alignas(64) unsigned char tmap_p[128];
+            const int ps = gemm_pilot_stride(N);
+            e = make_tmap_bf16(tmap_p, db, (uint64_t)np, (uint64_t)d, 256, (uint64_t)ps * d);
+            if (e != cudaSuccess) return e;
+            GemmLaunch P = G;
+            int pg = 1;
+            P.tmap_b = tmap_p;
+            P.ncols = np; P.b_part_rows = np;
+            gemm_grid(nq, np, sm_count(), &P.mg, &P.nsplit, &pg);
+            P.mode = 1; P.scores = pilot_scores;
+            e = launch_gemm_select(P, s);
+            if (e == cudaSuccess) e = launch_row_tau(pilot_scores, nq, np, G.nsel, row_tau, s);
+            if (e != cudaSuccess) return e;
+            G.row_tau = row_tau;
+        }
         e = launch_gemm_select(G, s);
         if (e != cudaSuccess) return e;
         flat_merge_kernel<<<nq, FSEL_THREADS, 0, s>>>(nsplit, k, cap, cand_cnt, cand, out_ids, out_scores);

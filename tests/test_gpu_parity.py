@@ -148,6 +148,7 @@ def test_results_do_not_depend_on_run():
 
 @pytest.mark.parametrize("N,d,nq,k", [(5000, 64, 7, 10), (70_000, 128, 33, 100), (3, 64, 2, 5),
                                       (200_000, 64, 200, 100),   # two row tiles, lists compacted while streaming
+                                      (300_000, 64, 40, 50),     # large enough for the pilot-threshold pass
                                       (40_000, 64, 9, 300),      # wide candidate lists
                                       (30_000, 64, 5, 1000)])    # k above the fused selection: fp32-pipe fallback
 def test_flat_search_matches_oracle(N, d, nq, k):
