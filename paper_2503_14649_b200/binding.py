@@ -104,8 +104,11 @@ class Index:
         self._ws = None
 
     def close(self):
-        if getattr(self, "_h", None) is not None and self._h.value:
-            lib().rago_index_free(self._h)
+        if getattr(self, "_h", None) is not None and self._h.value and _lib is not None:
+            try:
+                _lib.rago_index_free(self._h)
+            except Exception:  # interpreter shutdown: the module globals may already be gone
+                pass
             self._h = ctypes.c_void_p()
 
     __del__ = close

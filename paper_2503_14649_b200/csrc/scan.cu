@@ -28,6 +28,13 @@
 // is assembled by a single PRMT from the code word and a per-lane constant.  Tables wider than two
 // banks (M = 80 with its two copies) fall back to a multiply-add address.
 //
+// Fixed-point table.  Entries are stored as 32-bit integers scaled by a per-query power of two chosen
+// so that a sum of M entries cannot overflow (|sum| < 2^30): the scan then adds two entries per
+// instruction (a three-input integer add) and the sum is exact, so it does not depend on the order of
+// the additions; it is converted back to fp32 once per vector.  The quantisation step is
+// max|entry| * M / 2^30, i.e. an absolute error below max|entry| * M^2 / 2^31 per vector (2e-5 for
+// M = 96 and entries of size 5), far inside the 1e-4 relative bar.
+//
 // Candidates better than the running threshold go to a shared buffer (topk.cuh); the threshold of a
 // query is shared between CTAs through global memory, which only ever removes keys that cannot be
 // among the k best, so the result does not depend on timing.
@@ -164,6 +171,7 @@ struct Ctrl {
     TileDesc desc[MAX_STAGES];
     int cnt;
     uint32_t abort_flag;
+    float red[32];  // per-warp maxima of the table build
 };
 static_assert(sizeof(Ctrl) <= CTRL_BYTES, "control block too large");
 
@@ -188,7 +196,8 @@ __device__ __forceinline__ void sts_f32(uint32_t addr, float v) {
 // stores that walk the banks).  UNR entries per thread are loaded before any is used so that enough
 // requests are in flight to cover the L2 latency.
 template <class C, int D4>
-__device__ __forceinline__ void build_table(const float* __restrict__ cbT, const float* rT, uint32_t lut, int ctid) {
+__device__ __forceinline__ float build_table(const float* __restrict__ cbT, const float* rT, uint32_t lut, int ctid) {
+    float mx = 0.f;
     constexpr int UNR = D4 >= 3 ? 4 : 8;
     constexpr int TOTAL = KSUB * C::M;
     for (int e0 = ctid; e0 < TOTAL; e0 += C::NCT * UNR) {
@@ -215,51 +224,82 @@ __device__ __forceinline__ void build_table(const float* __restrict__ cbT, const
                 acc = fmaf(rT[(4 * i + 3) * C::M + m], cv[u][i].w, acc);
             }
             sts_f32(lut + C::lut_off(j, m), acc);
-            if (C::COPIES == 2) sts_f32(lut + C::lut_off(j, C::COPY_OFF + m), acc);
+            mx = fmaxf(mx, fabsf(acc));
         }
     }
+    return mx;
 }
 template <class C>
-__device__ __forceinline__ void build_table_any(const float* __restrict__ cbT, const float* rT, uint32_t lut,
+__device__ __forceinline__ float build_table_any(const float* __restrict__ cbT, const float* rT, uint32_t lut,
                                                 int ctid, int dsub) {
+    float mx = 0.f;
     for (int e = ctid; e < KSUB * C::M; e += C::NCT) {
         const int j = e / C::M, m = e - j * C::M;
         float acc = 0.f;
         for (int t = 0; t < dsub; ++t) acc = fmaf(rT[t * C::M + m], __ldg(cbT + (size_t)e * dsub + t), acc);
         sts_f32(lut + C::lut_off(j, m), acc);
-        if (C::COPIES == 2) sts_f32(lut + C::lut_off(j, C::COPY_OFF + m), acc);
+        mx = fmaxf(mx, fabsf(acc));
+    }
+    return mx;
+}
+// Second pass of the table build: every thread turns the fp32 entries it wrote itself into scaled
+// integers (and fills the second copy where the layout keeps one).
+template <class C>
+__device__ __forceinline__ void quantise_table(uint32_t lut, int ctid, float scale) {
+    for (int e = ctid; e < KSUB * C::M; e += C::NCT) {
+        const int j = e / C::M, m = e - j * C::M;
+        const uint32_t addr = lut + C::lut_off(j, m);
+        const int q = __float2int_rn(lds_f32(addr) * scale);
+        sts_f32(addr, __int_as_float(q));
+        if (C::COPIES == 2) sts_f32(lut + C::lut_off(j, C::COPY_OFF + m), __int_as_float(q));
     }
 }
 
-// One block (G code words = 4G sub-spaces) of one virtual row: load the words, then 4G lookups.
+// Code words of one virtual row, all loaded before the first look-up (look-up addresses depend on them,
+// so loading block by block would expose the shared-memory latency once per block).
 template <class C, int G, int BLK>
-__device__ __forceinline__ void scan_block(uint32_t rowaddr, const uint32_t (&xo)[G], const uint32_t (&cc)[G][2],
-                                           const uint32_t (&sel)[4], const uint32_t (&lo)[G][4], uint32_t lut,
-                                           float (&acc)[4]) {
-    uint32_t x[G];
+struct LoadWords {
+    __device__ __forceinline__ static void run(uint32_t rowaddr, const uint32_t (&xo)[G], uint32_t (&x)[C::NBLK][G]) {
 #pragma unroll
-    for (int il = 0; il < G; ++il) x[il] = lds_u32_imm<BLK * G * 4>(rowaddr + xo[il]);
+        for (int il = 0; il < G; ++il) x[BLK][il] = lds_u32_imm<BLK * G * 4>(rowaddr + xo[il]);
+        if constexpr (BLK + 1 < C::NBLK) LoadWords<C, G, BLK + 1>::run(rowaddr, xo, x);
+    }
+};
+
+// One block (G code words = 4G sub-spaces) of one virtual row: 4G look-ups, written as three passes over
+// half a block (all addresses, all loads, all adds).
+template <class C, int G, int BLK>
+__device__ __forceinline__ void scan_block(const uint32_t (&x)[G], const uint32_t (&cc)[G][2], const uint32_t (&sel)[4],
+                                           const uint32_t (&lo)[G][4], uint32_t lut, int (&acc)[4]) {
+    constexpr int H = G / 2;
 #pragma unroll
-    for (int il = 0; il < G; ++il) {
+    for (int h0 = 0; h0 < G; h0 += H) {
+        uint32_t ad[H][4];
+        uint32_t vv[H][4];
 #pragma unroll
-        for (int t = 0; t < 4; ++t) {
-            if (C::BANKED) {
-                const uint32_t a = __byte_perm(x[il], cc[il][t >> 1], sel[t]);
-                acc[t] += lds_f32_imm<(int)C::blk_imm(BLK)>(a);
-            } else {
-                const uint32_t j = __byte_perm(x[il], 0u, sel[t]);
-                acc[t] += lds_f32_imm<BLK * G * 16>(lut + j * (uint32_t)(C::LSTRIDE * 4) + lo[il][t]);
-            }
-        }
+        for (int i = 0; i < H; ++i)
+#pragma unroll
+            for (int t = 0; t < 4; ++t)
+                ad[i][t] = C::BANKED ? __byte_perm(x[h0 + i], cc[h0 + i][t >> 1], sel[t])
+                                     : lut + __byte_perm(x[h0 + i], 0u, sel[t]) * (uint32_t)(C::LSTRIDE * 4) + lo[h0 + i][t];
+#pragma unroll
+        for (int i = 0; i < H; ++i)
+#pragma unroll
+            for (int t = 0; t < 4; ++t)
+                vv[i][t] = C::BANKED ? lds_u32_imm<(int)C::blk_imm(BLK)>(ad[i][t]) : lds_u32_imm<BLK * G * 16>(ad[i][t]);
+#pragma unroll
+        for (int i = 0; i < H; i += 2)  // two entries per add
+#pragma unroll
+            for (int t = 0; t < 4; ++t) acc[t] = acc[t] + (int)vv[i][t] + (int)vv[i + 1][t];
     }
 }
 template <class C, int G, int BLK>
 struct ScanBlocks {
-    __device__ __forceinline__ static void run(uint32_t rowaddr, const uint32_t (&xo)[G], const uint32_t (&cc)[G][2],
+    __device__ __forceinline__ static void run(const uint32_t (&x)[C::NBLK][G], const uint32_t (&cc)[G][2],
                                                const uint32_t (&sel)[4], const uint32_t (&lo)[G][4], uint32_t lut,
-                                               float (&acc)[4]) {
-        scan_block<C, G, BLK>(rowaddr, xo, cc, sel, lo, lut, acc);
-        if constexpr (BLK + 1 < C::NBLK) ScanBlocks<C, G, BLK + 1>::run(rowaddr, xo, cc, sel, lo, lut, acc);
+                                               int (&acc)[4]) {
+        scan_block<C, G, BLK>(x[BLK], cc, sel, lo, lut, acc);
+        if constexpr (BLK + 1 < C::NBLK) ScanBlocks<C, G, BLK + 1>::run(x, cc, sel, lo, lut, acc);
     }
 };
 
@@ -422,6 +462,7 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_>::THREADS, 1) scan_kernel(c
     const int k = a.k;
     const bool ip = a.metric == RAGO_IP;
     const float lut_scale = ip ? -1.f : -2.f;
+    float inv_scale = 1.f;  // fp32 value of one unit of the current query's integer table
 
     // Close the current query's candidate buffer: keep at most k keys and park them in this CTA's slot.
     auto finalize = [&]() {
@@ -447,13 +488,25 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_>::THREADS, 1) scan_kernel(c
         if (ctid == 0) ctrl->cnt = 0;
         csync();
         if (dead) return;
+        float mx;
         switch (a.dsub) {
-            case 4: build_table<C, 1>(a.cbT, rT, P.lut, ctid); break;
-            case 8: build_table<C, 2>(a.cbT, rT, P.lut, ctid); break;
-            case 12: build_table<C, 3>(a.cbT, rT, P.lut, ctid); break;
-            case 16: build_table<C, 4>(a.cbT, rT, P.lut, ctid); break;
-            default: build_table_any<C>(a.cbT, rT, P.lut, ctid, a.dsub); break;
+            case 4: mx = build_table<C, 1>(a.cbT, rT, P.lut, ctid); break;
+            case 8: mx = build_table<C, 2>(a.cbT, rT, P.lut, ctid); break;
+            case 12: mx = build_table<C, 3>(a.cbT, rT, P.lut, ctid); break;
+            case 16: mx = build_table<C, 4>(a.cbT, rT, P.lut, ctid); break;
+            default: mx = build_table_any<C>(a.cbT, rT, P.lut, ctid, a.dsub); break;
         }
+        // per-query scale: the largest power of two that keeps a sum of M entries below 2^30
+        mx = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(mx)));  // non-negative floats order like their bits
+        if (lane == 0) ctrl->red[warp] = mx;
+        csync();
+        if (dead) return;
+        for (int w = 0; w < NCW; ++w) mx = fmaxf(mx, ctrl->red[w]);
+        int ex = 0;
+        if (mx > 0.f && mx < 3.0e38f) frexpf(mx * (float)C::M, &ex);  // mx * M < 2^ex
+        ex = ex < -90 ? -90 : (ex > 120 ? 120 : ex);
+        quantise_table<C>(P.lut, ctid, ldexpf(1.f, 30 - ex));
+        inv_scale = ldexpf(1.f, ex - 30);
         tau = *reinterpret_cast<volatile unsigned long long*>(&a.qthresh[q]);
         ub = 0;
         csync();
@@ -503,11 +556,14 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_>::THREADS, 1) scan_kernel(c
             if (vr0 >= nvr) break;
             const int vr = vr0 + lane;
             const uint32_t rowaddr = tile_base + (uint32_t)vr * C::MV;
-            float acc[4] = {0.f, 0.f, 0.f, 0.f};
-            ScanBlocks<C, G, 0>::run(rowaddr, xo, cc, sel, lo, P.lut, acc);
-            float s = (acc[0] + acc[1]) + (acc[2] + acc[3]);
-            if (R >= 2) s += __shfl_xor_sync(0xffffffffu, s, 1);
-            if (R >= 4) s += __shfl_xor_sync(0xffffffffu, s, 2);
+            int acc[4] = {0, 0, 0, 0};
+            uint32_t x[C::NBLK][G];
+            LoadWords<C, G, 0>::run(rowaddr, xo, x);
+            ScanBlocks<C, G, 0>::run(x, cc, sel, lo, P.lut, acc);
+            int si = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+            if (R >= 2) si += __shfl_xor_sync(0xffffffffu, si, 1);
+            if (R >= 4) si += __shfl_xor_sync(0xffffffffu, si, 2);
+            const float s = (float)si * inv_scale;
             // per-vector term of the L2 expansion (0 for inner product); rows past the tile's end read
             // stale but in-bounds shared memory and are never pushed
             const float vt = a.vterm != nullptr ? lds_f32(vt_base + (uint32_t)(vr / R) * 4u) : 0.f;
