@@ -49,3 +49,31 @@ def match_results(ids_a, d_a, ids_o, d_o, rel=1e-4, floor=1e-6):
             if not ok:
                 problems.append((t, "id", int(ids_a[t]), float(d_a[t]), int(ids_o[t]), float(d_o[t])))
     return problems
+
+
+def compact_hashed_subindex(oracle, data, lists):
+    """Host-side oracle.Index holding only the given inverted lists of a hash-coded synth index.
+
+    The lists' codes and ids are regenerated on the CPU from (seed, position), so nothing comes from
+    the device; every other list is empty.  Used for sampled parity at sizes whose codes do not fit
+    host memory: a query whose probed lists are all in `lists` gets the same answer as on the full index.
+    """
+    from paper_2503_14649_b200 import synth
+    off = data.list_offsets.cpu().numpy()
+    lists = sorted(set(int(l) for l in lists))
+    lens = np.zeros(data.nlist, np.int64)
+    codes, ids = [], []
+    for l in lists:
+        n = int(off[l + 1] - off[l])
+        lens[l] = n
+        if n:
+            codes.append(synth.hash_codes(data.seed, int(off[l]), n, data.M).numpy())
+            ids.append(synth.hash_ids(int(off[l]), n).numpy())
+    new_off = np.zeros(data.nlist + 1, np.int64)
+    new_off[1:] = np.cumsum(lens)
+    codes = np.concatenate(codes) if codes else np.zeros((0, data.M), np.uint8)
+    ids = np.concatenate(ids) if ids else np.zeros((0,), np.int64)
+    cen = data.centroids
+    cen_h = cen.cpu().view(torch.uint16).numpy() if cen.dtype == torch.bfloat16 else cen.cpu().numpy()
+    return oracle.Index(cen_h, data.codebooks.cpu().numpy(), codes, new_off, ids, data.metric,
+                        coarse_bf16=cen.dtype == torch.bfloat16)
