@@ -402,6 +402,115 @@ def run_coarse_hyper(args):
         "step_ms_p50": float(np.median(step_ms))}))
 
 
+def run_hyper(args):
+    """Secondary workload: the whole Hyperscale shape: 1e9 hash-coded vectors (64 GB of codes), 65 536 bf16
+    centroids, 4096 queries, nprobe = 64, k = 100, inner product."""
+    from paper_2503_14649_b200 import binding, synth
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    c = synth.CONFIGS[3]
+    nq, nprobe, k = c["nq"], c["nprobe"], c["k"]
+    data = synth.make_config(3, device=dev, scale=args.scale)
+    ix = binding.rago_index_load(data.centroids, data.codebooks, data.codes, data.list_offsets.to(dev), data.ids, data.metric)
+    q = data.queries.contiguous()
+    ws = torch.empty(ix.search_workspace_bytes(nq, nprobe, k), dtype=torch.uint8, device=dev)
+    out_i = torch.empty((nq, k), dtype=torch.int64, device=dev)
+    out_d = torch.empty((nq, k), dtype=torch.float32, device=dev)
+    lists, _ = ix.rago_search_probes(q, nprobe, workspace=ws)
+    Ln = (data.list_offsets[1:] - data.list_offsets[:-1]).to(dev)
+    scan_bytes = int(Ln[lists.long()].sum().item()) * c["M"]
+    sampler = ClockSampler(0)
+    sampler.start()
+    t0 = time.time()
+    total_ms, step_ms = _time_steps(lambda: ix.rago_search(q, nprobe, k, out_i, out_d, ws), args.steps, args.warmup)
+    t1 = time.time()
+    clocks = sampler.stop(t0, t1)
+    ix.rago_check(ws)
+    ix.rago_profile_enable(True)
+    stage = []
+    for _ in range(3):
+        ix.rago_search(q, nprobe, k, out_i, out_d, ws)
+        stage.append(ix.rago_profile_read())
+    st = {kk: float(np.median([s_[kk] for s_ in stage])) for kk in stage[0]}
+    ms = total_ms / args.steps
+    hbm, kind = _peaks()
+    achieved = scan_bytes / (st["table_scan"] / 1e3) / 1e9
+    print(json.dumps({
+        "metric": METRIC, "value": nq / (ms / 1e3), "unit": UNIT, "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic",
+        "config": {"workload": "Hyperscale IVF-PQ (configs[2]): N=%d d=%d nlist=%d M=%d nq=%d nprobe=%d k=%d IP, bf16 centroids"
+                   % (data.N, c["d"], c["nlist"], c["M"], nq, nprobe, k),
+                   "l2_policy": "inputs larger than L2 (%.0f GB of codes)" % (data.N * c["M"] / 1e9), "scale": args.scale},
+        "clocks": clocks,
+        "roofline": {"bound": "hbm", "kernel": "scan_kernel (table build + ADC scan)", "achieved": achieved, "peak": hbm,
+                     "peak_kind": kind, "unit": "GB/s", "frac": achieved / hbm, "traffic": None,
+                     "algorithmic_bytes_per_launch": scan_bytes, "kernel_ms": st["table_scan"]},
+        "stage_ms": st, "step_ms_p50": float(np.median(step_ms))}))
+
+
+def run_iter(args):
+    """Secondary workload: the iterative-retrieval latency shape: N = 1e8, d = 512, nlist = 16 384, M = 32; a stream
+    of 256 batches of 1, 4 or 16 queries issued back to back on one stream, nprobe = 16, k = 20; per-batch latency
+    from CUDA events between the batches."""
+    from paper_2503_14649_b200 import binding, synth
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    c = synth.CONFIGS[4]
+    nprobe, k = c["nprobe"], c["k"]
+    sizes = synth.batch_size_stream(synth.MASTER_SEED, 256)
+    data = synth.make_config(4, device=dev, scale=args.scale, nq=sum(sizes))
+    ix = binding.rago_index_load(data.centroids, data.codebooks, data.codes, data.list_offsets.to(dev), data.ids, data.metric)
+    q = data.queries.contiguous()
+    ws = torch.empty(ix.search_workspace_bytes(16, nprobe, k), dtype=torch.uint8, device=dev)
+    out_i = torch.empty((16, k), dtype=torch.int64, device=dev)
+    out_d = torch.empty((16, k), dtype=torch.float32, device=dev)
+    starts = np.concatenate([[0], np.cumsum(sizes)[:-1]])
+
+    def stream(ev=None):
+        for b, nb in enumerate(sizes):
+            if ev is not None:
+                ev[b].record()
+            ix.rago_search(q[starts[b]:starts[b] + nb], nprobe, k, out_i[:nb], out_d[:nb], ws)
+        if ev is not None:
+            ev[len(sizes)].record()
+
+    for _ in range(max(3, args.warmup)):
+        stream()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    sampler.start()
+    t0 = time.time()
+    lat = {1: [], 4: [], 16: []}
+    tot = []
+    for _ in range(args.steps):
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(len(sizes) + 1)]
+        stream(ev)
+        torch.cuda.synchronize()
+        for b, nb in enumerate(sizes):
+            lat[nb].append(ev[b].elapsed_time(ev[b + 1]))
+        tot.append(ev[0].elapsed_time(ev[-1]))
+    t1 = time.time()
+    clocks = sampler.stop(t0, t1)
+    ix.rago_check(ws)
+    ms = float(np.mean(tot))
+    alll = np.concatenate([lat[1], lat[4], lat[16]])
+    print(json.dumps({
+        "metric": METRIC, "value": sum(sizes) / (ms / 1e3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "Iterative-retrieval stream (configs[3]): N=%d d=%d nlist=%d M=%d, 256 batches of 1/4/16 "
+                   "queries back to back on one stream, nprobe=%d k=%d L2" % (data.N, c["d"], c["nlist"], c["M"], nprobe, k),
+                   "step": "one pass over the 256-batch stream (%d queries)" % sum(sizes), "scale": args.scale},
+        "clocks": clocks,
+        "latency_ms": {"p50": float(np.percentile(alll, 50)), "p99": float(np.percentile(alll, 99)),
+                       "by_batch_size": {str(nb): {"p50": float(np.percentile(v, 50)), "p99": float(np.percentile(v, 99))}
+                                         for nb, v in lat.items()},
+                       "note": "device time between consecutive batches' start events (launch-to-launch on a busy stream)"},
+        "roofline": {"bound": "latency", "kernel": "whole call", "achieved": None, "peak": None,
+                     "unit": None, "frac": None, "traffic": None}}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -410,7 +519,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--scale", type=float, default=1.0, help="shrink N (development only; 1.0 = the named workload)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="mid", choices=["mid", "flat", "coarse_hyper"],
+    ap.add_argument("--workload", default="mid", choices=["mid", "flat", "coarse_hyper", "hyper", "iter"],
                     help="mid = the headline Mid IVF-PQ workload (default); the others are secondary measurements")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -419,6 +528,10 @@ def main():
         run_flat(args)
     elif args.workload == "coarse_hyper":
         run_coarse_hyper(args)
+    elif args.workload == "hyper":
+        run_hyper(args)
+    elif args.workload == "iter":
+        run_iter(args)
     else:
         run_ours(args)
 
