@@ -100,7 +100,66 @@ __global__ void __launch_bounds__(256) coarse_scores_kernel(const float* __restr
     }
 }
 
+// ---- score matrix for tiny batches (the latency-bound iterative-retrieval shape) -------------------
+// Up to CS_MAXQ queries sit in shared memory; one warp per centroid streams the centroid row once
+// (16-byte loads) and keeps one partial sum per query, so the centroid table is read exactly once per
+// batch however few queries there are.
+constexpr int CS_MAXQ = 16;
+template <bool BF16>
+__global__ void __launch_bounds__(256) coarse_small_kernel(const float* __restrict__ Q, const void* __restrict__ C,
+                                                           const float* __restrict__ cnorm, int nq, int nlist, int d,
+                                                           int metric, float* __restrict__ scores) {
+    extern __shared__ __align__(16) float qs[];  // [nq][d]
+    for (int i = threadIdx.x; i < nq * d; i += blockDim.x) qs[i] = BF16 ? round_bf16(Q[i]) : Q[i];
+    __syncthreads();
+    const int lane = threadIdx.x & 31;
+    const int warps = (gridDim.x * blockDim.x) >> 5;
+    for (int c = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; c < nlist; c += warps) {
+        float acc[CS_MAXQ];
+#pragma unroll
+        for (int qi = 0; qi < CS_MAXQ; ++qi) acc[qi] = 0.f;
+        for (int j0 = lane * 4; j0 < d; j0 += 128) {
+            float4 cv;
+            if (BF16) {
+                const uint2 raw = *reinterpret_cast<const uint2*>(static_cast<const __nv_bfloat16*>(C) + (size_t)c * d + j0);
+                cv.x = __uint_as_float(raw.x << 16); cv.y = __uint_as_float(raw.x & 0xFFFF0000u);
+                cv.z = __uint_as_float(raw.y << 16); cv.w = __uint_as_float(raw.y & 0xFFFF0000u);
+            } else {
+                cv = *reinterpret_cast<const float4*>(static_cast<const float*>(C) + (size_t)c * d + j0);
+            }
+#pragma unroll
+            for (int qi = 0; qi < CS_MAXQ; ++qi) {
+                if (qi < nq) {  // uniform
+                    const float4 qv = *reinterpret_cast<const float4*>(qs + qi * d + j0);
+                    acc[qi] = fmaf(qv.x, cv.x, fmaf(qv.y, cv.y, fmaf(qv.z, cv.z, fmaf(qv.w, cv.w, acc[qi]))));
+                }
+            }
+        }
+#pragma unroll
+        for (int qi = 0; qi < CS_MAXQ; ++qi) {
+            if (qi < nq) {
+                float v = acc[qi];
+                for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                if (lane == 0) scores[(size_t)qi * nlist + c] = metric == RAGO_L2 ? fmaf(-2.f, v, cnorm[c]) : -v;
+            }
+        }
+    }
+}
+
 cudaError_t launch_coarse_scores(const IndexImpl* ix, const float* queries, int nq, float* scores, cudaStream_t s) {
+    const size_t qbytes = (size_t)nq * ix->d * 4;
+    if (nq <= CS_MAXQ && qbytes <= 48 * 1024) {
+        const int want = (ix->nlist + 7) / 8;
+        const int blocks = want < ix->num_sms * 8 ? want : ix->num_sms * 8;
+        if (ix->coarse_bf16)
+            coarse_small_kernel<true><<<blocks, 256, qbytes, s>>>(queries, ix->centroids, ix->cnorm, nq, ix->nlist, ix->d,
+                                                                   ix->metric, scores);
+        else
+            coarse_small_kernel<false><<<blocks, 256, qbytes, s>>>(queries, ix->centroids, ix->cnorm, nq, ix->nlist, ix->d,
+                                                                    ix->metric, scores);
+        count_launch();
+        return cudaGetLastError();
+    }
     dim3 grid((ix->nlist + BN - 1) / BN, (nq + BM - 1) / BM);
     if (ix->coarse_bf16)
         coarse_scores_kernel<true><<<grid, 256, 0, s>>>(queries, ix->centroids, ix->cnorm, nq, ix->nlist, ix->d,
@@ -113,11 +172,16 @@ cudaError_t launch_coarse_scores(const IndexImpl* ix, const float* queries, int 
 }
 
 // ---- per-query selection of the nprobe best lists ----------------------------------------------
-constexpr int SEL_THREADS = 256;
+constexpr int SEL_MAX_SPLIT = 512;  // candidate lists per query the kernel can index (one per column range of the GEMM)
 
 // Candidates come either from a score row (scores != null: all nlist lists) or from the candidate
 // lists the tensor-core kernel left behind (cand[q][split][cap] keys with counts cand_cnt[q][split]).
-template <bool BF16>
+// First a cut value is found by bisection on the ordered score bits (CTA-wide counts, items held in
+// registers when they fit, re-read from memory otherwise) such that between nsel and nsel + slack items
+// lie at or below it; only those go to shared memory, are sorted, re-scored exactly and sorted again.
+// SEL_THREADS threads per query keep up to SEL_REG item scores each in registers: a big CTA for tiny
+// batches (latency), a small one when there are enough queries to fill the GPU.
+template <bool BF16, int SEL_THREADS, int SEL_REG>
 __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
     const float* __restrict__ Q, const void* __restrict__ C, const float* __restrict__ scores,
     const unsigned long long* __restrict__ cand, const int32_t* __restrict__ cand_cnt, int nsplit, int cap, int nlist,
@@ -125,42 +189,116 @@ __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
     float* __restrict__ probe_bias) {
     __shared__ unsigned long long keys[TOPK_CAP];
     __shared__ unsigned long long keys2[MAX_K + PROBE_GUARD];
+    __shared__ uint32_t red[2][SEL_THREADS / 32];
+    __shared__ int pre[SEL_MAX_SPLIT + 1];  // candidate path: exclusive prefix of the lists' counts
     __shared__ int cnt;
     const int q = blockIdx.x, tid = threadIdx.x;
+    const int warp = tid >> 5, lane = tid & 31;
     auto sync = [] { __syncthreads(); };
     int nsel = nprobe + PROBE_GUARD;
     if (nsel > nlist) nsel = nlist;
     if (tid == 0) cnt = 0;
-    __syncthreads();
-    unsigned long long tau = KEY_MAX;
-    int ub = 0;  // upper bound of cnt, identical in every thread
     const float* srow = scores ? scores + (size_t)q * nlist : nullptr;
-    const int nitems = scores ? nlist : nsplit * cap;
-    for (int l0 = 0; l0 < nitems; l0 += SEL_THREADS) {
-        const int l = l0 + tid;
-        unsigned long long key = KEY_MAX;
-        if (l < nitems) {
-            if (scores) {
-                key = make_key(srow[l], (uint32_t)l);
-            } else {
-                const int sp = l / cap, i = l - sp * cap;
-                if (i < cand_cnt[(size_t)q * nsplit + sp]) key = cand[((size_t)q * nsplit + sp) * cap + i];
+    if (!scores) {  // the valid entries of the query's lists, numbered consecutively
+        if (tid == 0) {
+            int acc = 0;
+            for (int sp = 0; sp < nsplit; ++sp) { pre[sp] = acc; acc += cand_cnt[(size_t)q * nsplit + sp]; }
+            pre[nsplit] = acc;
+        }
+        __syncthreads();
+    }
+    const int nitems = scores ? nlist : pre[nsplit];
+    // key of item l
+    auto item = [&](int l) -> unsigned long long {
+        if (scores) return make_key(srow[l], (uint32_t)l);
+        int lo_s = 0, hi_s = nsplit;  // pre[lo_s] <= l < pre[hi_s]
+        while (hi_s - lo_s > 1) {
+            const int mid_s = (lo_s + hi_s) >> 1;
+            if (pre[mid_s] <= l) lo_s = mid_s; else hi_s = mid_s;
+        }
+        return cand[((size_t)q * nsplit + lo_s) * cap + (l - pre[lo_s])];
+    };
+    const bool in_regs = nitems <= SEL_REG * SEL_THREADS;
+    uint32_t mine[SEL_REG];  // ordered score bits; 0xFFFFFFFF marks an empty slot
+    uint32_t mn = 0xFFFFFFFFu, mx = 0u, nvalid = 0;
+    if (in_regs) {
+#pragma unroll
+        for (int j = 0; j < SEL_REG; ++j) {
+            const int l = tid + j * SEL_THREADS;
+            const unsigned long long k = l < nitems ? item(l) : KEY_MAX;
+            mine[j] = k == KEY_MAX ? 0xFFFFFFFFu : (uint32_t)(k >> 32);
+            if (k != KEY_MAX) {
+                mn = mine[j] < mn ? mine[j] : mn; mx = mine[j] > mx ? mine[j] : mx; ++nvalid;
             }
         }
-        warp_push(keys, &cnt, key < tau, key);
-        ub += SEL_THREADS;
-        if (ub + SEL_THREADS > TOPK_CAP) {
-            __syncthreads();
-            const int kept = block_select(keys, &cnt, nsel, tid, SEL_THREADS, sync);
-            if (kept == nsel) tau = keys[nsel - 1];
-            ub = kept;
-            __syncthreads();
+    } else {
+        for (int l = tid; l < nitems; l += SEL_THREADS) {
+            const unsigned long long k = item(l);
+            if (k != KEY_MAX) {
+                const uint32_t o = (uint32_t)(k >> 32);
+                mn = o < mn ? o : mn; mx = o > mx ? o : mx; ++nvalid;
+            }
+        }
+    }
+    // CTA-wide minimum, maximum and count
+    mn = __reduce_min_sync(0xffffffffu, mn);
+    mx = __reduce_max_sync(0xffffffffu, mx);
+    nvalid = __reduce_add_sync(0xffffffffu, nvalid);
+    if (lane == 0) { red[0][warp] = mn; red[1][warp] = mx; }
+    __syncthreads();
+    mn = red[0][0]; mx = red[1][0];
+    for (int w = 1; w < SEL_THREADS / 32; ++w) { mn = red[0][w] < mn ? red[0][w] : mn; mx = red[1][w] > mx ? red[1][w] : mx; }
+    __syncthreads();
+    if (lane == 0) red[0][warp] = nvalid;
+    __syncthreads();
+    nvalid = 0;
+    for (int w = 0; w < SEL_THREADS / 32; ++w) nvalid += red[0][w];
+    __syncthreads();
+    if ((int)nvalid < nsel) nsel = (int)nvalid;  // cannot happen for a well-formed candidate set; stay safe
+    // bisection: #(score <= lo) < nsel <= #(score <= hi)
+    long long lo = (long long)mn - 1, hi = mx;
+    uint32_t c_hi = nvalid;
+    int slack = nsel / 4 > 8 ? nsel / 4 : 8;
+    if (nsel + slack > TOPK_CAP) slack = TOPK_CAP - nsel;
+    int round = 0;
+    while (hi - lo > 1 && c_hi > (uint32_t)(nsel + slack)) {  // uniform
+        const uint32_t mid = (uint32_t)(lo + (hi - lo) / 2);
+        uint32_t c = 0;
+        if (in_regs) {
+#pragma unroll
+            for (int j = 0; j < SEL_REG; ++j) c += mine[j] <= mid ? 1u : 0u;  // mid <= mx < the empty-slot pattern
+        } else {
+            for (int l = tid; l < nitems; l += SEL_THREADS) {
+                const unsigned long long k = item(l);
+                c += (k != KEY_MAX && (uint32_t)(k >> 32) <= mid) ? 1u : 0u;
+            }
+        }
+        c = __reduce_add_sync(0xffffffffu, c);
+        if (lane == 0) red[round & 1][warp] = c;
+        __syncthreads();
+        c = 0;
+        for (int w = 0; w < SEL_THREADS / 32; ++w) c += red[round & 1][w];
+        if (c < (uint32_t)nsel) lo = mid; else { hi = mid; c_hi = c; }
+        ++round;
+    }
+    const uint32_t T = (uint32_t)hi;
+    // collect the items at or below the cut (a tie group larger than the buffer is cut arbitrarily)
+    if (in_regs) {
+#pragma unroll
+        for (int j = 0; j < SEL_REG; ++j) {
+            const bool take = mine[j] != 0xFFFFFFFFu && mine[j] <= T;
+            warp_push(keys, &cnt, take, take ? item(tid + j * SEL_THREADS) : KEY_MAX);
+        }
+    } else {
+        for (int l0 = 0; l0 < nitems; l0 += SEL_THREADS) {
+            const int l = l0 + tid;
+            const unsigned long long k = l < nitems ? item(l) : KEY_MAX;
+            warp_push(keys, &cnt, k != KEY_MAX && (uint32_t)(k >> 32) <= T, k);
         }
     }
     __syncthreads();
-    const int kept = block_select(keys, &cnt, nsel, tid, SEL_THREADS, sync);  // kept == nsel (nsel <= nlist)
+    const int kept = block_select(keys, &cnt, nsel, tid, SEL_THREADS, sync);
     // exact re-score of the survivors, one warp per candidate
-    const int warp = tid >> 5, lane = tid & 31;
     const float* qrow = Q + (size_t)q * d;
     for (int i = warp; i < kept; i += SEL_THREADS / 32) {
         const uint32_t l = (uint32_t)(keys[i] & 0xFFFFFFFFull);
@@ -208,18 +346,30 @@ __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
     }
 }
 
+template <int THREADS, int REG>
+static void launch_select_shape(const IndexImpl* ix, const float* queries, const float* scores,
+                                const unsigned long long* cand, const int32_t* cand_cnt, int nsplit, int cap, int nq,
+                                int nprobe, int32_t* probe_list, float* probe_term, float* probe_bias, cudaStream_t s) {
+    if (ix->coarse_bf16)
+        select_probes_kernel<true, THREADS, REG><<<nq, THREADS, 0, s>>>(queries, ix->centroids, scores, cand, cand_cnt,
+                                                                         nsplit, cap, ix->nlist, ix->d, ix->metric, nprobe,
+                                                                         probe_list, probe_term, probe_bias);
+    else
+        select_probes_kernel<false, THREADS, REG><<<nq, THREADS, 0, s>>>(queries, ix->centroids, scores, cand, cand_cnt,
+                                                                          nsplit, cap, ix->nlist, ix->d, ix->metric, nprobe,
+                                                                          probe_list, probe_term, probe_bias);
+}
 static cudaError_t launch_select_any(const IndexImpl* ix, const float* queries, const float* scores,
                                      const unsigned long long* cand, const int32_t* cand_cnt, int nsplit, int cap, int nq,
                                      int nprobe, int32_t* probe_list, float* probe_term, float* probe_bias,
                                      cudaStream_t s) {
-    if (ix->coarse_bf16)
-        select_probes_kernel<true><<<nq, SEL_THREADS, 0, s>>>(queries, ix->centroids, scores, cand, cand_cnt, nsplit, cap,
-                                                              ix->nlist, ix->d, ix->metric, nprobe, probe_list,
-                                                              probe_term, probe_bias);
+    if (nsplit > SEL_MAX_SPLIT) return cudaErrorInvalidValue;
+    if (nq <= 64)
+        launch_select_shape<1024, 16>(ix, queries, scores, cand, cand_cnt, nsplit, cap, nq, nprobe, probe_list, probe_term,
+                                      probe_bias, s);
     else
-        select_probes_kernel<false><<<nq, SEL_THREADS, 0, s>>>(queries, ix->centroids, scores, cand, cand_cnt, nsplit,
-                                                               cap, ix->nlist, ix->d, ix->metric, nprobe, probe_list,
-                                                               probe_term, probe_bias);
+        launch_select_shape<256, 20>(ix, queries, scores, cand, cand_cnt, nsplit, cap, nq, nprobe, probe_list, probe_term,
+                                     probe_bias, s);
     count_launch();
     return cudaGetLastError();
 }

@@ -30,21 +30,26 @@ __global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(
     if (u1 > u0) {
         const long long s0 = (long long)q + cta_of_unit(u0, W, ctas);
         const long long s1 = (long long)q + cta_of_unit(u1 - 1, W, ctas);
-        for (long long s = s0; s <= s1; ++s) {
-            const int c = slot_cnt[s];  // <= k
-            if (c == 0) continue;       // uniform: every thread reads the same word
-            if (cnt + c > TOPK_CAP) {
+        // all slots of the query side by side: entry e = (slot, i); empty entries are skipped
+        const long long total = (s1 - s0 + 1) * (long long)k;
+        int ub = 0;  // upper bound of cnt, identical in every thread
+        for (long long e0 = 0; e0 < total; e0 += MERGE_THREADS) {
+            const long long e = e0 + tid;
+            unsigned long long key = KEY_MAX;
+            if (e < total) {
+                const long long s = s0 + e / k;
+                const int i = (int)(e % k);
+                if (i < slot_cnt[s]) key = slot_keys[(size_t)s * k + i];
+            }
+            warp_push(keys, &cnt, key < tau, key);
+            ub += MERGE_THREADS;
+            if (ub + MERGE_THREADS > TOPK_CAP) {
+                __syncthreads();
                 const int kept = block_select(keys, &cnt, k, tid, MERGE_THREADS, sync);
                 if (kept == k) tau = keys[k - 1];
+                ub = kept;
                 __syncthreads();
             }
-            for (int i0 = 0; i0 < c; i0 += MERGE_THREADS) {
-                const int i = i0 + tid;
-                unsigned long long key = KEY_MAX;
-                if (i < c) key = slot_keys[(size_t)s * k + i];
-                warp_push(keys, &cnt, i < c && key < tau, key);
-            }
-            __syncthreads();
         }
     }
     __syncthreads();
