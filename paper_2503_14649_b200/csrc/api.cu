@@ -372,16 +372,14 @@ rago_status rago_search(const rago_index* index, const float* queries, int32_t n
     unsigned long long* slot_keys = reinterpret_cast<unsigned long long*>(ws + L.slot_keys);
 
     e = launch_plan_work(ix, probe_list, npairs, ix->plan.tile_vecs, reinterpret_cast<int32_t*>(ws + L.pair_tiles),
-                         work_prefix, s);
-    if (e == cudaSuccess) e = launch_fill_u64(qthresh, (size_t)nq, KEY_MAX, s);
-    if (e == cudaSuccess) e = cudaMemsetAsync(slot_cnt, 0, L.nslots * 4, s);
+                         work_prefix, qthresh, nq, slot_cnt, (int)L.nslots, s);
     if (e != cudaSuccess) return cuda_fail(e, "work planning");
     record(mix, 3, s);
     e = launch_scan(ix, ix->plan, queries, probe_list, probe_term, work_prefix, nq, nprobe, k, qthresh, slot_cnt,
                     slot_keys, reinterpret_cast<uint32_t*>(ws + L.err), s);
     if (e != cudaSuccess) return cuda_fail(e, "scan kernel");
     record(mix, 4, s);
-    e = launch_merge(ix, work_prefix, nq, nprobe, k, ix->plan.ctas, slot_cnt, slot_keys, out_ids, out_dists, s);
+    e = launch_merge(ix, work_prefix, nq, nprobe, k, ix->plan.ctas, slot_cnt, slot_keys, qthresh, out_ids, out_dists, s);
     if (e != cudaSuccess) return cuda_fail(e, "merge kernel");
     record(mix, 5, s);
     return RAGO_OK;

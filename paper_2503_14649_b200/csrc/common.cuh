@@ -204,15 +204,16 @@ cudaError_t scan_plan(const IndexImpl* ix, ScanPlan* plan);
 cudaError_t launch_vector_terms(const IndexImpl* ix, float* vterm, cudaStream_t s);
 cudaError_t launch_transpose_codebook(const float* cb, int M, int dsub, float* cbT, cudaStream_t s);
 cudaError_t launch_plan_work(const IndexImpl* ix, const int32_t* probe_list, int npairs, int tile_vecs,
-                             int32_t* pair_tiles, int64_t* work_prefix, cudaStream_t s);
+                             int32_t* pair_tiles, int64_t* work_prefix, unsigned long long* qthresh, int nq,
+                             int32_t* slot_cnt, int nslots, cudaStream_t s);
 cudaError_t launch_scan(const IndexImpl* ix, const ScanPlan& plan, const float* queries, const int32_t* probe_list,
                         const float* probe_term, const int64_t* work_prefix, int nq, int nprobe, int k,
                         unsigned long long* qthresh, int32_t* slot_cnt, unsigned long long* slot_keys,
                         uint32_t* err_word, cudaStream_t s);
 // merge.cu
 cudaError_t launch_merge(const IndexImpl* ix, const int64_t* work_prefix, int nq, int nprobe, int k, int ctas,
-                         const int32_t* slot_cnt, const unsigned long long* slot_keys, int64_t* out_ids,
-                         float* out_dists, cudaStream_t s);
+                         const int32_t* slot_cnt, const unsigned long long* slot_keys, const unsigned long long* qthresh,
+                         int64_t* out_ids, float* out_dists, cudaStream_t s);
 cudaError_t launch_fill_u64(unsigned long long* p, size_t n, unsigned long long v, cudaStream_t s);
 // flat.cu
 size_t flat_workspace_bytes(int64_t N, int d, int nq, int k);

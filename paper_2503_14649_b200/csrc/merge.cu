@@ -17,6 +17,7 @@ __device__ __forceinline__ long long cta_of_unit(long long u, long long W, int c
 __global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(
     const int64_t* __restrict__ work_prefix, const int64_t* __restrict__ ids, int npairs, int nprobe, int k, int ctas,
     int metric, const int32_t* __restrict__ slot_cnt, const unsigned long long* __restrict__ slot_keys,
+    const unsigned long long* __restrict__ qthresh,
     int64_t* __restrict__ out_ids, float* __restrict__ out_dists) {
     __shared__ unsigned long long keys[TOPK_CAP];
     __shared__ int cnt;
@@ -26,13 +27,14 @@ __global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(
     __syncthreads();
     const long long W = work_prefix[npairs];
     const long long u0 = work_prefix[(size_t)q * nprobe], u1 = work_prefix[(size_t)(q + 1) * nprobe];
-    unsigned long long tau = KEY_MAX;
+    // a key above the threshold the scan CTAs agreed on is not among the k best (it is some CTA's k-th key)
+    unsigned long long tau = qthresh[q];
+    if (tau != KEY_MAX) ++tau;  // the threshold key itself is a result
     if (u1 > u0) {
         const long long s0 = (long long)q + cta_of_unit(u0, W, ctas);
         const long long s1 = (long long)q + cta_of_unit(u1 - 1, W, ctas);
         // all slots of the query side by side: entry e = (slot, i); empty entries are skipped
         const long long total = (s1 - s0 + 1) * (long long)k;
-        int ub = 0;  // upper bound of cnt, identical in every thread
         for (long long e0 = 0; e0 < total; e0 += MERGE_THREADS) {
             const long long e = e0 + tid;
             unsigned long long key = KEY_MAX;
@@ -42,14 +44,12 @@ __global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(
                 if (i < slot_cnt[s]) key = slot_keys[(size_t)s * k + i];
             }
             warp_push(keys, &cnt, key < tau, key);
-            ub += MERGE_THREADS;
-            if (ub + MERGE_THREADS > TOPK_CAP) {
-                __syncthreads();
+            __syncthreads();
+            if (cnt + MERGE_THREADS > TOPK_CAP) {  // uniform: cnt is stable between the barriers
                 const int kept = block_select(keys, &cnt, k, tid, MERGE_THREADS, sync);
                 if (kept == k) tau = keys[k - 1];
-                ub = kept;
-                __syncthreads();
             }
+            __syncthreads();
         }
     }
     __syncthreads();
@@ -69,10 +69,10 @@ __global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(
 }
 
 cudaError_t launch_merge(const IndexImpl* ix, const int64_t* work_prefix, int nq, int nprobe, int k, int ctas,
-                         const int32_t* slot_cnt, const unsigned long long* slot_keys, int64_t* out_ids,
-                         float* out_dists, cudaStream_t s) {
+                         const int32_t* slot_cnt, const unsigned long long* slot_keys, const unsigned long long* qthresh,
+                         int64_t* out_ids, float* out_dists, cudaStream_t s) {
     merge_kernel<<<nq, MERGE_THREADS, 0, s>>>(work_prefix, ix->ids, nq * nprobe, nprobe, k, ctas, ix->metric,
-                                              slot_cnt, slot_keys, out_ids, out_dists);
+                                              slot_cnt, slot_keys, qthresh, out_ids, out_dists);
     count_launch();
     return cudaGetLastError();
 }

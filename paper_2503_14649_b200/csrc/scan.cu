@@ -750,13 +750,60 @@ __global__ void __launch_bounds__(PFX_THREADS) prefix_kernel(const int32_t* __re
     if (tid == 0) prefix[npairs] = carry_s;
 }
 
+// Small batches: one CTA does the whole preparation of a search (tiles per pair, their prefix sum,
+// threshold and slot-counter reset), which would otherwise be four launches of a few microseconds each.
+__global__ void __launch_bounds__(PFX_THREADS) plan_small_kernel(const int32_t* __restrict__ probe_list,
+                                                                 const int64_t* __restrict__ offsets, int npairs,
+                                                                 int tile_vecs, int64_t* __restrict__ prefix,
+                                                                 unsigned long long* __restrict__ qthresh, int nq,
+                                                                 int32_t* __restrict__ slot_cnt, int nslots) {
+    __shared__ long long warp_sums[32];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    long long v = 0;
+    if (tid < npairs) {
+        const int l = probe_list[tid];
+        v = (offsets[l + 1] - offsets[l] + tile_vecs - 1) / tile_vecs;
+    }
+    long long incl = v;
+    for (int o = 1; o < 32; o <<= 1) {
+        const long long y = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += y;
+    }
+    if (lane == 31) warp_sums[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        long long w = warp_sums[lane];
+        for (int o = 1; o < 32; o <<= 1) {
+            const long long y = __shfl_up_sync(0xffffffffu, w, o);
+            if (lane >= o) w += y;
+        }
+        warp_sums[lane] = w;
+    }
+    __syncthreads();
+    const long long before = (warp ? warp_sums[warp - 1] : 0) + incl - v;
+    if (tid < npairs) prefix[tid] = before;
+    if (tid == npairs - 1) prefix[npairs] = before + v;
+    for (int i = tid; i < nq; i += PFX_THREADS) qthresh[i] = KEY_MAX;
+    for (int i = tid; i < nslots; i += PFX_THREADS) slot_cnt[i] = 0;
+}
+
 cudaError_t launch_plan_work(const IndexImpl* ix, const int32_t* probe_list, int npairs, int tile_vecs,
-                             int32_t* pair_tiles, int64_t* work_prefix, cudaStream_t s) {
+                             int32_t* pair_tiles, int64_t* work_prefix, unsigned long long* qthresh, int nq,
+                             int32_t* slot_cnt, int nslots, cudaStream_t s) {
+    if (npairs <= PFX_THREADS) {
+        plan_small_kernel<<<1, PFX_THREADS, 0, s>>>(probe_list, ix->list_offsets, npairs, tile_vecs, work_prefix, qthresh,
+                                                    nq, slot_cnt, nslots);
+        count_launch();
+        return cudaGetLastError();
+    }
     pair_tiles_kernel<<<(npairs + 255) / 256, 256, 0, s>>>(probe_list, ix->list_offsets, npairs, tile_vecs,
                                                           pair_tiles);
     prefix_kernel<<<1, PFX_THREADS, 0, s>>>(pair_tiles, npairs, work_prefix);
     count_launch(2);
-    return cudaGetLastError();
+    cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess) e = launch_fill_u64(qthresh, (size_t)nq, KEY_MAX, s);
+    if (e == cudaSuccess) e = cudaMemsetAsync(slot_cnt, 0, (size_t)nslots * 4, s);
+    return e;
 }
 
 }  // namespace rago
