@@ -89,6 +89,29 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def rank_batch_permutation(nq: int, rank: int) -> torch.Tensor:
+    """Which of the workload's queries, in which order, rank `rank` searches: a seeded permutation, so every
+    replica works on its own batch and any rank's batch can be rebuilt elsewhere (CPU generator: the same on
+    every device)."""
+    g = torch.Generator(device="cpu")
+    g.manual_seed(1000 + rank)
+    return torch.randperm(nq, generator=g)
+
+
+def max_over_ranks(value_ms: float, world: int, device) -> float:
+    """The slowest rank's time (the job is as slow as its slowest replica); a no-op for one rank."""
+    if world <= 1:
+        return float(value_ms)
+    t = torch.tensor([value_ms], device=device, dtype=torch.float64)
+    torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_qps(nq_per_rank: int, world: int, steps: int, total_ms: float) -> float:
+    """Queries per second of all replicas together (weak scaling: every rank searches nq_per_rank per step)."""
+    return nq_per_rank * world * steps / (total_ms / 1e3)
+
+
 def _dist_env():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -166,12 +189,9 @@ def run_ours(args):
     nq, nprobe, k = cfg["nq"], cfg["nprobe"], cfg["k"]
     data = synth.make_config(WORKLOAD, device=dev, scale=args.scale)
     if world > 1:  # every rank searches its own batch against its replica
-        g = torch.Generator(device=dev)
-        g.manual_seed(1000 + rank)
-        comp = data.extra["query_component"].to(dev)
-        perm = torch.randperm(nq, generator=g, device=dev)
-        data.queries = data.queries[perm].contiguous()
-        data.extra["query_component"] = comp[perm].cpu()
+        perm = rank_batch_permutation(nq, rank)
+        data.queries = data.queries[perm.to(dev)].contiguous()
+        data.extra["query_component"] = data.extra["query_component"][perm]
     ix = binding.rago_index_load(data.centroids, data.codebooks, data.codes, data.list_offsets.to(dev), data.ids,
                                  data.metric)
     q = data.queries.contiguous()
@@ -226,11 +246,8 @@ def run_ours(args):
     ix.rago_profile_enable(False)
     scan_ms = float(np.mean([s["table_scan"] for s in stage_ms]))
 
-    if world > 1:
-        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        total_ms = float(t.item())
-    qps = nq * world * args.steps / (total_ms / 1e3)
+    total_ms = max_over_ranks(total_ms, world, dev)
+    qps = whole_job_qps(nq, world, args.steps, total_ms)
 
     # end to end through the host-buffer entry point: pinned queries in, pinned results out
     hq = q.cpu().pin_memory()
@@ -247,11 +264,8 @@ def run_ours(args):
     e1.record()
     barrier()
     e2e_ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e_qps = nq * world * args.steps / (e2e_ms / 1e3)
+    e2e_ms = max_over_ranks(e2e_ms, world, dev)
+    e2e_qps = whole_job_qps(nq, world, args.steps, e2e_ms)
     assert torch.equal(hids, out_ids.cpu()), "host-buffer path disagrees with the device path"
 
     if rank != 0:
