@@ -714,40 +714,40 @@ __global__ void pair_tiles_kernel(const int32_t* __restrict__ probe_list, const 
 }
 
 constexpr int PFX_THREADS = 1024;
+// Exclusive prefix sum of the tiles per pair by one CTA: every thread owns a contiguous run of pairs
+// (summed, scanned across the CTA, then written out), so the cost is two passes over the pairs instead
+// of one CTA-wide scan per 1024 pairs.
 __global__ void __launch_bounds__(PFX_THREADS) prefix_kernel(const int32_t* __restrict__ tiles, int npairs,
                                                              int64_t* __restrict__ prefix) {
     __shared__ long long warp_sums[32];
-    __shared__ long long carry_s;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    if (tid == 0) carry_s = 0;
-    __syncthreads();
-    for (int base = 0; base < npairs; base += PFX_THREADS) {
-        const int i = base + tid;
-        const long long v = i < npairs ? tiles[i] : 0;
-        long long incl = v;
-        for (int o = 1; o < 32; o <<= 1) {
-            const long long y = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += y;
-        }
-        if (lane == 31) warp_sums[warp] = incl;
-        __syncthreads();
-        if (warp == 0) {
-            long long w = warp_sums[lane];
-            for (int o = 1; o < 32; o <<= 1) {
-                const long long y = __shfl_up_sync(0xffffffffu, w, o);
-                if (lane >= o) w += y;
-            }
-            warp_sums[lane] = w;  // inclusive over warps
-        }
-        __syncthreads();
-        const long long carry = carry_s;
-        const long long before = carry + (warp ? warp_sums[warp - 1] : 0) + incl - v;
-        if (i < npairs) prefix[i] = before;
-        __syncthreads();
-        if (tid == PFX_THREADS - 1) carry_s = before + v;
-        __syncthreads();
+    const int per = (npairs + PFX_THREADS - 1) / PFX_THREADS;
+    const int i0 = tid * per;
+    const int i1 = i0 + per < npairs ? i0 + per : npairs;
+    long long v = 0;
+    for (int i = i0; i < i1; ++i) v += tiles[i];
+    long long incl = v;
+    for (int o = 1; o < 32; o <<= 1) {
+        const long long y = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += y;
     }
-    if (tid == 0) prefix[npairs] = carry_s;
+    if (lane == 31) warp_sums[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        long long w = warp_sums[lane];
+        for (int o = 1; o < 32; o <<= 1) {
+            const long long y = __shfl_up_sync(0xffffffffu, w, o);
+            if (lane >= o) w += y;
+        }
+        warp_sums[lane] = w;  // inclusive over warps
+    }
+    __syncthreads();
+    long long run = (warp ? warp_sums[warp - 1] : 0) + incl - v;
+    for (int i = i0; i < i1; ++i) {
+        prefix[i] = run;
+        run += tiles[i];
+    }
+    if (tid == PFX_THREADS - 1) prefix[npairs] = warp_sums[31];
 }
 
 // Small batches: one CTA does the whole preparation of a search (tiles per pair, their prefix sum,
