@@ -704,28 +704,20 @@ cudaError_t launch_vector_terms(const IndexImpl* ix, float* vterm, cudaStream_t 
 }
 
 // ---- work planning: tiles per pair and their exclusive prefix sum ------------------------------
-__global__ void pair_tiles_kernel(const int32_t* __restrict__ probe_list, const int64_t* __restrict__ offsets,
-                                  int npairs, int tile_vecs, int32_t* __restrict__ tiles) {
-    const int p = blockIdx.x * blockDim.x + threadIdx.x;
-    if (p >= npairs) return;
-    const int l = probe_list[p];
-    const long long len = offsets[l + 1] - offsets[l];
-    tiles[p] = (int32_t)((len + tile_vecs - 1) / tile_vecs);
-}
-
-constexpr int PFX_THREADS = 1024;
-// Exclusive prefix sum of the tiles per pair by one CTA: every thread owns a contiguous run of pairs
-// (summed, scanned across the CTA, then written out), so the cost is two passes over the pairs instead
-// of one CTA-wide scan per 1024 pairs.
-__global__ void __launch_bounds__(PFX_THREADS) prefix_kernel(const int32_t* __restrict__ tiles, int npairs,
-                                                             int64_t* __restrict__ prefix) {
-    __shared__ long long warp_sums[32];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int per = (npairs + PFX_THREADS - 1) / PFX_THREADS;
-    const int i0 = tid * per;
-    const int i1 = i0 + per < npairs ? i0 + per : npairs;
+// Three small launches: (1) tiles per pair with a CTA-local exclusive scan and one total per CTA,
+// (2) one CTA scans the totals, (3) every CTA adds its offset.
+constexpr int PT_THREADS = 256;
+__global__ void __launch_bounds__(PT_THREADS) pair_tiles_kernel(const int32_t* __restrict__ probe_list,
+                                                                const int64_t* __restrict__ offsets, int npairs,
+                                                                int tile_vecs, int64_t* __restrict__ prefix,
+                                                                long long* __restrict__ block_sums) {
+    __shared__ long long warp_sums[PT_THREADS / 32];
+    const int p = blockIdx.x * PT_THREADS + threadIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     long long v = 0;
-    for (int i = i0; i < i1; ++i) v += tiles[i];
+    if (p < npairs) {
+        const int l = probe_list[p];
+        v = (offsets[l + 1] - offsets[l] + tile_vecs - 1) / tile_vecs;
+    }
     long long incl = v;
     for (int o = 1; o < 32; o <<= 1) {
         const long long y = __shfl_up_sync(0xffffffffu, incl, o);
@@ -733,21 +725,53 @@ __global__ void __launch_bounds__(PFX_THREADS) prefix_kernel(const int32_t* __re
     }
     if (lane == 31) warp_sums[warp] = incl;
     __syncthreads();
-    if (warp == 0) {
-        long long w = warp_sums[lane];
-        for (int o = 1; o < 32; o <<= 1) {
-            const long long y = __shfl_up_sync(0xffffffffu, w, o);
-            if (lane >= o) w += y;
-        }
-        warp_sums[lane] = w;  // inclusive over warps
-    }
+    long long before = incl - v;
+    for (int w = 0; w < warp; ++w) before += warp_sums[w];
+    if (p < npairs) prefix[p] = before;
+    if (threadIdx.x == PT_THREADS - 1) block_sums[blockIdx.x] = before + v;
+}
+
+constexpr int PFX_THREADS = 1024;
+// In-place exclusive scan of n totals by one CTA; the grand total goes to *total_out.
+__global__ void __launch_bounds__(PFX_THREADS) scan_totals_kernel(long long* __restrict__ sums, int n,
+                                                                  int64_t* __restrict__ total_out) {
+    __shared__ long long warp_sums[32];
+    __shared__ long long carry_s;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) carry_s = 0;
     __syncthreads();
-    long long run = (warp ? warp_sums[warp - 1] : 0) + incl - v;
-    for (int i = i0; i < i1; ++i) {
-        prefix[i] = run;
-        run += tiles[i];
+    for (int base = 0; base < n; base += PFX_THREADS) {
+        const int i = base + tid;
+        const long long v = i < n ? sums[i] : 0;
+        long long incl = v;
+        for (int o = 1; o < 32; o <<= 1) {
+            const long long y = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += y;
+        }
+        if (lane == 31) warp_sums[warp] = incl;
+        __syncthreads();
+        if (warp == 0) {
+            long long w = warp_sums[lane];
+            for (int o = 1; o < 32; o <<= 1) {
+                const long long y = __shfl_up_sync(0xffffffffu, w, o);
+                if (lane >= o) w += y;
+            }
+            warp_sums[lane] = w;  // inclusive over warps
+        }
+        __syncthreads();
+        const long long before = carry_s + (warp ? warp_sums[warp - 1] : 0) + incl - v;
+        if (i < n) sums[i] = before;
+        __syncthreads();
+        if (tid == PFX_THREADS - 1) carry_s = before + v;
+        __syncthreads();
     }
-    if (tid == PFX_THREADS - 1) prefix[npairs] = warp_sums[31];
+    if (tid == 0) *total_out = carry_s;
+}
+
+__global__ void __launch_bounds__(PT_THREADS) add_offsets_kernel(int64_t* __restrict__ prefix, int npairs,
+                                                                 const long long* __restrict__ block_sums) {
+    const int p = blockIdx.x * PT_THREADS + threadIdx.x;
+    if (p < npairs) prefix[p] += block_sums[blockIdx.x];
 }
 
 // Small batches: one CTA does the whole preparation of a search (tiles per pair, their prefix sum,
@@ -796,10 +820,14 @@ cudaError_t launch_plan_work(const IndexImpl* ix, const int32_t* probe_list, int
         count_launch();
         return cudaGetLastError();
     }
-    pair_tiles_kernel<<<(npairs + 255) / 256, 256, 0, s>>>(probe_list, ix->list_offsets, npairs, tile_vecs,
-                                                          pair_tiles);
-    prefix_kernel<<<1, PFX_THREADS, 0, s>>>(pair_tiles, npairs, work_prefix);
-    count_launch(2);
+    // pair_tiles (npairs int32 of scratch) holds the per-CTA totals: one 64-bit word per 256 pairs
+    const int nblocks = (npairs + PT_THREADS - 1) / PT_THREADS;
+    long long* block_sums = reinterpret_cast<long long*>(pair_tiles);
+    pair_tiles_kernel<<<nblocks, PT_THREADS, 0, s>>>(probe_list, ix->list_offsets, npairs, tile_vecs, work_prefix,
+                                                    block_sums);
+    scan_totals_kernel<<<1, PFX_THREADS, 0, s>>>(block_sums, nblocks, work_prefix + npairs);
+    add_offsets_kernel<<<nblocks, PT_THREADS, 0, s>>>(work_prefix, npairs, block_sums);
+    count_launch(3);
     cudaError_t e = cudaGetLastError();
     if (e == cudaSuccess) e = launch_fill_u64(qthresh, (size_t)nq, KEY_MAX, s);
     if (e == cudaSuccess) e = cudaMemsetAsync(slot_cnt, 0, (size_t)nslots * 4, s);
