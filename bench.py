@@ -31,6 +31,7 @@ import numpy as np  # noqa: E402
 import torch  # noqa: E402
 
 WORKLOAD = 2  # index into synth.CONFIGS
+SCAN_DRAM_PER_LOGICAL = 3.639e9 / 11.126e9
 METRIC = "retrieval_qps"
 UNIT = "queries/s"
 
@@ -275,6 +276,10 @@ def run_ours(args):
 
     peak, peak_kind = _peaks()
     achieved = scan_bytes / (scan_ms / 1e3) / 1e9
+    # DRAM bytes of one scan launch: ncu capture at 1/4 of the vectors (profiles/scan_kernel_mid_quarter_scale.md:
+    # 3.639 GB for 11.126 GB of logical code bytes), scaled by this launch's logical bytes.  Valid for the scan
+    # kernel that capture was taken from; set SCAN_DRAM_PER_LOGICAL to None after changing the kernel.
+    traffic = None if SCAN_DRAM_PER_LOGICAL is None else SCAN_DRAM_PER_LOGICAL * scan_bytes
     out = {
         "metric": METRIC, "value": qps, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -284,7 +289,7 @@ def run_ours(args):
                 "d2h_bytes_per_step": nq * k * 12},
         "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "kernel": "scan_kernel (table build + ADC scan)", "achieved": achieved,
-                     "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+                     "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak, "traffic": traffic,
                      "algorithmic_bytes_per_launch": scan_bytes, "kernel_ms": scan_ms,
                      "scanned_vectors_per_query": scanned_vectors / nq},
         "stage_ms": {kk: float(np.mean([s[kk] for s in stage_ms])) for kk in stage_ms[0]},
