@@ -300,6 +300,8 @@ def run_ours(args):
         from tests.helpers import match_results
         threads = oracle.default_threads()
         nsample = min(nq, 4 * threads)
+        dt, oi, od = _oracle_sample(data, cfg, nsample, threads)  # a first, small sample sizes the real one (~15 s)
+        nsample = int(min(nq, max(nsample, (nsample / dt) * 15.0)))
         dt, oi, od = _oracle_sample(data, cfg, nsample, threads)
         gi, gd = out_ids[:nsample].cpu().numpy(), out_d[:nsample].cpu().numpy()
         mism = sum(1 for i in range(nsample) if match_results(gi[i], gd[i], oi[i], od[i], rel=1e-4))
