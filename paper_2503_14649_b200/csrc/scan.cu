@@ -53,7 +53,7 @@ struct TileDesc {
     int32_t list;      // inverted list number
     uint32_t pos0;     // storage position of the tile's first vector
     int32_t nvec;      // vectors in this tile
-    int32_t newpair;   // first tile of this pair inside this CTA
+    int32_t newpair;   // bit 0: first tile of this pair inside this CTA; bit 1: cut the candidate buffer before this tile
     int32_t vrem;      // index of the first vector's term inside the staged term block (0..3)
     uint32_t tile_addr;  // shared address of the stage's code tile
     uint32_t vt_addr;    // shared address of the stage's per-vector terms
@@ -91,14 +91,19 @@ struct Cfg {
     static constexpr int NBANK = (NCOLS + 63) / 64;
     static constexpr int LSTRIDE = NCOLS;               // words per table row (multiply-add addressing)
     static constexpr int LUT_BYTES = BANKED ? NBANK * 65536 : KSUB * LSTRIDE * 4;
-    static constexpr int RGW = MV >= 80 ? 1 : 2;        // 32-row groups per warp per tile
+    static constexpr int RGW = MV >= 48 ? 1 : 2;        // 32-row groups per warp per tile
     static constexpr int TILE_VROWS = NCW * 32 * RGW;
     static constexpr int TV = TILE_VROWS / R;           // vectors per tile
     static constexpr int TILE_BYTES = TILE_VROWS * MV;
     static constexpr int VT_BYTES = (TV + 4) * 4;       // staged per-vector terms (start rounded down to 16 bytes)
+    static constexpr int KCAP = LUT_BYTES <= 65536 ? 2 * TOPK_CAP : TOPK_CAP;  // keys of the CTA's candidate buffer
     static_assert(WV % G == 0, "virtual rows are whole blocks");
     static_assert(TILE_VROWS % R == 0, "tile must hold whole vectors");
-    static_assert(TV + MAX_K <= TOPK_CAP, "one tile of pushes plus k kept keys must fit the candidate buffer");
+    // The producer asks for a cut of the candidate buffer when the count it sees plus everything the tiles in
+    // flight can still push would not fit; SMAX bounds the ring depth so that this leaves room to work in.
+    static constexpr int SMAX = KCAP / TV / 2 < MAX_STAGES ? KCAP / TV / 2 : MAX_STAGES;
+    static_assert(SMAX >= 2, "two tiles in flight must fit the candidate buffer twice over");
+    static_assert(MAX_K + SMAX * TV <= KCAP, "k kept keys plus the pushes of all tiles in flight must fit");
     static_assert(COPY_OFF % 32 == (COPIES == 2 ? 16 : 0), "second copy must sit 16 banks away");
     static_assert(LSTRIDE % 32 == 0 || BANKED, "table rows must keep bank = column mod 32");
     static_assert(VT_BYTES % 16 == 0 && TILE_BYTES % 16 == 0, "bulk-copy destinations are 16-byte granular");
@@ -156,7 +161,7 @@ __host__ __device__ inline SmemPlan plan_smem(uint32_t base, uint32_t dyn_bytes,
         return base;
     };
     p.ctrl = take(CTRL_BYTES, 16);
-    p.keys = take(TOPK_CAP * 8, 16);
+    p.keys = take(C::KCAP * 8, 16);
     p.rT = take((uint32_t)d * 4, 16);
     for (int s = 0; s < MAX_STAGES; ++s) p.vt[s] = s < stages ? take(C::VT_BYTES, 16) : base;
     for (int s = 0; s < MAX_STAGES; ++s) p.tile[s] = s < stages ? take(C::TILE_BYTES, 128) : base;
@@ -393,7 +398,10 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_>::THREADS, 1) scan_kernel(c
                 D.list = list;
                 D.pos0 = pos0;
                 D.nvec = (int32_t)nvec;
-                D.newpair = (n == 0 || t_in_pair == 0) ? 1 : 0;
+                // everything tiles n-S+1 .. n can still push must fit behind what is in the buffer now
+                const int cnt_seen = *reinterpret_cast<volatile int*>(&ctrl->cnt);
+                const int cut = cnt_seen + (S + 1) * C::TV > C::KCAP ? 2 : 0;
+                D.newpair = ((n == 0 || t_in_pair == 0) ? 1 : 0) | cut;
                 D.vrem = (int32_t)(pos0 & 3u);
                 D.tile_addr = P.tile[st];
                 D.vt_addr = P.vt[st];
@@ -458,7 +466,6 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_>::THREADS, 1) scan_kernel(c
     int cur_q = -1;
     unsigned long long tau = KEY_MAX;
     float bias = 0.f;
-    int ub = 0;
     const int k = a.k;
     const bool ip = a.metric == RAGO_IP;
     const float lut_scale = ip ? -1.f : -2.f;
@@ -470,7 +477,7 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_>::THREADS, 1) scan_kernel(c
         if (dead) return;
         int kept = ctrl->cnt;
         if (kept > k) {
-            kept = block_select(keys, &ctrl->cnt, k, ctid, NCT, csync);
+            kept = block_select(keys, &ctrl->cnt, k, ctid, NCT, csync, C::KCAP);
             if (dead) return;
             if (ctid == 0) atomicMin(&a.qthresh[cur_q], keys[k - 1]);
         }
@@ -508,7 +515,6 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_>::THREADS, 1) scan_kernel(c
         quantise_table<C>(P.lut, ctid, ldexpf(1.f, 30 - ex));
         inv_scale = ldexpf(1.f, ex - 30);
         tau = *reinterpret_cast<volatile unsigned long long*>(&a.qthresh[q]);
-        ub = 0;
         csync();
     };
 
@@ -517,7 +523,7 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_>::THREADS, 1) scan_kernel(c
         dead = dead || !mbar_wait(smem_u32(&ctrl->full[st]), (n / S) & 1, abort_flag, a.err);
         if (dead) break;
         const TileDesc D = ctrl->desc[st];
-        if (D.newpair) {
+        if (D.newpair & 1) {
             const int q = D.pair / a.nprobe;
             if (q != cur_q) {
                 if (cur_q >= 0) finalize();
@@ -528,11 +534,11 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_>::THREADS, 1) scan_kernel(c
             const float term = a.probe_term[D.pair];
             bias = ip ? -term : term;
         }
-        if (ub + C::TV > TOPK_CAP) {
+        if (D.newpair & 2) {  // the producer saw the buffer filling up: keep the k best, refresh the threshold
             csync();
             if (dead) break;
-            if (ctrl->cnt + C::TV > TOPK_CAP) {
-                const int kept = block_select(keys, &ctrl->cnt, k, ctid, NCT, csync);
+            if (ctrl->cnt > k) {
+                const int kept = block_select(keys, &ctrl->cnt, k, ctid, NCT, csync, C::KCAP);
                 if (dead) break;
                 if (kept == k) {
                     if (keys[k - 1] < tau) tau = keys[k - 1];
@@ -541,7 +547,6 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_>::THREADS, 1) scan_kernel(c
             }
             const unsigned long long g = *reinterpret_cast<volatile unsigned long long*>(&a.qthresh[cur_q]);
             if (g < tau) tau = g;
-            ub = ctrl->cnt;
             csync();
             if (dead) break;
         }
@@ -569,9 +574,8 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_>::THREADS, 1) scan_kernel(c
             const float vt = a.vterm != nullptr ? lds_f32(vt_base + (uint32_t)(vr / R) * 4u) : 0.f;
             const float score = (bias + vt) + s;  // smaller is better for both metrics
             const unsigned long long key = make_key(score, D.pos0 + (uint32_t)(vr / R));
-            warp_push(keys, &ctrl->cnt, vr < nvr && sr == 0 && key < tau, key);
+            warp_push(keys, &ctrl->cnt, vr < nvr && sr == 0 && key < tau, key, C::KCAP);
         }
-        ub += D.nvec;
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&ctrl->empty[st]));
     }
@@ -587,7 +591,7 @@ struct Variant {
 };
 template <class C>
 static int stages_for(int d) {
-    for (int s = MAX_STAGES; s >= 2; --s)
+    for (int s = C::SMAX; s >= 2; --s)
         if (plan_smem<C>(SMEM_BASE_EXPECTED, SMEM_OPTIN, d, s).ok) return s;
     return 0;
 }

@@ -37,9 +37,9 @@ __device__ __forceinline__ void block_bitonic_sort(unsigned long long* keys, int
 // Returns the new count; ends with a barrier.
 template <class Sync>
 __device__ __forceinline__ int block_select(unsigned long long* keys, int* cnt, int k, int tid, int nthreads,
-                                            Sync sync) {
+                                            Sync sync, int cap = TOPK_CAP) {
     int n = *cnt;
-    if (n > TOPK_CAP) n = TOPK_CAP;
+    if (n > cap) n = cap;
     int n2 = 2;
     while (n2 < n) n2 <<= 1;
     for (int i = n + tid; i < n2; i += nthreads) keys[i] = KEY_MAX;
@@ -52,7 +52,8 @@ __device__ __forceinline__ int block_select(unsigned long long* keys, int* cnt, 
 }
 
 // Append `key` for the lanes with pred set; one shared atomic per warp.  Whole warp must call.
-__device__ __forceinline__ void warp_push(unsigned long long* keys, int* cnt, bool pred, unsigned long long key) {
+__device__ __forceinline__ void warp_push(unsigned long long* keys, int* cnt, bool pred, unsigned long long key,
+                                          int cap = TOPK_CAP) {
     const unsigned mask = __ballot_sync(0xffffffffu, pred);
     if (mask == 0) return;
     const int lane = threadIdx.x & 31;
@@ -62,7 +63,7 @@ __device__ __forceinline__ void warp_push(unsigned long long* keys, int* cnt, bo
     base = __shfl_sync(0xffffffffu, base, leader);
     if (pred) {
         const int idx = base + __popc(mask & ((1u << lane) - 1u));
-        if (idx < TOPK_CAP) keys[idx] = key;
+        if (idx < cap) keys[idx] = key;
     }
 }
 
