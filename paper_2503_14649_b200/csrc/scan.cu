@@ -177,6 +177,7 @@ struct Ctrl {
     int cnt;
     uint32_t abort_flag;
     float red[32];  // per-warp maxima of the table build
+    uint32_t redu[2][32];  // per-warp minima / maxima / counts of the buffer cut
 };
 static_assert(sizeof(Ctrl) <= CTRL_BYTES, "control block too large");
 
@@ -471,6 +472,66 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_>::THREADS, 1) scan_kernel(c
     const float lut_scale = ip ? -1.f : -2.f;
     float inv_scale = 1.f;  // fp32 value of one unit of the current query's integer table
 
+    // Cut the candidate buffer (more than k keys, count stable, called by all consumer threads after a csync):
+    // every thread takes its share of the keys into registers, the CTA bisects on the ordered score bits for a
+    // value T with between k and k + k/4 keys at or below it (one barrier per step instead of the ~66 of a full
+    // sort), and the keys up to T are pushed back.  All keys of the k best are kept; T bounds the k-th best.
+    auto cut_buffer = [&]() {
+        constexpr int KPT = (C::KCAP + NCT - 1) / NCT;
+        const int n = ctrl->cnt < C::KCAP ? ctrl->cnt : C::KCAP;
+        unsigned long long mine[KPT];
+        uint32_t mn = 0xFFFFFFFFu, mx = 0u;
+#pragma unroll
+        for (int j = 0; j < KPT; ++j) {
+            const int i = ctid + j * NCT;
+            mine[j] = i < n ? keys[i] : KEY_MAX;
+            if (i < n) {
+                const uint32_t o = (uint32_t)(mine[j] >> 32);
+                mn = o < mn ? o : mn;
+                mx = o > mx ? o : mx;
+            }
+        }
+        mn = __reduce_min_sync(0xffffffffu, mn);
+        mx = __reduce_max_sync(0xffffffffu, mx);
+        if (lane == 0) { ctrl->redu[0][warp] = mn; ctrl->redu[1][warp] = mx; }
+        csync();
+        if (dead) return;
+        for (int w = 0; w < NCW; ++w) {
+            mn = ctrl->redu[0][w] < mn ? ctrl->redu[0][w] : mn;
+            mx = ctrl->redu[1][w] > mx ? ctrl->redu[1][w] : mx;
+        }
+        csync();  // the minima / maxima have been read; redu is free for the counts
+        if (dead) return;
+        long long lo = (long long)mn - 1, hi = mx;  // #(score <= lo) < k <= #(score <= hi)
+        uint32_t c_hi = (uint32_t)n;
+        const uint32_t want_max = (uint32_t)(k + (k >> 2) + 8);
+        int round = 0;
+        while (hi - lo > 1 && c_hi > want_max) {  // uniform across the CTA
+            const uint32_t mid = (uint32_t)(lo + (hi - lo) / 2);
+            uint32_t c = 0;
+#pragma unroll
+            for (int j = 0; j < KPT; ++j) c += (mine[j] != KEY_MAX && (uint32_t)(mine[j] >> 32) <= mid) ? 1u : 0u;
+            c = __reduce_add_sync(0xffffffffu, c);
+            if (lane == 0) ctrl->redu[round & 1][warp] = c;
+            csync();
+            if (dead) return;
+            c = 0;
+            for (int w = 0; w < NCW; ++w) c += ctrl->redu[round & 1][w];
+            if (c < (uint32_t)k) lo = mid; else { hi = mid; c_hi = c; }
+            ++round;
+        }
+        const uint32_t T = (uint32_t)hi;
+        if (ctid == 0) ctrl->cnt = 0;  // every thread holds its keys in registers since the first barrier above
+        csync();
+        if (dead) return;
+#pragma unroll
+        for (int j = 0; j < KPT; ++j)
+            warp_push(keys, &ctrl->cnt, mine[j] != KEY_MAX && (uint32_t)(mine[j] >> 32) <= T, mine[j], C::KCAP);
+        const unsigned long long bound = ((unsigned long long)T << 32) | 0xFFFFFFFFull;  // >= the k-th best key
+        if (bound < tau) tau = bound;
+        if (ctid == 0) atomicMin(&a.qthresh[cur_q], bound);
+    };
+
     // Close the current query's candidate buffer: keep at most k keys and park them in this CTA's slot.
     auto finalize = [&]() {
         csync();
@@ -534,17 +595,11 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_>::THREADS, 1) scan_kernel(c
             const float term = a.probe_term[D.pair];
             bias = ip ? -term : term;
         }
-        if (D.newpair & 2) {  // the producer saw the buffer filling up: keep the k best, refresh the threshold
+        if (D.newpair & 2) {  // the producer saw the buffer filling up: keep the best k (or a few more), lower the threshold
             csync();
             if (dead) break;
-            if (ctrl->cnt > k) {
-                const int kept = block_select(keys, &ctrl->cnt, k, ctid, NCT, csync, C::KCAP);
-                if (dead) break;
-                if (kept == k) {
-                    if (keys[k - 1] < tau) tau = keys[k - 1];
-                    if (ctid == 0) atomicMin(&a.qthresh[cur_q], keys[k - 1]);
-                }
-            }
+            if (ctrl->cnt > k) cut_buffer();
+            if (dead) break;
             const unsigned long long g = *reinterpret_cast<volatile unsigned long long*>(&a.qthresh[cur_q]);
             if (g < tau) tau = g;
             csync();
