@@ -215,11 +215,11 @@ def run_ours(args):
     def step():
         ix.rago_search(q, nprobe, k, out_ids, out_d, ws)
 
+    sampler = ClockSampler(local)
+    sampler.start()  # before the warm-up, so that nvidia-smi is already reporting when the timed region starts
     for _ in range(max(3, args.warmup)):
         step()
     ix.rago_check(ws)
-    sampler = ClockSampler(local)
-    sampler.start()
     ix.rago_profile_enable(True)
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     stage_ms = []
@@ -535,7 +535,7 @@ def run_iter(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--scale", type=float, default=1.0, help="shrink N (development only; 1.0 = the named workload)")
