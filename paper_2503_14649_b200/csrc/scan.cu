@@ -611,25 +611,34 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_>::THREADS, 1) scan_kernel(c
         const uint32_t tile_base = D.tile_addr;
         const uint32_t vt_base = D.vt_addr + (uint32_t)D.vrem * 4u;
 #pragma unroll 1
-        for (int rg = 0; rg < C::RGW; ++rg) {
+        // Row groups are taken MERGE at a time: with R lanes per vector every lane of an R-group ends up with
+        // the vector's sum, so lane slice g finishes row group g and one epilogue serves MERGE row groups.
+        constexpr int MERGE = R < C::RGW ? R : C::RGW;
+        for (int rg = 0; rg < C::RGW; rg += MERGE) {
             const int vr0 = (warp * C::RGW + rg) * 32;
             if (vr0 >= nvr) break;
-            const int vr = vr0 + lane;
-            const uint32_t rowaddr = tile_base + (uint32_t)vr * C::MV;
-            int acc[4] = {0, 0, 0, 0};
-            uint32_t x[C::NBLK][G];
-            LoadWords<C, G, 0>::run(rowaddr, xo, x);
-            ScanBlocks<C, G, 0>::run(x, cc, sel, lo, P.lut, acc);
-            int si = (acc[0] + acc[1]) + (acc[2] + acc[3]);
-            if (R >= 2) si += __shfl_xor_sync(0xffffffffu, si, 1);
-            if (R >= 4) si += __shfl_xor_sync(0xffffffffu, si, 2);
-            const float s = (float)si * inv_scale;
+            int mine = 0;
+#pragma unroll
+            for (int g = 0; g < MERGE; ++g) {
+                const uint32_t rowaddr = tile_base + (uint32_t)(vr0 + g * 32 + lane) * C::MV;
+                int acc[4] = {0, 0, 0, 0};
+                uint32_t x[C::NBLK][G];
+                LoadWords<C, G, 0>::run(rowaddr, xo, x);
+                ScanBlocks<C, G, 0>::run(x, cc, sel, lo, P.lut, acc);
+                int si = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+                if (R >= 2) si += __shfl_xor_sync(0xffffffffu, si, 1);
+                if (R >= 4) si += __shfl_xor_sync(0xffffffffu, si, 2);
+                if (MERGE == 1 || sr == g) mine = si;
+            }
+            const int vr = vr0 + (MERGE == 1 ? 0 : sr * 32) + lane;  // the virtual row whose vector this lane finishes
+            const float s = (float)mine * inv_scale;
             // per-vector term of the L2 expansion (0 for inner product); rows past the tile's end read
             // stale but in-bounds shared memory and are never pushed
             const float vt = a.vterm != nullptr ? lds_f32(vt_base + (uint32_t)(vr / R) * 4u) : 0.f;
             const float score = (bias + vt) + s;  // smaller is better for both metrics
             const unsigned long long key = make_key(score, D.pos0 + (uint32_t)(vr / R));
-            warp_push(keys, &ctrl->cnt, vr < nvr && sr == 0 && key < tau, key, C::KCAP);
+            const bool owner = MERGE == 1 ? sr == 0 : sr < MERGE;
+            warp_push(keys, &ctrl->cnt, vr < nvr && owner && key < tau, key, C::KCAP);
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&ctrl->empty[st]));
