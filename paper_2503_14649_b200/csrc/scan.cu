@@ -76,7 +76,7 @@ struct ScanArgs {
     uint32_t dyn_bytes;
 };
 
-template <int WV, int G, int R, int NCW_>
+template <int WV, int G, int R, int NCW_, int RGW_>
 struct Cfg {
     static constexpr int NCW = NCW_;                    // consumer warps
     static constexpr int NCT = NCW * 32;                // consumer threads
@@ -91,7 +91,7 @@ struct Cfg {
     static constexpr int NBANK = (NCOLS + 63) / 64;
     static constexpr int LSTRIDE = NCOLS;               // words per table row (multiply-add addressing)
     static constexpr int LUT_BYTES = BANKED ? NBANK * 65536 : KSUB * LSTRIDE * 4;
-    static constexpr int RGW = MV >= 48 ? 1 : 2;        // 32-row groups per warp per tile
+    static constexpr int RGW = RGW_;                    // 32-row groups per warp per tile (unrolled: independent work in flight)
     static constexpr int TILE_VROWS = NCW * 32 * RGW;
     static constexpr int TV = TILE_VROWS / R;           // vectors per tile
     static constexpr int TILE_BYTES = TILE_VROWS * MV;
@@ -309,9 +309,9 @@ struct ScanBlocks {
     }
 };
 
-template <int WV, int G, int R, int NCW_>
-__global__ void __launch_bounds__(Cfg<WV, G, R, NCW_>::THREADS, 1) scan_kernel(const ScanArgs a) {
-    using C = Cfg<WV, G, R, NCW_>;
+template <int WV, int G, int R, int NCW_, int RGW_>
+__global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_kernel(const ScanArgs a) {
+    using C = Cfg<WV, G, R, NCW_, RGW_>;
     constexpr int NCW = C::NCW, NCT = C::NCT;
     extern __shared__ __align__(1024) uint8_t smem[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -610,10 +610,10 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_>::THREADS, 1) scan_kernel(c
         const int nvr = D.nvec * R;
         const uint32_t tile_base = D.tile_addr;
         const uint32_t vt_base = D.vt_addr + (uint32_t)D.vrem * 4u;
-#pragma unroll 1
         // Row groups are taken MERGE at a time: with R lanes per vector every lane of an R-group ends up with
         // the vector's sum, so lane slice g finishes row group g and one epilogue serves MERGE row groups.
         constexpr int MERGE = R < C::RGW ? R : C::RGW;
+#pragma unroll
         for (int rg = 0; rg < C::RGW; rg += MERGE) {
             const int vr0 = (warp * C::RGW + rg) * 32;
             if (vr0 >= nvr) break;
@@ -659,17 +659,17 @@ static int stages_for(int d) {
         if (plan_smem<C>(SMEM_BASE_EXPECTED, SMEM_OPTIN, d, s).ok) return s;
     return 0;
 }
-#define RAGO_VARIANT(WV, G, R, NCW) \
-    { Cfg<WV, G, R, NCW>::M, scan_kernel<WV, G, R, NCW>, Cfg<WV, G, R, NCW>::THREADS, Cfg<WV, G, R, NCW>::TV, \
-      stages_for<Cfg<WV, G, R, NCW>> }
+#define RAGO_VARIANT(WV, G, R, NCW, RGW) \
+    { Cfg<WV, G, R, NCW, RGW>::M, scan_kernel<WV, G, R, NCW, RGW>, Cfg<WV, G, R, NCW, RGW>::THREADS, \
+      Cfg<WV, G, R, NCW, RGW>::TV, stages_for<Cfg<WV, G, R, NCW, RGW>> }
 static const Variant kVariants[] = {
-    RAGO_VARIANT(4, 4, 1, 16),   // M = 16
-    RAGO_VARIANT(8, 8, 1, 16),   // M = 32
-    RAGO_VARIANT(12, 4, 1, 12),  // M = 48
-    RAGO_VARIANT(8, 8, 2, 16),   // M = 64
-    RAGO_VARIANT(20, 4, 1, 8),   // M = 80
-    RAGO_VARIANT(24, 8, 1, 12),  // M = 96
-    RAGO_VARIANT(8, 8, 4, 12),   // M = 128
+    RAGO_VARIANT(4, 4, 1, 16, 2),   // M = 16
+    RAGO_VARIANT(8, 8, 1, 16, 2),   // M = 32
+    RAGO_VARIANT(12, 4, 1, 12, 1),  // M = 48
+    RAGO_VARIANT(8, 8, 2, 16, 2),   // M = 64
+    RAGO_VARIANT(20, 4, 1, 8, 1),   // M = 80
+    RAGO_VARIANT(24, 8, 1, 12, 1),  // M = 96
+    RAGO_VARIANT(8, 8, 4, 12, 2),   // M = 128
 };
 
 static const Variant* find_variant(int M) {
