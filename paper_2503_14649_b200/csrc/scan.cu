@@ -662,11 +662,13 @@ static int stages_for(int d) {
 #define RAGO_VARIANT(WV, G, R, NCW, RGW) \
     { Cfg<WV, G, R, NCW, RGW>::M, scan_kernel<WV, G, R, NCW, RGW>, Cfg<WV, G, R, NCW, RGW>::THREADS, \
       Cfg<WV, G, R, NCW, RGW>::TV, stages_for<Cfg<WV, G, R, NCW, RGW>> }
+// Warps x unrolled row groups per warp were chosen by measurement: independent row groups in flight inside a warp
+// hide the look-up latency better than more warps do (M = 64: 16 x 2 -> 12 x 4 gave +30%).
 static const Variant kVariants[] = {
     RAGO_VARIANT(4, 4, 1, 16, 2),   // M = 16
-    RAGO_VARIANT(8, 8, 1, 16, 2),   // M = 32
+    RAGO_VARIANT(8, 8, 1, 10, 3),   // M = 32
     RAGO_VARIANT(12, 4, 1, 12, 1),  // M = 48
-    RAGO_VARIANT(8, 8, 2, 16, 2),   // M = 64
+    RAGO_VARIANT(8, 8, 2, 12, 4),   // M = 64
     RAGO_VARIANT(20, 4, 1, 8, 1),   // M = 80
     RAGO_VARIANT(24, 8, 1, 12, 1),  // M = 96
     RAGO_VARIANT(8, 8, 4, 12, 2),   // M = 128
