@@ -303,15 +303,22 @@ __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
     for (int i = warp; i < kept; i += SEL_THREADS / 32) {
         const uint32_t l = (uint32_t)(keys[i] & 0xFFFFFFFFull);
         float acc = 0.f;
-        for (int j = lane; j < d; j += 32) {
-            float qv = qrow[j];
-            if (BF16) qv = round_bf16(qv);
-            const float c = load_c<BF16>(C, (size_t)l * d + j);
-            if (metric == RAGO_L2) {
-                const float t = qv - c;
-                acc = fmaf(t, t, acc);
+        for (int j = lane * 4; j < d; j += 128) {  // d is a multiple of 4: 16-byte (fp32) / 8-byte (bf16) loads
+            float4 qv = *reinterpret_cast<const float4*>(qrow + j);
+            float4 cv;
+            if (BF16) {
+                qv.x = round_bf16(qv.x); qv.y = round_bf16(qv.y); qv.z = round_bf16(qv.z); qv.w = round_bf16(qv.w);
+                const uint2 raw = *reinterpret_cast<const uint2*>(static_cast<const __nv_bfloat16*>(C) + (size_t)l * d + j);
+                cv.x = __uint_as_float(raw.x << 16); cv.y = __uint_as_float(raw.x & 0xFFFF0000u);
+                cv.z = __uint_as_float(raw.y << 16); cv.w = __uint_as_float(raw.y & 0xFFFF0000u);
             } else {
-                acc = fmaf(qv, c, acc);
+                cv = *reinterpret_cast<const float4*>(static_cast<const float*>(C) + (size_t)l * d + j);
+            }
+            if (metric == RAGO_L2) {
+                const float t0 = qv.x - cv.x, t1 = qv.y - cv.y, t2 = qv.z - cv.z, t3 = qv.w - cv.w;
+                acc = fmaf(t0, t0, fmaf(t1, t1, fmaf(t2, t2, fmaf(t3, t3, acc))));
+            } else {
+                acc = fmaf(qv.x, cv.x, fmaf(qv.y, cv.y, fmaf(qv.z, cv.z, fmaf(qv.w, cv.w, acc))));
             }
         }
         for (int o = 16; o; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);

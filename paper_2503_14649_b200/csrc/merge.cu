@@ -35,21 +35,30 @@ __global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(
         const long long s1 = (long long)q + cta_of_unit(u1 - 1, W, ctas);
         // all slots of the query side by side: entry e = (slot, i); empty entries are skipped
         const long long total = (s1 - s0 + 1) * (long long)k;
-        for (long long e0 = 0; e0 < total; e0 += MERGE_THREADS) {
-            const long long e = e0 + tid;
-            unsigned long long key = KEY_MAX;
-            if (e < total) {
-                const long long s = s0 + e / k;
-                const int i = (int)(e % k);
-                if (i < slot_cnt[s]) key = slot_keys[(size_t)s * k + i];
+        // entries are fetched MERGE_BATCH per thread at a time (independent loads in flight), then pushed
+        constexpr int MERGE_BATCH = 8;
+        for (long long e0 = 0; e0 < total; e0 += (long long)MERGE_THREADS * MERGE_BATCH) {
+            unsigned long long mine[MERGE_BATCH];
+#pragma unroll
+            for (int j = 0; j < MERGE_BATCH; ++j) {
+                const long long e = e0 + (long long)j * MERGE_THREADS + tid;
+                mine[j] = KEY_MAX;
+                if (e < total) {
+                    const long long s = s0 + e / k;
+                    const int i = (int)(e % k);
+                    if (i < slot_cnt[s]) mine[j] = slot_keys[(size_t)s * k + i];
+                }
             }
-            warp_push(keys, &cnt, key < tau, key);
-            __syncthreads();
-            if (cnt + MERGE_THREADS > TOPK_CAP) {  // uniform: cnt is stable between the barriers
-                const int kept = block_select(keys, &cnt, k, tid, MERGE_THREADS, sync);
-                if (kept == k) tau = keys[k - 1];
+#pragma unroll
+            for (int j = 0; j < MERGE_BATCH; ++j) {
+                warp_push(keys, &cnt, mine[j] < tau, mine[j]);
+                __syncthreads();
+                if (cnt + MERGE_THREADS > TOPK_CAP) {  // uniform: cnt is stable between the barriers
+                    const int kept = block_select(keys, &cnt, k, tid, MERGE_THREADS, sync);
+                    if (kept == k) tau = keys[k - 1];
+                }
+                __syncthreads();
             }
-            __syncthreads();
         }
     }
     __syncthreads();

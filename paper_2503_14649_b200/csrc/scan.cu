@@ -537,6 +537,13 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
         csync();
         if (dead) return;
         int kept = ctrl->cnt;
+        if (kept > 2 * k + 64) {  // a long buffer: bisect down to about k keys first, then sort only those
+            cut_buffer();
+            if (dead) return;
+            csync();
+            if (dead) return;
+            kept = ctrl->cnt;
+        }
         if (kept > k) {
             kept = block_select(keys, &ctrl->cnt, k, ctid, NCT, csync, C::KCAP);
             if (dead) return;
