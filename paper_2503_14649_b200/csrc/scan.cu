@@ -35,9 +35,16 @@
 // max|entry| * M / 2^30, i.e. an absolute error below max|entry| * M^2 / 2^31 per vector (2e-5 for
 // M = 96 and entries of size 5), far inside the 1e-4 relative bar.
 //
-// Candidates better than the running threshold go to a shared buffer (topk.cuh); the threshold of a
-// query is shared between CTAs through global memory, which only ever removes keys that cannot be
-// among the k best, so the result does not depend on timing.
+// Candidates better than the running threshold go to a shared buffer (topk.cuh).  The producer warp
+// watches the buffer count and marks a tile "cut first" when the tiles in flight could overflow it; a
+// cut is a CTA-wide bisection on the ordered score bits that keeps the k best keys and a few more (one
+// barrier per step), and the exact k best are sorted once, when the CTA leaves the query.  The
+// threshold of a query is shared between CTAs through global memory, which only ever removes keys that
+// cannot be among the k best, so the result does not depend on timing.
+//
+// A warp works on RGW row groups of 32 (virtual) rows per tile, unrolled, so that several independent
+// chains code word -> address -> table entry are in flight per warp; with R lanes per vector one
+// epilogue (term, bias, key, push) serves R row groups.
 #include "topk.cuh"
 
 namespace rago {
