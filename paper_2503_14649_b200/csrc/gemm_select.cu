@@ -474,12 +474,6 @@ void gemm_grid(int nrows, int64_t ncols, int num_sms, int* mg, int* nsplit, int*
     *mgroups = (mtiles + best_mg - 1) / best_mg;
 }
 
-cudaError_t gemm_select_init() {
-    cudaError_t e = cudaFuncSetAttribute(gemm_select_kernel<GEMM_CAP_SMALL / 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_SMEM_BYTES);
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(gemm_select_kernel<GEMM_CAP_LARGE / 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_SMEM_BYTES);
-    return e;
-}
 
 cudaError_t launch_gemm_select(const GemmLaunch& L, cudaStream_t s) {
     GemmArgs a;
@@ -577,17 +571,21 @@ cudaError_t launch_row_tau(const float* scores, int nrows, int n, int nsel, floa
     if (n <= RT_REG * RT_THREADS) {
         row_tau_kernel<true><<<nrows, RT_THREADS, 0, s>>>(scores, n, nsel, row_tau);
     } else {
-        static bool attr_set = false;
-        if (!attr_set) {
-            cudaError_t e = cudaFuncSetAttribute(row_tau_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-            if (e != cudaSuccess) return e;
-            attr_set = true;
-        }
         if ((size_t)n * 4 > 200 * 1024) return cudaErrorInvalidValue;
         row_tau_kernel<false><<<nrows, RT_THREADS, (size_t)n * 4, s>>>(scores, n, nsel, row_tau);
     }
     count_launch();
     return cudaGetLastError();
+}
+
+// Per-device set-up: the kernels' dynamic shared-memory limits (called at index load and by the flat search).
+cudaError_t gemm_select_init() {
+    cudaError_t e = cudaFuncSetAttribute(gemm_select_kernel<GEMM_CAP_SMALL / 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_SMEM_BYTES);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(gemm_select_kernel<GEMM_CAP_LARGE / 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_SMEM_BYTES);
+    if (e == cudaSuccess)  // rows of up to 51 200 pilot scores in shared memory
+        e = cudaFuncSetAttribute(row_tau_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    return e;
 }
 
 // ---- fp32 -> stacked bf16 parts: out[p][i] = bf16 part p of x[i] ---------------------------------

@@ -188,3 +188,30 @@ def test_argument_errors_are_reported_before_any_launch():
     with pytest.raises(binding.RagoError) as e:
         binding.load_index_from(data, "cuda")
     assert e.value.status == 1
+
+
+def test_search_replays_from_a_cuda_graph():
+    """rago_search only enqueues work on the caller's stream (no allocation, no synchronisation), so a call can be
+    captured once and replayed; the replay must give the eager call's results."""
+    data = synth.make_ivfpq(50_000, 128, 128, 32, 24, metric="l2", seed=12)
+    ix = binding.load_index_from(data, "cuda")
+    q = data.queries.cuda().contiguous()
+    ws = torch.empty(ix.search_workspace_bytes(24, 8, 20), dtype=torch.uint8, device="cuda")
+    ids = torch.empty((24, 20), dtype=torch.int64, device="cuda")
+    dists = torch.empty((24, 20), dtype=torch.float32, device="cuda")
+    ix.rago_search(q, 8, 20, ids, dists, ws)
+    torch.cuda.synchronize()
+    want_i, want_d = ids.clone(), dists.clone()
+    g = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(g, stream=side):
+            ix.rago_search(q, 8, 20, ids, dists, ws)
+    for _ in range(2):
+        ids.zero_()
+        dists.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(ids, want_i) and torch.equal(dists, want_d)
+    ix.rago_check(ws)
+    ix.close()
