@@ -159,3 +159,37 @@ def locate(ix: Index, ident: int):
     pos = int(np.nonzero(ix.ids == ident)[0][0])
     lst = int(np.searchsorted(ix.offsets, pos, side="right") - 1)
     return lst, pos
+
+
+def merge_results(part_ids, part_dists, k, metric):
+    """Aggregate the result lists of independently indexed database shards (paper, Sec. 4, retrieval
+    performance model: every shard answers every query and the results are aggregated).
+
+    part_ids / part_dists: [nparts][nq][k_in]; an entry with id -1 is padding.  For each query the
+    union of all real entries is ordered best first (smaller L2 distance, larger inner product;
+    equal scores by smaller id) and the first k are returned, padded with id -1 and +inf / -inf.
+    Plain definition, one query at a time.
+    """
+    ids = np.asarray(part_ids, np.int64)
+    dists = np.asarray(part_dists, np.float32)
+    m = _METRIC[metric]
+    nparts, nq, _ = ids.shape
+    out_ids = np.full((nq, k), -1, np.int64)
+    out_d = np.full((nq, k), np.inf if m == L2 else -np.inf, np.float32)
+    for q in range(nq):
+        entries = []
+        for p in range(nparts):
+            for ident, dist in zip(ids[p, q], dists[p, q]):
+                if ident >= 0:
+                    entries.append((float(dist) if m == L2 else -float(dist), int(ident), float(dist)))
+        entries.sort(key=lambda e: (e[0], e[1]))
+        for t, (_, ident, dist) in enumerate(entries[:k]):
+            out_ids[q, t] = ident
+            out_d[q, t] = dist
+    return out_ids, out_d
+
+
+def sharded_search(shards, queries, nprobe, k, nthreads=1):
+    """Search every shard's own index with the same queries, nprobe and k, then aggregate."""
+    parts = [ivfpq_search(ix, queries, nprobe, k, nthreads=nthreads) for ix in shards]
+    return merge_results(np.stack([p[0] for p in parts]), np.stack([p[1] for p in parts]), k, shards[0].metric)

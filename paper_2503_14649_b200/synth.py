@@ -218,6 +218,40 @@ def make_ivfpq(N: int, d: int, nlist: int, M: int, nq: int, *, metric: str = "l2
                      vectors=vectors, extra={"query_component": qcomp.cpu()})
 
 
+def make_ivfpq_shards(S: int, N_per: int, d: int, nlist: int, M: int, nq: int, *, metric: str = "l2",
+                      seed: int = MASTER_SEED, coarse_bf16: bool = False, device="cpu") -> list:
+    """S independently indexed shards of one Gaussian-mixture corpus, with one shared query batch.
+
+    The mixture centres ~ N(0,1)^d and the queries (centre + SIGMA * N(0,1)) come from `seed`.
+    Shard s draws its own N_per vectors from that mixture, its own coarse centroids (the centres
+    plus 0.25 * SIGMA * N(0,1), as if it had clustered its own sample) and its own codewords, files
+    a vector under its generating component and encodes the residual to that shard's centroid.
+    ids are disjoint across shards: s * N_per + a permutation of [0, N_per).
+    """
+    assert d % M == 0 and metric in ("l2", "ip")
+    dev = torch.device(device)
+    g = _generator(seed, dev)
+    centres = torch.randn((nlist, d), generator=g, device=dev, dtype=torch.float32)
+    qcomp = torch.randint(0, nlist, (nq,), generator=g, device=dev)
+    queries = centres[qcomp] + SIGMA * torch.randn((nq, d), generator=g, device=dev, dtype=torch.float32)
+    shards = []
+    for s in range(S):
+        gs = _generator(seed + 1000003 * (s + 1), dev)
+        cen = centres + 0.25 * SIGMA * torch.randn((nlist, d), generator=gs, device=dev, dtype=torch.float32)
+        centroids_q = cen.to(torch.bfloat16) if coarse_bf16 else cen
+        cen_f32 = centroids_q.float()
+        codebooks = SIGMA * torch.randn((M, 256, d // M), generator=gs, device=dev, dtype=torch.float32)
+        lab, _ = torch.sort(torch.randint(0, nlist, (N_per,), generator=gs, device=dev))
+        x = centres[lab] + SIGMA * torch.randn((N_per, d), generator=gs, device=dev, dtype=torch.float32)
+        codes = encode_residuals(x - cen_f32[lab], codebooks)
+        ids = (torch.randperm(N_per, generator=gs, device=dev) + s * N_per).to(torch.int64)
+        offsets = offsets_from_lengths(torch.bincount(lab, minlength=nlist).cpu())
+        shards.append(IvfPqData(N=N_per, d=d, nlist=nlist, M=M, metric=metric, centroids=centroids_q,
+                                codebooks=codebooks, codes=codes, list_offsets=offsets, ids=ids, queries=queries,
+                                seed=seed, extra={"shard": s}))
+    return shards
+
+
 def make_ivfpq_hashed(N: int, d: int, nlist: int, M: int, nq: int, *, metric: str, seed: int = MASTER_SEED,
                       coarse_bf16: bool = False, device="cpu", materialise: bool = True,
                       chunk: int = 1 << 22) -> IvfPqData:

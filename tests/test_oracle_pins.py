@@ -265,3 +265,48 @@ def test_bad_arguments_are_refused():
         oracle.ivfpq_search(ix, data.queries.numpy(), 5, 3)  # nprobe > nlist
     with pytest.raises(ValueError):
         oracle.ivfpq_search(ix, data.queries.numpy(), 1, 0)
+
+
+def _decoded_vectors(data):
+    lab, resid, cen = _decode_all(data)
+    return cen[lab] + resid
+
+
+@pytest.mark.parametrize("metric", ["l2", "ip"])
+def test_sharded_full_probe_equals_bruteforce_over_the_union_of_shards(metric):
+    """Independent indexes per shard, results aggregated (paper, Sec. 4, retrieval model): with every
+    list of every shard probed, the aggregate is the exact kNN over all decoded vectors of all
+    shards, whichever shard holds them."""
+    S, k = 3, 17
+    shards = synth.make_ivfpq_shards(S, 700, 16, 8, 4, 6, metric=metric, seed=77)
+    q = shards[0].queries.double().numpy()
+    got_i, got_d = oracle.sharded_search([host_index(oracle, sh) for sh in shards], shards[0].queries.numpy(), 8, k)
+    y = np.concatenate([_decoded_vectors(sh) for sh in shards])
+    ids = np.concatenate([sh.ids.numpy() for sh in shards])
+    assert np.unique(ids).size == ids.size
+    if metric == "l2":
+        s = ((q[:, None, :] - y[None]) ** 2).sum(2)
+        order = np.argsort(s, axis=1, kind="stable")[:, :k]
+    else:
+        s = q @ y.T
+        order = np.argsort(-s, axis=1, kind="stable")[:, :k]
+    assert np.array_equal(got_i, ids[order])
+    assert np.allclose(got_d, np.take_along_axis(s, order, 1), rtol=2e-6, atol=1e-6)
+    # every shard contributes to some query's answer, so no part is dropped silently
+    assert set(np.unique(got_i // 700)) == set(range(S))
+
+
+def test_merge_results_by_hand():
+    """Two shards, two queries, worked by hand: padding is skipped, ties go to the smaller id, short
+    unions are padded."""
+    inf = np.inf
+    ids = np.array([[[5, 9, -1], [4, -1, -1]],
+                    [[7, 2, 8], [-1, -1, -1]]], np.int64)
+    l2 = np.array([[[0.5, 2.0, inf], [1.0, inf, inf]],
+                   [[0.25, 2.0, 3.0], [inf, inf, inf]]], np.float32)
+    oi, od = oracle.merge_results(ids, l2, 4, "l2")
+    assert oi.tolist() == [[7, 5, 2, 9], [4, -1, -1, -1]]
+    assert od[0].tolist() == [0.25, 0.5, 2.0, 2.0] and od[1, 0] == 1.0 and np.isposinf(od[1, 1:]).all()
+    ip = np.where(np.isinf(l2), -inf, -l2).astype(np.float32)   # same order under inner product
+    oi2, od2 = oracle.merge_results(ids, ip, 2, "ip")
+    assert oi2.tolist() == [[7, 5], [4, -1]] and od2[0].tolist() == [-0.25, -0.5] and np.isneginf(od2[1, 1])
