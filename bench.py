@@ -532,6 +532,77 @@ def run_iter(args):
                      "unit": None, "frac": None, "traffic": None}}))
 
 
+def run_sharded(args):
+    """Secondary workload: database-sharded search.  Every rank holds its own Mid-shape shard with an independent
+    index (its own seed); all ranks answer rank 0's query batch, exchange their [nq, k] answers with one all-gather
+    and aggregate them.  The database grows with the number of ranks, the query batch does not."""
+    from paper_2503_14649_b200 import binding, sharded, synth
+    rank, world, local = _dist_env()
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    else:
+        torch.cuda.set_device(0)
+        local = 0
+    dev = torch.device("cuda", local)
+    c = synth.CONFIGS[WORKLOAD]
+    nq, nprobe, k = c["nq"], c["nprobe"], c["k"]
+    data = synth.make_config(WORKLOAD, device=dev, scale=args.scale, seed=synth.MASTER_SEED + 7919 * rank)
+    ix = binding.rago_index_load(data.centroids, data.codebooks, data.codes, data.list_offsets.to(dev), data.ids,
+                                 data.metric)
+    q = data.queries.contiguous()
+    if world > 1:
+        torch.distributed.broadcast(q, 0)
+    ws = torch.empty(ix.search_workspace_bytes(nq, nprobe, k), dtype=torch.uint8, device=dev)
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+
+    def step():
+        return sharded.rago_search_sharded(ix, q, nprobe, k, workspace=ws)
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    for _ in range(max(3, args.warmup)):
+        step()
+    barrier()
+    launches0 = binding.rago_kernel_launches()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    t0 = time.time()
+    ev[0].record()
+    for _ in range(args.steps):
+        step()
+    ev[1].record()
+    barrier()
+    t1 = time.time()
+    launches = binding.rago_kernel_launches() - launches0
+    clocks = sampler.stop(t0, t1)
+    ix.rago_check(ws)
+    total_ms = max_over_ranks(ev[0].elapsed_time(ev[1]), world, dev)
+    # the aggregation kernel alone, on gathered answers already in place
+    ids, dists = ix.rago_search(q, nprobe, k, workspace=ws)
+    parts = sharded.gather_parts(ids, dists)
+    agg_ms, _ = _time_steps(lambda: binding.rago_merge_results(parts[0], parts[1], k, ix.metric), 20, 3)
+    if rank == 0:
+        ms = total_ms / args.steps
+        print(json.dumps({
+            "metric": METRIC, "value": nq / (ms / 1e3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak (database grows with ranks, one shared query batch)", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic",
+            "config": {"workload": "Sharded Mid IVF-PQ: %d shard(s) of N=%d d=%d nlist=%d M=%d, independent indexes; nq=%d "
+                                   "nprobe=%d k=%d L2; all-gather + aggregation every step"
+                                   % (world, data.N, c["d"], c["nlist"], c["M"], nq, nprobe, k),
+                       "l2_policy": "inputs larger than L2", "scale": args.scale},
+            "clocks": clocks, "gpu_launches": launches, "aggregate_kernel_ms": agg_ms / 20,
+            "exchange_bytes_per_rank": nq * k * 12}))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -540,7 +611,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--scale", type=float, default=1.0, help="shrink N (development only; 1.0 = the named workload)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="mid", choices=["mid", "flat", "coarse_hyper", "hyper", "iter"],
+    ap.add_argument("--workload", default="mid", choices=["mid", "flat", "coarse_hyper", "hyper", "iter", "sharded"],
                     help="mid = the headline Mid IVF-PQ workload (default); the others are secondary measurements")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -553,6 +624,8 @@ def main():
         run_hyper(args)
     elif args.workload == "iter":
         run_iter(args)
+    elif args.workload == "sharded":
+        run_sharded(args)
     else:
         run_ours(args)
 

@@ -193,6 +193,27 @@ rago_status rago_check(void* workspace, void* cuda_stream);
  */
 rago_status rago_set_coarse_mode(rago_index* index, int32_t mode);
 
+/*
+ * Aggregation step of a database that is split into shards with independent indexes (paper, Sec. 4,
+ * retrieval performance model: queries go to every shard, results are aggregated).  Every shard has
+ * answered the same nq queries with k_in results each (rago_search's output layout, padding id -1
+ * allowed anywhere); for each query the k_out best entries of the union are written best first.
+ *
+ *   part_ids    device, int64: shard p's row of query q starts at part_ids[p * part_stride + q * k_in];
+ *               the gathered buffers of nparts ranks laid end to end have part_stride = nq * k_in
+ *   part_dists  device, fp32, same layout: L2 distances or inner products as rago_search returns them
+ *   out_ids     device, int64 [nq][k_out]; out_dists device, fp32 [nq][k_out]; short unions are padded with
+ *               id -1 and +inf (L2) / -inf (IP); entries with equal scores keep the order (shard, rank)
+ *   metric      RAGO_L2 or RAGO_IP, the metric of the shards' indexes
+ *
+ * ids are copied through unchanged: they should be unique across shards, which is the caller's
+ * business.  1 <= k_out <= 1024, nparts * k_in < 2^31.  Needs no workspace, borrows every pointer, is
+ * asynchronous on cuda_stream.  RAGO_EINVAL / RAGO_EUNSUPPORTED on bad sizes, nothing is launched then.
+ */
+rago_status rago_merge_results(const int64_t* part_ids, const float* part_dists, int32_t nparts,
+                               int64_t part_stride, int32_t nq, int32_t k_in, int32_t k_out, int32_t metric,
+                               int64_t* out_ids, float* out_dists, void* cuda_stream);
+
 /* Per-stage device timings of rago_search.  When enabled, rago_search records CUDA events on the
  * caller's stream around each stage; rago_profile_read synchronises and returns the last call's
  * stage times in milliseconds (out_ms[RAGO_NUM_STAGES]). */

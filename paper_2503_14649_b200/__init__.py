@@ -7,4 +7,4 @@ opened on first use of the binding and a missing library is an error, never a
 fallback.
 """
 
-__all__ = ["binding", "synth"]
+__all__ = ["binding", "sharded", "synth"]

@@ -27,7 +27,7 @@ STAGE_NAMES = ("coarse_scores", "probe_select", "plan", "table_scan", "merge")
 EXPORTS = ("rago_index_load", "rago_index_free", "rago_search_workspace_bytes", "rago_search",
            "rago_search_probes", "rago_search_probes_noalloc", "rago_search_host", "rago_host_staging_bytes", "rago_flat_search",
            "rago_flat_workspace_bytes", "rago_check", "rago_set_coarse_mode", "rago_profile_enable", "rago_profile_read",
-           "rago_kernel_launches", "rago_last_error")
+           "rago_merge_results", "rago_kernel_launches", "rago_last_error")
 
 
 class RagoError(RuntimeError):
@@ -56,6 +56,7 @@ def lib() -> ctypes.CDLL:
         L.rago_search_host.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, sz, vp]
         L.rago_flat_search.argtypes = [vp, i64, i32, vp, i32, i32, vp, vp, vp, sz, vp]
         L.rago_flat_workspace_bytes.argtypes = [i64, i32, i32, i32, ctypes.POINTER(sz)]
+        L.rago_merge_results.argtypes = [vp, vp, i32, i64, i32, i32, i32, i32, vp, vp, vp]
         L.rago_check.argtypes = [vp, vp]
         L.rago_set_coarse_mode.argtypes = [vp, i32]
         L.rago_profile_enable.argtypes = [vp, i32]
@@ -209,6 +210,23 @@ def rago_flat_search(db: torch.Tensor, queries: torch.Tensor, k: int, workspace:
     _check(lib().rago_flat_search(_ptr(db), N, d, _ptr(queries), nq, k, _ptr(out_ids), _ptr(out_scores),
                                   _ptr(workspace), workspace.numel(), _stream()))
     return out_ids, out_scores
+
+
+def rago_merge_results(part_ids: torch.Tensor, part_dists: torch.Tensor, k_out: int, metric,
+                       out_ids: Optional[torch.Tensor] = None, out_dists: Optional[torch.Tensor] = None):
+    """part_ids / part_dists: contiguous [nparts, nq, k_in] device tensors (the shards' answers side by side)."""
+    metric = {"l2": RAGO_L2, "ip": RAGO_IP}.get(metric, metric)
+    nparts, nq, k_in = part_ids.shape
+    if part_dists.shape != part_ids.shape or not (part_ids.is_contiguous() and part_dists.is_contiguous()):
+        raise ValueError("part_ids and part_dists must be contiguous tensors of one shape [nparts, nq, k_in]")
+    dev = part_ids.device
+    if out_ids is None:
+        out_ids = torch.empty((nq, k_out), dtype=torch.int64, device=dev)
+    if out_dists is None:
+        out_dists = torch.empty((nq, k_out), dtype=torch.float32, device=dev)
+    _check(lib().rago_merge_results(_ptr(part_ids), _ptr(part_dists), nparts, nq * k_in, nq, k_in, k_out, metric,
+                                    _ptr(out_ids), _ptr(out_dists), _stream()))
+    return out_ids, out_dists
 
 
 def load_index_from(data, device="cuda") -> Index:
