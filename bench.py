@@ -31,7 +31,7 @@ import numpy as np  # noqa: E402
 import torch  # noqa: E402
 
 WORKLOAD = 2  # index into synth.CONFIGS
-SCAN_DRAM_PER_LOGICAL = 3.532e9 / 11.126e9
+SCAN_DRAM_PER_LOGICAL = 30.867e9 / 42.427e9  # full-size Mid workload only (see run_ours)
 METRIC = "retrieval_qps"
 UNIT = "queries/s"
 
@@ -276,10 +276,12 @@ def run_ours(args):
 
     peak, peak_kind = _peaks()
     achieved = scan_bytes / (scan_ms / 1e3) / 1e9
-    # DRAM bytes of one scan launch: ncu capture at 1/4 of the vectors (profiles/scan_kernel_mid_quarter_scale.md:
-    # 3.639 GB for 11.126 GB of logical code bytes), scaled by this launch's logical bytes.  Valid for the scan
-    # kernel that capture was taken from; set SCAN_DRAM_PER_LOGICAL to None after changing the kernel.
-    traffic = None if SCAN_DRAM_PER_LOGICAL is None else SCAN_DRAM_PER_LOGICAL * scan_bytes
+    # DRAM bytes of one scan launch: dram__bytes_read.sum + dram__bytes_write.sum of one launch of this very
+    # workload at full size (profiles/scan_kernel_mid_quarter_scale.md: 30.867 GB for 42.427 GB of logical code
+    # bytes; hot lists are shared through L2).  The ratio does not carry over to other sizes (at 1/4 of the vectors
+    # it is 0.31), so scaled-down runs report null.  Valid for the scan kernel the capture was taken from: set
+    # SCAN_DRAM_PER_LOGICAL to None after changing the kernel.
+    traffic = SCAN_DRAM_PER_LOGICAL * scan_bytes if SCAN_DRAM_PER_LOGICAL is not None and args.scale == 1.0 else None
     out = {
         "metric": METRIC, "value": qps, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
