@@ -605,6 +605,53 @@ def run_sharded(args):
         torch.distributed.destroy_process_group()
 
 
+def run_sweep(args):
+    """Secondary measurement: batch-size sweep on the Mid index, the data a retrieval cost model needs.  The paper
+    models a scan operator as T = max(D / P_comp(Q), D / B_mem) with D the bytes scanned and Q the batch size
+    (Sec. 4); here every batch size gets its measured time and scanned bytes, and a least-squares line
+    T = T0 + D / B_eff over the sweep gives the two constants of the same model on this GPU (T0: the launch-bound
+    floor the paper's model does not have)."""
+    from paper_2503_14649_b200 import binding, synth
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    c = synth.CONFIGS[WORKLOAD]
+    nprobe, k = c["nprobe"], c["k"]
+    data = synth.make_config(WORKLOAD, device=dev, scale=args.scale)
+    ix = binding.rago_index_load(data.centroids, data.codebooks, data.codes, data.list_offsets.to(dev), data.ids,
+                                 data.metric)
+    Ln = (data.list_offsets[1:] - data.list_offsets[:-1]).to(dev)
+    rows = []
+    sampler = ClockSampler(0)
+    sampler.start()
+    t0 = time.time()
+    for nq in (1, 2, 4, 8, 16, 32, 64, 128, 256, 512, 1024):
+        q = data.queries[:nq].contiguous()
+        ws = torch.empty(ix.search_workspace_bytes(nq, nprobe, k), dtype=torch.uint8, device=dev)
+        out_i = torch.empty((nq, k), dtype=torch.int64, device=dev)
+        out_d = torch.empty((nq, k), dtype=torch.float32, device=dev)
+        lists, _ = ix.rago_search_probes(q, nprobe, workspace=ws)
+        D = int(Ln[lists.long()].sum().item()) * c["M"]
+        steps = max(10, min(200, int(2000 / nq)))
+        total_ms, step_ms = _time_steps(lambda: ix.rago_search(q, nprobe, k, out_i, out_d, ws), steps, 3)
+        ix.rago_check(ws)
+        ms = float(np.median(step_ms))
+        rows.append({"nq": nq, "ms": ms, "qps": nq / (ms / 1e3), "scanned_bytes": D, "gbs": D / (ms / 1e3) / 1e9})
+    t1 = time.time()
+    clocks = sampler.stop(t0, t1)
+    Dv = np.array([r["scanned_bytes"] for r in rows], np.float64)
+    Tv = np.array([r["ms"] for r in rows], np.float64) * 1e-3
+    A = np.stack([np.ones_like(Dv), Dv], 1)
+    # relative least squares, so that the small batches weigh as much as the large ones
+    coef, *_ = np.linalg.lstsq(A / Tv[:, None], np.ones_like(Tv), rcond=None)
+    print(json.dumps({
+        "metric": "retrieval_cost_model", "unit": "s = T0 + D / B_eff", "n_gpus": 1, "data": "synthetic",
+        "config": {"workload": "Mid IVF-PQ index (configs[1]), batch sizes 1..1024, nprobe=%d k=%d" % (nprobe, k),
+                   "scale": args.scale},
+        "fit": {"T0_us": coef[0] * 1e6, "B_eff_GBs": 1.0 / coef[1] / 1e9,
+                "max_rel_err": float(np.max(np.abs(A @ coef - Tv) / Tv))},
+        "rows": rows, "clocks": clocks}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -613,7 +660,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--scale", type=float, default=1.0, help="shrink N (development only; 1.0 = the named workload)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="mid", choices=["mid", "flat", "coarse_hyper", "hyper", "iter", "sharded"],
+    ap.add_argument("--workload", default="mid", choices=["mid", "flat", "coarse_hyper", "hyper", "iter", "sharded", "sweep"],
                     help="mid = the headline Mid IVF-PQ workload (default); the others are secondary measurements")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -628,6 +675,8 @@ def main():
         run_iter(args)
     elif args.workload == "sharded":
         run_sharded(args)
+    elif args.workload == "sweep":
+        run_sweep(args)
     else:
         run_ours(args)
 

@@ -551,11 +551,11 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
             if (dead) return;
             kept = ctrl->cnt;
         }
-        if (kept > k) {
+        if (kept > 1) {  // the slot is left in ascending order, which the merge relies on
             kept = block_select(keys, &ctrl->cnt, k, ctid, NCT, csync, C::KCAP);
             if (dead) return;
-            if (ctid == 0) atomicMin(&a.qthresh[cur_q], keys[k - 1]);
         }
+        if (kept == k && ctid == 0) atomicMin(&a.qthresh[cur_q], keys[k - 1]);
         const size_t slot = (size_t)cur_q + blockIdx.x;
         for (int i = ctid; i < kept; i += NCT) a.slot_keys[slot * k + i] = keys[i];
         if (ctid == 0) a.slot_cnt[slot] = kept;

@@ -215,3 +215,48 @@ def test_search_replays_from_a_cuda_graph():
         assert torch.equal(ids, want_i) and torch.equal(dists, want_d)
     ix.rago_check(ws)
     ix.close()
+
+
+def test_concurrent_searches_on_two_streams_do_not_interfere():
+    """Calls on one index from different streams, each with its own workspace and outputs, may overlap on the GPU:
+    the index is read-only during a search and all per-call state lives in the workspace."""
+    data = synth.make_ivfpq(150_000, 128, 256, 32, 96, metric="ip", seed=19, zipf=1.0)
+    ix = binding.load_index_from(data, "cuda")
+    qa = data.queries[:64].cuda().contiguous()
+    qb = data.queries[64:].cuda().contiguous()
+    want_a = [t.clone() for t in ix.rago_search(qa, 12, 30)]
+    want_b = [t.clone() for t in ix.rago_search(qb, 20, 50)]
+    torch.cuda.synchronize()
+    sa, sb = torch.cuda.Stream(), torch.cuda.Stream()
+    wa = torch.empty(ix.search_workspace_bytes(64, 12, 30), dtype=torch.uint8, device="cuda")
+    wb = torch.empty(ix.search_workspace_bytes(32, 20, 50), dtype=torch.uint8, device="cuda")
+    outs_a, outs_b = [], []
+    for _ in range(6):
+        oa = (torch.empty((64, 30), dtype=torch.int64, device="cuda"), torch.empty((64, 30), device="cuda"))
+        ob = (torch.empty((32, 50), dtype=torch.int64, device="cuda"), torch.empty((32, 50), device="cuda"))
+        with torch.cuda.stream(sa):
+            ix.rago_search(qa, 12, 30, oa[0], oa[1], wa)
+        with torch.cuda.stream(sb):
+            ix.rago_search(qb, 20, 50, ob[0], ob[1], wb)
+        outs_a.append(oa)
+        outs_b.append(ob)
+    torch.cuda.synchronize()
+    ix.rago_check(wa)
+    ix.rago_check(wb)
+    for oa, ob in zip(outs_a, outs_b):
+        assert torch.equal(oa[0], want_a[0]) and torch.equal(oa[1], want_a[1])
+        assert torch.equal(ob[0], want_b[0]) and torch.equal(ob[1], want_b[1])
+    ix.close()
+
+
+@pytest.mark.parametrize("k", [1000, 100])
+def test_single_query_whose_best_list_is_spread_over_many_ctas(k):
+    """One query, k large: every scan CTA leaves a partial top-k, and the CTAs that worked on the query's own list
+    hold far more than k keys below every other CTA's best one, so the merge cannot finish from the slots' leading
+    keys alone and has to select in several rounds."""
+    data = synth.make_ivfpq(200_000, 32, 8, 16, 1, metric="l2", seed=23)
+    cen = torch.zeros((8, 32))
+    cen[1:] = 10.0 * torch.nn.functional.normalize(data.centroids[1:], dim=1)   # list 0 around the origin, the rest far
+    data.centroids = cen
+    data.queries = 0.01 * data.queries / data.queries.norm()
+    _compare(data, 8, k)
