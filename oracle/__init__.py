@@ -193,3 +193,69 @@ def sharded_search(shards, queries, nprobe, k, nthreads=1):
     """Search every shard's own index with the same queries, nprobe and k, then aggregate."""
     parts = [ivfpq_search(ix, queries, nprobe, k, nthreads=nthreads) for ix in shards]
     return merge_results(np.stack([p[0] for p in parts]), np.stack([p[1] for p in parts]), k, shards[0].metric)
+
+
+# ---- 4-bit product quantisation (the paper's "low-precision" PQ variant, Sec. 2: 4-bit vs 8-bit codes) ----
+# Definition, in numpy fp64: each sub-space has 16 codewords, two codes share a byte (sub-space 2j in the low
+# nibble of byte j, sub-space 2j + 1 in the high nibble).  Pins in tests/test_oracle_pins.py: a hand-worked
+# example, brute force over the decoded vectors, and agreement with the 8-bit oracle on the index whose
+# sub-spaces are the pairs and whose 256 codewords per pair are all concatenations.
+
+def unpack_pq4(packed):
+    """uint8 [N, M4/2] -> uint8 [N, M4]: code of sub-space 2j = byte j & 15, of sub-space 2j + 1 = byte j >> 4."""
+    p = np.asarray(packed, np.uint8)
+    out = np.empty((p.shape[0], p.shape[1] * 2), np.uint8)
+    out[:, 0::2] = p & 15
+    out[:, 1::2] = p >> 4
+    return out
+
+
+def ivfpq4_search(centroids, codebooks4, packed_codes, list_offsets, ids, metric, queries, nprobe, k,
+                  coarse_bf16=False):
+    """IVF-PQ search with 4-bit codes.  centroids fp32 [nlist, d] (or bf16 bit patterns, uint16, with
+    coarse_bf16), codebooks4 fp32 [M4, 16, d / M4], packed_codes uint8 [N, M4 / 2] in list order.
+
+    The nprobe lists come from the same coarse step as the 8-bit search.  A stored vector stands for
+    y = centroid + concatenated codewords; its score is ||q - y||^2, or <q, y> with the centroid part
+    taken from the coarse step's value (so that a bf16 coarse quantiser enters the same way as in the
+    8-bit search).  Best first, ties to the smaller id, padding (-1, +inf / -inf).
+    """
+    m = _METRIC[metric]
+    q = _c(queries, np.float32)
+    cb = np.asarray(codebooks4, np.float64)
+    M4, ksub, dsub = cb.shape
+    assert ksub == 16
+    codes = unpack_pq4(packed_codes)
+    off = np.asarray(list_offsets, np.int64)
+    ids = np.asarray(ids, np.int64)
+    lists, cvals = coarse(centroids, q, nprobe, m, coarse_bf16=coarse_bf16)
+    if coarse_bf16:
+        cen = (np.asarray(centroids, np.uint16).astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    else:
+        cen = np.asarray(centroids, np.float64)
+    nq = q.shape[0]
+    out_ids = np.full((nq, k), -1, np.int64)
+    out_d = np.full((nq, k), np.inf if m == L2 else -np.inf, np.float32)
+    for i in range(nq):
+        qi = q[i].astype(np.float64)
+        cand_s, cand_id = [], []
+        for p in range(nprobe):
+            l = int(lists[i, p])
+            a, b = int(off[l]), int(off[l + 1])
+            if b == a:
+                continue
+            r = np.concatenate([cb[s][codes[a:b, s]] for s in range(M4)], axis=1)   # [n, d] decoded residuals
+            if m == L2:
+                s_ = ((qi[None, :] - (cen[l][None, :] + r)) ** 2).sum(1)
+            else:
+                s_ = float(cvals[i, p]) + r @ qi
+            cand_s.append(s_)
+            cand_id.append(ids[a:b])
+        if not cand_s:
+            continue
+        s_ = np.concatenate(cand_s)
+        id_ = np.concatenate(cand_id)
+        order = np.lexsort((id_, s_ if m == L2 else -s_))[:k]
+        out_ids[i, :order.size] = id_[order]
+        out_d[i, :order.size] = s_[order]
+    return out_ids, out_d

@@ -218,6 +218,42 @@ def make_ivfpq(N: int, d: int, nlist: int, M: int, nq: int, *, metric: str = "l2
                      vectors=vectors, extra={"query_component": qcomp.cpu()})
 
 
+def pack_pq4(codes: torch.Tensor) -> torch.Tensor:
+    """uint8 [N, M4] codes below 16 -> uint8 [N, M4/2]: sub-space 2j in the low nibble of byte j, 2j+1 in the high."""
+    return (codes[:, 0::2] | (codes[:, 1::2] << 4)).contiguous()
+
+
+def make_ivfpq4(N: int, d: int, nlist: int, M4: int, nq: int, *, metric: str = "l2", seed: int = MASTER_SEED,
+                zipf: Optional[float] = None, coarse_bf16: bool = False, device="cpu",
+                chunk: int = 1 << 16) -> IvfPqData:
+    """The corpus of make_ivfpq (vectors filed under their generating component) encoded with 4-bit codes:
+    M4 sub-spaces of 16 codewords ~ N(0, SIGMA^2) each, two codes per byte.  The returned record has
+    M = M4 / 2 code bytes per vector, codebooks [M4, 16, d/M4] and extra["pq4"] = True."""
+    assert d % M4 == 0 and M4 % 2 == 0 and metric in ("l2", "ip")
+    dev = torch.device(device)
+    g = _generator(seed, dev)
+    centres = torch.randn((nlist, d), generator=g, device=dev, dtype=torch.float32)
+    codebooks = SIGMA * torch.randn((M4, 16, d // M4), generator=g, device=dev, dtype=torch.float32)
+    w = (zipf_weights(nlist, zipf) if zipf else torch.full((nlist,), 1.0 / nlist, dtype=torch.float64)).to(dev)
+    comp = torch.multinomial(w.float(), N, replacement=True, generator=g) if N > 0 else \
+        torch.zeros(0, dtype=torch.int64, device=dev)
+    centroids_q = centres.to(torch.bfloat16) if coarse_bf16 else centres
+    cen_f32 = centroids_q.float()
+    lab, _ = torch.sort(comp)
+    codes = torch.empty((N, M4 // 2), dtype=torch.uint8, device=dev)
+    for s in range(0, N, chunk):
+        c = cen_f32[lab[s:s + chunk]]
+        x = c + SIGMA * torch.randn(c.shape, generator=g, device=dev, dtype=torch.float32)
+        codes[s:s + chunk] = pack_pq4(encode_residuals(x - c, codebooks, chunk=min(chunk, 8192)))
+    list_offsets = offsets_from_lengths(torch.bincount(lab, minlength=nlist).cpu())
+    ids = torch.randperm(N, generator=g, device=dev).to(torch.int64)
+    qcomp = torch.multinomial(w.float(), nq, replacement=True, generator=g)
+    queries = centres[qcomp] + SIGMA * torch.randn((nq, d), generator=g, device=dev, dtype=torch.float32)
+    return IvfPqData(N=N, d=d, nlist=nlist, M=M4 // 2, metric=metric, centroids=centroids_q, codebooks=codebooks,
+                     codes=codes, list_offsets=list_offsets, ids=ids, queries=queries, seed=seed,
+                     extra={"pq4": True, "M4": M4})
+
+
 def make_ivfpq_shards(S: int, N_per: int, d: int, nlist: int, M: int, nq: int, *, metric: str = "l2",
                       seed: int = MASTER_SEED, coarse_bf16: bool = False, device="cpu") -> list:
     """S independently indexed shards of one Gaussian-mixture corpus, with one shared query batch.

@@ -310,3 +310,44 @@ def test_merge_results_by_hand():
     ip = np.where(np.isinf(l2), -inf, -l2).astype(np.float32)   # same order under inner product
     oi2, od2 = oracle.merge_results(ids, ip, 2, "ip")
     assert oi2.tolist() == [[7, 5], [4, -1]] and od2[0].tolist() == [-0.25, -0.5] and np.isneginf(od2[1, 1])
+
+
+@pytest.mark.parametrize("metric", ["l2", "ip"])
+def test_pq4_handworked_example(metric):
+    g = json.load(open(os.path.join(GOLD, "handworked_pq4.json")))
+    cb = np.zeros((2, 16, 1), np.float32)
+    cb[0, :, 0] = np.arange(16)
+    cb[1, :, 0] = -np.arange(16)
+    for case in g[metric]["cases"]:
+        ids, dists = oracle.ivfpq4_search(np.asarray(g["centroids"], np.float32), cb,
+                                          np.asarray(g["packed_codes"], np.uint8), g["list_offsets"], g["ids"], metric,
+                                          np.asarray([g["query"]], np.float32), case["nprobe"], case["k"])
+        assert ids[0].tolist() == case["ids"], case
+        assert dists[0].tolist() == [_inf(v) for v in case["dists"]], case
+
+
+def _pair_codebooks(cb4):
+    """[M4, 16, ds] -> [M4/2, 256, 2 ds]: codeword `byte` of pair j = codeword byte & 15 of sub-space 2j followed
+    by codeword byte >> 4 of sub-space 2j + 1."""
+    M4, _, ds = cb4.shape
+    byte = np.arange(256)
+    return np.concatenate([cb4[0::2][:, byte & 15, :], cb4[1::2][:, byte >> 4, :]], axis=2).astype(np.float32)
+
+
+@pytest.mark.parametrize("metric,bf16", [("l2", False), ("ip", False), ("l2", True), ("ip", True)])
+def test_pq4_equals_8bit_search_over_paired_subspaces(metric, bf16):
+    """A 4-bit index is an 8-bit index in disguise: pairs of sub-spaces with all 256 concatenated codewords, the
+    packed byte as the code.  The numpy 4-bit definition and the 8-bit oracle (different code) must agree on it."""
+    data = synth.make_ivfpq4(4000, 32, 16, 16, 9, metric=metric, seed=61, coarse_bf16=bf16)
+    cen = data.centroids.view(torch.uint16).numpy() if bf16 else data.centroids.numpy()
+    cb4 = data.codebooks.numpy()
+    a_i, a_d = oracle.ivfpq4_search(cen, cb4, data.codes.numpy(), data.list_offsets.numpy(), data.ids.numpy(), metric,
+                                    data.queries.numpy(), 5, 12, coarse_bf16=bf16)
+    ix8 = oracle.Index(cen, _pair_codebooks(cb4), data.codes.numpy(), data.list_offsets.numpy(), data.ids.numpy(),
+                       metric, coarse_bf16=bf16)
+    b_i, b_d = oracle.ivfpq_search(ix8, data.queries.numpy(), 5, 12)
+    assert np.array_equal(a_i, b_i)
+    assert np.allclose(a_d, b_d, rtol=2e-6, atol=1e-6)
+    # and the codes really are nibbles of the nearest codewords: unpack(pack(x)) == x
+    codes = torch.randint(0, 16, (50, 8), dtype=torch.uint8)
+    assert np.array_equal(oracle.unpack_pq4(synth.pack_pq4(codes).numpy()), codes.numpy())
