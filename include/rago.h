@@ -81,6 +81,27 @@ rago_status rago_index_load(rago_index** out, const void* coarse_centroids, rago
                             const int64_t* ids, int64_t N, int32_t d, int32_t nlist, int32_t M,
                             rago_metric metric, void* cuda_stream);
 
+/*
+ * Load an index whose product quantiser uses 4-bit codes: the paper's low-precision PQ variant (Sec. 2,
+ * vector search background: 4-bit codes make the scan memory-bound, 8-bit codes compute-bound on CPUs).
+ * M4 sub-spaces of 16 codewords each; two codes share a byte, sub-space 2j in the low nibble of byte j and
+ * sub-space 2j + 1 in the high nibble, so a vector occupies M4 / 2 bytes.
+ *
+ *   pq4_codebooks  device, fp32 [M4][16][d / M4], 16-byte aligned; read during the call only
+ *   packed_codes   device, uint8 [N][M4 / 2], list-contiguous like rago_index_load's codes; borrowed
+ *   everything else as in rago_index_load
+ *
+ * The result is an ordinary rago_index with M = M4 / 2 code bytes per vector: every search call takes it, and
+ * scores follow the same definitions with the decoded vector centroid + concatenated 4-bit codewords.
+ * M4 / 2 must be one of the supported code sizes (16, 32, 48, 64, 80, 96, 128).  Allocates and frees a
+ * temporary of 1024 * d bytes and synchronises cuda_stream.  Errors as rago_index_load, plus RAGO_EINVAL for an
+ * odd M4.
+ */
+rago_status rago_index_load_pq4(rago_index** out, const void* coarse_centroids, rago_dtype coarse_dtype,
+                                const float* pq4_codebooks, const uint8_t* packed_codes, const int64_t* list_offsets,
+                                const int64_t* ids, int64_t N, int32_t d, int32_t nlist, int32_t M4,
+                                rago_metric metric, void* cuda_stream);
+
 /* Release the handle and the arrays the library allocated for it (never the borrowed ones).
  * Synchronises the device first.  NULL is accepted. */
 rago_status rago_index_free(rago_index* index);

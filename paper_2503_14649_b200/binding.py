@@ -24,7 +24,7 @@ RAGO_F32, RAGO_BF16 = 0, 1
 NUM_STAGES = 5
 STAGE_NAMES = ("coarse_scores", "probe_select", "plan", "table_scan", "merge")
 
-EXPORTS = ("rago_index_load", "rago_index_free", "rago_search_workspace_bytes", "rago_search",
+EXPORTS = ("rago_index_load", "rago_index_load_pq4", "rago_index_free", "rago_search_workspace_bytes", "rago_search",
            "rago_search_probes", "rago_search_probes_noalloc", "rago_search_host", "rago_host_staging_bytes", "rago_flat_search",
            "rago_flat_workspace_bytes", "rago_check", "rago_set_coarse_mode", "rago_profile_enable", "rago_profile_read",
            "rago_merge_results", "rago_kernel_launches", "rago_last_error")
@@ -47,6 +47,7 @@ def lib() -> ctypes.CDLL:
         vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
         L.rago_index_load.argtypes = [ctypes.POINTER(vp), vp, ctypes.c_int, vp, vp, vp, vp, i64, i32, i32, i32,
                                       ctypes.c_int, vp]
+        L.rago_index_load_pq4.argtypes = L.rago_index_load.argtypes
         L.rago_index_free.argtypes = [vp]
         L.rago_search_workspace_bytes.argtypes = [vp, i32, i32, i32, ctypes.POINTER(sz)]
         L.rago_host_staging_bytes.argtypes = [vp, i32, i32, ctypes.POINTER(sz)]
@@ -95,13 +96,20 @@ class Index:
         metric = {"l2": RAGO_L2, "ip": RAGO_IP}.get(metric, metric)
         dtype = RAGO_BF16 if centroids.dtype == torch.bfloat16 else RAGO_F32
         nlist, d = centroids.shape
-        M = codebooks.shape[0]
         N = codes.shape[0]
         self._keep = (centroids, codebooks, codes, list_offsets, ids)
-        self.nlist, self.d, self.M, self.N, self.metric = nlist, d, M, N, metric
         self._h = ctypes.c_void_p()
-        _check(lib().rago_index_load(ctypes.byref(self._h), _ptr(centroids), dtype, _ptr(codebooks), _ptr(codes),
-                                     _ptr(list_offsets), _ptr(ids), N, d, nlist, M, metric, _stream()))
+        if codebooks.shape[1] == 16:  # 4-bit codes, two per byte: rago_index_load_pq4
+            M4 = codebooks.shape[0]
+            M = M4 // 2
+            _check(lib().rago_index_load_pq4(ctypes.byref(self._h), _ptr(centroids), dtype, _ptr(codebooks),
+                                             _ptr(codes), _ptr(list_offsets), _ptr(ids), N, d, nlist, M4, metric,
+                                             _stream()))
+        else:
+            M = codebooks.shape[0]
+            _check(lib().rago_index_load(ctypes.byref(self._h), _ptr(centroids), dtype, _ptr(codebooks), _ptr(codes),
+                                         _ptr(list_offsets), _ptr(ids), N, d, nlist, M, metric, _stream()))
+        self.nlist, self.d, self.M, self.N, self.metric = nlist, d, M, N, metric
         self._ws = None
 
     def close(self):
@@ -191,6 +199,13 @@ class Index:
 
 def rago_index_load(centroids, codebooks, codes, list_offsets, ids, metric) -> Index:
     return Index(centroids, codebooks, codes, list_offsets, ids, metric)
+
+
+def rago_index_load_pq4(centroids, pq4_codebooks, packed_codes, list_offsets, ids, metric) -> Index:
+    """pq4_codebooks [M4, 16, d / M4], packed_codes uint8 [N, M4 / 2] (low nibble = even sub-space)."""
+    if pq4_codebooks.shape[1] != 16:
+        raise ValueError("4-bit codebooks have 16 codewords per sub-space")
+    return Index(centroids, pq4_codebooks, packed_codes, list_offsets, ids, metric)
 
 
 def rago_flat_workspace_bytes(N: int, d: int, nq: int, k: int) -> int:
