@@ -681,11 +681,11 @@ static int stages_for(int d) {
 static const Variant kVariants[] = {
     RAGO_VARIANT(4, 4, 1, 16, 2),   // M = 16
     RAGO_VARIANT(8, 8, 1, 10, 3),   // M = 32
-    RAGO_VARIANT(12, 4, 1, 12, 1),  // M = 48
+    RAGO_VARIANT(12, 4, 1, 8, 2),   // M = 48
     RAGO_VARIANT(8, 8, 2, 12, 4),   // M = 64
     RAGO_VARIANT(20, 4, 1, 8, 1),   // M = 80
     RAGO_VARIANT(24, 8, 1, 12, 1),  // M = 96
-    RAGO_VARIANT(8, 8, 4, 12, 2),   // M = 128
+    RAGO_VARIANT(8, 8, 4, 12, 3),   // M = 128
 };
 
 static const Variant* find_variant(int M) {
