@@ -101,47 +101,81 @@ __global__ void __launch_bounds__(256) coarse_scores_kernel(const float* __restr
 }
 
 // ---- score matrix for tiny batches (the latency-bound iterative-retrieval shape) -------------------
-// Up to CS_MAXQ queries sit in shared memory; one warp per centroid streams the centroid row once
-// (16-byte loads) and keeps one partial sum per query, so the centroid table is read exactly once per
-// batch however few queries there are.
+// For up to CS_MAXQ queries: a warp streams CS_CPW centroid rows at a time (16-byte loads) and keeps one partial sum
+// per (row, query), so the centroid table is read exactly once per batch however few queries there are.
 constexpr int CS_MAXQ = 16;
+constexpr int CS_CPW = 4;  // centroids per warp per step
 template <bool BF16>
 __global__ void __launch_bounds__(256) coarse_small_kernel(const float* __restrict__ Q, const void* __restrict__ C,
                                                            const float* __restrict__ cnorm, int nq, int nlist, int d,
                                                            int metric, float* __restrict__ scores) {
-    extern __shared__ __align__(16) float qs[];  // [nq][d]
+    extern __shared__ __align__(16) float qs[];  // [nq][d], rounded to bf16 values for a bf16 index
     for (int i = threadIdx.x; i < nq * d; i += blockDim.x) qs[i] = BF16 ? round_bf16(Q[i]) : Q[i];
     __syncthreads();
     const int lane = threadIdx.x & 31;
     const int warps = (gridDim.x * blockDim.x) >> 5;
-    for (int c = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; c < nlist; c += warps) {
-        float acc[CS_MAXQ];
+    // A warp takes CS_CPW consecutive centroids at a time: each query value read from shared memory serves CS_CPW
+    // rows, and the next slice of the rows is already in flight while the current one is multiplied.
+    for (int c0 = ((blockIdx.x * blockDim.x + threadIdx.x) >> 5) * CS_CPW; c0 < nlist; c0 += warps * CS_CPW) {
+        float acc[CS_CPW][CS_MAXQ];
+        float cn[CS_CPW];
 #pragma unroll
-        for (int qi = 0; qi < CS_MAXQ; ++qi) acc[qi] = 0.f;
-        for (int j0 = lane * 4; j0 < d; j0 += 128) {
-            float4 cv;
-            if (BF16) {
-                const uint2 raw = *reinterpret_cast<const uint2*>(static_cast<const __nv_bfloat16*>(C) + (size_t)c * d + j0);
-                cv.x = __uint_as_float(raw.x << 16); cv.y = __uint_as_float(raw.x & 0xFFFF0000u);
-                cv.z = __uint_as_float(raw.y << 16); cv.w = __uint_as_float(raw.y & 0xFFFF0000u);
-            } else {
-                cv = *reinterpret_cast<const float4*>(static_cast<const float*>(C) + (size_t)c * d + j0);
+        for (int u = 0; u < CS_CPW; ++u) {
+            cn[u] = metric == RAGO_L2 ? __ldg(cnorm + (c0 + u < nlist ? c0 + u : nlist - 1)) : 0.f;
+#pragma unroll
+            for (int qi = 0; qi < CS_MAXQ; ++qi) acc[u][qi] = 0.f;
+        }
+        auto load_rows = [&](float4 (&cv)[CS_CPW], int j0) {
+#pragma unroll
+            for (int u = 0; u < CS_CPW; ++u) {
+                const int c = c0 + u < nlist ? c0 + u : nlist - 1;  // rows past the end repeat the last one, unused
+                if (BF16) {
+                    const uint2 raw = *reinterpret_cast<const uint2*>(static_cast<const __nv_bfloat16*>(C) + (size_t)c * d + j0);
+                    cv[u].x = __uint_as_float(raw.x << 16); cv[u].y = __uint_as_float(raw.x & 0xFFFF0000u);
+                    cv[u].z = __uint_as_float(raw.y << 16); cv[u].w = __uint_as_float(raw.y & 0xFFFF0000u);
+                } else {
+                    cv[u] = *reinterpret_cast<const float4*>(static_cast<const float*>(C) + (size_t)c * d + j0);
+                }
             }
+        };
+        float4 cv[CS_CPW], nx[CS_CPW];
+        if (lane * 4 < d) load_rows(cv, lane * 4);
+        for (int j0 = lane * 4; j0 < d; j0 += 128) {
+            const bool more = j0 + 128 < d;
+            if (more) load_rows(nx, j0 + 128);
 #pragma unroll
             for (int qi = 0; qi < CS_MAXQ; ++qi) {
                 if (qi < nq) {  // uniform
                     const float4 qv = *reinterpret_cast<const float4*>(qs + qi * d + j0);
-                    acc[qi] = fmaf(qv.x, cv.x, fmaf(qv.y, cv.y, fmaf(qv.z, cv.z, fmaf(qv.w, cv.w, acc[qi]))));
+#pragma unroll
+                    for (int u = 0; u < CS_CPW; ++u)
+                        acc[u][qi] = fmaf(qv.x, cv[u].x, fmaf(qv.y, cv[u].y, fmaf(qv.z, cv[u].z, fmaf(qv.w, cv[u].w, acc[u][qi]))));
                 }
             }
-        }
+            if (more) {
 #pragma unroll
-        for (int qi = 0; qi < CS_MAXQ; ++qi) {
-            if (qi < nq) {
-                float v = acc[qi];
-                for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-                if (lane == 0) scores[(size_t)qi * nlist + c] = metric == RAGO_L2 ? fmaf(-2.f, v, cnorm[c]) : -v;
+                for (int u = 0; u < CS_CPW; ++u) cv[u] = nx[u];
             }
+        }
+        // Sum over the lanes, all CS_MAXQ queries of a row at once: at each halving a lane keeps the half of its
+        // values that its lane-number bit selects and hands over the other half, so 16 + 1 exchanges do the work of
+        // 16 x 5, and the total of query 8 b4 + 4 b3 + 2 b2 + b1 (lane bits) ends in the lanes with bit 0 clear.
+#pragma unroll
+        for (int u = 0; u < CS_CPW; ++u) {
+#pragma unroll
+            for (int half = CS_MAXQ / 2, o = 16; half >= 1; half >>= 1, o >>= 1) {
+                const bool upper = (lane & o) != 0;
+#pragma unroll
+                for (int i = 0; i < half; ++i) {
+                    const float keep = upper ? acc[u][i + half] : acc[u][i];
+                    const float send = upper ? acc[u][i] : acc[u][i + half];
+                    acc[u][i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+                }
+            }
+            const float v = acc[u][0] + __shfl_xor_sync(0xffffffffu, acc[u][0], 1);
+            const int qi = (lane >> 1) & 15;  // bits 4..1 of the lane, most significant first: 8 b4 + 4 b3 + 2 b2 + b1
+            if ((lane & 1) == 0 && qi < nq && c0 + u < nlist)
+                scores[(size_t)qi * nlist + c0 + u] = metric == RAGO_L2 ? fmaf(-2.f, v, cn[u]) : -v;
         }
     }
 }
@@ -149,8 +183,8 @@ __global__ void __launch_bounds__(256) coarse_small_kernel(const float* __restri
 cudaError_t launch_coarse_scores(const IndexImpl* ix, const float* queries, int nq, float* scores, cudaStream_t s) {
     const size_t qbytes = (size_t)nq * ix->d * 4;
     if (nq <= CS_MAXQ && qbytes <= 48 * 1024) {
-        const int want = (ix->nlist + 7) / 8;
-        const int blocks = want < ix->num_sms * 8 ? want : ix->num_sms * 8;
+        const int want = (ix->nlist + 8 * CS_CPW - 1) / (8 * CS_CPW);  // 8 warps per CTA, CS_CPW rows per warp step
+        const int blocks = want < ix->num_sms * 2 ? want : ix->num_sms * 2;
         if (ix->coarse_bf16)
             coarse_small_kernel<true><<<blocks, 256, qbytes, s>>>(queries, ix->centroids, ix->cnorm, nq, ix->nlist, ix->d,
                                                                    ix->metric, scores);
@@ -181,7 +215,10 @@ constexpr int SEL_MAX_SPLIT = 512;  // candidate lists per query the kernel can 
 // lie at or below it; only those go to shared memory, are sorted, re-scored exactly and sorted again.
 // SEL_THREADS threads per query keep up to SEL_REG item scores each in registers: a big CTA for tiny
 // batches (latency), a small one when there are enough queries to fill the GPU.
-template <bool BF16, int SEL_THREADS, int SEL_REG>
+// FROM_SCORES: the items are a row of the score matrix (else the candidate lists the GEMM left).  The two sources
+// are separate instantiations because the kernel body runs once per CTA, largely unrolled: its size is what a
+// small batch pays for, in instruction fetches.
+template <bool BF16, int SEL_THREADS, int SEL_REG, bool FROM_SCORES>
 __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
     const float* __restrict__ Q, const void* __restrict__ C, const float* __restrict__ scores,
     const unsigned long long* __restrict__ cand, const int32_t* __restrict__ cand_cnt, int nsplit, int cap, int nlist,
@@ -189,28 +226,32 @@ __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
     float* __restrict__ probe_bias) {
     __shared__ unsigned long long keys[TOPK_CAP];
     __shared__ unsigned long long keys2[MAX_K + PROBE_GUARD];
-    __shared__ uint32_t red[2][SEL_THREADS / 32];
     __shared__ int pre[SEL_MAX_SPLIT + 1];  // candidate path: exclusive prefix of the lists' counts
+    __shared__ uint32_t hist[256];           // items per slice of the score range
+    __shared__ uint32_t s_mn, s_mx, s_nv;    // CTA-wide minimum, maximum, count of the ordered score bits
+    __shared__ uint32_t s_round[3];          // bisection counts, one word per round in rotation
+    __shared__ uint32_t s_bin[3];            // slice holding the cut, items of the range up to and including / before it
     __shared__ int cnt;
     const int q = blockIdx.x, tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
     auto sync = [] { __syncthreads(); };
     int nsel = nprobe + PROBE_GUARD;
     if (nsel > nlist) nsel = nlist;
-    if (tid == 0) cnt = 0;
-    const float* srow = scores ? scores + (size_t)q * nlist : nullptr;
-    if (!scores) {  // the valid entries of the query's lists, numbered consecutively
+    if (tid == 0) { cnt = 0; s_mn = 0xFFFFFFFFu; s_mx = 0u; s_nv = 0u; s_round[0] = s_round[1] = s_round[2] = 0u; }
+    for (int i = tid; i < 256; i += SEL_THREADS) hist[i] = 0u;
+    const float* srow = FROM_SCORES ? scores + (size_t)q * nlist : nullptr;
+    if (!FROM_SCORES) {  // the valid entries of the query's lists, numbered consecutively
         if (tid == 0) {
             int acc = 0;
             for (int sp = 0; sp < nsplit; ++sp) { pre[sp] = acc; acc += cand_cnt[(size_t)q * nsplit + sp]; }
             pre[nsplit] = acc;
         }
-        __syncthreads();
     }
-    const int nitems = scores ? nlist : pre[nsplit];
+    __syncthreads();
+    const int nitems = FROM_SCORES ? nlist : pre[nsplit];
     // key of item l
     auto item = [&](int l) -> unsigned long long {
-        if (scores) return make_key(srow[l], (uint32_t)l);
+        if constexpr (FROM_SCORES) return make_key(srow[l], (uint32_t)l);
         int lo_s = 0, hi_s = nsplit;  // pre[lo_s] <= l < pre[hi_s]
         while (hi_s - lo_s > 1) {
             const int mid_s = (lo_s + hi_s) >> 1;
@@ -244,22 +285,64 @@ __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
     mn = __reduce_min_sync(0xffffffffu, mn);
     mx = __reduce_max_sync(0xffffffffu, mx);
     nvalid = __reduce_add_sync(0xffffffffu, nvalid);
-    if (lane == 0) { red[0][warp] = mn; red[1][warp] = mx; }
+    if (lane == 0) { atomicMin(&s_mn, mn); atomicMax(&s_mx, mx); atomicAdd(&s_nv, nvalid); }
     __syncthreads();
-    mn = red[0][0]; mx = red[1][0];
-    for (int w = 1; w < SEL_THREADS / 32; ++w) { mn = red[0][w] < mn ? red[0][w] : mn; mx = red[1][w] > mx ? red[1][w] : mx; }
-    __syncthreads();
-    if (lane == 0) red[0][warp] = nvalid;
-    __syncthreads();
-    nvalid = 0;
-    for (int w = 0; w < SEL_THREADS / 32; ++w) nvalid += red[0][w];
-    __syncthreads();
+    mn = s_mn; mx = s_mx; nvalid = s_nv;
     if ((int)nvalid < nsel) nsel = (int)nvalid;  // cannot happen for a well-formed candidate set; stay safe
-    // bisection: #(score <= lo) < nsel <= #(score <= hi)
-    long long lo = (long long)mn - 1, hi = mx;
-    uint32_t c_hi = nvalid;
     int slack = nsel / 4 > 8 ? nsel / 4 : 8;
     if (nsel + slack > TOPK_CAP) slack = TOPK_CAP - nsel;
+    // Narrow the range first: 256 equal slices of (lo, hi] (in ordered score bits), one shared-memory count each;
+    // the slice that holds the nsel-th smallest item becomes the new range.  Two passes usually leave at most
+    // nsel + slack items at or below hi; ties and odd distributions are finished by the bisection below.
+    long long lo = (long long)mn - 1, hi = mx;  // invariant: #(score <= lo) < nsel <= #(score <= hi)
+    uint32_t c_hi = nvalid, below = 0;          // below = #(score <= lo)
+    for (int pass = 0; pass < 3 && hi - lo > 1 && c_hi > (uint32_t)(nsel + slack); ++pass) {  // uniform
+        const uint32_t first = (uint32_t)(lo + 1), range = (uint32_t)(hi - lo - 1);
+        const int shift = range < 256u ? 0 : 24 - __clz(range);  // (range >> shift) < 256
+        if (in_regs) {
+#pragma unroll
+            for (int j = 0; j < SEL_REG; ++j)  // hi <= mx < the empty-slot pattern
+                if (mine[j] >= first && mine[j] <= (uint32_t)hi) atomicAdd(&hist[(mine[j] - first) >> shift], 1u);
+        } else {
+            for (int l = tid; l < nitems; l += SEL_THREADS) {
+                const unsigned long long k = item(l);
+                const uint32_t o = (uint32_t)(k >> 32);
+                if (k != KEY_MAX && o >= first && o <= (uint32_t)hi) atomicAdd(&hist[(o - first) >> shift], 1u);
+            }
+        }
+        __syncthreads();
+        if (warp == 0) {  // lane i owns slices 8 i .. 8 i + 7
+            const uint32_t want = (uint32_t)nsel - below;  // rank of the cut inside the range, >= 1
+            uint32_t h[8], tot = 0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) { h[j] = hist[lane * 8 + j]; tot += h[j]; }
+            uint32_t before = tot;  // inclusive scan over the lanes, then made exclusive
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t v = __shfl_up_sync(0xffffffffu, before, o);
+                if (lane >= o) before += v;
+            }
+            before -= tot;
+            if (before < want && before + tot >= want) {  // exactly one lane
+                uint32_t c = before, prev = before;
+                int bsel = 0;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    if (c < want) { bsel = j; prev = c; c += h[j]; }
+                }
+                s_bin[0] = (uint32_t)(lane * 8 + bsel); s_bin[1] = c; s_bin[2] = prev;
+            }
+        }
+        __syncthreads();
+        const uint32_t bsel = s_bin[0];
+        const long long top = (long long)first + (((long long)bsel + 1) << shift) - 1;
+        c_hi = below + s_bin[1];
+        below += s_bin[2];
+        hi = top < hi ? top : hi;
+        lo = (long long)first + ((long long)bsel << shift) - 1;
+        for (int i = tid; i < 256; i += SEL_THREADS) hist[i] = 0u;
+        __syncthreads();
+    }
+    // bisection inside the slice: #(score <= lo) < nsel <= #(score <= hi)
     int round = 0;
     while (hi - lo > 1 && c_hi > (uint32_t)(nsel + slack)) {  // uniform
         const uint32_t mid = (uint32_t)(lo + (hi - lo) / 2);
@@ -274,10 +357,11 @@ __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
             }
         }
         c = __reduce_add_sync(0xffffffffu, c);
-        if (lane == 0) red[round & 1][warp] = c;
+        const int slot = round % 3;
+        if (lane == 0 && c) atomicAdd(&s_round[slot], c);
+        if (tid == 0) s_round[(slot + 1) % 3] = 0u;  // next round's word; its last readers passed two barriers ago
         __syncthreads();
-        c = 0;
-        for (int w = 0; w < SEL_THREADS / 32; ++w) c += red[round & 1][w];
+        c = s_round[slot];
         if (c < (uint32_t)nsel) lo = mid; else { hi = mid; c_hi = c; }
         ++round;
     }
@@ -287,7 +371,10 @@ __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
 #pragma unroll
         for (int j = 0; j < SEL_REG; ++j) {
             const bool take = mine[j] != 0xFFFFFFFFu && mine[j] <= T;
-            warp_push(keys, &cnt, take, take ? item(tid + j * SEL_THREADS) : KEY_MAX);
+            unsigned long long key = KEY_MAX;
+            if (FROM_SCORES) key = ((unsigned long long)mine[j] << 32) | (uint32_t)(tid + j * SEL_THREADS);
+            else if (take) key = item(tid + j * SEL_THREADS);
+            warp_push(keys, &cnt, take, key);
         }
     } else {
         for (int l0 = 0; l0 < nitems; l0 += SEL_THREADS) {
@@ -297,7 +384,7 @@ __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
         }
     }
     __syncthreads();
-    const int kept = block_select(keys, &cnt, nsel, tid, SEL_THREADS, sync);
+    const int kept = block_select_short(keys, &cnt, nsel, tid, SEL_THREADS, sync);
     // exact re-score of the survivors, one warp per candidate
     const float* qrow = Q + (size_t)q * d;
     for (int i = warp; i < kept; i += SEL_THREADS / 32) {
@@ -325,11 +412,20 @@ __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
         if (lane == 0) keys2[i] = make_key(metric == RAGO_L2 ? acc : -acc, l);
     }
     __syncthreads();
-    for (int i = tid; i < TOPK_CAP; i += SEL_THREADS) keys[i] = i < kept ? keys2[i] : KEY_MAX;
-    __syncthreads();
     int n2 = 2;
     while (n2 < kept) n2 <<= 1;
-    block_bitonic_sort(keys, n2, tid, SEL_THREADS, sync);
+    if (kept <= WARP_SORT_MAX) {  // the usual case: one warp orders the few survivors
+        if (warp == 0) {
+            for (int i = lane; i < n2; i += 32) keys[i] = i < kept ? keys2[i] : KEY_MAX;
+            __syncwarp();
+            warp_bitonic_sort(keys, n2, lane);
+        }
+        __syncthreads();
+    } else {
+        for (int i = tid; i < n2; i += SEL_THREADS) keys[i] = i < kept ? keys2[i] : KEY_MAX;
+        __syncthreads();
+        block_bitonic_sort(keys, n2, tid, SEL_THREADS, sync);
+    }
     for (int i = tid; i < nprobe; i += SEL_THREADS) {
         const unsigned long long key = keys[i];
         const float sc = orderable_f32((uint32_t)(key >> 32));
@@ -353,18 +449,29 @@ __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
     }
 }
 
+template <bool BF16, int THREADS, int REG>
+static void launch_select_source(const IndexImpl* ix, const float* queries, const float* scores,
+                                 const unsigned long long* cand, const int32_t* cand_cnt, int nsplit, int cap, int nq,
+                                 int nprobe, int32_t* probe_list, float* probe_term, float* probe_bias, cudaStream_t s) {
+    if (scores)
+        select_probes_kernel<BF16, THREADS, REG, true><<<nq, THREADS, 0, s>>>(
+            queries, ix->centroids, scores, cand, cand_cnt, nsplit, cap, ix->nlist, ix->d, ix->metric, nprobe, probe_list,
+            probe_term, probe_bias);
+    else
+        select_probes_kernel<BF16, THREADS, REG, false><<<nq, THREADS, 0, s>>>(
+            queries, ix->centroids, scores, cand, cand_cnt, nsplit, cap, ix->nlist, ix->d, ix->metric, nprobe, probe_list,
+            probe_term, probe_bias);
+}
 template <int THREADS, int REG>
 static void launch_select_shape(const IndexImpl* ix, const float* queries, const float* scores,
                                 const unsigned long long* cand, const int32_t* cand_cnt, int nsplit, int cap, int nq,
                                 int nprobe, int32_t* probe_list, float* probe_term, float* probe_bias, cudaStream_t s) {
     if (ix->coarse_bf16)
-        select_probes_kernel<true, THREADS, REG><<<nq, THREADS, 0, s>>>(queries, ix->centroids, scores, cand, cand_cnt,
-                                                                         nsplit, cap, ix->nlist, ix->d, ix->metric, nprobe,
-                                                                         probe_list, probe_term, probe_bias);
+        launch_select_source<true, THREADS, REG>(ix, queries, scores, cand, cand_cnt, nsplit, cap, nq, nprobe, probe_list,
+                                                 probe_term, probe_bias, s);
     else
-        select_probes_kernel<false, THREADS, REG><<<nq, THREADS, 0, s>>>(queries, ix->centroids, scores, cand, cand_cnt,
-                                                                          nsplit, cap, ix->nlist, ix->d, ix->metric, nprobe,
-                                                                          probe_list, probe_term, probe_bias);
+        launch_select_source<false, THREADS, REG>(ix, queries, scores, cand, cand_cnt, nsplit, cap, nq, nprobe, probe_list,
+                                                  probe_term, probe_bias, s);
 }
 static cudaError_t launch_select_any(const IndexImpl* ix, const float* queries, const float* scores,
                                      const unsigned long long* cand, const int32_t* cand_cnt, int nsplit, int cap, int nq,

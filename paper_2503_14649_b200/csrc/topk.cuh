@@ -51,6 +51,61 @@ __device__ __forceinline__ int block_select(unsigned long long* keys, int* cnt, 
     return kept;
 }
 
+// Ascending sort of n2 <= 64 keys (n2 a power of two) in shared memory by ONE warp, in registers: lane L holds
+// elements L and L + 32 and the bitonic network's exchanges are shuffles, so no step waits on shared memory.
+__device__ __forceinline__ unsigned long long shfl_xor_u64(unsigned long long v, int m) {
+    const uint32_t lo = __shfl_xor_sync(0xffffffffu, (uint32_t)v, m);
+    const uint32_t hi = __shfl_xor_sync(0xffffffffu, (uint32_t)(v >> 32), m);
+    return ((unsigned long long)hi << 32) | lo;
+}
+__device__ __forceinline__ void warp_bitonic_sort(unsigned long long* keys, int n2, int lane) {
+    unsigned long long k0 = lane < n2 ? keys[lane] : KEY_MAX;
+    unsigned long long k1 = lane + 32 < n2 ? keys[lane + 32] : KEY_MAX;
+    const int top = n2 > 32 ? 64 : 32;  // padding keys are maximal, so sorting more slots than n2 is harmless
+    for (int size = 2; size <= top; size <<= 1) {
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            if (stride == 32) {  // size 64: element L against element L + 32, ascending
+                if (k0 > k1) { const unsigned long long t = k0; k0 = k1; k1 = t; }
+            } else {
+                const bool lower = (lane & stride) == 0;
+                const unsigned long long o0 = shfl_xor_u64(k0, stride);
+                const bool min0 = lower == ((lane & size) == 0);
+                k0 = (min0 == (k0 < o0)) ? k0 : o0;
+                if (top == 64) {
+                    const unsigned long long o1 = shfl_xor_u64(k1, stride);
+                    const bool min1 = lower == (((lane + 32) & size) == 0);
+                    k1 = (min1 == (k1 < o1)) ? k1 : o1;
+                }
+            }
+        }
+    }
+    if (lane < n2) keys[lane] = k0;
+    if (lane + 32 < n2) keys[lane + 32] = k1;
+    __syncwarp();
+}
+constexpr int WARP_SORT_MAX = 64;
+
+// block_select for short buffers: when at most WARP_SORT_MAX keys are buffered, warp 0 sorts them alone while the
+// other warps wait at one barrier.  Same contract as block_select.
+template <class Sync>
+__device__ __forceinline__ int block_select_short(unsigned long long* keys, int* cnt, int k, int tid, int nthreads,
+                                                  Sync sync, int cap = TOPK_CAP) {
+    int n = *cnt;
+    if (n > cap) n = cap;
+    if (n > WARP_SORT_MAX) return block_select(keys, cnt, k, tid, nthreads, sync, cap);
+    const int kept = n < k ? n : k;
+    if (tid < 32) {
+        int n2 = 2;
+        while (n2 < n) n2 <<= 1;
+        for (int i = n + tid; i < n2; i += 32) keys[i] = KEY_MAX;
+        __syncwarp();
+        warp_bitonic_sort(keys, n2, tid);
+        if (tid == 0) *cnt = kept;
+    }
+    sync();
+    return kept;
+}
+
 // Append `key` for the lanes with pred set; one shared atomic per warp.  Whole warp must call.
 __device__ __forceinline__ void warp_push(unsigned long long* keys, int* cnt, bool pred, unsigned long long key,
                                           int cap = TOPK_CAP) {
