@@ -42,6 +42,8 @@ struct Layout {
     size_t err, probe_list, probe_term, probe_bias, scores, pair_tiles, work_prefix, qthresh, slot_cnt, slot_keys, total;
     size_t qparts, cand, cand_cnt;  // tensor-core coarse step: query parts, candidate lists and their counts
     size_t pilot_scores, row_tau;   // pilot pass: scores of the sampled lists, per-query starting thresholds
+    size_t lut_img, lut_inv;        // small batches: lookup tables built ahead of the scan, and their scales
+    int prebuilt;
     int pilot_cols;                 // 0: no pilot pass
     size_t nslots;
     int tc, tc_mode, tc_cap, tc_mg, tc_nsplit;  // coarse plan for this (nq, nprobe)
@@ -99,6 +101,11 @@ static Layout make_layout(const IndexImpl* ix, int nq, int nprobe, int k) {
     L.qthresh = take((size_t)nq * 8);
     L.slot_cnt = take(L.nslots * 4);
     L.slot_keys = take(L.nslots * (size_t)k * 8);
+    L.prebuilt = nq <= PREBUILT_MAX_NQ ? 1 : 0;
+    // reserved for larger batches too, so that a workspace sized for nq queries also serves fewer
+    const size_t nlut = nq < PREBUILT_MAX_NQ ? nq : PREBUILT_MAX_NQ;
+    L.lut_img = take(nlut * ix->plan.lut_bytes);
+    L.lut_inv = take(nlut * 4);
     L.total = o;
     return L;
 }
@@ -244,6 +251,7 @@ rago_status rago_index_load(rago_index** out, const void* coarse_centroids, rago
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ix->num_sms, cudaDevAttrMultiProcessorCount, ix->device);
     if (e == cudaSuccess) e = cudaMalloc(&ix->cnorm, (size_t)nlist * 4);
     if (e == cudaSuccess) e = cudaMalloc(&ix->cbT, (size_t)KSUB * d * 4);
+    if (e == cudaSuccess) e = cudaMalloc(&ix->cwmax, (size_t)M * 4);
     if (e == cudaSuccess && metric == RAGO_L2 && N > 0) e = cudaMalloc(&ix->vterm, ((size_t)N + 4) * 4);  // + slack: tiles copy whole 16-byte groups
     if (e != cudaSuccess) {
         rago_status st = e == cudaErrorMemoryAllocation ? fail(RAGO_ENOMEM, "device allocation failed")
@@ -255,6 +263,7 @@ rago_status rago_index_load(rago_index** out, const void* coarse_centroids, rago
     if (e == cudaSuccess) { ix->ev_valid = 1; e = scan_plan(ix, &ix->plan); }
     if (e == cudaSuccess) e = launch_centroid_norms(coarse_centroids, ix->coarse_bf16, nlist, d, ix->cnorm, s);
     if (e == cudaSuccess) e = launch_transpose_codebook(pq_codebooks, M, ix->dsub, ix->cbT, s);
+    if (e == cudaSuccess) e = launch_codeword_norms(pq_codebooks, M, ix->dsub, ix->cwmax, s);
     if (e == cudaSuccess && ix->vterm) e = launch_vector_terms(ix, ix->vterm, s);
     // tensor-core coarse operand: the centroids as stacked bf16 parts, and their tensor map
     if (e == cudaSuccess && d % 8 == 0) {
@@ -292,6 +301,7 @@ rago_status rago_index_free(rago_index* index) {
     cudaDeviceSynchronize();
     if (ix->cnorm) cudaFree(ix->cnorm);
     if (ix->cbT) cudaFree(ix->cbT);
+    if (ix->cwmax) cudaFree(ix->cwmax);
     if (ix->vterm) cudaFree(ix->vterm);
     if (ix->cparts) cudaFree(ix->cparts);
     if (ix->ev_valid)
@@ -371,12 +381,15 @@ rago_status rago_search(const rago_index* index, const float* queries, int32_t n
     int32_t* slot_cnt = reinterpret_cast<int32_t*>(ws + L.slot_cnt);
     unsigned long long* slot_keys = reinterpret_cast<unsigned long long*>(ws + L.slot_keys);
 
+    // small batches: the lookup tables are built ahead of the scan, by CTAs of the planning launch
+    uint8_t* lut_img = L.prebuilt ? ws + L.lut_img : nullptr;
+    float* lut_inv = L.prebuilt ? reinterpret_cast<float*>(ws + L.lut_inv) : nullptr;
     e = launch_plan_work(ix, probe_list, npairs, ix->plan.tile_vecs, reinterpret_cast<int32_t*>(ws + L.pair_tiles),
-                         work_prefix, qthresh, nq, slot_cnt, (int)L.nslots, s);
+                         work_prefix, qthresh, nq, slot_cnt, (int)L.nslots, queries, lut_img, lut_inv, s);
     if (e != cudaSuccess) return cuda_fail(e, "work planning");
     record(mix, 3, s);
     e = launch_scan(ix, ix->plan, queries, probe_list, probe_term, work_prefix, nq, nprobe, k, qthresh, slot_cnt,
-                    slot_keys, reinterpret_cast<uint32_t*>(ws + L.err), s);
+                    slot_keys, reinterpret_cast<uint32_t*>(ws + L.err), lut_img, lut_inv, s);
     if (e != cudaSuccess) return cuda_fail(e, "scan kernel");
     record(mix, 4, s);
     e = launch_merge(ix, work_prefix, nq, nprobe, k, ix->plan.ctas, slot_cnt, slot_keys, qthresh, out_ids, out_dists, s);

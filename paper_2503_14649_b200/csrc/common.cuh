@@ -24,7 +24,13 @@ struct ScanPlan {
     int stages;        // tiles in flight per CTA
     int ctas;          // persistent CTAs (one per SM)
     size_t smem_bytes;
+    // shared-memory image of a query's lookup table, as the scan variant of this index lays it out
+    int lut_bytes, lut_banked, lut_copies, lut_copy_off, lut_stride;
 };
+
+// Batches of at most this many queries get their lookup tables from a kernel of their own, spread over the whole
+// GPU, instead of every scan CTA building the table of each query it meets.
+constexpr int PREBUILT_MAX_NQ = 32;
 
 // Index handle.  Borrowed pointers first, then what the library owns.
 struct IndexImpl {
@@ -40,6 +46,7 @@ struct IndexImpl {
     float* cnorm;  // [nlist] squared centroid norms (L2 coarse ranking)
     float* cbT;    // [256][M][dsub] codebook with the codeword index outermost
     float* vterm;  // [N] per-vector term of the L2 expansion (null for inner product)
+    float* cwmax;  // [M] largest codeword norm of every sub-space (bounds a table entry without building the table)
     void* cparts;  // bf16 [parts][nlist][d]: the centroids as a sum of bf16 parts (fp32 index); null for a bf16 index
     int cparts_n;  // parts of the tensor-core coarse operand: 3 (fp32 index) or 1 (bf16 index, borrowed array)
     int tc_ok;     // tensor-core coarse path available (tensor map encoded)
@@ -205,11 +212,15 @@ cudaError_t launch_vector_terms(const IndexImpl* ix, float* vterm, cudaStream_t 
 cudaError_t launch_transpose_codebook(const float* cb, int M, int dsub, float* cbT, cudaStream_t s);
 cudaError_t launch_plan_work(const IndexImpl* ix, const int32_t* probe_list, int npairs, int tile_vecs,
                              int32_t* pair_tiles, int64_t* work_prefix, unsigned long long* qthresh, int nq,
-                             int32_t* slot_cnt, int nslots, cudaStream_t s);
+                             int32_t* slot_cnt, int nslots, const float* queries, uint8_t* lut_img, float* lut_inv,
+                             cudaStream_t s);
 cudaError_t launch_scan(const IndexImpl* ix, const ScanPlan& plan, const float* queries, const int32_t* probe_list,
                         const float* probe_term, const int64_t* work_prefix, int nq, int nprobe, int k,
                         unsigned long long* qthresh, int32_t* slot_cnt, unsigned long long* slot_keys,
-                        uint32_t* err_word, cudaStream_t s);
+                        uint32_t* err_word, const uint8_t* lut_img, const float* lut_inv, cudaStream_t s);
+cudaError_t launch_codeword_norms(const float* codebooks, int M, int dsub, float* cwmax, cudaStream_t s);
+cudaError_t launch_build_tables(const IndexImpl* ix, const float* queries, int nq, uint8_t* lut_img, float* lut_inv,
+                                cudaStream_t s);
 // merge.cu
 cudaError_t launch_merge(const IndexImpl* ix, const int64_t* work_prefix, int nq, int nprobe, int k, int ctas,
                          const int32_t* slot_cnt, const unsigned long long* slot_keys, const unsigned long long* qthresh,

@@ -50,6 +50,7 @@
 namespace rago {
 
 constexpr int MAX_STAGES = 4;
+constexpr int CUT_PASSES = 3;               // range-narrowing passes of a buffer cut before it falls back to bisection
 constexpr int SMEM_OPTIN = 227 * 1024;          // dynamic shared memory asked for (the sm_100 per-block limit)
 constexpr uint32_t SMEM_BASE_EXPECTED = 1024;   // shared-window address of dynamic shared memory when the kernel has no static part
 constexpr int CTRL_BYTES = 1024;
@@ -79,6 +80,8 @@ struct ScanArgs {
     int32_t* slot_cnt;
     unsigned long long* slot_keys;
     uint32_t* err;
+    const uint8_t* lut_img;  // [nq][LUT_BYTES] tables built ahead of the scan (small batches), or null
+    const float* lut_inv;    // [nq] fp32 value of one integer unit of each such table
     int32_t npairs, nprobe, d, dsub, metric, k, stages;
     uint32_t dyn_bytes;
 };
@@ -507,11 +510,58 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
             mn = ctrl->redu[0][w] < mn ? ctrl->redu[0][w] : mn;
             mx = ctrl->redu[1][w] > mx ? ctrl->redu[1][w] : mx;
         }
-        csync();  // the minima / maxima have been read; redu is free for the counts
+        // All keys sit in registers now, so the buffer's memory is free until they are pushed back: its first words
+        // hold the slice counts of the passes below (one array per pass, cleared here).
+        uint32_t* hist = reinterpret_cast<uint32_t*>(keys);
+        for (int i = ctid; i < CUT_PASSES * 256; i += NCT) hist[i] = 0u;
+        csync();  // the minima / maxima have been read (redu is free for the counts), the slice counts are clear
         if (dead) return;
         long long lo = (long long)mn - 1, hi = mx;  // #(score <= lo) < k <= #(score <= hi)
-        uint32_t c_hi = (uint32_t)n;
+        uint32_t c_hi = (uint32_t)n, below = 0;     // below = #(score <= lo)
         const uint32_t want_max = (uint32_t)(k + (k >> 2) + 8);
+        // Narrow (lo, hi] by 256 equal slices per pass: the slice that holds the k-th smallest key becomes the new
+        // range (two barriers per pass).  What the passes leave undecided (ties, odd distributions) is bisected.
+        for (int pass = 0; pass < CUT_PASSES && hi - lo > 1 && c_hi > want_max; ++pass) {  // uniform across the CTA
+            uint32_t* h = hist + pass * 256;
+            const uint32_t first = (uint32_t)(lo + 1), range = (uint32_t)(hi - lo - 1);
+            const int shift = range < 256u ? 0 : 24 - __clz(range);  // (range >> shift) < 256
+#pragma unroll
+            for (int j = 0; j < KPT; ++j) {
+                const uint32_t o = (uint32_t)(mine[j] >> 32);
+                if (mine[j] != KEY_MAX && o >= first && o <= (uint32_t)hi) atomicAdd(&h[(o - first) >> shift], 1u);
+            }
+            csync();
+            if (dead) return;
+            if (warp == 0) {  // lane i owns slices 8 i .. 8 i + 7
+                const uint32_t want = (uint32_t)k - below;  // rank of the cut inside the range, >= 1
+                uint32_t hv[8], tot = 0;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) { hv[j] = h[lane * 8 + j]; tot += hv[j]; }
+                uint32_t before = tot;  // inclusive scan over the lanes, then made exclusive
+                for (int o = 1; o < 32; o <<= 1) {
+                    const uint32_t v = __shfl_up_sync(0xffffffffu, before, o);
+                    if (lane >= o) before += v;
+                }
+                before -= tot;
+                if (before < want && before + tot >= want) {  // exactly one lane
+                    uint32_t c = before, prev = before;
+                    int bsel = 0;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        if (c < want) { bsel = j; prev = c; c += hv[j]; }
+                    }
+                    ctrl->redu[1][0] = (uint32_t)(lane * 8 + bsel); ctrl->redu[1][1] = c; ctrl->redu[1][2] = prev;
+                }
+            }
+            csync();
+            if (dead) return;
+            const uint32_t bsel = ctrl->redu[1][0];
+            const long long top = (long long)first + (((long long)bsel + 1) << shift) - 1;
+            c_hi = below + ctrl->redu[1][1];
+            below += ctrl->redu[1][2];
+            hi = top < hi ? top : hi;
+            lo = (long long)first + ((long long)bsel << shift) - 1;
+        }
         int round = 0;
         while (hi - lo > 1 && c_hi > want_max) {  // uniform across the CTA
             const uint32_t mid = (uint32_t)(lo + (hi - lo) / 2);
@@ -565,6 +615,17 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
     // Table of a query: entry (j, m) = lut_scale * <q_m, codeword j of sub-space m>.
     auto begin_query = [&](int q) {
         cur_q = q;
+        if (a.lut_img != nullptr) {  // the table was built ahead of the scan: fetch its shared-memory image
+            const uint4* src = reinterpret_cast<const uint4*>(a.lut_img + (size_t)q * C::LUT_BYTES);
+            uint4* dst = reinterpret_cast<uint4*>(smem + (P.lut - base));
+#pragma unroll 4
+            for (int i = ctid; i < C::LUT_BYTES / 16; i += NCT) dst[i] = __ldg(src + i);
+            inv_scale = __ldg(a.lut_inv + q);
+            if (ctid == 0) ctrl->cnt = 0;
+            tau = *reinterpret_cast<volatile unsigned long long*>(&a.qthresh[q]);
+            csync();
+            return;
+        }
         const float* qrow = a.queries + (size_t)q * a.d;
         for (int j = ctid; j < a.d; j += NCT) rT[(j % a.dsub) * C::M + j / a.dsub] = lut_scale * qrow[j];
         if (ctid == 0) ctrl->cnt = 0;
@@ -666,6 +727,7 @@ struct Variant {
     void (*kernel)(const ScanArgs);
     int threads, tile_vecs;
     int (*stages_for)(int d);
+    int lut_bytes, lut_banked, lut_copies, lut_copy_off, lut_stride;
 };
 template <class C>
 static int stages_for(int d) {
@@ -675,7 +737,9 @@ static int stages_for(int d) {
 }
 #define RAGO_VARIANT(WV, G, R, NCW, RGW) \
     { Cfg<WV, G, R, NCW, RGW>::M, scan_kernel<WV, G, R, NCW, RGW>, Cfg<WV, G, R, NCW, RGW>::THREADS, \
-      Cfg<WV, G, R, NCW, RGW>::TV, stages_for<Cfg<WV, G, R, NCW, RGW>> }
+      Cfg<WV, G, R, NCW, RGW>::TV, stages_for<Cfg<WV, G, R, NCW, RGW>>, Cfg<WV, G, R, NCW, RGW>::LUT_BYTES, \
+      Cfg<WV, G, R, NCW, RGW>::BANKED ? 1 : 0, Cfg<WV, G, R, NCW, RGW>::COPIES, Cfg<WV, G, R, NCW, RGW>::COPY_OFF, \
+      Cfg<WV, G, R, NCW, RGW>::LSTRIDE }
 // Warps x unrolled row groups per warp were chosen by measurement: independent row groups in flight inside a warp
 // hide the look-up latency better than more warps do (M = 64: 16 x 2 -> 12 x 4 gave +30%).
 static const Variant kVariants[] = {
@@ -705,13 +769,15 @@ cudaError_t scan_plan(const IndexImpl* ix, ScanPlan* plan) {
     plan->stages = stages;
     plan->ctas = ix->num_sms;
     plan->smem_bytes = SMEM_OPTIN;
+    plan->lut_bytes = v->lut_bytes; plan->lut_banked = v->lut_banked; plan->lut_copies = v->lut_copies;
+    plan->lut_copy_off = v->lut_copy_off; plan->lut_stride = v->lut_stride;
     return cudaFuncSetAttribute(v->kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_OPTIN);
 }
 
 cudaError_t launch_scan(const IndexImpl* ix, const ScanPlan& plan, const float* queries, const int32_t* probe_list,
                         const float* probe_term, const int64_t* work_prefix, int nq, int nprobe, int k,
                         unsigned long long* qthresh, int32_t* slot_cnt, unsigned long long* slot_keys,
-                        uint32_t* err_word, cudaStream_t s) {
+                        uint32_t* err_word, const uint8_t* lut_img, const float* lut_inv, cudaStream_t s) {
     const Variant* v = find_variant(ix->M);
     if (!v) return cudaErrorInvalidValue;
     ScanArgs a;
@@ -719,9 +785,107 @@ cudaError_t launch_scan(const IndexImpl* ix, const ScanPlan& plan, const float* 
     a.queries = queries; a.cbT = ix->cbT; a.work_prefix = work_prefix;
     a.vterm = ix->vterm;
     a.qthresh = qthresh; a.slot_cnt = slot_cnt; a.slot_keys = slot_keys; a.err = err_word;
+    a.lut_img = lut_img; a.lut_inv = lut_inv;
     a.npairs = nq * nprobe; a.nprobe = nprobe; a.d = ix->d; a.dsub = ix->dsub;
     a.metric = ix->metric; a.k = k; a.stages = plan.stages; a.dyn_bytes = (uint32_t)plan.smem_bytes;
     v->kernel<<<plan.ctas, v->threads, plan.smem_bytes, s>>>(a);
+    count_launch();
+    return cudaGetLastError();
+}
+
+// ---- lookup tables of a small batch, built ahead of the scan ---------------------------------------
+// With few queries every scan CTA would build the same handful of tables, each reading the whole codebook; here
+// the tables are built once, by many CTAs per query, and stored as the exact shared-memory image the scan variant
+// uses (padding included), so a scan CTA fetches a table with one linear copy.
+//
+// The fixed-point scale cannot wait for the largest entry (the CTAs of a query do not meet), so it comes from a
+// bound: |entry(j, m)| = |s <q_m, cw_mj>| <= |s| ||q_m|| max_j ||cw_mj||.  The bound costs a bit or two of the 30
+// the sum may use, which leaves the quantisation error far below the tolerance.
+__global__ void codeword_norms_kernel(const float* __restrict__ cb, int dsub, float* __restrict__ cwmax) {
+    __shared__ float red[KSUB / 32];
+    const int m = blockIdx.x, j = threadIdx.x;  // KSUB threads: one codeword each
+    float n2 = 0.f;
+    for (int t = 0; t < dsub; ++t) { const float v = cb[((size_t)m * KSUB + j) * dsub + t]; n2 = fmaf(v, v, n2); }
+    float n = sqrtf(n2);
+    for (int o = 16; o; o >>= 1) n = fmaxf(n, __shfl_xor_sync(0xffffffffu, n, o));
+    if ((j & 31) == 0) red[j >> 5] = n;
+    __syncthreads();
+    if (j == 0) {
+        for (int w = 1; w < KSUB / 32; ++w) n = fmaxf(n, red[w]);
+        cwmax[m] = n;
+    }
+}
+cudaError_t launch_codeword_norms(const float* codebooks, int M, int dsub, float* cwmax, cudaStream_t s) {
+    codeword_norms_kernel<<<M, KSUB, 0, s>>>(codebooks, dsub, cwmax);
+    count_launch();
+    return cudaGetLastError();
+}
+
+constexpr int BT_THREADS = 256;
+struct TableArgs {
+    const float* queries; const float* cbT; const float* cwmax;
+    int d, dsub, M, metric, lut_bytes, banked, copies, copy_off, lstride;
+    uint8_t* lut_img; float* lut_inv;
+};
+// Part `part` of `parts` of query q's table, by all threads of the CTA.  sm: d + M floats of shared memory.
+__device__ __forceinline__ void build_table_part(const TableArgs& t, int q, int part, int parts, float* sm) {
+    const int d = t.d, dsub = t.dsub, M = t.M, tid = threadIdx.x, nthreads = blockDim.x;
+    float* rT = sm;       // the scaled query with the sub-space index innermost
+    float* bnd = sm + d;  // bound of the entries of every sub-space
+    const float lut_scale = t.metric == RAGO_IP ? -1.f : -2.f;
+    const float* qrow = t.queries + (size_t)q * d;
+    for (int j = tid; j < d; j += nthreads) rT[(j % dsub) * M + j / dsub] = lut_scale * qrow[j];
+    for (int m = tid; m < M; m += nthreads) {
+        float n2 = 0.f;
+        for (int u = 0; u < dsub; ++u) { const float v = qrow[m * dsub + u]; n2 = fmaf(v, v, n2); }
+        bnd[m] = 2.0002f * sqrtf(n2) * t.cwmax[m];  // |s| <= 2, and a margin for the rounding of the norms
+    }
+    __syncthreads();
+    float mx = 0.f;
+    for (int m = 0; m < M; ++m) mx = fmaxf(mx, bnd[m]);
+    int ex = 0;
+    if (mx > 0.f && mx < 3.0e38f) frexpf(mx * (float)M, &ex);  // mx * M < 2^ex
+    ex = ex < -90 ? -90 : (ex > 120 ? 120 : ex);
+    const float scale = ldexpf(1.f, 30 - ex);
+    if (part == 0 && tid == 0) t.lut_inv[q] = ldexpf(1.f, ex - 30);
+    uint8_t* img = t.lut_img + (size_t)q * t.lut_bytes;
+    auto off = [&](int j, int col) -> uint32_t {
+        return t.banked ? (uint32_t)(col / 64) * 65536u + (uint32_t)j * 256u + (uint32_t)(col % 64) * 4u
+                        : ((uint32_t)j * t.lstride + (uint32_t)col) * 4u;
+    };
+    const int total = KSUB * M;
+    const int per = (total + parts - 1) / parts;
+    const int e1 = (part + 1) * per < total ? (part + 1) * per : total;
+    for (int e = part * per + tid; e < e1; e += nthreads) {
+        const int j = e / M, m = e - j * M;
+        float acc = 0.f;
+        for (int u = 0; u < dsub; ++u) acc = fmaf(rT[u * M + m], __ldg(t.cbT + (size_t)e * dsub + u), acc);
+        const int v = __float2int_rn(acc * scale);
+        *reinterpret_cast<int*>(img + off(j, m)) = v;
+        if (t.copies == 2) *reinterpret_cast<int*>(img + off(j, t.copy_off + m)) = v;
+    }
+}
+__global__ void __launch_bounds__(BT_THREADS) build_tables_kernel(const TableArgs t) {
+    extern __shared__ float bt_smem[];
+    build_table_part(t, blockIdx.y, blockIdx.x, gridDim.x, bt_smem);
+}
+static TableArgs table_args(const IndexImpl* ix, const float* queries, uint8_t* lut_img, float* lut_inv) {
+    const ScanPlan& pl = ix->plan;
+    TableArgs t;
+    t.queries = queries; t.cbT = ix->cbT; t.cwmax = ix->cwmax;
+    t.d = ix->d; t.dsub = ix->dsub; t.M = ix->M; t.metric = ix->metric;
+    t.lut_bytes = pl.lut_bytes; t.banked = pl.lut_banked; t.copies = pl.lut_copies; t.copy_off = pl.lut_copy_off;
+    t.lstride = pl.lut_stride; t.lut_img = lut_img; t.lut_inv = lut_inv;
+    return t;
+}
+static int table_parts(const IndexImpl* ix, int nq) {
+    const int parts = 2 * ix->num_sms / nq;
+    return parts < 1 ? 1 : (parts > 64 ? 64 : parts);
+}
+cudaError_t launch_build_tables(const IndexImpl* ix, const float* queries, int nq, uint8_t* lut_img, float* lut_inv,
+                                cudaStream_t s) {
+    build_tables_kernel<<<dim3(table_parts(ix, nq), nq), BT_THREADS, (size_t)(ix->d + ix->M) * 4, s>>>(
+        table_args(ix, queries, lut_img, lut_inv));
     count_launch();
     return cudaGetLastError();
 }
@@ -860,11 +1024,20 @@ __global__ void __launch_bounds__(PT_THREADS) add_offsets_kernel(int64_t* __rest
 
 // Small batches: one CTA does the whole preparation of a search (tiles per pair, their prefix sum,
 // threshold and slot-counter reset), which would otherwise be four launches of a few microseconds each.
+// With table_parts > 0 the CTAs after the first build the batch's lookup tables meanwhile (the tables depend on the
+// queries only, so nothing orders them against the planning).
 __global__ void __launch_bounds__(PFX_THREADS) plan_small_kernel(const int32_t* __restrict__ probe_list,
                                                                  const int64_t* __restrict__ offsets, int npairs,
                                                                  int tile_vecs, int64_t* __restrict__ prefix,
                                                                  unsigned long long* __restrict__ qthresh, int nq,
-                                                                 int32_t* __restrict__ slot_cnt, int nslots) {
+                                                                 int32_t* __restrict__ slot_cnt, int nslots,
+                                                                 const TableArgs tables, int table_parts) {
+    extern __shared__ float bt_smem[];
+    if (blockIdx.x > 0) {
+        const int b = blockIdx.x - 1;
+        build_table_part(tables, b / table_parts, b % table_parts, table_parts, bt_smem);
+        return;
+    }
     __shared__ long long warp_sums[32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     long long v = 0;
@@ -897,12 +1070,19 @@ __global__ void __launch_bounds__(PFX_THREADS) plan_small_kernel(const int32_t* 
 
 cudaError_t launch_plan_work(const IndexImpl* ix, const int32_t* probe_list, int npairs, int tile_vecs,
                              int32_t* pair_tiles, int64_t* work_prefix, unsigned long long* qthresh, int nq,
-                             int32_t* slot_cnt, int nslots, cudaStream_t s) {
+                             int32_t* slot_cnt, int nslots, const float* queries, uint8_t* lut_img, float* lut_inv,
+                             cudaStream_t s) {
     if (npairs <= PFX_THREADS) {
-        plan_small_kernel<<<1, PFX_THREADS, 0, s>>>(probe_list, ix->list_offsets, npairs, tile_vecs, work_prefix, qthresh,
-                                                    nq, slot_cnt, nslots);
+        const int parts = lut_img ? table_parts(ix, nq) : 0;
+        plan_small_kernel<<<1 + parts * nq, PFX_THREADS, parts ? (size_t)(ix->d + ix->M) * 4 : 0, s>>>(
+            probe_list, ix->list_offsets, npairs, tile_vecs, work_prefix, qthresh, nq, slot_cnt, nslots,
+            table_args(ix, queries, lut_img, lut_inv), parts);
         count_launch();
         return cudaGetLastError();
+    }
+    if (lut_img) {
+        const cudaError_t et = launch_build_tables(ix, queries, nq, lut_img, lut_inv, s);
+        if (et != cudaSuccess) return et;
     }
     // pair_tiles (npairs int32 of scratch) holds the per-CTA totals: one 64-bit word per 256 pairs
     const int nblocks = (npairs + PT_THREADS - 1) / PT_THREADS;
