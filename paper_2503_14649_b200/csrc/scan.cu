@@ -50,7 +50,6 @@
 namespace rago {
 
 constexpr int MAX_STAGES = 4;
-constexpr int CUT_PASSES = 3;               // range-narrowing passes of a buffer cut before it falls back to bisection
 constexpr int SMEM_OPTIN = 227 * 1024;          // dynamic shared memory asked for (the sm_100 per-block limit)
 constexpr uint32_t SMEM_BASE_EXPECTED = 1024;   // shared-window address of dynamic shared memory when the kernel has no static part
 constexpr int CTRL_BYTES = 1024;
@@ -510,58 +509,11 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
             mn = ctrl->redu[0][w] < mn ? ctrl->redu[0][w] : mn;
             mx = ctrl->redu[1][w] > mx ? ctrl->redu[1][w] : mx;
         }
-        // All keys sit in registers now, so the buffer's memory is free until they are pushed back: its first words
-        // hold the slice counts of the passes below (one array per pass, cleared here).
-        uint32_t* hist = reinterpret_cast<uint32_t*>(keys);
-        for (int i = ctid; i < CUT_PASSES * 256; i += NCT) hist[i] = 0u;
-        csync();  // the minima / maxima have been read (redu is free for the counts), the slice counts are clear
+        csync();  // the minima / maxima have been read; redu is free for the counts
         if (dead) return;
         long long lo = (long long)mn - 1, hi = mx;  // #(score <= lo) < k <= #(score <= hi)
-        uint32_t c_hi = (uint32_t)n, below = 0;     // below = #(score <= lo)
+        uint32_t c_hi = (uint32_t)n;
         const uint32_t want_max = (uint32_t)(k + (k >> 2) + 8);
-        // Narrow (lo, hi] by 256 equal slices per pass: the slice that holds the k-th smallest key becomes the new
-        // range (two barriers per pass).  What the passes leave undecided (ties, odd distributions) is bisected.
-        for (int pass = 0; pass < CUT_PASSES && hi - lo > 1 && c_hi > want_max; ++pass) {  // uniform across the CTA
-            uint32_t* h = hist + pass * 256;
-            const uint32_t first = (uint32_t)(lo + 1), range = (uint32_t)(hi - lo - 1);
-            const int shift = range < 256u ? 0 : 24 - __clz(range);  // (range >> shift) < 256
-#pragma unroll
-            for (int j = 0; j < KPT; ++j) {
-                const uint32_t o = (uint32_t)(mine[j] >> 32);
-                if (mine[j] != KEY_MAX && o >= first && o <= (uint32_t)hi) atomicAdd(&h[(o - first) >> shift], 1u);
-            }
-            csync();
-            if (dead) return;
-            if (warp == 0) {  // lane i owns slices 8 i .. 8 i + 7
-                const uint32_t want = (uint32_t)k - below;  // rank of the cut inside the range, >= 1
-                uint32_t hv[8], tot = 0;
-#pragma unroll
-                for (int j = 0; j < 8; ++j) { hv[j] = h[lane * 8 + j]; tot += hv[j]; }
-                uint32_t before = tot;  // inclusive scan over the lanes, then made exclusive
-                for (int o = 1; o < 32; o <<= 1) {
-                    const uint32_t v = __shfl_up_sync(0xffffffffu, before, o);
-                    if (lane >= o) before += v;
-                }
-                before -= tot;
-                if (before < want && before + tot >= want) {  // exactly one lane
-                    uint32_t c = before, prev = before;
-                    int bsel = 0;
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        if (c < want) { bsel = j; prev = c; c += hv[j]; }
-                    }
-                    ctrl->redu[1][0] = (uint32_t)(lane * 8 + bsel); ctrl->redu[1][1] = c; ctrl->redu[1][2] = prev;
-                }
-            }
-            csync();
-            if (dead) return;
-            const uint32_t bsel = ctrl->redu[1][0];
-            const long long top = (long long)first + (((long long)bsel + 1) << shift) - 1;
-            c_hi = below + ctrl->redu[1][1];
-            below += ctrl->redu[1][2];
-            hi = top < hi ? top : hi;
-            lo = (long long)first + ((long long)bsel << shift) - 1;
-        }
         int round = 0;
         while (hi - lo > 1 && c_hi > want_max) {  // uniform across the CTA
             const uint32_t mid = (uint32_t)(lo + (hi - lo) / 2);
