@@ -110,6 +110,8 @@ __global__ void __launch_bounds__(256) coarse_small_kernel(const float* __restri
                                                            const float* __restrict__ cnorm, int nq, int nlist, int d,
                                                            int metric, float* __restrict__ scores) {
     extern __shared__ __align__(16) float qs[];  // [nq][d], rounded to bf16 values for a bf16 index
+    grid_dependency_wait();
+    grid_dependents_may_launch();
     for (int i = threadIdx.x; i < nq * d; i += blockDim.x) qs[i] = BF16 ? round_bf16(Q[i]) : Q[i];
     __syncthreads();
     const int lane = threadIdx.x & 31;
@@ -186,11 +188,11 @@ cudaError_t launch_coarse_scores(const IndexImpl* ix, const float* queries, int 
         const int want = (ix->nlist + 8 * CS_CPW - 1) / (8 * CS_CPW);  // 8 warps per CTA, CS_CPW rows per warp step
         const int blocks = want < ix->num_sms * 2 ? want : ix->num_sms * 2;
         if (ix->coarse_bf16)
-            coarse_small_kernel<true><<<blocks, 256, qbytes, s>>>(queries, ix->centroids, ix->cnorm, nq, ix->nlist, ix->d,
-                                                                   ix->metric, scores);
+            launch_overlapped(coarse_small_kernel<true>, dim3(blocks), dim3(256), qbytes, s, queries, ix->centroids, ix->cnorm,
+                              nq, ix->nlist, ix->d, ix->metric, scores);
         else
-            coarse_small_kernel<false><<<blocks, 256, qbytes, s>>>(queries, ix->centroids, ix->cnorm, nq, ix->nlist, ix->d,
-                                                                    ix->metric, scores);
+            launch_overlapped(coarse_small_kernel<false>, dim3(blocks), dim3(256), qbytes, s, queries, ix->centroids, ix->cnorm,
+                              nq, ix->nlist, ix->d, ix->metric, scores);
         count_launch();
         return cudaGetLastError();
     }
@@ -235,6 +237,8 @@ __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
     const int q = blockIdx.x, tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
     auto sync = [] { __syncthreads(); };
+    grid_dependency_wait();
+    grid_dependents_may_launch();
     int nsel = nprobe + PROBE_GUARD;
     if (nsel > nlist) nsel = nlist;
     if (tid == 0) { cnt = 0; s_mn = 0xFFFFFFFFu; s_mx = 0u; s_nv = 0u; s_round[0] = s_round[1] = s_round[2] = 0u; }
@@ -454,11 +458,11 @@ static void launch_select_source(const IndexImpl* ix, const float* queries, cons
                                  const unsigned long long* cand, const int32_t* cand_cnt, int nsplit, int cap, int nq,
                                  int nprobe, int32_t* probe_list, float* probe_term, float* probe_bias, cudaStream_t s) {
     if (scores)
-        select_probes_kernel<BF16, THREADS, REG, true><<<nq, THREADS, 0, s>>>(
+        launch_overlapped(select_probes_kernel<BF16, THREADS, REG, true>, dim3(nq), dim3(THREADS), 0, s,
             queries, ix->centroids, scores, cand, cand_cnt, nsplit, cap, ix->nlist, ix->d, ix->metric, nprobe, probe_list,
             probe_term, probe_bias);
     else
-        select_probes_kernel<BF16, THREADS, REG, false><<<nq, THREADS, 0, s>>>(
+        launch_overlapped(select_probes_kernel<BF16, THREADS, REG, false>, dim3(nq), dim3(THREADS), 0, s,
             queries, ix->centroids, scores, cand, cand_cnt, nsplit, cap, ix->nlist, ix->d, ix->metric, nprobe, probe_list,
             probe_term, probe_bias);
 }

@@ -169,6 +169,25 @@ __device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
 
 // ---- host-side launch bookkeeping -------------------------------------------------------------
 void count_launch(int n = 1);
+
+// ---- back-to-back kernels of one search -------------------------------------------------------------
+// A kernel launched with launch_overlapped may be scheduled while the kernel before it on the stream is still
+// draining; it must not touch global memory before grid_dependency_wait(), which returns once that kernel has
+// completed and its writes are visible.  Every kernel of the chain waits first thing and then lets its own
+// successor be scheduled, so the order of all memory accesses is the stream order; what overlaps is launch
+// latency.  In a kernel launched the ordinary way both calls do nothing.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependents_may_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+template <class... P, class... A>
+inline cudaError_t launch_overlapped(void (*kernel)(P...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, A... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, P(args)...);
+}
 void set_error(const char* fmt, ...);
 
 // ---- kernel launchers (one per .cu file) ------------------------------------------------------

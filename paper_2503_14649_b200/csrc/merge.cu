@@ -24,6 +24,8 @@ __global__ void __launch_bounds__(THREADS) merge_kernel(
     __shared__ int cnt;
     const int q = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     auto sync = [] { __syncthreads(); };
+    grid_dependency_wait();
+    grid_dependents_may_launch();
     if (tid == 0) cnt = 0;
     __syncthreads();
     const long long W = work_prefix[npairs];
@@ -126,11 +128,11 @@ cudaError_t launch_merge(const IndexImpl* ix, const int64_t* work_prefix, int nq
                          const int32_t* slot_cnt, const unsigned long long* slot_keys, const unsigned long long* qthresh,
                          int64_t* out_ids, float* out_dists, cudaStream_t s) {
     if (nq <= 64)
-        merge_kernel<1024><<<nq, 1024, 0, s>>>(work_prefix, ix->ids, nq * nprobe, nprobe, k, ctas, ix->metric,
-                                               slot_cnt, slot_keys, qthresh, out_ids, out_dists);
+        launch_overlapped(merge_kernel<1024>, dim3(nq), dim3(1024), 0, s, work_prefix, ix->ids, nq * nprobe, nprobe, k, ctas,
+                          ix->metric, slot_cnt, slot_keys, qthresh, out_ids, out_dists);
     else
-        merge_kernel<256><<<nq, 256, 0, s>>>(work_prefix, ix->ids, nq * nprobe, nprobe, k, ctas, ix->metric,
-                                             slot_cnt, slot_keys, qthresh, out_ids, out_dists);
+        launch_overlapped(merge_kernel<256>, dim3(nq), dim3(256), 0, s, work_prefix, ix->ids, nq * nprobe, nprobe, k, ctas,
+                          ix->metric, slot_cnt, slot_keys, qthresh, out_ids, out_dists);
     count_launch();
     return cudaGetLastError();
 }

@@ -325,6 +325,8 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
     extern __shared__ __align__(1024) uint8_t smem[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int S = a.stages;
+    grid_dependency_wait();
+    grid_dependents_may_launch();
     const uint32_t base = smem_u32(smem);
     const SmemPlan P = plan_smem<C>(base, a.dyn_bytes, a.d, S);
     if (!P.ok) {  // uniform: every thread sees the same plan
@@ -740,9 +742,9 @@ cudaError_t launch_scan(const IndexImpl* ix, const ScanPlan& plan, const float* 
     a.lut_img = lut_img; a.lut_inv = lut_inv;
     a.npairs = nq * nprobe; a.nprobe = nprobe; a.d = ix->d; a.dsub = ix->dsub;
     a.metric = ix->metric; a.k = k; a.stages = plan.stages; a.dyn_bytes = (uint32_t)plan.smem_bytes;
-    v->kernel<<<plan.ctas, v->threads, plan.smem_bytes, s>>>(a);
+    const cudaError_t e = launch_overlapped(v->kernel, dim3(plan.ctas), dim3(v->threads), plan.smem_bytes, s, a);
     count_launch();
-    return cudaGetLastError();
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 // ---- lookup tables of a small batch, built ahead of the scan ---------------------------------------
@@ -985,6 +987,8 @@ __global__ void __launch_bounds__(PFX_THREADS) plan_small_kernel(const int32_t* 
                                                                  int32_t* __restrict__ slot_cnt, int nslots,
                                                                  const TableArgs tables, int table_parts) {
     extern __shared__ float bt_smem[];
+    grid_dependency_wait();
+    grid_dependents_may_launch();
     if (blockIdx.x > 0) {
         const int b = blockIdx.x - 1;
         build_table_part(tables, b / table_parts, b % table_parts, table_parts, bt_smem);
@@ -1026,7 +1030,8 @@ cudaError_t launch_plan_work(const IndexImpl* ix, const int32_t* probe_list, int
                              cudaStream_t s) {
     if (npairs <= PFX_THREADS) {
         const int parts = lut_img ? table_parts(ix, nq) : 0;
-        plan_small_kernel<<<1 + parts * nq, PFX_THREADS, parts ? (size_t)(ix->d + ix->M) * 4 : 0, s>>>(
+        launch_overlapped(plan_small_kernel, dim3(1 + parts * nq), dim3(PFX_THREADS),
+                          parts ? (size_t)(ix->d + ix->M) * 4 : 0, s,
             probe_list, ix->list_offsets, npairs, tile_vecs, work_prefix, qthresh, nq, slot_cnt, nslots,
             table_args(ix, queries, lut_img, lut_inv), parts);
         count_launch();
