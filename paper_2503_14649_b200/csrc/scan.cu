@@ -325,8 +325,6 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
     extern __shared__ __align__(1024) uint8_t smem[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int S = a.stages;
-    grid_dependency_wait();
-    grid_dependents_may_launch();
     const uint32_t base = smem_u32(smem);
     const SmemPlan P = plan_smem<C>(base, a.dyn_bytes, a.d, S);
     if (!P.ok) {  // uniform: every thread sees the same plan
@@ -351,6 +349,10 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
     }
     __syncthreads();
 
+    // Everything above touched shared memory and kernel arguments only; from here on the kernel reads what the
+    // kernels before it wrote.
+    grid_dependency_wait();
+    grid_dependents_may_launch();
     // This CTA's share of the work units (tiles).
     const long long W = a.work_prefix[a.npairs];
     const long long u_begin = (long long)blockIdx.x * W / gridDim.x;
