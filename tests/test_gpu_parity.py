@@ -260,3 +260,19 @@ def test_single_query_whose_best_list_is_spread_over_many_ctas(k):
     data.centroids = cen
     data.queries = 0.01 * data.queries / data.queries.norm()
     _compare(data, 8, k)
+
+
+@pytest.mark.parametrize("metric", ["l2", "ip"])
+@pytest.mark.parametrize("nq", [5, 40])     # tables built ahead of the scan / inside it
+def test_query_magnitudes_from_zero_to_huge(metric, nq):
+    """The lookup table is fixed-point with a per-query scale: a zero query, tiny and huge queries and one with an
+    empty sub-vector must all come out within tolerance."""
+    data = synth.make_ivfpq(30_000, 64, 32, 16, nq, metric=metric, seed=77)
+    q = data.queries.clone()
+    q[0] = 0.0
+    q[1] *= 1e-6
+    q[2] *= 1e5
+    q[3, :8] = 0.0
+    q[4, 4:] = 0.0
+    data.queries = q
+    _compare(data, 6, 15, max_probe_mismatch=1)
