@@ -50,6 +50,11 @@
 namespace rago {
 
 constexpr int MAX_STAGES = 4;
+constexpr int SCAN_PF = 2;                  // tiles ahead of the one being copied that are prefetched into L2 (measured: 1-2 best)
+// Prefetch of a contiguous global range into L2 (16-byte aligned start, size a multiple of 16 bytes).
+__device__ __forceinline__ void l2_prefetch(const void* g, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(g), "r"(bytes) : "memory");
+}
 constexpr int SMEM_OPTIN = 227 * 1024;          // dynamic shared memory asked for (the sm_100 per-block limit)
 constexpr uint32_t SMEM_BASE_EXPECTED = 1024;   // shared-window address of dynamic shared memory when the kernel has no static part
 constexpr int CTRL_BYTES = 1024;
@@ -426,6 +431,14 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
                 mbar_arrive_expect_tx(bar, bytes + vbytes);
                 bulk_g2s(P.tile[st], a.codes + (size_t)pos0 * C::M, bytes, bar);
                 if (vbytes) bulk_g2s(P.vt[st], a.vterm + (pos0 & ~3u), vbytes, bar);
+                // pull the tiles a few steps ahead in this list into L2, so that their copies find them there
+                for (int ahead = (t_in_pair == 0 ? 1 : SCAN_PF); ahead <= SCAN_PF; ++ahead) {
+                    const long long vp = v0 + (long long)ahead * C::TV;
+                    if (vp >= len) break;
+                    long long np = len - vp;
+                    if (np > C::TV) np = C::TV;
+                    l2_prefetch(a.codes + (size_t)(off + vp) * C::M, (uint32_t)np * C::M);
+                }
             }
             issued = n + 1;
         }
