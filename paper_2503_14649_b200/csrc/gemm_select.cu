@@ -59,12 +59,6 @@ __device__ __forceinline__ void tma_load_2d(const CUtensorMap* map, uint32_t bar
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
         : "memory");
 }
-// Pull a tile into L2 ahead of its load (no shared memory, no completion to wait for).
-__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* map, int x, int y) {
-    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(reinterpret_cast<uint64_t>(map)),
-                 "r"(x), "r"(y)
-                 : "memory");
-}
 __device__ __forceinline__ void tmem_alloc(uint32_t slot_smem, uint32_t ncols) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(ncols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -256,7 +250,6 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
     if (warp == 0) {
         // ================= TMA producer =================
         if (lane == 0) {
-            constexpr int PF = 2 * G_STAGES;  // B tiles are pulled into L2 this many k-blocks ahead of their load
             const int total = nunits * kiters;
             auto coords = [&](int gi, int& kx, int& ya, int& yb) {
                 const int u = gi / kiters, r = gi - u * kiters;
@@ -267,17 +260,9 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                 yb = a.term_b[t] * a.b_part_rows + nt * GBN;
             };
             int kx, ya, yb;
-            for (int gi = 0; gi < PF && gi < total; ++gi) {
-                coords(gi, kx, ya, yb);
-                tma_prefetch_2d(&tmB, kx, yb);
-            }
             for (int gi = 0; gi < total; ++gi) {
                 const int s = gi % G_STAGES;
                 const uint32_t ph = (uint32_t)(gi / G_STAGES) & 1u;
-                if (gi + PF < total) {
-                    coords(gi + PF, kx, ya, yb);
-                    tma_prefetch_2d(&tmB, kx, yb);
-                }
                 coords(gi, kx, ya, yb);
                 if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, a.err, 64)) break;
                 mbar_arrive_expect_tx(full_bar(s), G_STAGE_BYTES);
