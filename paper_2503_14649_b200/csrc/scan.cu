@@ -3,8 +3,10 @@
 // One persistent CTA per SM walks a contiguous, equally sized share of the batch's code tiles
 // (pairs (query, probed list) in probe order, each list cut into tiles of TV vectors).  A producer
 // warp streams code tiles global -> shared with 1-D bulk copies (cp.async.bulk + mbarrier, a ring of
-// S tiles in flight); consumer warps build the fp32 lookup table of the current QUERY in shared
-// memory, then every lane owns one (virtual) code row of the tile and sums table entries.
+// S tiles in flight, the tiles two steps further down the list prefetched into L2); consumer warps
+// build the lookup table of the current QUERY in shared memory (or, for small batches, fetch the
+// image a kernel before the scan has built), then every lane owns one (virtual) code row of the tile
+// and sums table entries.
 //
 // Score, smaller is better for both metrics:
 //   inner product:  -<q, c_p>  +  sum_m -<q_m, cw_m>
