@@ -276,3 +276,10 @@ def test_query_magnitudes_from_zero_to_huge(metric, nq):
     q[4, 4:] = 0.0
     data.queries = q
     _compare(data, 6, 15, max_probe_mismatch=1)
+
+
+def test_small_batch_with_many_probes_builds_tables_in_their_own_launch():
+    """24 queries x 64 probes: few enough queries for tables built ahead of the scan, too many (query, list) pairs
+    for the single planning launch that otherwise hosts the table CTAs."""
+    data = synth.make_ivfpq(60_000, 96, 128, 48, 24, metric="ip", seed=41, zipf=0.8)
+    _compare(data, 64, 40, max_probe_mismatch=1)
