@@ -212,9 +212,10 @@ constexpr int SEL_MAX_SPLIT = 512;  // candidate lists per query the kernel can 
 
 // Candidates come either from a score row (scores != null: all nlist lists) or from the candidate
 // lists the tensor-core kernel left behind (cand[q][split][cap] keys with counts cand_cnt[q][split]).
-// First a cut value is found by bisection on the ordered score bits (CTA-wide counts, items held in
-// registers when they fit, re-read from memory otherwise) such that between nsel and nsel + slack items
-// lie at or below it; only those go to shared memory, are sorted, re-scored exactly and sorted again.
+// First a cut value is found on the ordered score bits (the range is narrowed by counting items per slice in
+// shared memory, then bisected if ties or an odd distribution leave it open; items are held in registers when
+// they fit, re-read from memory otherwise) such that between nsel and nsel + slack items lie at or below it;
+// only those go to shared memory, are sorted, re-scored exactly and sorted again.
 // SEL_THREADS threads per query keep up to SEL_REG item scores each in registers: a big CTA for tiny
 // batches (latency), a small one when there are enough queries to fill the GPU.
 // FROM_SCORES: the items are a row of the score matrix (else the candidate lists the GEMM left).  The two sources
