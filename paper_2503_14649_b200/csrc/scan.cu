@@ -951,6 +951,8 @@ __global__ void __launch_bounds__(PT_THREADS) pair_tiles_kernel(const int32_t* _
 }
 
 constexpr int PFX_THREADS = 1024;
+constexpr int PLAN_PER_THREAD = 4;       // pairs per thread of the single-CTA planning kernel
+constexpr int PLAN_SMALL_MAX = PFX_THREADS * PLAN_PER_THREAD;
 // In-place exclusive scan of n totals by one CTA; the grand total goes to *total_out.
 __global__ void __launch_bounds__(PFX_THREADS) scan_totals_kernel(long long* __restrict__ sums, int n,
                                                                   int64_t* __restrict__ total_out) {
@@ -1013,10 +1015,18 @@ __global__ void __launch_bounds__(PFX_THREADS) plan_small_kernel(const int32_t* 
     }
     __shared__ long long warp_sums[32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    // thread t owns pairs PLAN_PER_THREAD * t .. + PLAN_PER_THREAD - 1
+    long long mine[PLAN_PER_THREAD];
     long long v = 0;
-    if (tid < npairs) {
-        const int l = probe_list[tid];
-        v = (offsets[l + 1] - offsets[l] + tile_vecs - 1) / tile_vecs;
+#pragma unroll
+    for (int j = 0; j < PLAN_PER_THREAD; ++j) {
+        const int p = tid * PLAN_PER_THREAD + j;
+        mine[j] = 0;
+        if (p < npairs) {
+            const int l = probe_list[p];
+            mine[j] = (offsets[l + 1] - offsets[l] + tile_vecs - 1) / tile_vecs;
+        }
+        v += mine[j];
     }
     long long incl = v;
     for (int o = 1; o < 32; o <<= 1) {
@@ -1034,9 +1044,14 @@ __global__ void __launch_bounds__(PFX_THREADS) plan_small_kernel(const int32_t* 
         warp_sums[lane] = w;
     }
     __syncthreads();
-    const long long before = (warp ? warp_sums[warp - 1] : 0) + incl - v;
-    if (tid < npairs) prefix[tid] = before;
-    if (tid == npairs - 1) prefix[npairs] = before + v;
+    long long before = (warp ? warp_sums[warp - 1] : 0) + incl - v;
+#pragma unroll
+    for (int j = 0; j < PLAN_PER_THREAD; ++j) {
+        const int p = tid * PLAN_PER_THREAD + j;
+        if (p < npairs) prefix[p] = before;
+        before += mine[j];
+        if (p == npairs - 1) prefix[npairs] = before;
+    }
     for (int i = tid; i < nq; i += PFX_THREADS) qthresh[i] = KEY_MAX;
     for (int i = tid; i < nslots; i += PFX_THREADS) slot_cnt[i] = 0;
 }
@@ -1045,7 +1060,7 @@ cudaError_t launch_plan_work(const IndexImpl* ix, const int32_t* probe_list, int
                              int32_t* pair_tiles, int64_t* work_prefix, unsigned long long* qthresh, int nq,
                              int32_t* slot_cnt, int nslots, const float* queries, uint8_t* lut_img, float* lut_inv,
                              cudaStream_t s) {
-    if (npairs <= PFX_THREADS) {
+    if (npairs <= PLAN_SMALL_MAX) {
         const int parts = lut_img ? table_parts(ix, nq) : 0;
         launch_overlapped(plan_small_kernel, dim3(1 + parts * nq), dim3(PFX_THREADS),
                           parts ? (size_t)(ix->d + ix->M) * 4 : 0, s,

@@ -279,7 +279,7 @@ def test_query_magnitudes_from_zero_to_huge(metric, nq):
 
 
 def test_small_batch_with_many_probes_builds_tables_in_their_own_launch():
-    """24 queries x 64 probes: few enough queries for tables built ahead of the scan, too many (query, list) pairs
-    for the single planning launch that otherwise hosts the table CTAs."""
-    data = synth.make_ivfpq(60_000, 96, 128, 48, 24, metric="ip", seed=41, zipf=0.8)
-    _compare(data, 64, 40, max_probe_mismatch=1)
+    """30 queries x 150 probes: few enough queries for tables built ahead of the scan, too many (query, list) pairs
+    (4 500) for the single planning launch that otherwise hosts the table CTAs."""
+    data = synth.make_ivfpq(60_000, 96, 256, 48, 30, metric="ip", seed=41, zipf=0.8)
+    _compare(data, 150, 40, max_probe_mismatch=1)
