@@ -30,7 +30,7 @@ struct ScanPlan {
 
 // Batches of at most this many queries get their lookup tables from a kernel of their own, spread over the whole
 // GPU, instead of every scan CTA building the table of each query it meets.
-constexpr int PREBUILT_MAX_NQ = 32;
+constexpr int PREBUILT_MAX_NQ = 256;
 
 // Index handle.  Borrowed pointers first, then what the library owns.
 struct IndexImpl {
