@@ -77,10 +77,18 @@ def test_hyperscale_full_size_sampled():
     torch.cuda.synchronize()
     ix.rago_check()
     gi, gd, gl = ids.cpu().numpy(), dists.cpu().numpy(), lists.cpu().numpy()
-    ix.close()
     sample = [0, 1023, 2048, 4095]
+    # the same four queries as a batch of their own: the small-batch path (tables built ahead of the scan)
+    qs = q[sample].contiguous()
+    ids4, dists4 = ix.rago_search(qs, c["nprobe"], c["k"])
+    lists4, _ = ix.rago_search_probes(qs, c["nprobe"])
+    torch.cuda.synchronize()
+    ix.rago_check()
+    gi4, gd4, gl4 = ids4.cpu().numpy(), dists4.cpu().numpy(), lists4.cpu().numpy()
+    ix.close()
     hix = compact_hashed_subindex(oracle, data, np.unique(gl[sample]))
     _check_sample(data, hix, data.queries, sample, gi, gd, gl, c["nprobe"], c["k"])
+    _check_sample(data, hix, data.queries[sample], [0, 1, 2, 3], gi4, gd4, gl4, c["nprobe"], c["k"])
     del data, ix, q, ids, dists, lists
     _free()
 
