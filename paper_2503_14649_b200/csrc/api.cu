@@ -42,7 +42,7 @@ struct Layout {
     size_t err, probe_list, probe_term, probe_bias, scores, pair_tiles, work_prefix, qthresh, slot_cnt, slot_keys, total;
     size_t qparts, cand, cand_cnt;  // tensor-core coarse step: query parts, candidate lists and their counts
     size_t pilot_scores, row_tau;   // pilot pass: scores of the sampled lists, per-query starting thresholds
-    size_t lut_img, lut_inv;        // small batches: lookup tables built ahead of the scan, and their scales
+    size_t lut_img, lut_inv, lut_scale;        // small batches: lookup tables built ahead of the scan, and their scales
     int prebuilt;
     int pilot_cols;                 // 0: no pilot pass
     size_t nslots;
@@ -106,6 +106,7 @@ static Layout make_layout(const IndexImpl* ix, int nq, int nprobe, int k) {
     const size_t nlut = nq < PREBUILT_MAX_NQ ? nq : PREBUILT_MAX_NQ;
     L.lut_img = take(nlut * ix->plan.lut_bytes);
     L.lut_inv = take(nlut * 4);
+    L.lut_scale = take(nlut * 4);
     L.total = o;
     return L;
 }
@@ -385,7 +386,8 @@ rago_status rago_search(const rago_index* index, const float* queries, int32_t n
     uint8_t* lut_img = L.prebuilt ? ws + L.lut_img : nullptr;
     float* lut_inv = L.prebuilt ? reinterpret_cast<float*>(ws + L.lut_inv) : nullptr;
     e = launch_plan_work(ix, probe_list, npairs, ix->plan.tile_vecs, reinterpret_cast<int32_t*>(ws + L.pair_tiles),
-                         work_prefix, qthresh, nq, slot_cnt, (int)L.nslots, queries, lut_img, lut_inv, s);
+                         work_prefix, qthresh, nq, slot_cnt, (int)L.nslots, queries, lut_img, lut_inv,
+                         L.prebuilt ? reinterpret_cast<float*>(ws + L.lut_scale) : nullptr, s);
     if (e != cudaSuccess) return cuda_fail(e, "work planning");
     record(mix, 3, s);
     e = launch_scan(ix, ix->plan, queries, probe_list, probe_term, work_prefix, nq, nprobe, k, qthresh, slot_cnt,

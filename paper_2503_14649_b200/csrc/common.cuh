@@ -28,9 +28,9 @@ struct ScanPlan {
     int lut_bytes, lut_banked, lut_copies, lut_copy_off, lut_stride;
 };
 
-// Batches of at most this many queries get their lookup tables from a kernel of their own, spread over the whole
+// Batches of at most this many queries get their lookup tables from kernels of their own, spread over the whole
 // GPU, instead of every scan CTA building the table of each query it meets.
-constexpr int PREBUILT_MAX_NQ = 256;
+constexpr int PREBUILT_MAX_NQ = 4096;
 
 // Index handle.  Borrowed pointers first, then what the library owns.
 struct IndexImpl {
@@ -232,14 +232,14 @@ cudaError_t launch_transpose_codebook(const float* cb, int M, int dsub, float* c
 cudaError_t launch_plan_work(const IndexImpl* ix, const int32_t* probe_list, int npairs, int tile_vecs,
                              int32_t* pair_tiles, int64_t* work_prefix, unsigned long long* qthresh, int nq,
                              int32_t* slot_cnt, int nslots, const float* queries, uint8_t* lut_img, float* lut_inv,
-                             cudaStream_t s);
+                             float* lut_scale, cudaStream_t s);
 cudaError_t launch_scan(const IndexImpl* ix, const ScanPlan& plan, const float* queries, const int32_t* probe_list,
                         const float* probe_term, const int64_t* work_prefix, int nq, int nprobe, int k,
                         unsigned long long* qthresh, int32_t* slot_cnt, unsigned long long* slot_keys,
                         uint32_t* err_word, const uint8_t* lut_img, const float* lut_inv, cudaStream_t s);
 cudaError_t launch_codeword_norms(const float* codebooks, int M, int dsub, float* cwmax, cudaStream_t s);
 cudaError_t launch_build_tables(const IndexImpl* ix, const float* queries, int nq, uint8_t* lut_img, float* lut_inv,
-                                cudaStream_t s);
+                                float* lut_scale, cudaStream_t s);
 // merge.cu
 cudaError_t launch_merge(const IndexImpl* ix, const int64_t* work_prefix, int nq, int nprobe, int k, int ctas,
                          const int32_t* slot_cnt, const unsigned long long* slot_keys, const unsigned long long* qthresh,

@@ -853,10 +853,149 @@ static int table_parts(const IndexImpl* ix, int nq) {
     const int parts = 2 * ix->num_sms / nq;
     return parts < 1 ? 1 : (parts > 64 ? 64 : parts);
 }
+// Large batches.  One CTA per (slice of the table's entries, chunk of queries): every thread keeps the codewords of
+// its EPT entries in registers and walks the chunk's queries, so the codebook crosses L2 once per chunk of
+// queries instead of once per query.  The scale of each query (same bound as above) comes from a kernel of
+// its own, because a CTA sees only a slice of the sub-spaces.
+__global__ void __launch_bounds__(128) table_scales_kernel(const float* __restrict__ queries,
+                                                            const float* __restrict__ cwmax, int d, int dsub, int M,
+                                                            float* __restrict__ lut_scale, float* __restrict__ lut_inv) {
+    __shared__ float red[4];
+    const int q = blockIdx.x, tid = threadIdx.x;
+    const float* qrow = queries + (size_t)q * d;
+    float mx = 0.f;
+    for (int m = tid; m < M; m += 128) {
+        float n2 = 0.f;
+        for (int u = 0; u < dsub; ++u) { const float v = qrow[m * dsub + u]; n2 = fmaf(v, v, n2); }
+        mx = fmaxf(mx, 2.0002f * sqrtf(n2) * cwmax[m]);
+    }
+    for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    if ((tid & 31) == 0) red[tid >> 5] = mx;
+    __syncthreads();
+    if (tid == 0) {
+        mx = fmaxf(fmaxf(red[0], red[1]), fmaxf(red[2], red[3]));
+        int ex = 0;
+        if (mx > 0.f && mx < 3.0e38f) frexpf(mx * (float)M, &ex);
+        ex = ex < -90 ? -90 : (ex > 120 ? 120 : ex);
+        lut_scale[q] = ldexpf(1.f, 30 - ex);
+        lut_inv[q] = ldexpf(1.f, ex - 30);
+    }
+}
+
+constexpr int BTB_THREADS = 256;
+constexpr int BTB_CW_FLOATS = 96;  // codeword floats a thread keeps in registers
+template <int DSUB>
+__global__ void __launch_bounds__(BTB_THREADS) build_tables_batch_kernel(const TableArgs t,
+                                                                          const float* __restrict__ lut_scale, int nq,
+                                                                          int qchunk) {
+    constexpr int EPT = BTB_CW_FLOATS / DSUB;  // entries per thread
+    extern __shared__ float btb_smem[];        // two buffers of d floats: the scaled query, sub-space index innermost
+    const int d = t.d, M = t.M, tid = threadIdx.x;
+    const int total = KSUB * M;
+    const int per = (total + gridDim.x - 1) / gridDim.x;
+    const int e0 = blockIdx.x * per;
+    const int e1 = e0 + per < total ? e0 + per : total;
+    float cw[EPT][DSUB];
+    uint32_t off[EPT];  // byte offset of the entry in a table image, 0xFFFFFFFF for an unused slot
+    int col[EPT];       // its sub-space
+#pragma unroll
+    for (int i = 0; i < EPT; ++i) {
+        const int e = e0 + tid + i * BTB_THREADS;
+        off[i] = 0xFFFFFFFFu;
+        col[i] = 0;
+#pragma unroll
+        for (int u = 0; u < DSUB; ++u) cw[i][u] = 0.f;
+        if (e < e1) {
+            const int j = e / M, m = e - j * M;
+            col[i] = m;
+            off[i] = t.banked ? (uint32_t)(m / 64) * 65536u + (uint32_t)j * 256u + (uint32_t)(m % 64) * 4u
+                              : ((uint32_t)j * t.lstride + (uint32_t)m) * 4u;
+#pragma unroll
+            for (int u = 0; u < DSUB; u += 4) {
+                const float4 v = __ldg(reinterpret_cast<const float4*>(t.cbT + (size_t)e * DSUB + u));
+                cw[i][u] = v.x; cw[i][u + 1] = v.y; cw[i][u + 2] = v.z; cw[i][u + 3] = v.w;
+            }
+        }
+    }
+    const uint32_t copy_delta = t.copies == 2
+        ? (t.banked ? (uint32_t)((t.copy_off / 64) * 65536 + (t.copy_off % 64) * 4) : (uint32_t)t.copy_off * 4u) : 0u;
+    const float lut_s = t.metric == RAGO_IP ? -1.f : -2.f;
+    const int q0 = blockIdx.y * qchunk;
+    const int q1 = q0 + qchunk < nq ? q0 + qchunk : nq;
+    // The next query's values are fetched into registers before the current query's entries are computed and
+    // written to the other buffer afterwards, so their latency hides behind the arithmetic (d <= 16 * 256).
+    constexpr int QPT = 16;  // query floats per thread, at most
+    float nxt[QPT];
+    auto fetch = [&](int q) {
+        const float* qrow = t.queries + (size_t)q * d;
+#pragma unroll
+        for (int r = 0; r < QPT; ++r) {
+            const int j = tid + r * BTB_THREADS;
+            nxt[r] = j < d ? lut_s * __ldg(qrow + j) : 0.f;
+        }
+    };
+    auto stage = [&](float* rT) {
+#pragma unroll
+        for (int r = 0; r < QPT; ++r) {
+            const int j = tid + r * BTB_THREADS;
+            if (j < d) rT[(j % DSUB) * M + j / DSUB] = nxt[r];
+        }
+    };
+    if (q0 < q1) { fetch(q0); stage(btb_smem); }
+    __syncthreads();
+    for (int q = q0; q < q1; ++q) {
+        const float* rT = btb_smem + ((q - q0) & 1) * d;
+        if (q + 1 < q1) fetch(q + 1);
+        const float scale = __ldg(lut_scale + q);
+        uint8_t* img = t.lut_img + (size_t)q * t.lut_bytes;
+        // all entries of the thread advance together, one sub-space coordinate at a time: EPT independent chains
+        float acc[EPT];
+#pragma unroll
+        for (int i = 0; i < EPT; ++i) acc[i] = 0.f;
+#pragma unroll
+        for (int u = 0; u < DSUB; ++u) {
+            const float* row = rT + u * M;
+#pragma unroll
+            for (int i = 0; i < EPT; ++i) acc[i] = fmaf(row[col[i]], cw[i][u], acc[i]);
+        }
+#pragma unroll
+        for (int i = 0; i < EPT; ++i) {
+            if (off[i] != 0xFFFFFFFFu) {
+                const int v = __float2int_rn(acc[i] * scale);
+                *reinterpret_cast<int*>(img + off[i]) = v;
+                if (copy_delta) *reinterpret_cast<int*>(img + off[i] + copy_delta) = v;
+            }
+        }
+        // the other buffer was last read for query q - 1, which every thread finished before the barrier that
+        // ended the previous iteration
+        if (q + 1 < q1) stage(btb_smem + ((q + 1 - q0) & 1) * d);
+        __syncthreads();
+    }
+}
+
 cudaError_t launch_build_tables(const IndexImpl* ix, const float* queries, int nq, uint8_t* lut_img, float* lut_inv,
-                                cudaStream_t s) {
-    build_tables_kernel<<<dim3(table_parts(ix, nq), nq), BT_THREADS, (size_t)(ix->d + ix->M) * 4, s>>>(
-        table_args(ix, queries, lut_img, lut_inv));
+                                float* lut_scale, cudaStream_t s) {
+    const int dsub = ix->dsub;
+    const TableArgs t = table_args(ix, queries, lut_img, lut_inv);
+    if (nq > 64 && lut_scale && (dsub == 4 || dsub == 8 || dsub == 12 || dsub == 16)) {
+        table_scales_kernel<<<nq, 128, 0, s>>>(queries, ix->cwmax, ix->d, dsub, ix->M, lut_scale, lut_inv);
+        const int ept = BTB_CW_FLOATS / dsub;
+        const int total = KSUB * ix->M;
+        const int parts = (total + BTB_THREADS * ept - 1) / (BTB_THREADS * ept);
+        int qchunk = (int)(((long long)nq * parts + 2 * ix->num_sms - 1) / (2 * ix->num_sms));
+        if (qchunk < 1) qchunk = 1;
+        const dim3 grid(parts, (nq + qchunk - 1) / qchunk);
+        const size_t smem = (size_t)2 * ix->d * 4;
+        switch (dsub) {
+            case 4: build_tables_batch_kernel<4><<<grid, BTB_THREADS, smem, s>>>(t, lut_scale, nq, qchunk); break;
+            case 8: build_tables_batch_kernel<8><<<grid, BTB_THREADS, smem, s>>>(t, lut_scale, nq, qchunk); break;
+            case 12: build_tables_batch_kernel<12><<<grid, BTB_THREADS, smem, s>>>(t, lut_scale, nq, qchunk); break;
+            default: build_tables_batch_kernel<16><<<grid, BTB_THREADS, smem, s>>>(t, lut_scale, nq, qchunk); break;
+        }
+        count_launch(2);
+        return cudaGetLastError();
+    }
+    build_tables_kernel<<<dim3(table_parts(ix, nq), nq), BT_THREADS, (size_t)(ix->d + ix->M) * 4, s>>>(t);
     count_launch();
     return cudaGetLastError();
 }
@@ -1059,19 +1198,20 @@ __global__ void __launch_bounds__(PFX_THREADS) plan_small_kernel(const int32_t* 
 cudaError_t launch_plan_work(const IndexImpl* ix, const int32_t* probe_list, int npairs, int tile_vecs,
                              int32_t* pair_tiles, int64_t* work_prefix, unsigned long long* qthresh, int nq,
                              int32_t* slot_cnt, int nslots, const float* queries, uint8_t* lut_img, float* lut_inv,
-                             cudaStream_t s) {
+                             float* lut_scale, cudaStream_t s) {
+    const bool fused_tables = lut_img && npairs <= PLAN_SMALL_MAX && nq <= 64;
+    if (lut_img && !fused_tables) {
+        const cudaError_t et = launch_build_tables(ix, queries, nq, lut_img, lut_inv, lut_scale, s);
+        if (et != cudaSuccess) return et;
+    }
     if (npairs <= PLAN_SMALL_MAX) {
-        const int parts = lut_img ? table_parts(ix, nq) : 0;
+        const int parts = fused_tables ? table_parts(ix, nq) : 0;
         launch_overlapped(plan_small_kernel, dim3(1 + parts * nq), dim3(PFX_THREADS),
                           parts ? (size_t)(ix->d + ix->M) * 4 : 0, s,
             probe_list, ix->list_offsets, npairs, tile_vecs, work_prefix, qthresh, nq, slot_cnt, nslots,
             table_args(ix, queries, lut_img, lut_inv), parts);
         count_launch();
         return cudaGetLastError();
-    }
-    if (lut_img) {
-        const cudaError_t et = launch_build_tables(ix, queries, nq, lut_img, lut_inv, s);
-        if (et != cudaSuccess) return et;
     }
     // pair_tiles (npairs int32 of scratch) holds the per-CTA totals: one 64-bit word per 256 pairs
     const int nblocks = (npairs + PT_THREADS - 1) / PT_THREADS;
