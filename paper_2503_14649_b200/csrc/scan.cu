@@ -853,9 +853,9 @@ static int table_parts(const IndexImpl* ix, int nq) {
     const int parts = 2 * ix->num_sms / nq;
     return parts < 1 ? 1 : (parts > 64 ? 64 : parts);
 }
-// Large batches.  One CTA per (slice of the table's entries, chunk of queries): every thread keeps the codewords of
-// its EPT entries in registers and walks the chunk's queries, so the codebook crosses L2 once per chunk of
-// queries instead of once per query.  The scale of each query (same bound as above) comes from a kernel of
+// Large batches.  One CTA per (range of code values, chunk of queries): every thread keeps the codewords of its EPT
+// entries in registers and walks the chunk's queries, so the codebook crosses L2 once per chunk of queries
+// instead of once per query.  The scale of each query (same bound as above) comes from a kernel of
 // its own, because a CTA sees only a slice of the sub-spaces.
 __global__ void __launch_bounds__(128) table_scales_kernel(const float* __restrict__ queries,
                                                             const float* __restrict__ cwmax, int d, int dsub, int M,
@@ -882,94 +882,72 @@ __global__ void __launch_bounds__(128) table_scales_kernel(const float* __restri
     }
 }
 
-constexpr int BTB_THREADS = 256;
 constexpr int BTB_CW_FLOATS = 96;  // codeword floats a thread keeps in registers
+// blockDim.x = M * G: thread (m, g) owns sub-space m of the code values j = j0 + g + G i, i < EPT, so everything it
+// needs of a query is the DSUB values of one sub-space, fetched straight into registers (the next query's while the
+// current one is multiplied): no shared memory and no barrier.  Threads with consecutive m read consecutive
+// codewords and write consecutive table columns.
 template <int DSUB>
-__global__ void __launch_bounds__(BTB_THREADS) build_tables_batch_kernel(const TableArgs t,
-                                                                          const float* __restrict__ lut_scale, int nq,
-                                                                          int qchunk) {
+__global__ void __launch_bounds__(256) build_tables_batch_kernel(const TableArgs t, const float* __restrict__ lut_scale,
+                                                                  int nq, int qchunk) {
     constexpr int EPT = BTB_CW_FLOATS / DSUB;  // entries per thread
-    extern __shared__ float btb_smem[];        // two buffers of d floats: the scaled query, sub-space index innermost
     const int d = t.d, M = t.M, tid = threadIdx.x;
-    const int total = KSUB * M;
-    const int per = (total + gridDim.x - 1) / gridDim.x;
-    const int e0 = blockIdx.x * per;
-    const int e1 = e0 + per < total ? e0 + per : total;
+    const int G = blockDim.x / M;
+    const int m = tid % M, g = tid / M;
+    const int j0 = blockIdx.x * (G * EPT);
     float cw[EPT][DSUB];
     uint32_t off[EPT];  // byte offset of the entry in a table image, 0xFFFFFFFF for an unused slot
-    int col[EPT];       // its sub-space
 #pragma unroll
     for (int i = 0; i < EPT; ++i) {
-        const int e = e0 + tid + i * BTB_THREADS;
+        const int j = j0 + g + G * i;
         off[i] = 0xFFFFFFFFu;
-        col[i] = 0;
 #pragma unroll
         for (int u = 0; u < DSUB; ++u) cw[i][u] = 0.f;
-        if (e < e1) {
-            const int j = e / M, m = e - j * M;
-            col[i] = m;
+        if (j < KSUB) {
             off[i] = t.banked ? (uint32_t)(m / 64) * 65536u + (uint32_t)j * 256u + (uint32_t)(m % 64) * 4u
                               : ((uint32_t)j * t.lstride + (uint32_t)m) * 4u;
+            const float* src = t.cbT + ((size_t)j * M + m) * DSUB;
 #pragma unroll
             for (int u = 0; u < DSUB; u += 4) {
-                const float4 v = __ldg(reinterpret_cast<const float4*>(t.cbT + (size_t)e * DSUB + u));
+                const float4 v = __ldg(reinterpret_cast<const float4*>(src + u));
                 cw[i][u] = v.x; cw[i][u + 1] = v.y; cw[i][u + 2] = v.z; cw[i][u + 3] = v.w;
             }
         }
     }
+    // second copy of a column (layouts that keep one), as a byte distance inside the image
     const uint32_t copy_delta = t.copies == 2
         ? (t.banked ? (uint32_t)((t.copy_off / 64) * 65536 + (t.copy_off % 64) * 4) : (uint32_t)t.copy_off * 4u) : 0u;
     const float lut_s = t.metric == RAGO_IP ? -1.f : -2.f;
     const int q0 = blockIdx.y * qchunk;
     const int q1 = q0 + qchunk < nq ? q0 + qchunk : nq;
-    // The next query's values are fetched into registers before the current query's entries are computed and
-    // written to the other buffer afterwards, so their latency hides behind the arithmetic (d <= 16 * 256).
-    constexpr int QPT = 16;  // query floats per thread, at most
-    float nxt[QPT];
+    float qn[DSUB];
     auto fetch = [&](int q) {
-        const float* qrow = t.queries + (size_t)q * d;
+        const float* src = t.queries + (size_t)q * d + m * DSUB;
 #pragma unroll
-        for (int r = 0; r < QPT; ++r) {
-            const int j = tid + r * BTB_THREADS;
-            nxt[r] = j < d ? lut_s * __ldg(qrow + j) : 0.f;
+        for (int u = 0; u < DSUB; u += 4) {
+            const float4 v = __ldg(reinterpret_cast<const float4*>(src + u));
+            qn[u] = v.x; qn[u + 1] = v.y; qn[u + 2] = v.z; qn[u + 3] = v.w;
         }
     };
-    auto stage = [&](float* rT) {
-#pragma unroll
-        for (int r = 0; r < QPT; ++r) {
-            const int j = tid + r * BTB_THREADS;
-            if (j < d) rT[(j % DSUB) * M + j / DSUB] = nxt[r];
-        }
-    };
-    if (q0 < q1) { fetch(q0); stage(btb_smem); }
-    __syncthreads();
+    if (q0 < q1) fetch(q0);
     for (int q = q0; q < q1; ++q) {
-        const float* rT = btb_smem + ((q - q0) & 1) * d;
+        float qv[DSUB];
+#pragma unroll
+        for (int u = 0; u < DSUB; ++u) qv[u] = lut_s * qn[u];
         if (q + 1 < q1) fetch(q + 1);
         const float scale = __ldg(lut_scale + q);
         uint8_t* img = t.lut_img + (size_t)q * t.lut_bytes;
-        // all entries of the thread advance together, one sub-space coordinate at a time: EPT independent chains
-        float acc[EPT];
-#pragma unroll
-        for (int i = 0; i < EPT; ++i) acc[i] = 0.f;
-#pragma unroll
-        for (int u = 0; u < DSUB; ++u) {
-            const float* row = rT + u * M;
-#pragma unroll
-            for (int i = 0; i < EPT; ++i) acc[i] = fmaf(row[col[i]], cw[i][u], acc[i]);
-        }
 #pragma unroll
         for (int i = 0; i < EPT; ++i) {
+            float acc = 0.f;
+#pragma unroll
+            for (int u = 0; u < DSUB; ++u) acc = fmaf(qv[u], cw[i][u], acc);
             if (off[i] != 0xFFFFFFFFu) {
-                const int v = __float2int_rn(acc[i] * scale);
+                const int v = __float2int_rn(acc * scale);
                 *reinterpret_cast<int*>(img + off[i]) = v;
                 if (copy_delta) *reinterpret_cast<int*>(img + off[i] + copy_delta) = v;
             }
         }
-        // the other buffer was last read for query q - 1, which every thread finished before the barrier that
-        // ended the previous iteration
-        if (q + 1 < q1) stage(btb_smem + ((q + 1 - q0) & 1) * d);
-        __syncthreads();
     }
 }
 
@@ -980,17 +958,17 @@ cudaError_t launch_build_tables(const IndexImpl* ix, const float* queries, int n
     if (nq > 64 && lut_scale && (dsub == 4 || dsub == 8 || dsub == 12 || dsub == 16)) {
         table_scales_kernel<<<nq, 128, 0, s>>>(queries, ix->cwmax, ix->d, dsub, ix->M, lut_scale, lut_inv);
         const int ept = BTB_CW_FLOATS / dsub;
-        const int total = KSUB * ix->M;
-        const int parts = (total + BTB_THREADS * ept - 1) / (BTB_THREADS * ept);
-        int qchunk = (int)(((long long)nq * parts + 2 * ix->num_sms - 1) / (2 * ix->num_sms));
+        const int G = 256 / ix->M;  // >= 2: the scan supports M <= 128
+        const int threads = ix->M * G;
+        const int parts = (KSUB + G * ept - 1) / (G * ept);
+        int qchunk = (int)(((long long)nq * parts + 4 * ix->num_sms - 1) / (4 * ix->num_sms));
         if (qchunk < 1) qchunk = 1;
         const dim3 grid(parts, (nq + qchunk - 1) / qchunk);
-        const size_t smem = (size_t)2 * ix->d * 4;
         switch (dsub) {
-            case 4: build_tables_batch_kernel<4><<<grid, BTB_THREADS, smem, s>>>(t, lut_scale, nq, qchunk); break;
-            case 8: build_tables_batch_kernel<8><<<grid, BTB_THREADS, smem, s>>>(t, lut_scale, nq, qchunk); break;
-            case 12: build_tables_batch_kernel<12><<<grid, BTB_THREADS, smem, s>>>(t, lut_scale, nq, qchunk); break;
-            default: build_tables_batch_kernel<16><<<grid, BTB_THREADS, smem, s>>>(t, lut_scale, nq, qchunk); break;
+            case 4: build_tables_batch_kernel<4><<<grid, threads, 0, s>>>(t, lut_scale, nq, qchunk); break;
+            case 8: build_tables_batch_kernel<8><<<grid, threads, 0, s>>>(t, lut_scale, nq, qchunk); break;
+            case 12: build_tables_batch_kernel<12><<<grid, threads, 0, s>>>(t, lut_scale, nq, qchunk); break;
+            default: build_tables_batch_kernel<16><<<grid, threads, 0, s>>>(t, lut_scale, nq, qchunk); break;
         }
         count_launch(2);
         return cudaGetLastError();
