@@ -107,8 +107,7 @@ rago_status rago_index_load_pq4(rago_index** out, const void* coarse_centroids, 
 rago_status rago_index_free(rago_index* index);
 
 /* Bytes of device scratch rago_search / rago_search_probes / rago_search_host need for a batch
- * of up to nq queries with these nprobe and k (1 <= nprobe <= nlist, 1 <= k <= 1024).  The size does
- * not decrease with nq, so scratch sized for a batch also serves smaller ones.  Its largest parts are
+ * of nq queries with these nprobe and k (1 <= nprobe <= nlist, 1 <= k <= 1024).  Its largest parts are
  * the per-query lookup tables (64 to 160 KB each, for at most 4096 queries of a batch: 128 KB per
  * query at M = 96) and, for batches the tensor-core coarse step does not take, nq * nlist scores. */
 rago_status rago_search_workspace_bytes(const rago_index* index, int32_t nq, int32_t nprobe, int32_t k,
