@@ -283,3 +283,11 @@ def test_small_batch_with_many_probes_builds_tables_in_their_own_launch():
     (4 500) for the single planning launch that otherwise hosts the table CTAs."""
     data = synth.make_ivfpq(60_000, 96, 256, 48, 30, metric="ip", seed=41, zipf=0.8)
     _compare(data, 150, 40, max_probe_mismatch=1)
+
+
+@pytest.mark.parametrize("metric,M,d", [("l2", 16, 64), ("ip", 32, 256)])
+def test_batch_beyond_the_prebuilt_table_limit_builds_tables_in_the_scan(metric, M, d):
+    """More than 4 096 queries: the scan CTAs build each query's table themselves (exact largest entry for the
+    fixed-point scale) instead of fetching an image built ahead."""
+    data = synth.make_ivfpq(20_000, d, 64, M, 4200, metric=metric, seed=5)
+    _compare(data, 4, 10, max_probe_mismatch=8)
