@@ -277,7 +277,7 @@ def run_ours(args):
     peak, peak_kind = _peaks()
     achieved = scan_bytes / (scan_ms / 1e3) / 1e9
     # DRAM bytes of one scan launch: dram__bytes_read.sum + dram__bytes_write.sum of one launch of this very
-    # workload at full size (profiles/scan_kernel_mid_quarter_scale.md: 34.106 GB for 42.427 GB of logical code
+    # workload at full size (one-pass ncu capture: 34.106 GB for 42.427 GB of logical code
     # bytes; hot lists are shared through L2).  The ratio does not carry over to other sizes (at 1/4 of the vectors
     # it is 0.31), so scaled-down runs report null.  Valid for the scan kernel the capture was taken from: set
     # SCAN_DRAM_PER_LOGICAL to None after changing the kernel.
