@@ -351,3 +351,27 @@ def test_pq4_equals_8bit_search_over_paired_subspaces(metric, bf16):
     # and the codes really are nibbles of the nearest codewords: unpack(pack(x)) == x
     codes = torch.randint(0, 16, (50, 8), dtype=torch.uint8)
     assert np.array_equal(oracle.unpack_pq4(synth.pack_pq4(codes).numpy()), codes.numpy())
+
+
+def test_merge_results_invariants():
+    """Aggregation does not depend on the order of the shards, a single shard is returned as it is (cut to k), and
+    merging in two steps equals merging at once."""
+    rng = np.random.default_rng(11)
+    nparts, nq, k = 5, 7, 12
+    d = np.sort(rng.permutation(nparts * nq * k).astype(np.float32).reshape(nparts, nq, k) * 0.5, axis=2)
+    ids = rng.permutation(nparts * nq * k).astype(np.int64).reshape(nparts, nq, k)
+    ids[3, :, 8:] = -1
+    d[3, :, 8:] = np.inf
+    a = oracle.merge_results(ids, d, k, "l2")
+    perm = [4, 0, 3, 1, 2]
+    b = oracle.merge_results(ids[perm], d[perm], k, "l2")
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
+    one = oracle.merge_results(ids[:1], d[:1], 5, "l2")
+    assert np.array_equal(one[0], ids[0][:, :5]) and np.array_equal(one[1], d[0][:, :5])
+    left = oracle.merge_results(ids[:2], d[:2], k, "l2")
+    right = oracle.merge_results(ids[2:], d[2:], k, "l2")
+    two = oracle.merge_results(np.stack([left[0], right[0]]), np.stack([left[1], right[1]]), k, "l2")
+    assert np.array_equal(two[0], a[0]) and np.array_equal(two[1], a[1])
+    # inner product: the same lists with the sign flipped rank the same way
+    c = oracle.merge_results(ids, np.where(np.isinf(d), -np.inf, -d).astype(np.float32), k, "ip")
+    assert np.array_equal(c[0], a[0])
