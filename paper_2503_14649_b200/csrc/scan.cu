@@ -659,7 +659,6 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
         // Row groups are taken MERGE at a time: with R lanes per vector every lane of an R-group ends up with
         // the vector's sum, so lane slice g finishes row group g and one epilogue serves MERGE row groups.
         constexpr int MERGE = R < C::RGW ? R : C::RGW;
-        constexpr bool EARLY_RELEASE = MERGE == C::RGW;  // the loop below runs once
         bool released = false;
 #pragma unroll
         for (int rg = 0; rg < C::RGW; rg += MERGE) {
@@ -683,10 +682,9 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
             // per-vector term of the L2 expansion (0 for inner product); rows past the tile's end read
             // stale but in-bounds shared memory and are never pushed
             const float vt = a.vterm != nullptr ? lds_f32(vt_base + (uint32_t)(vr / R) * 4u) : 0.f;
-            // With a single pass over the tile that was this warp's last read of the stage: hand the stage back
-            // before the rest of the epilogue, so that the refill starts that much earlier (M = 96: -1%; with
-            // several passes per tile the extra bookkeeping costs more than it returns).
-            if constexpr (EARLY_RELEASE) {
+            // In the last pass over the tile that was this warp's last read of the stage: hand the stage back
+            // before the rest of the epilogue, so that the refill starts that much earlier (M = 96: -1%).
+            if (rg + MERGE >= C::RGW) {  // compile-time under the unrolled loop
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&ctrl->empty[st]));
                 released = true;
@@ -696,7 +694,7 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
             const bool owner = MERGE == 1 ? sr == 0 : sr < MERGE;
             warp_push(keys, &ctrl->cnt, vr < nvr && owner && key < tau, key, C::KCAP);
         }
-        if (!released) {  // no early release, or a warp without rows in this tile
+        if (!released) {  // a warp that left the loop early: no rows of this tile are its own
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ctrl->empty[st]));
         }
