@@ -396,9 +396,8 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
         int issued = 0;
         for (int n = 0; n < T && !dead; ++n, ++u) {
             const int st = n % S;
-            if (n >= S) dead = !mbar_wait(smem_u32(&ctrl->empty[st]), ((n / S) - 1) & 1, abort_flag, a.err);
-            if (dead) break;
-            // advance to the pair that owns unit u (skips empty pairs)
+            // advance to the pair that owns unit u (skips empty pairs); all of this before the wait for the
+            // stage, so that as little as possible stands between a stage coming free and its refill
             for (;;) {
                 const long long we = __shfl_sync(0xffffffffu, c_we, cur);
                 if (u < we) break;
@@ -408,6 +407,8 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
             const long long off = __shfl_sync(0xffffffffu, c_off, cur);
             const long long len = __shfl_sync(0xffffffffu, c_len, cur);
             const int list = __shfl_sync(0xffffffffu, c_list, cur);
+            if (n >= S) dead = !mbar_wait(smem_u32(&ctrl->empty[st]), ((n / S) - 1) & 1, abort_flag, a.err);
+            if (dead) break;
             if (lane == 0) {
                 const long long t_in_pair = u - ws;
                 const long long v0 = t_in_pair * C::TV;
