@@ -394,8 +394,12 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
         long long u = u_begin;
         bool dead = false;
         int issued = 0;
+        int pst = 0;          // n % S, kept by counting (S is a run-time value: no division per tile)
+        uint32_t pround = 0;  // n / S
         for (int n = 0; n < T && !dead; ++n, ++u) {
-            const int st = n % S;
+            const int st = pst;
+            const uint32_t round = pround;
+            if (++pst == S) { pst = 0; ++pround; }
             // advance to the pair that owns unit u (skips empty pairs); all of this before the wait for the
             // stage, so that as little as possible stands between a stage coming free and its refill
             for (;;) {
@@ -407,7 +411,7 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
             const long long off = __shfl_sync(0xffffffffu, c_off, cur);
             const long long len = __shfl_sync(0xffffffffu, c_len, cur);
             const int list = __shfl_sync(0xffffffffu, c_list, cur);
-            if (n >= S) dead = !mbar_wait(smem_u32(&ctrl->empty[st]), ((n / S) - 1) & 1, abort_flag, a.err);
+            if (round > 0) dead = !mbar_wait(smem_u32(&ctrl->empty[st]), (round - 1) & 1, abort_flag, a.err);
             if (dead) break;
             if (lane == 0) {
                 const long long t_in_pair = u - ws;
@@ -626,9 +630,13 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
         csync();
     };
 
+    int cst = 0;            // n % S and the parity of n / S, kept by counting
+    uint32_t cparity = 0;
     for (int n = 0; n < T; ++n) {
-        const int st = n % S;
-        dead = dead || !mbar_wait(smem_u32(&ctrl->full[st]), (n / S) & 1, abort_flag, a.err);
+        const int st = cst;
+        const uint32_t parity = cparity;
+        if (++cst == S) { cst = 0; cparity ^= 1u; }
+        dead = dead || !mbar_wait(smem_u32(&ctrl->full[st]), parity, abort_flag, a.err);
         if (dead) break;
         const TileDesc D = ctrl->desc[st];
         if (D.newpair & 1) {
