@@ -250,20 +250,23 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
     if (warp == 0) {
         // ================= TMA producer =================
         if (lane == 0) {
+            // unit u = (column tile nt, row tile m), m fastest; inside it the terms, inside a term the k-blocks:
+            // kept by counting, no division per load
             const int total = nunits * kiters;
-            auto coords = [&](int gi, int& kx, int& ya, int& yb) {
-                const int u = gi / kiters, r = gi - u * kiters;
-                const int t = r / a.kblocks, kb = r - t * a.kblocks;
-                const int nt = nt_begin + u / mcount, m = m0 + u % mcount;
-                kx = kb * GBK;
-                ya = a.term_a[t] * a.a_part_rows + m * GBM;
-                yb = a.term_b[t] * a.b_part_rows + nt * GBN;
-            };
-            int kx, ya, yb;
+            int nt = nt_begin, mi = 0, t = 0, kb = 0;
             for (int gi = 0; gi < total; ++gi) {
                 const int s = gi % G_STAGES;
                 const uint32_t ph = (uint32_t)(gi / G_STAGES) & 1u;
-                coords(gi, kx, ya, yb);
+                const int kx = kb * GBK;
+                const int ya = a.term_a[t] * a.a_part_rows + (m0 + mi) * GBM;
+                const int yb = a.term_b[t] * a.b_part_rows + nt * GBN;
+                if (++kb == a.kblocks) {
+                    kb = 0;
+                    if (++t == a.nterms) {
+                        t = 0;
+                        if (++mi == mcount) { mi = 0; ++nt; }
+                    }
+                }
                 if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, a.err, 64)) break;
                 mbar_arrive_expect_tx(full_bar(s), G_STAGE_BYTES);
                 tma_load_2d(&tmA, full_bar(s), base + s * G_STAGE_BYTES, kx, ya);
@@ -310,7 +313,7 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         }
         bool dead = false;
         for (int u = 0; u < nunits && !dead; ++u) {
-            const int nt = nt_begin + u / mcount, g = u % mcount;
+            const int nt = nt_begin + (mcount == 2 ? u >> 1 : u), g = mcount == 2 ? u & 1 : 0;  // mcount is 1 or 2
             const int buf = u & 1;
             const uint32_t uph = (u >> 1) & 1u;
             for (int i = lane; i < GBN; i += 32) {
