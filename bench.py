@@ -31,7 +31,7 @@ import numpy as np  # noqa: E402
 import torch  # noqa: E402
 
 WORKLOAD = 2  # index into synth.CONFIGS
-SCAN_DRAM_PER_LOGICAL = 34.106e9 / 42.427e9  # full-size Mid workload only (see run_ours)
+SCAN_DRAM_PER_LOGICAL = 34.217e9 / 42.427e9  # full-size Mid workload only (see run_ours)
 METRIC = "retrieval_qps"
 UNIT = "queries/s"
 
@@ -277,7 +277,7 @@ def run_ours(args):
     peak, peak_kind = _peaks()
     achieved = scan_bytes / (scan_ms / 1e3) / 1e9
     # DRAM bytes of one scan launch: dram__bytes_read.sum + dram__bytes_write.sum of one launch of this very
-    # workload at full size (one-pass ncu capture: 34.106 GB for 42.427 GB of logical code
+    # workload at full size (one-pass ncu capture: 34.217 GB for 42.427 GB of logical code
     # bytes; hot lists are shared through L2).  The ratio does not carry over to other sizes (at 1/4 of the vectors
     # it is 0.31), so scaled-down runs report null.  Valid for the scan kernel the capture was taken from: set
     # SCAN_DRAM_PER_LOGICAL to None after changing the kernel.
