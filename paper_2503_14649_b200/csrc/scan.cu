@@ -846,13 +846,19 @@ __device__ __forceinline__ void build_table_part(const TableArgs& t, int q, int 
     const int total = KSUB * M;
     const int per = (total + parts - 1) / parts;
     const int e1 = (part + 1) * per < total ? (part + 1) * per : total;
-    for (int e = part * per + tid; e < e1; e += nthreads) {
-        const int j = e / M, m = e - j * M;
+    // entry e = (code value j, sub-space m), m fastest; (j, m) follow e by counting, not by dividing per entry
+    const int step_j = nthreads / M, step_m = nthreads - step_j * M;
+    int e = part * per + tid;
+    int j = e / M, m = e - j * M;
+    for (; e < e1; e += nthreads) {
         float acc = 0.f;
         for (int u = 0; u < dsub; ++u) acc = fmaf(rT[u * M + m], __ldg(t.cbT + (size_t)e * dsub + u), acc);
         const int v = __float2int_rn(acc * scale);
         *reinterpret_cast<int*>(img + off(j, m)) = v;
         if (t.copies == 2) *reinterpret_cast<int*>(img + off(j, t.copy_off + m)) = v;
+        j += step_j;
+        m += step_m;
+        if (m >= M) { m -= M; ++j; }
     }
 }
 __global__ void __launch_bounds__(BT_THREADS) build_tables_kernel(const TableArgs t) {
