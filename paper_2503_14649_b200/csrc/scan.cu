@@ -115,6 +115,7 @@ struct Cfg {
     static constexpr int KCAP = LUT_BYTES <= 65536 ? 2 * TOPK_CAP : TOPK_CAP;  // keys of the CTA's candidate buffer
     static_assert(WV % G == 0, "virtual rows are whole blocks");
     static_assert(TILE_VROWS % R == 0, "tile must hold whole vectors");
+    static_assert(RGW % (R < RGW ? R : RGW) == 0, "row groups are taken min(R, RGW) at a time");
     // The producer asks for a cut of the candidate buffer when the count it sees plus everything the tiles in
     // flight can still push would not fit; SMAX bounds the ring depth so that this leaves room to work in.
     static constexpr int SMAX = KCAP / TV / 2 < MAX_STAGES ? KCAP / TV / 2 : MAX_STAGES;
