@@ -15,14 +15,18 @@
  *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL = default stream)
  *     and the call returns without synchronising, unless stated otherwise.
  *   - The caller owns every buffer it passes.  An index BORROWS its arrays: they must stay valid
- *     and unchanged until rago_index_free.  Scratch memory is caller-provided ("workspace"); the
+ *     and unchanged until rago_index_free.  Scratch memory is caller-provided ("workspace"), with
+ *     one exception (rago_search_probes_noalloc, which uses an array built into the library); the
  *     search calls allocate nothing.
+ *   - An index belongs to the device that was current when it was loaded; every call that takes an
+ *     index must be made with that device current, otherwise it returns RAGO_EINVAL.
  *   - Errors are return codes.  Argument errors are found on the host before anything is
  *     launched.  rago_last_error() returns a thread-local description of the last failure.
  *   - L2 means SQUARED Euclidean distance, smaller is better, results ascending.  IP means inner
  *     product, larger is better, results descending.  Missing results (fewer than k candidates)
  *     are id -1 with +INFINITY (L2) or -INFINITY (IP).
- *   - 8-bit product quantisation only (256 codewords per sub-space).
+ *   - Product-quantisation codes are 8 bits (256 codewords per sub-space, rago_index_load) or 4 bits
+ *     (16 codewords, two codes per byte, rago_index_load_pq4).
  */
 #ifndef RAGO_H
 #define RAGO_H
@@ -152,15 +156,19 @@ rago_status rago_search_probes(const rago_index* index, const float* queries, in
  *
  * Same inputs, outputs and results as rago_search_probes, but there is no workspace argument:
  * the query-by-list score matrix is kept in an array of RAGO_NOALLOC_SCRATCH_BYTES that is part
- * of the library image (each GPU that loads the library gives up that much memory until the
- * process ends).  The call itself allocates and frees nothing.
+ * of the library image.  A GPU gives up that much memory from the first rago_index_load on it
+ * (which looks the array up, so the CUDA runtime loads it then; a failure shows there as
+ * RAGO_ECUDA) until the process ends.  The call itself allocates and frees nothing.
  *
  *   limit     align256(nq * nlist * 4) + align256(nq * nprobe * 4) <= RAGO_NOALLOC_SCRATCH_BYTES;
  *             a larger batch is refused with RAGO_ENOMEM and a message that names the limit
  *             (split the batch, or use rago_search_probes).
- *   set-up    the first call on each device looks up the array's device address
- *             (cudaGetSymbolAddress) with that device current; make that first call before
- *             starting any stream capture.
+ *   set-up    rago_index_load looks up the array's device address (cudaGetSymbolAddress) with the
+ *             index's device current, once per device, and this call reuses it.  Should that
+ *             look-up have failed, the first call here repeats it; such a first call must come
+ *             before any stream capture.
+ *   device    the array's address differs per device: the call returns RAGO_EINVAL unless the
+ *             current device is the index's.
  *   sharing   all calls on a device use the same array and find the previous call's contents in
  *             it.  Nothing needs clearing (every word read is written first by the same call),
  *             but two calls that overlap on the GPU - different streams, or different host

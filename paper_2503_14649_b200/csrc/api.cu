@@ -84,8 +84,8 @@ static Layout make_layout(const IndexImpl* ix, int nq, int nprobe, int k) {
         L.tc_mode = L.tc_cap ? 0 : 1;
         L.qparts = take((size_t)ix->cparts_n * nq * ix->d * 2);
         if (L.tc_mode == 0) {
-            L.cand = take((size_t)nq * L.tc_nsplit * L.tc_cap * 8);
-            L.cand_cnt = take((size_t)nq * L.tc_nsplit * 4);
+            L.cand = take((size_t)nq * L.tc_nsplit * GEMM_COL_HALVES * L.tc_cap * 8);
+            L.cand_cnt = take((size_t)nq * L.tc_nsplit * GEMM_COL_HALVES * 4);
             // a pilot pass pays off when a CTA sees many column tiles per row and the sample can hold nsel values
             const int np = ix->pilot_stride ? ix->nlist / ix->pilot_stride : 0;
             if (np >= 4 * nsel && ix->nlist >= 8192) {
@@ -109,6 +109,16 @@ static Layout make_layout(const IndexImpl* ix, int nq, int nprobe, int k) {
     L.lut_scale = take(nlut * 4);
     L.total = o;
     return L;
+}
+
+// Every pointer an index holds, and everything derived at load, belongs to one device.
+static rago_status check_device(const IndexImpl* ix) {
+    int dev = -1;
+    const cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+    if (dev != ix->device)
+        return fail(RAGO_EINVAL, "the current device (%d) is not the index's device (%d)", dev, ix->device);
+    return RAGO_OK;
 }
 
 static rago_status check_search_args(const IndexImpl* ix, int nq, int nprobe, int k) {
@@ -186,7 +196,7 @@ static rago_status run_coarse(const IndexImpl* ix, const float* queries, int nq,
         if (e != cudaSuccess) return cuda_fail(e, "tensor-core coarse kernel");
         record(mix, 1, s);
         if (L.tc_mode == 0)
-            e = launch_select_probes_cand(ix, queries, G.cand, G.cand_cnt, L.tc_nsplit, L.tc_cap, nq, nprobe, probe_list,
+            e = launch_select_probes_cand(ix, queries, G.cand, G.cand_cnt, L.tc_nsplit * GEMM_COL_HALVES, L.tc_cap, nq, nprobe, probe_list,
                                           probe_term, probe_bias, s);
         else
             e = launch_select_probes(ix, queries, scores, nq, nprobe, probe_list, probe_term, probe_bias, s);
@@ -286,6 +296,7 @@ rago_status rago_index_load(rago_index** out, const void* coarse_centroids, rago
             ix->pilot_stride = ps;
         cudaGetLastError();  // a missing tensor-core path is not an error: the fp32 kernel serves every batch
     }
+    if (e == cudaSuccess) e = noalloc_prepare();  // the built-in scratch of rago_search_probes_noalloc becomes resident now
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) {
         rago_status st = cuda_fail(e, "index setup kernels");
@@ -338,6 +349,8 @@ rago_status rago_search_probes(const rago_index* index, const float* queries, in
     if (nq == 0) return RAGO_OK;
     if (!queries || !out_lists || !out_coarse || !workspace) return fail(RAGO_EINVAL, "null pointer");
     if (!aligned(queries, 16) || !aligned(workspace, 256)) return fail(RAGO_EALIGN, "queries need 16-byte, workspace 256-byte alignment");
+    st = check_device(ix);
+    if (st != RAGO_OK) return st;
     const Layout L = make_layout(ix, nq, nprobe, 1);
     if (workspace_bytes < L.total) return fail(RAGO_ENOMEM, "workspace holds %zu bytes, %zu needed", workspace_bytes, L.total);
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
@@ -363,6 +376,8 @@ rago_status rago_search(const rago_index* index, const float* queries, int32_t n
     if (!queries || !out_ids || !out_dists || !workspace) return fail(RAGO_EINVAL, "null pointer");
     if (!aligned(queries, 16) || !aligned(workspace, 256) || !aligned(out_ids, 8) || !aligned(out_dists, 4))
         return fail(RAGO_EALIGN, "queries need 16-byte, workspace 256-byte alignment");
+    st = check_device(ix);
+    if (st != RAGO_OK) return st;
     const Layout L = make_layout(ix, nq, nprobe, k);
     if (workspace_bytes < L.total) return fail(RAGO_ENOMEM, "workspace holds %zu bytes, %zu needed", workspace_bytes, L.total);
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
@@ -409,6 +424,8 @@ rago_status rago_search_host(const rago_index* index, const float* host_queries,
     if (nq == 0) return RAGO_OK;
     if (!host_queries || !host_out_ids || !host_out_dists || !workspace) return fail(RAGO_EINVAL, "null pointer");
     if (!aligned(workspace, 256)) return fail(RAGO_EALIGN, "workspace needs 256-byte alignment");
+    st = check_device(ix);
+    if (st != RAGO_OK) return st;
     const Layout L = make_layout(ix, nq, nprobe, k);
     size_t staging = 0;
     rago_host_staging_bytes(index, nq, k, &staging);

@@ -201,18 +201,20 @@ cudaError_t launch_select_probes_cand(const IndexImpl* ix, const float* queries,
                                       const int32_t* cand_cnt, int nsplit, int cap, int nq, int nprobe,
                                       int32_t* probe_list, float* probe_term, float* probe_bias, cudaStream_t s);
 // gemm_select.cu
-constexpr int GEMM_CAP_SMALL = 512, GEMM_CAP_LARGE = 1024;  // candidate-list capacities (keys per row and column range)
+constexpr int GEMM_CAP_SMALL = 512, GEMM_CAP_LARGE = 1024;  // candidate-list capacities (keys per list)
+constexpr int GEMM_COL_HALVES = 2;  // a row has one candidate list per column range of the grid AND per half of a 256-column tile
 struct GemmLaunch {
     const void* tmap_a;          // CUtensorMap of A: bf16 [a parts * a_part_rows][d]
     const void* tmap_b;          // CUtensorMap of B: bf16 [b parts * b_part_rows][d]
     int nrows; int64_t ncols; int d;
     int a_part_rows; int64_t b_part_rows;
     int nterms; int term_a[6], term_b[6];
-    int mg, nsplit;              // from gemm_grid
+    int mg, nsplit;              // from gemm_grid: row tiles per CTA (2 = both share each B tile), column ranges
     float alpha; const float* colterm; int colterm_stride;
     const float* row_tau;        // initial per-row thresholds (mode 0) or null
     int mode, nsel, cap;
-    unsigned long long* cand; int32_t* cand_cnt; float* scores; uint32_t* err;
+    unsigned long long* cand; int32_t* cand_cnt;  // [nrows][nsplit * GEMM_COL_HALVES][cap] keys and their counts
+    float* scores; uint32_t* err;
 };
 cudaError_t gemm_select_init();
 cudaError_t make_tmap_bf16(void* out_map, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows,
@@ -240,6 +242,8 @@ cudaError_t launch_scan(const IndexImpl* ix, const ScanPlan& plan, const float* 
 cudaError_t launch_codeword_norms(const float* codebooks, int M, int dsub, float* cwmax, cudaStream_t s);
 cudaError_t launch_build_tables(const IndexImpl* ix, const float* queries, int nq, uint8_t* lut_img, float* lut_inv,
                                 float* lut_scale, cudaStream_t s);
+// no_alloc.cu
+cudaError_t noalloc_prepare();  // with the index's device current: look up (and make resident) the built-in scratch array
 // merge.cu
 cudaError_t launch_merge(const IndexImpl* ix, const int64_t* work_prefix, int nq, int nprobe, int k, int ctas,
                          const int32_t* slot_cnt, const unsigned long long* slot_keys, const unsigned long long* qthresh,

@@ -173,13 +173,15 @@ static int flat_pilot_cols(int64_t N, int k) {
     return np >= 4LL * k ? (int)np : 0;
 }
 
-// Workspace, tensor-core path: [err 256 B][cand nq*nsplit*cap u64][cand_cnt nq*nsplit i32][pilot scores nq*np f32][row_tau nq f32]
+// Workspace, tensor-core path: [err 256 B][cand nq*nlists*cap u64][cand_cnt nq*nlists i32][pilot scores nq*np f32][row_tau nq f32]
+//            (nlists = column ranges of the grid x GEMM_COL_HALVES candidate lists per query)
 //            fallback:         [err 256 B][scores nq*PANEL f32][slot_cnt nq*nchunks i32][slot_keys nq*nchunks*k u64]
 size_t flat_workspace_bytes(int64_t N, int d, int nq, int k) {
     if (flat_on_tensor_cores(d, k)) {
         int mg, nsplit, mgroups;
         gemm_grid(nq > 0 ? nq : 1, N > 0 ? N : 1, sm_count(), &mg, &nsplit, &mgroups);
-        return 256 + align_up((size_t)nq * nsplit * gemm_cand_cap(k) * 8, 256) + align_up((size_t)nq * nsplit * 4, 256) +
+        const size_t nlists = (size_t)nsplit * GEMM_COL_HALVES;
+        return 256 + align_up((size_t)nq * nlists * gemm_cand_cap(k) * 8, 256) + align_up((size_t)nq * nlists * 4, 256) +
                align_up((size_t)nq * flat_pilot_cols(N, k) * 4, 256) + align_up((size_t)nq * 4, 256);
     }
     const size_t nchunks = (size_t)((N + FLAT_CHUNK - 1) / FLAT_CHUNK);
@@ -198,11 +200,12 @@ cudaError_t launch_flat_search(const void* db, int64_t N, int d, const void* que
         int mg, nsplit, mgroups;
         gemm_grid(nq, N, sm_count(), &mg, &nsplit, &mgroups);
         const int cap = gemm_cand_cap(k);
+        const int nlists = nsplit * GEMM_COL_HALVES;
         uint8_t* w = static_cast<uint8_t*>(workspace) + 256;
         unsigned long long* cand = reinterpret_cast<unsigned long long*>(w);
-        w += align_up((size_t)nq * nsplit * cap * 8, 256);
+        w += align_up((size_t)nq * nlists * cap * 8, 256);
         int32_t* cand_cnt = reinterpret_cast<int32_t*>(w);
-        w += align_up((size_t)nq * nsplit * 4, 256);
+        w += align_up((size_t)nq * nlists * 4, 256);
         const int np = flat_pilot_cols(N, k);
         float* pilot_scores = reinterpret_cast<float*>(w);
         w += align_up((size_t)nq * np * 4, 256);
@@ -243,7 +246,7 @@ cudaError_t launch_flat_search(const void* db, int64_t N, int d, const void* que
         }
         e = launch_gemm_select(G, s);
         if (e != cudaSuccess) return e;
-        flat_merge_kernel<<<nq, FSEL_THREADS, 0, s>>>(nsplit, k, cap, cand_cnt, cand, out_ids, out_scores);
+        flat_merge_kernel<<<nq, FSEL_THREADS, 0, s>>>(nlists, k, cap, cand_cnt, cand, out_ids, out_scores);
         count_launch();
         return cudaGetLastError();
     }

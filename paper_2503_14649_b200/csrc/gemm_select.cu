@@ -7,22 +7,29 @@
 // (x = x0 + x1 + x2 exactly up to 24 bits) and the product as the six part pairs whose weight is at
 // least 2^-16 relative; each pair is simply more K-blocks accumulated into the same TMEM tile.
 //
-// One CTA = 128 x 256 output tile, K-blocks of 64 bf16 (one 128-byte swizzle span):
-//   warp 0   TMA producer: cp.async.bulk.tensor (tiled, 128B swizzle) into a 4-stage ring, mbarrier tx counts
-//   warp 1   one lane issues tcgen05.mma (M128 N256 K16, bf16 -> fp32 in TMEM), tcgen05.commit frees stages
-//   warps 2-5 epilogue: tcgen05.ld 32 columns at a time, thread = output row; two TMEM accumulators
-//            (2 x 256 columns) let the epilogue of one tile overlap the MMAs of the next; the warps never
-//            wait for each other
-// A CTA owns a contiguous range of column tiles for one or two row tiles, so a row's running state
-// (threshold, candidate count) lives in the registers of the thread that owns the row.
+// One CTA works on 128 x 256 output tiles, K-blocks of 64 bf16 (one 128-byte swizzle span):
+//   warp 0    TMA producer: cp.async.bulk.tensor (tiled, 128B swizzle) into a ring of stages, mbarrier tx counts
+//   warp 1    one lane issues tcgen05.mma (M128 N256 K16, bf16 -> fp32 in TMEM), tcgen05.commit frees stages
+//   warps 2-9 epilogue: tcgen05.ld 32 columns at a time, thread = output row; warp w reads TMEM lane quarter
+//             w mod 4 and the column half (w - 2) / 4 of the tile, and never waits for another warp
+// Two shapes of the main loop (template parameter PAIR):
+//   PAIR = false   one row tile per CTA.  A stage holds A (16 KB) and B (32 KB), four stages; the two 256-column
+//                  TMEM accumulators alternate, so the epilogue of one tile overlaps the MMAs of the next.
+//   PAIR = true    two row tiles per CTA (256 queries).  A stage holds A0, A1 and ONE B tile (64 KB), three
+//                  stages; every K-block feeds two MMA chains, A0.B into accumulator 0 and A1.B into accumulator
+//                  1, so a B tile crosses L2 -> shared memory once per 256 queries and the operand traffic per
+//                  flop drops by a third.  Both accumulators belong to the same column tile, so the epilogue
+//                  does not overlap the next tile's MMAs; eight epilogue warps keep it short.
+// A CTA owns a contiguous range of column tiles, so a row's running state (threshold, candidate count) lives in
+// the registers of the thread that owns the (row, column half).
 //
-// Fused selection (mode 0).  A value below the row's threshold is appended to the row's candidate
-// list in global memory (capacity CAP = 32*NK keys, 64-bit key = ordered score bits << 32 | column).
-// When a list could overflow, its warp loads it into registers (NK keys per lane), bisects for a cut
-// value that keeps between nsel and nsel + slack keys (a few warp-wide counts), writes the kept keys
-// back and lowers the threshold.  The threshold is always at least the nsel-th smallest of a subset of
-// the row, so no key that belongs to the row's nsel best is ever dropped; the lists of all column ranges are merged
-// by the caller.  Mode 1 writes the score matrix instead.
+// Fused selection (mode 0).  A value below the row's threshold is appended to a candidate list in global memory
+// (one list per row, column range and column half; capacity CAP = 32*NK keys, 64-bit key = ordered score bits
+// << 32 | column).  When a list could overflow, its warp loads it into registers (NK keys per lane), bisects for
+// a cut value that keeps between nsel and nsel + slack keys (a few warp-wide counts), writes the kept keys back
+// and lowers the threshold.  The threshold is always at least the nsel-th smallest of a subset of the row, so no
+// key that belongs to the row's nsel best is ever dropped; the lists are merged by the caller.  Mode 1 writes
+// the score matrix instead.
 //
 // Pilot thresholds.  A row may start with a threshold instead of +inf: the caller first runs mode 1
 // over every 16th column (a tensor map with a 16-row stride: 6% more work) and takes, per row, the
@@ -39,14 +46,17 @@
 namespace rago {
 
 constexpr int GBM = 128, GBN = 256, GBK = 64;
-constexpr int G_STAGES = 4;
 constexpr int G_A_BYTES = GBM * GBK * 2;
 constexpr int G_B_BYTES = GBN * GBK * 2;
-constexpr int G_STAGE_BYTES = G_A_BYTES + G_B_BYTES;
-constexpr int G_THREADS = 192;
+constexpr int G_RING_BYTES = 4 * (G_A_BYTES + G_B_BYTES);  // four stages of A + B, or three of A0 + A1 + B
+constexpr int G_MAX_STAGES = 4;
+constexpr int G_EPI_WARPS = 8;                       // 4 TMEM lane quarters x 2 column halves
+constexpr int G_THREADS = 32 * (2 + G_EPI_WARPS);
+constexpr int G_HALF = GBN / GEMM_COL_HALVES;        // columns of a tile one epilogue warp reads
 constexpr int G_TMEM_COLS = 512;
-constexpr int G_CN_BYTES = 4 * 2 * GBN * 4;  // column terms: one copy per epilogue warp and accumulator
-constexpr int G_SMEM_BYTES = G_STAGES * G_STAGE_BYTES + G_CN_BYTES + 256 + 1024;  // + barriers + alignment slack
+constexpr int G_CN_BYTES = G_EPI_WARPS * 2 * G_HALF * 4;  // column terms: two copies per epilogue warp
+constexpr int G_SMEM_BYTES = G_RING_BYTES + G_CN_BYTES + 256 + 1024;  // + barriers + alignment slack
+static_assert(3 * (2 * G_A_BYTES + G_B_BYTES) <= G_RING_BYTES, "three paired stages fit the ring");
 
 // tcgen05 instruction descriptor, kind::f16: D = f32 (bits 4-5 = 1), A = B = bf16 (bits 7-9, 10-12 = 1),
 // both operands K-major (bits 15, 16 = 0), N >> 3 in bits 17-22, M >> 4 in bits 24-28.
@@ -105,19 +115,34 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
            ((uint64_t)2 << 61);
 }
 
-// if (score < tau) { *slot = key(score, col); ++cnt; }  without a branch
-__device__ __forceinline__ void push_if_below(unsigned long long* slot, float score, float tau, uint32_t col, int& cnt) {
-    const uint32_t u = __float_as_uint(score);
-    const uint32_t ord = u ^ ((uint32_t)((int32_t)u >> 31) | 0x80000000u);  // order-preserving bits (f32_orderable)
+// While the kernel runs, a candidate list holds RAW entries: low word = column, high word = the fp32 bits of the
+// score xor `sign` (sign = 0x80000000 on the alpha = -1 path, where the accumulator value itself is stored and
+// the score is its negation).  Appending is then a compare, a predicated 8-byte store and a predicated pointer
+// bump per value; the order-preserving key bits are formed once per kept entry when the CTA finishes.
+//   if (value > thr) { *ptr++ = {col, bits(value)}; }          (alpha = -1, no column term: score = -value)
+__device__ __forceinline__ void push_if_above(unsigned long long*& ptr, float value, float thr, uint32_t col) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.gt.f32 p, %1, %2;\n\t"
+        "@p st.global.v2.u32 [%0], {%3, %4};\n\t"
+        "@p add.u64 %0, %0, 8;\n\t}"
+        : "+l"(ptr)
+        : "f"(value), "f"(thr), "r"(col), "r"(__float_as_uint(value))
+        : "memory");
+}
+//   if (score < tau) { *ptr++ = {col, bits}; }
+__device__ __forceinline__ void push_if_below(unsigned long long*& ptr, float score, float tau, uint32_t col, uint32_t bits) {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.lt.f32 p, %1, %2;\n\t"
-        "@p st.global.v2.u32 [%3], {%4, %5};\n\t"
-        "@p add.s32 %0, %0, 1;\n\t}"
-        : "+r"(cnt)
-        : "f"(score), "f"(tau), "l"(slot), "r"(col), "r"(ord)
+        "@p st.global.v2.u32 [%0], {%3, %4};\n\t"
+        "@p add.u64 %0, %0, 8;\n\t}"
+        : "+l"(ptr)
+        : "f"(score), "f"(tau), "r"(col), "r"(bits)
         : "memory");
 }
+__device__ __forceinline__ uint32_t ord_bits(uint32_t u) { return u ^ ((uint32_t)((int32_t)u >> 31) | 0x80000000u); }
+__device__ __forceinline__ uint32_t unord_bits(uint32_t o) { return (o & 0x80000000u) ? (o & 0x7FFFFFFFu) : ~o; }
 
 struct GemmArgs {
     int nrows, ncols;            // valid rows of A (queries) and of B (lists / database rows)
@@ -125,15 +150,15 @@ struct GemmArgs {
     int kblocks;                 // ceil(d / 64)
     int nterms;
     int term_a[6], term_b[6];    // part pair of each term
-    int mtiles, ntiles, mg;      // row tiles, column tiles, row tiles per CTA (1 or 2)
+    int mtiles, ntiles;          // row tiles, column tiles
     float alpha;
     const float* colterm;        // [ncols * colterm_stride] or null: column c adds colterm[c * colterm_stride]
     int colterm_stride;
     const float* row_tau;        // [nrows] initial thresholds (mode 0) or null for +inf
     int mode;                    // 0: candidate lists, 1: score matrix
     int nsel;                    // keys a row must keep (mode 0)
-    unsigned long long* cand;    // [nrows][nsplit][CAP]
-    int32_t* cand_cnt;           // [nrows][nsplit]
+    unsigned long long* cand;    // [nrows][nsplit][GEMM_COL_HALVES][CAP]
+    int32_t* cand_cnt;           // [nrows][nsplit][GEMM_COL_HALVES]
     float* scores;               // [nrows][ncols] (mode 1)
     uint32_t* err;
 };
@@ -144,16 +169,18 @@ struct GemmArgs {
 // counts instead of one per bit; if it runs down to a single value (a tie group larger than the slack)
 // only as many of the tied keys are kept as are needed to reach nsel.  Every kept set contains the
 // nsel smallest keys of the list, and the threshold is the largest kept score.
+// The list is in the raw format described above (sign: see push_if_above) and stays in it.
 template <int NK>
-__device__ __forceinline__ float compact_list(unsigned long long* list, int n, int nsel, int nkeep, int lane, int* kept) {
+__device__ __forceinline__ float compact_list(unsigned long long* list, int n, int nsel, int nkeep, int lane, int* kept,
+                                              uint32_t sign) {
     uint32_t s[NK];
     uint32_t pl[NK];
     uint32_t mn = 0xFFFFFFFFu, mx = 0u;
 #pragma unroll
     for (int j = 0; j < NK; ++j) {
         const int idx = lane + 32 * j;
-        const unsigned long long k = idx < n ? list[idx] : KEY_MAX;
-        s[j] = (uint32_t)(k >> 32);
+        const unsigned long long k = idx < n ? list[idx] : 0ull;
+        s[j] = idx < n ? ord_bits((uint32_t)(k >> 32) ^ sign) : 0xFFFFFFFFu;
         pl[j] = (uint32_t)k;
         if (idx < n) {
             mn = s[j] < mn ? s[j] : mn;
@@ -191,7 +218,7 @@ __device__ __forceinline__ float compact_list(unsigned long long* list, int n, i
         const uint32_t meq = __ballot_sync(0xffffffffu, eq);
         const bool keep = valid && (s[j] < T || (eq && __popc(meq & lt_mask) < need));
         const uint32_t mk = __ballot_sync(0xffffffffu, keep);
-        if (keep) list[base + __popc(mk & lt_mask)] = ((unsigned long long)s[j] << 32) | pl[j];
+        if (keep) list[base + __popc(mk & lt_mask)] = ((unsigned long long)(unord_bits(s[j]) ^ sign) << 32) | pl[j];
         base += __popc(mk);
         const int eq_kept = __popc(meq) < need ? __popc(meq) : need;
         need -= eq_kept;
@@ -201,33 +228,128 @@ __device__ __forceinline__ float compact_list(unsigned long long* list, int n, i
     return orderable_f32(T);
 }
 
-template <int NK>
+// Epilogue of one accumulator half in mode 0: G_HALF columns starting at TMEM address taddr, global column col_g.
+// NEG1: alpha = -1 and no column term, so "score < tau" is "value > -tau" on the accumulator value itself and
+// nothing but the compare stands between the TMEM load and the store (chunks that reach past the last valid
+// column take the general path, whose column terms are +inf there).
+// (Measured and dropped: skipping pairs of columns behind a warp-wide vote when none of their 64 values passes.
+// Even at the flat search's pass rate of 0.3% the votes and branches cost more than the predicated stores save.)
+template <int NK, bool NEG1>
+__device__ __forceinline__ void epilogue_select(uint32_t taddr, const float* cn, float alpha, uint32_t col_g, int ncols,
+                                                unsigned long long* list, float& tau, int& cnt, int nsel, int nkeep,
+                                                int lane) {
+    constexpr int CAP = NK * 32;
+    constexpr uint32_t SIGN = NEG1 ? 0x80000000u : 0u;
+    unsigned long long* ptr = list + cnt;
+    unsigned long long* const full = list + (CAP - 32);
+#pragma unroll 1
+    for (int c0 = 0; c0 < G_HALF; c0 += 32) {
+        float v[32];
+        tmem_ld32(taddr + c0, v);
+        const uint32_t colc = col_g + c0;
+        if (NEG1 && (int)colc + 32 <= ncols) {
+            const float thr = -tau;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) push_if_above(ptr, v[j], thr, colc + j);
+        } else {
+            // all 32 scores first (their column-term loads must not queue behind the stores), then one
+            // predicated store per value: no branches, the only serial dependence is the list cursor
+            float sc[32];
+#pragma unroll
+            for (int j = 0; j < 32; j += 4) {
+                const float4 c4 = *reinterpret_cast<const float4*>(cn + c0 + j);
+                sc[j + 0] = fmaf(alpha, v[j + 0], c4.x);
+                sc[j + 1] = fmaf(alpha, v[j + 1], c4.y);
+                sc[j + 2] = fmaf(alpha, v[j + 2], c4.z);
+                sc[j + 3] = fmaf(alpha, v[j + 3], c4.w);
+            }
+#pragma unroll
+            for (int j = 0; j < 32; ++j) push_if_below(ptr, sc[j], tau, colc + j, __float_as_uint(sc[j]) ^ SIGN);
+        }
+        uint32_t todo = __ballot_sync(0xffffffffu, ptr > full);
+        while (todo) {  // warp-uniform
+            const int r = __ffs(todo) - 1;
+            todo &= todo - 1;
+            const int n = __shfl_sync(0xffffffffu, (int)(ptr - list), r);
+            const unsigned long long lp = __shfl_sync(0xffffffffu, (unsigned long long)list, r);
+            __syncwarp();
+            int kept = 0;
+            const float nt_tau =
+                compact_list<NK>(reinterpret_cast<unsigned long long*>(lp), n, nsel, nkeep, lane, &kept, SIGN);
+            if (lane == r) { ptr = list + kept; tau = nt_tau; }
+        }
+    }
+    cnt = (int)(ptr - list);
+}
+
+// Raw entries -> keys (ordered score bits << 32 | column), by the thread that owns the list.
+__device__ __forceinline__ void finish_list(unsigned long long* list, int cnt, uint32_t sign) {
+    for (int i = 0; i < cnt; ++i) {
+        const unsigned long long e = list[i];
+        list[i] = ((unsigned long long)ord_bits((uint32_t)(e >> 32) ^ sign) << 32) | (uint32_t)e;
+    }
+}
+
+// The same in mode 1: scores of row `row`, columns colb .. colb + G_HALF - 1, to the score matrix.
+__device__ __forceinline__ void epilogue_store(uint32_t taddr, const float* cn, float alpha, int row, int nrows,
+                                               int ncols, int colb0, float* scores) {
+#pragma unroll 1
+    for (int c0 = 0; c0 < G_HALF; c0 += 32) {
+        float v[32];
+        tmem_ld32(taddr + c0, v);
+        if (row < nrows) {
+            const int colb = colb0 + c0;
+            float* out = scores + (size_t)row * ncols + colb;
+            if ((ncols & 3) == 0 && colb + 32 <= ncols) {  // 16-byte stores: rows start on 16-byte boundaries
+#pragma unroll
+                for (int j = 0; j < 32; j += 4) {
+                    const float4 c4 = *reinterpret_cast<const float4*>(cn + c0 + j);
+                    float4 o;
+                    o.x = fmaf(alpha, v[j + 0], c4.x);
+                    o.y = fmaf(alpha, v[j + 1], c4.y);
+                    o.z = fmaf(alpha, v[j + 2], c4.z);
+                    o.w = fmaf(alpha, v[j + 3], c4.w);
+                    *reinterpret_cast<float4*>(out + j) = o;
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j)
+                    if (colb + j < ncols) out[j] = fmaf(alpha, v[j], cn[c0 + j]);
+            }
+        }
+    }
+}
+
+template <int NK, bool PAIR>
 __global__ void __launch_bounds__(G_THREADS, 1)
 gemm_select_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmArgs a) {
     constexpr int CAP = NK * 32;
+    constexpr int STAGES = PAIR ? 3 : 4;
+    constexpr int STAGE_BYTES = PAIR ? 2 * G_A_BYTES + G_B_BYTES : G_A_BYTES + G_B_BYTES;
+    constexpr int B_OFF = STAGE_BYTES - G_B_BYTES;  // B follows the A tile(s) of its stage
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;  // swizzled tiles need 1024-byte alignment
     uint8_t* smem = smem_raw + (base - raw);
-    float* cn_all = reinterpret_cast<float*>(smem + G_STAGES * G_STAGE_BYTES);  // [4 warps][2][GBN] column terms
-    unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + G_STAGES * G_STAGE_BYTES + G_CN_BYTES);
-    const uint32_t bar0 = base + G_STAGES * G_STAGE_BYTES + G_CN_BYTES;
+    float* cn_all = reinterpret_cast<float*>(smem + G_RING_BYTES);  // [8 warps][2][G_HALF] column terms
+    unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + G_RING_BYTES + G_CN_BYTES);
+    const uint32_t bar0 = base + G_RING_BYTES + G_CN_BYTES;
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
-    auto empty_bar = [&](int s) { return bar0 + 8u * (G_STAGES + s); };
-    auto tfull_bar = [&](int b) { return bar0 + 8u * (2 * G_STAGES + b); };
-    auto tempty_bar = [&](int b) { return bar0 + 8u * (2 * G_STAGES + 2 + b); };
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * G_STAGES + 4);
+    auto empty_bar = [&](int s) { return bar0 + 8u * (G_MAX_STAGES + s); };
+    auto tfull_bar = [&](int b) { return bar0 + 8u * (2 * G_MAX_STAGES + b); };
+    auto tempty_bar = [&](int b) { return bar0 + 8u * (2 * G_MAX_STAGES + 2 + b); };
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * G_MAX_STAGES + 4);
     volatile uint32_t* abort_flag = tmem_slot + 1;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
-        for (int s = 0; s < G_STAGES; ++s) {
+        for (int s = 0; s < STAGES; ++s) {
             mbar_init(full_bar(s), 1);
             mbar_init(empty_bar(s), 1);
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(tfull_bar(b), 1);
-            mbar_init(tempty_bar(b), 4);
+            mbar_init(tempty_bar(b), G_EPI_WARPS);
         }
         *abort_flag = 0;
         fence_barrier_init();
@@ -239,149 +361,126 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
+    // PAIR: blockIdx.y counts pairs of row tiles (the last pair may hold one tile); else row tiles.
     const int split = blockIdx.x, nsplit = gridDim.x;
-    const int m0 = blockIdx.y * a.mg;
-    const int mcount = (a.mtiles - m0) < a.mg ? (a.mtiles - m0) : a.mg;
+    const int m0 = PAIR ? blockIdx.y * 2 : blockIdx.y;
+    const int mcount = PAIR ? ((a.mtiles - m0) < 2 ? (a.mtiles - m0) : 2) : 1;
     const int nt_begin = (int)((long long)split * a.ntiles / nsplit);
     const int nt_end = (int)((long long)(split + 1) * a.ntiles / nsplit);
-    const int nunits = (nt_end - nt_begin) * mcount;
+    const int nunits = nt_end - nt_begin;  // column tiles of this CTA
     const int kiters = a.nterms * a.kblocks;
 
     if (warp == 0) {
         // ================= TMA producer =================
         if (lane == 0) {
-            // unit u = (column tile nt, row tile m), m fastest; inside it the terms, inside a term the k-blocks:
-            // kept by counting, no division per load
+            // unit = column tile; inside it the terms, inside a term the k-blocks: kept by counting, no division per load
             const int total = nunits * kiters;
-            int nt = nt_begin, mi = 0, t = 0, kb = 0;
+            const uint32_t tx_bytes = (uint32_t)(mcount == 2 ? STAGE_BYTES : G_A_BYTES + G_B_BYTES);
+            int nt = nt_begin, t = 0, kb = 0, s = 0;
+            uint32_t ph = 0;
             for (int gi = 0; gi < total; ++gi) {
-                const int s = gi % G_STAGES;
-                const uint32_t ph = (uint32_t)(gi / G_STAGES) & 1u;
                 const int kx = kb * GBK;
-                const int ya = a.term_a[t] * a.a_part_rows + (m0 + mi) * GBM;
+                const int ya = a.term_a[t] * a.a_part_rows + m0 * GBM;
                 const int yb = a.term_b[t] * a.b_part_rows + nt * GBN;
                 if (++kb == a.kblocks) {
                     kb = 0;
-                    if (++t == a.nterms) {
-                        t = 0;
-                        if (++mi == mcount) { mi = 0; ++nt; }
-                    }
+                    if (++t == a.nterms) { t = 0; ++nt; }
                 }
                 if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, a.err, 64)) break;
-                mbar_arrive_expect_tx(full_bar(s), G_STAGE_BYTES);
-                tma_load_2d(&tmA, full_bar(s), base + s * G_STAGE_BYTES, kx, ya);
-                tma_load_2d(&tmB, full_bar(s), base + s * G_STAGE_BYTES + G_A_BYTES, kx, yb);
+                const uint32_t st = base + s * STAGE_BYTES;
+                mbar_arrive_expect_tx(full_bar(s), tx_bytes);
+                tma_load_2d(&tmA, full_bar(s), st, kx, ya);
+                if (PAIR && mcount == 2) tma_load_2d(&tmA, full_bar(s), st + G_A_BYTES, kx, ya + GBM);
+                tma_load_2d(&tmB, full_bar(s), st + B_OFF, kx, yb);
+                if (++s == STAGES) { s = 0; ph ^= 1u; }
             }
         }
     } else if (warp == 1) {
         // ================= MMA issuer =================
         if (lane == 0) {
-            uint32_t it = 0;
+            int s = 0;
+            uint32_t ph = 0;
             bool dead = false;
             for (int u = 0; u < nunits && !dead; ++u) {
-                const int buf = u & 1;
-                const uint32_t uph = (u >> 1) & 1u;
+                // PAIR: both accumulators belong to this unit, one barrier pair; else the accumulators alternate
+                const int buf = PAIR ? 0 : (u & 1);
+                const uint32_t uph = PAIR ? (u & 1u) : ((u >> 1) & 1u);
                 if (!mbar_wait(tempty_bar(buf), uph ^ 1u, abort_flag, a.err, 64)) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * GBN);
-                for (int ki = 0; ki < kiters; ++ki, ++it) {
-                    const int s = it % G_STAGES;
-                    const uint32_t ph = (it / G_STAGES) & 1u;
+                for (int ki = 0; ki < kiters; ++ki) {
                     if (!mbar_wait(full_bar(s), ph, abort_flag, a.err, 32)) { dead = true; break; }
                     tc_fence_after();
-                    const uint64_t da = smem_desc_sw128(base + s * G_STAGE_BYTES);
-                    const uint64_t db = smem_desc_sw128(base + s * G_STAGE_BYTES + G_A_BYTES);
+                    const uint32_t st = base + s * STAGE_BYTES;
+                    const uint64_t da = smem_desc_sw128(st);
+                    const uint64_t db = smem_desc_sw128(st + B_OFF);
 #pragma unroll
                     for (int k = 0; k < GBK / 16; ++k)
                         tc_mma_bf16(d_tmem, da + 2u * k, db + 2u * k, G_IDESC, (ki | k) != 0 ? 1u : 0u);
+                    if (PAIR && mcount == 2) {
+                        const uint64_t da1 = smem_desc_sw128(st + G_A_BYTES);
+#pragma unroll
+                        for (int k = 0; k < GBK / 16; ++k)
+                            tc_mma_bf16(d_tmem + GBN, da1 + 2u * k, db + 2u * k, G_IDESC, (ki | k) != 0 ? 1u : 0u);
+                    }
                     tc_commit(empty_bar(s));  // frees the stage once these MMAs have read it
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
-                if (!dead) tc_commit(tfull_bar(buf));  // accumulator complete
+                if (!dead) tc_commit(tfull_bar(buf));  // accumulator(s) complete
             }
         }
     } else {
         // ================= epilogue warps =================
-        const int q4 = warp & 3;  // TMEM lane quarter this warp may read
-        float* cn = cn_all + (warp - 2) * 2 * GBN;  // this warp's own copy: no cross-warp barrier needed
+        const int ew = warp - 2;
+        const int q4 = warp & 3;   // TMEM lane quarter this warp may read
+        const int half = ew >> 2;  // column half of the tile: warps 2-5 take half 0, warps 6-9 half 1
+        float* cn = cn_all + ew * 2 * G_HALF;  // this warp's own copies: no cross-warp barrier needed
         const float inf = __int_as_float(0x7f800000);
-        float tau0 = inf, tau1 = inf;
-        int cnt0 = 0, cnt1 = 0;
-        {
-            const int r0 = m0 * GBM + q4 * 32 + lane, r1 = r0 + GBM;
-            if (r0 >= a.nrows) tau0 = -inf; else if (a.row_tau) tau0 = a.row_tau[r0];
-            if (r1 >= a.nrows || mcount < 2) tau1 = -inf; else if (a.row_tau) tau1 = a.row_tau[r1];
+        float tau[2] = {inf, inf};
+        int cnt[2] = {0, 0};
+#pragma unroll
+        for (int g = 0; g < 2; ++g) {
+            const int r = (m0 + g) * GBM + q4 * 32 + lane;
+            if (r >= a.nrows || g >= mcount) tau[g] = -inf; else if (a.row_tau) tau[g] = a.row_tau[r];
+        }
+        const int slack = a.nsel / 4 > 8 ? a.nsel / 4 : 8;
+        const int nkeep = a.nsel + slack < CAP - 64 ? a.nsel + slack : CAP - 64;  // what the bisection may leave in a list
+        const bool neg1 = a.alpha == -1.f && a.colterm == nullptr;  // accumulator values are compared and stored as they are
+        unsigned long long* lists[2];
+#pragma unroll
+        for (int g = 0; g < 2; ++g) {  // never written for padding rows
+            const int r = (m0 + g) * GBM + q4 * 32 + lane;
+            lists[g] = a.cand + (((size_t)(r < a.nrows ? r : 0) * nsplit + split) * GEMM_COL_HALVES + half) * CAP;
         }
         bool dead = false;
         for (int u = 0; u < nunits && !dead; ++u) {
-            const int nt = nt_begin + (mcount == 2 ? u >> 1 : u), g = mcount == 2 ? u & 1 : 0;  // mcount is 1 or 2
-            const int buf = u & 1;
-            const uint32_t uph = (u >> 1) & 1u;
-            for (int i = lane; i < GBN; i += 32) {
-                const int col = nt * GBN + i;
-                cn[buf * GBN + i] = col < a.ncols ? (a.colterm ? __ldg(a.colterm + (size_t)col * a.colterm_stride) : 0.f) : inf;
+            const int nt = nt_begin + u;
+            const int buf = PAIR ? 0 : (u & 1);
+            const uint32_t uph = PAIR ? (u & 1u) : ((u >> 1) & 1u);
+            float* cnu = cn + (u & 1) * G_HALF;
+            const int colb = nt * GBN + half * G_HALF;
+            for (int i = lane; i < G_HALF; i += 32) {
+                const int col = colb + i;
+                cnu[i] = col < a.ncols ? (a.colterm ? __ldg(a.colterm + (size_t)col * a.colterm_stride) : 0.f) : inf;
             }
             __syncwarp();
             if (!mbar_wait(tfull_bar(buf), uph, abort_flag, a.err)) { dead = true; break; }
             tc_fence_after();
-            const int row = (m0 + g) * GBM + q4 * 32 + lane;
-            const uint32_t taddr = tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(buf * GBN);
-            if (a.mode == 0) {
-                float tau = g ? tau1 : tau0;
-                int cnt = g ? cnt1 : cnt0;
-                unsigned long long* list =
-                    a.cand + ((size_t)(row < a.nrows ? row : 0) * nsplit + split) * CAP;  // never written for padding rows
-                const int slack = a.nsel / 4 > 8 ? a.nsel / 4 : 8;
-                const int nkeep = a.nsel + slack < CAP - 64 ? a.nsel + slack : CAP - 64;  // what the bisection may leave in a list
-#pragma unroll 1
-                for (int c0 = 0; c0 < GBN; c0 += 32) {
-                    float v[32];
-                    tmem_ld32(taddr + c0, v);
-                    // all 32 scores first (their column-term loads must not queue behind the stores), then one
-                    // predicated store per value: no branches, the only serial dependence is the list cursor
-                    const uint32_t col0 = (uint32_t)(nt * GBN + c0);
-                    float sc[32];
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) sc[j] = fmaf(a.alpha, v[j], cn[buf * GBN + c0 + j]);
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) push_if_below(list + cnt, sc[j], tau, col0 + j, cnt);
-                    uint32_t todo = __ballot_sync(0xffffffffu, cnt > CAP - 32);
-                    while (todo) {  // warp-uniform
-                        const int r = __ffs(todo) - 1;
-                        todo &= todo - 1;
-                        const int n = __shfl_sync(0xffffffffu, cnt, r);
-                        const unsigned long long lp = __shfl_sync(0xffffffffu, (unsigned long long)list, r);
-                        __syncwarp();
-                        int kept = 0;
-                        const float nt_tau =
-                            compact_list<NK>(reinterpret_cast<unsigned long long*>(lp), n, a.nsel, nkeep, lane, &kept);
-                        if (lane == r) { cnt = kept; tau = nt_tau; }
-                    }
-                }
-                if (g) { tau1 = tau; cnt1 = cnt; } else { tau0 = tau; cnt0 = cnt; }
-            } else {
-#pragma unroll 1
-                for (int c0 = 0; c0 < GBN; c0 += 32) {
-                    float v[32];
-                    tmem_ld32(taddr + c0, v);
-                    if (row < a.nrows) {
-                        const int colb = nt * GBN + c0;
-                        float* out = a.scores + (size_t)row * a.ncols + colb;
-                        if ((a.ncols & 3) == 0 && colb + 32 <= a.ncols) {  // 16-byte stores: rows start on 16-byte boundaries
-#pragma unroll
-                            for (int j = 0; j < 32; j += 4) {
-                                float4 o;
-                                o.x = fmaf(a.alpha, v[j + 0], cn[buf * GBN + c0 + j + 0]);
-                                o.y = fmaf(a.alpha, v[j + 1], cn[buf * GBN + c0 + j + 1]);
-                                o.z = fmaf(a.alpha, v[j + 2], cn[buf * GBN + c0 + j + 2]);
-                                o.w = fmaf(a.alpha, v[j + 3], cn[buf * GBN + c0 + j + 3]);
-                                *reinterpret_cast<float4*>(out + j) = o;
-                            }
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 32; ++j)
-                                if (colb + j < a.ncols) out[j] = fmaf(a.alpha, v[j], cn[buf * GBN + c0 + j]);
-                        }
-                    }
+            for (int g = 0; g < (PAIR ? 2 : 1); ++g) {
+                if (g >= mcount) break;
+                const int row = (m0 + g) * GBM + q4 * 32 + lane;
+                const uint32_t taddr = tmem_base + ((uint32_t)(q4 * 32) << 16) +
+                                       (uint32_t)((PAIR ? g : buf) * GBN + half * G_HALF);
+                if (a.mode == 0) {
+                    if (neg1)
+                        epilogue_select<NK, true>(taddr, cnu, a.alpha, (uint32_t)colb, a.ncols, lists[g], tau[g], cnt[g],
+                                                  a.nsel, nkeep, lane);
+                    else
+                        epilogue_select<NK, false>(taddr, cnu, a.alpha, (uint32_t)colb, a.ncols, lists[g], tau[g], cnt[g],
+                                                   a.nsel, nkeep, lane);
+                } else {
+                    epilogue_store(taddr, cnu, a.alpha, row, a.nrows, a.ncols, colb, a.scores);
                 }
             }
             tc_fence_before();
@@ -389,9 +488,14 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             if (lane == 0) mbar_arrive(tempty_bar(buf));
         }
         if (a.mode == 0 && !dead) {
-            const int r0 = m0 * GBM + q4 * 32 + lane, r1 = r0 + GBM;
-            if (r0 < a.nrows) a.cand_cnt[(size_t)r0 * nsplit + split] = cnt0;
-            if (mcount == 2 && r1 < a.nrows) a.cand_cnt[(size_t)r1 * nsplit + split] = cnt1;
+#pragma unroll
+            for (int g = 0; g < 2; ++g) {
+                const int r = (m0 + g) * GBM + q4 * 32 + lane;
+                if (g < mcount && r < a.nrows) {
+                    finish_list(lists[g], cnt[g], neg1 ? 0x80000000u : 0u);
+                    a.cand_cnt[((size_t)r * nsplit + split) * GEMM_COL_HALVES + half] = cnt[g];
+                }
+            }
         }
     }
 
@@ -472,18 +576,23 @@ cudaError_t launch_gemm_select(const GemmLaunch& L, cudaStream_t s) {
     for (int t = 0; t < 6; ++t) { a.term_a[t] = L.term_a[t]; a.term_b[t] = L.term_b[t]; }
     a.mtiles = (L.nrows + GBM - 1) / GBM;
     a.ntiles = (int)((L.ncols + GBN - 1) / GBN);
-    a.mg = L.mg;
     a.alpha = L.alpha; a.colterm = L.colterm; a.colterm_stride = L.colterm_stride > 0 ? L.colterm_stride : 1;
     a.row_tau = L.row_tau;
     a.mode = L.mode; a.nsel = L.nsel;
     a.cand = L.cand; a.cand_cnt = L.cand_cnt; a.scores = L.scores; a.err = L.err;
-    const dim3 grid(L.nsplit, (a.mtiles + L.mg - 1) / L.mg);
+    const bool pair = L.mg == 2;
+    const dim3 grid(L.nsplit, pair ? (a.mtiles + 1) / 2 : a.mtiles);
     const CUtensorMap* ma = reinterpret_cast<const CUtensorMap*>(L.tmap_a);
     const CUtensorMap* mb = reinterpret_cast<const CUtensorMap*>(L.tmap_b);
-    if (L.mode == 0 && L.cap == GEMM_CAP_LARGE)
-        gemm_select_kernel<GEMM_CAP_LARGE / 32><<<grid, G_THREADS, G_SMEM_BYTES, s>>>(*ma, *mb, a);
+    const bool large = L.mode == 0 && L.cap == GEMM_CAP_LARGE;
+    if (large && pair)
+        gemm_select_kernel<GEMM_CAP_LARGE / 32, true><<<grid, G_THREADS, G_SMEM_BYTES, s>>>(*ma, *mb, a);
+    else if (large)
+        gemm_select_kernel<GEMM_CAP_LARGE / 32, false><<<grid, G_THREADS, G_SMEM_BYTES, s>>>(*ma, *mb, a);
+    else if (pair)
+        gemm_select_kernel<GEMM_CAP_SMALL / 32, true><<<grid, G_THREADS, G_SMEM_BYTES, s>>>(*ma, *mb, a);
     else
-        gemm_select_kernel<GEMM_CAP_SMALL / 32><<<grid, G_THREADS, G_SMEM_BYTES, s>>>(*ma, *mb, a);
+        gemm_select_kernel<GEMM_CAP_SMALL / 32, false><<<grid, G_THREADS, G_SMEM_BYTES, s>>>(*ma, *mb, a);
     count_launch();
     return cudaGetLastError();
 }
@@ -568,9 +677,13 @@ cudaError_t launch_row_tau(const float* scores, int nrows, int n, int nsel, floa
 
 // Per-device set-up: the kernels' dynamic shared-memory limits (called at index load and by the flat search).
 cudaError_t gemm_select_init() {
-    cudaError_t e = cudaFuncSetAttribute(gemm_select_kernel<GEMM_CAP_SMALL / 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(gemm_select_kernel<GEMM_CAP_SMALL / 32, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_SMEM_BYTES);
     if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(gemm_select_kernel<GEMM_CAP_LARGE / 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_SMEM_BYTES);
+        e = cudaFuncSetAttribute(gemm_select_kernel<GEMM_CAP_SMALL / 32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_SMEM_BYTES);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(gemm_select_kernel<GEMM_CAP_LARGE / 32, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_SMEM_BYTES);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(gemm_select_kernel<GEMM_CAP_LARGE / 32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_SMEM_BYTES);
     if (e == cudaSuccess)  // rows of up to 51 200 pilot scores in shared memory
         e = cudaFuncSetAttribute(row_tau_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     return e;

@@ -7,8 +7,11 @@
 
 namespace rago {
 
-// Scratch of the no-allocation entry point.  Every GPU that loads the library reserves these bytes
-// until the process exits, whether or not the entry point is ever called.
+// Scratch of the no-allocation entry point.  The array is part of the library image: a GPU holds these bytes
+// from the moment the runtime loads this module on it until the process exits.  The runtime loads modules on
+// first use, so that moment is the first look-up of the array's address on the device, which rago_index_load
+// does (noalloc_prepare below): the memory is claimed, and a failure reported, when an index is loaded, not
+// in the middle of serving.
 static __device__ __align__(256) unsigned char g_static_scratch[RAGO_NOALLOC_SCRATCH_BYTES];
 
 constexpr int MAX_DEVICES = 64;
@@ -33,6 +36,12 @@ static cudaError_t scratch_address(void** out) {
     return cudaSuccess;
 }
 
+// Called by rago_index_load with the index's device current: resolves (and thereby makes resident) the array.
+cudaError_t noalloc_prepare() {
+    void* p = nullptr;
+    return scratch_address(&p);
+}
+
 }  // namespace rago
 
 using namespace rago;
@@ -50,6 +59,11 @@ extern "C" rago_status rago_search_probes_noalloc(const rago_index* index, const
     if (nprobe > MAX_K) { set_error("nprobe = %d exceeds %d", nprobe, MAX_K); return RAGO_EUNSUPPORTED; }
     if (nq == 0) return RAGO_OK;
     if (!queries || !out_lists || !out_coarse) { set_error("null pointer"); return RAGO_EINVAL; }
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev != ix->device) {  // the array's address is per device
+        set_error("the current device (%d) is not the index's device (%d)", dev, ix->device);
+        return RAGO_EINVAL;
+    }
     if (reinterpret_cast<uintptr_t>(queries) % 16) { set_error("queries need 16-byte alignment"); return RAGO_EALIGN; }
     // layout inside the fixed array: [scores nq*nlist f32][bias nq*nprobe f32], each 256-byte aligned
     const size_t scores_bytes = align_up((size_t)nq * ix->nlist * 4, 256);
@@ -61,7 +75,7 @@ extern "C" rago_status rago_search_probes_noalloc(const rago_index* index, const
                   (long long)nq * ix->nlist, need, (int)RAGO_NOALLOC_SCRATCH_BYTES);
         return RAGO_ENOMEM;
     }
-    void* base = nullptr;
+    void* base = nullptr;  // cached since rago_index_load; the look-up below only runs if that one failed
     cudaError_t e = scratch_address(&base);
     if (e != cudaSuccess) { set_error("cudaGetSymbolAddress(scratch): %s", cudaGetErrorString(e)); return RAGO_ECUDA; }
     float* scores = reinterpret_cast<float*>(base);

@@ -16,17 +16,22 @@ def host_index(oracle, data):
                         coarse_bf16=cen.dtype == torch.bfloat16)
 
 
-def match_results(ids_a, d_a, ids_o, d_o, rel=1e-4, floor=1e-6):
+def match_results(ids_a, d_a, ids_o, d_o, rel=1e-4, floor=1e-6, rescore=None):
     """Compare one query's result list (a) with the oracle's (o).
 
-    Distances must agree position by position within `rel` (relative, with an
-    absolute floor); ids must be equal except inside groups of oracle
-    distances that tie within the same tolerance, where any order and any
-    member of the tie group at the list's tail is accepted.
+    Distances (smaller = better) must agree position by position within `rel` (relative, with an
+    absolute floor).  ids must be equal except inside groups of oracle distances that tie within the
+    same tolerance: an id the oracle lists elsewhere must sit in such a tie group with position t; an
+    id the oracle does not list at all (the tie group cut by k) is scored by the ORACLE through
+    `rescore(id) -> distance` and that value must tie with the oracle's entry at t.  Without a
+    `rescore` such an id is reported as unverified.  No id may appear twice (padding excepted).
     Returns a list of problems (empty = match).
     """
     problems = []
     k = len(ids_o)
+    real = [int(i) for i, d in zip(ids_a, d_a) if not np.isinf(d)]
+    if len(set(real)) != len(real):
+        problems.append((-1, "duplicate ids", 0, 0.0, 0, 0.0))
     scale = max(floor, float(np.max(np.abs(d_o[np.isfinite(d_o)]))) if np.isfinite(d_o).any() else floor)
     for t in range(k):
         if np.isinf(d_o[t]) or np.isinf(d_a[t]):
@@ -38,17 +43,56 @@ def match_results(ids_a, d_a, ids_o, d_o, rel=1e-4, floor=1e-6):
             problems.append((t, "dist", int(ids_a[t]), float(d_a[t]), int(ids_o[t]), float(d_o[t])))
             continue
         if ids_a[t] != ids_o[t]:
-            # accept when the oracle has this id at a position whose distance ties with position t,
-            # or when position t ties with the last oracle entry (tie group cut by k)
             where = np.nonzero(ids_o == ids_a[t])[0]
-            ok = False
-            if where.size and abs(float(d_o[where[0]]) - float(d_o[t])) <= 2 * tol:
-                ok = True
-            elif not where.size and abs(float(d_o[k - 1]) - float(d_o[t])) <= 2 * tol:
-                ok = True
+            if where.size:
+                ok = abs(float(d_o[where[0]]) - float(d_o[t])) <= 2 * tol
+                what = "id"
+            elif rescore is None:
+                ok, what = False, "id not in the oracle's list and no rescore given"
+            else:
+                try:
+                    own = float(rescore(int(ids_a[t])))
+                    ok = abs(own - float(d_o[t])) <= 2 * tol and abs(own - float(d_o[k - 1])) <= 2 * tol
+                    what = "id outside the oracle's list: oracle distance %r" % own
+                except KeyError:
+                    ok, what = False, "id unknown to the oracle"
             if not ok:
-                problems.append((t, "id", int(ids_a[t]), float(d_a[t]), int(ids_o[t]), float(d_o[t])))
+                problems.append((t, what, int(ids_a[t]), float(d_a[t]), int(ids_o[t]), float(d_o[t])))
     return problems
+
+
+class IvfPqRescorer:
+    """Oracle distance of a single stored vector, looked up by id: what match_results needs for ids the
+    oracle's own list does not contain.  Built over an oracle.Index (ids are unique)."""
+
+    def __init__(self, oracle, hix):
+        self.oracle, self.hix = oracle, hix
+        self.order = np.argsort(hix.ids, kind="stable")
+        self.sorted_ids = hix.ids[self.order]
+
+    def position(self, ident):
+        j = int(np.searchsorted(self.sorted_ids, ident))
+        if j >= self.sorted_ids.size or int(self.sorted_ids[j]) != int(ident):
+            raise KeyError(ident)
+        pos = int(self.order[j])
+        return int(np.searchsorted(self.hix.offsets, pos, side="right") - 1), pos
+
+    def for_query(self, query, sign=1.0):
+        """callable id -> sign * oracle score of that vector for `query` (KeyError for an unknown id)."""
+        def f(ident):
+            lst, pos = self.position(ident)
+            return sign * self.oracle.adc_score(self.hix, query, lst, pos)
+        return f
+
+
+def coarse_rescorer(oracle, centroids_host, query, metric, coarse_bf16, sign=1.0):
+    """callable list number -> sign * oracle coarse score of that list for `query`."""
+    def f(lst):
+        if lst < 0 or lst >= centroids_host.shape[0]:
+            raise KeyError(lst)
+        _, sc = oracle.coarse(centroids_host[lst:lst + 1], query[None, :], 1, metric, coarse_bf16=coarse_bf16)
+        return sign * float(sc[0, 0])
+    return f
 
 
 def compact_hashed_subindex(oracle, data, lists):

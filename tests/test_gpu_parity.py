@@ -8,7 +8,7 @@ import torch
 
 import oracle
 from paper_2503_14649_b200 import binding, synth
-from tests.helpers import host_index, match_results
+from tests.helpers import IvfPqRescorer, coarse_rescorer, host_index, match_results
 
 pytestmark = pytest.mark.gpu
 
@@ -35,18 +35,20 @@ def _compare(data, nprobe, k, rel=REL, max_probe_mismatch=0):
                           nthreads=oracle.default_threads())
     gi, gd, gl, gc = _gpu_search(data, nprobe, k)
     bad_probe_queries = 0
+    rs = IvfPqRescorer(oracle, hix)
     for i in range(q.shape[0]):
         # probe lists: same lists in the same order, except where coarse scores tie within tolerance
         if not np.array_equal(gl[i], op[i]):
             sgn = 1.0 if data.metric == "l2" else -1.0
-            assert not match_results(gl[i].astype(np.int64), sgn * gc[i], op[i].astype(np.int64), sgn * oc[i],
-                                     rel=rel), ("probe order", i, gl[i], op[i])
+            assert not match_results(gl[i].astype(np.int64), sgn * gc[i], op[i].astype(np.int64), sgn * oc[i], rel=rel,
+                                     rescore=coarse_rescorer(oracle, hix.centroids, q[i], data.metric, data.coarse_bf16, sgn)
+                                     ), ("probe order", i, gl[i], op[i])
             if set(gl[i].tolist()) != set(op[i].tolist()):
                 bad_probe_queries += 1
                 continue  # a different list was probed at a coarse tie: final results legitimately differ
         assert np.allclose(gc[i], oc[i], rtol=rel, atol=rel * max(1.0, np.abs(oc[i]).max())), ("coarse", i)
         sgn = 1.0 if data.metric == "l2" else -1.0
-        problems = match_results(gi[i], sgn * gd[i], oi[i], sgn * od[i], rel=rel)
+        problems = match_results(gi[i], sgn * gd[i], oi[i], sgn * od[i], rel=rel, rescore=rs.for_query(q[i], sgn))
         assert not problems, ("query %d" % i, problems[:5])
     assert bad_probe_queries <= max_probe_mismatch
     return gi, gd
@@ -116,6 +118,7 @@ def test_iterative_small_batches_back_to_back():
     workspace; each must equal the oracle's answer for its own queries."""
     data = synth.make_ivfpq_hashed(300_000, 512, 256, 32, 64, metric="l2", seed=41)
     hix = host_index(oracle, data)
+    rs = IvfPqRescorer(oracle, hix)
     ix = binding.load_index_from(data, "cuda")
     q = data.queries.cuda()
     outs = []
@@ -127,9 +130,11 @@ def test_iterative_small_batches_back_to_back():
     torch.cuda.synchronize()
     ix.rago_check()
     for pos, nb, gi, gd in outs:
-        oi, od = oracle.ivfpq_search(hix, data.queries[pos:pos + nb].numpy(), 16, 20)
+        qh = data.queries[pos:pos + nb].numpy()
+        oi, od = oracle.ivfpq_search(hix, qh, 16, 20)
         for i in range(nb):
-            assert not match_results(gi[i].cpu().numpy(), gd[i].cpu().numpy(), oi[i], od[i], rel=REL)
+            assert not match_results(gi[i].cpu().numpy(), gd[i].cpu().numpy(), oi[i], od[i], rel=REL,
+                                     rescore=rs.for_query(qh[i]))
     ix.close()
 
 
@@ -158,8 +163,13 @@ def test_flat_search_matches_oracle(N, d, nq, k):
     oi, osc = oracle.flat_search(db.view(torch.uint16).numpy(), q.view(torch.uint16).numpy(), k,
                                  nthreads=oracle.default_threads())
     gi, gs = gi.cpu().numpy(), gs.cpu().numpy()
+    db_bits, q_bits = db.view(torch.uint16).numpy(), q.view(torch.uint16).numpy()
     for i in range(nq):
-        assert not match_results(gi[i], -gs[i], oi[i], -osc[i], rel=1e-3), i
+        def rescore(row, i=i):
+            if row < 0 or row >= N:
+                raise KeyError(row)
+            return -float(oracle.flat_scores(db_bits, q_bits[i], np.array([row], np.int64))[0])
+        assert not match_results(gi[i], -gs[i], oi[i], -osc[i], rel=1e-3, rescore=rescore), i
 
 
 def test_argument_errors_are_reported_before_any_launch():

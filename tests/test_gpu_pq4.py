@@ -25,8 +25,23 @@ def _compare(data, nprobe, k):
     gi, gd = gi.cpu().numpy(), gd.cpu().numpy()
     ix.close()
     sgn = 1.0 if data.metric == "l2" else -1.0
+    ids_h, off_h, qh = data.ids.numpy(), data.list_offsets.numpy(), data.queries.numpy()
+    order = np.argsort(ids_h, kind="stable")
     for i in range(gi.shape[0]):
-        assert not match_results(gi[i], sgn * gd[i], oi[i], sgn * od[i], rel=1e-4), i
+        def rescore(ident, i=i):
+            # the oracle's score of that one vector: a search of its own list alone, restricted to the vector
+            j = int(np.searchsorted(ids_h[order], ident))
+            if j >= ids_h.size or int(ids_h[order][j]) != ident:
+                raise KeyError(ident)
+            pos = int(order[j])
+            lst = int(np.searchsorted(off_h, pos, side="right") - 1)
+            one_off = np.zeros_like(off_h)
+            one_off[lst + 1:] = 1
+            si, sd = oracle.ivfpq4_search(cen, data.codebooks.numpy(), data.codes.numpy()[pos:pos + 1], one_off,
+                                          ids_h[pos:pos + 1], data.metric, qh[i:i + 1], cen.shape[0], 1, coarse_bf16=bf16)
+            assert int(si[0, 0]) == ident
+            return sgn * float(sd[0, 0])
+        assert not match_results(gi[i], sgn * gd[i], oi[i], sgn * od[i], rel=1e-4, rescore=rescore), i
 
 
 @pytest.mark.parametrize("N,d,nlist,M4,nq,nprobe,k,metric,bf16", [

@@ -8,7 +8,7 @@ import torch
 
 import oracle
 from paper_2503_14649_b200 import binding, sharded, synth
-from tests.helpers import host_index, match_results
+from tests.helpers import IvfPqRescorer, host_index, match_results
 
 pytestmark = pytest.mark.gpu
 
@@ -98,11 +98,17 @@ def test_sharded_search_on_one_gpu_matches_oracle(metric, S, nprobe, k):
         ix.close()
     gi, gd = binding.rago_merge_results(torch.stack(parts_i), torch.stack(parts_d), k, metric)
     gi, gd = gi.cpu().numpy(), gd.cpu().numpy()
-    oi, od = oracle.sharded_search([host_index(oracle, sh) for sh in shards], shards[0].queries.numpy(), nprobe, k,
-                                   nthreads=oracle.default_threads())
+    hixs = [host_index(oracle, sh) for sh in shards]
+    oi, od = oracle.sharded_search(hixs, shards[0].queries.numpy(), nprobe, k, nthreads=oracle.default_threads())
     sgn = 1.0 if metric == "l2" else -1.0
+    rss = [IvfPqRescorer(oracle, h) for h in hixs]
+    qh = shards[0].queries.numpy()
     for i in range(q.shape[0]):
-        assert not match_results(gi[i], sgn * gd[i], oi[i], sgn * od[i], rel=1e-4), i
+        def rescore(ident, i=i):  # ids are s * 30 000 + a permutation: the owning shard scores its vector
+            if ident < 0 or ident >= S * 30_000:
+                raise KeyError(ident)
+            return rss[ident // 30_000].for_query(qh[i], sgn)(ident)
+        assert not match_results(gi[i], sgn * gd[i], oi[i], sgn * od[i], rel=1e-4, rescore=rescore), i
     owners = np.unique(oi[oi >= 0] // 30_000)
     assert owners.size == S                                  # every shard contributes to the answers
 
