@@ -1,21 +1,25 @@
 #!/usr/bin/env python
-"""Benchmark of the retrieval hot path on the Mid IVF-PQ workload.
+"""Benchmark of the retrieval hot path.
 
-A step is one rago_search over a batch of 1024 queries (coarse distances + nprobe selection,
-table build, list scan, top-k merge) against a seeded synthetic index of 10 M vectors
-(d = 768, nlist = 4096 Zipf(1.1)-skewed lists, 96-byte PQ codes), nprobe = 32, k = 100.
+Headline workload: the Hyperscale-shaped IVF-PQ index, the largest of the five shapes that one B200 holds
+(1e9 vectors stored as 64-byte PQ codes = 64 GB, 65 536 bf16 coarse centroids, inner product).  A step is one
+rago_search over a batch of 4096 queries (coarse distances on the tensor cores + nprobe selection, table build,
+list scan, top-k merge), nprobe = 64, k = 100.  The other four shapes (Mid IVF-PQ, flat search, the Hyperscale
+coarse step alone, the iterative-retrieval stream) are measured in the same run and nested under "secondary".
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
 
-With N > 1 (under torchrun) every rank holds a replica of the index and searches its own batch:
-query batches are independent, so there is no data-path collective and scaling is weak.
-`--impl reference` times the CPU oracle, as it stands, on a bounded sample of the same workload.
+With N > 1 every rank holds a replica of the index and searches its own batch: query batches are independent, so
+there is no data-path collective and scaling is weak.  Started without torchrun, `--gpus N` starts the N ranks
+itself.  `--impl reference` times the CPU oracle, as it stands, on a bounded sample of the same workload.
 Prints one JSON line on rank 0.
 """
 
 from __future__ import annotations
 
 import argparse
+import gc
+import hashlib
 import json
 import os
 import subprocess
@@ -30,10 +34,35 @@ if ROOT not in sys.path:
 import numpy as np  # noqa: E402
 import torch  # noqa: E402
 
-WORKLOAD = 2  # index into synth.CONFIGS
-SCAN_DRAM_PER_LOGICAL = 34.217e9 / 42.427e9  # full-size Mid workload only (see run_ours)
 METRIC = "retrieval_qps"
 UNIT = "queries/s"
+HEADLINE = "hyper"
+SECONDARY = ("mid", "flat", "coarse_hyper", "iter")
+
+# DRAM bytes per logical (algorithmic) code byte of one scan_kernel launch, from ncu one-pass captures of
+# dram__bytes_read.sum + dram__bytes_write.sum (profiles/scan_kernel_dram_traffic.md).  A figure is only valid for
+# the kernel source it was captured from: each entry names the SHA-256 of csrc/scan.cu (first 16 hex digits) and a
+# run whose scan.cu hashes differently reports traffic = null.  "hyper" was captured at 1/16 of the vectors (4 GB
+# of codes; the capture-size rule) and carries over to the full size because the lists are uniform and no list is
+# shared through L2 at either size; "mid" was captured at full size and is not scaled to other sizes.
+SCAN_TRAFFIC = {
+    "hyper": {"scan_sha": None, "dram_per_logical": None},
+    "mid": {"scan_sha": None, "dram_per_logical": None},
+}
+
+
+def _scan_sha():
+    with open(os.path.join(ROOT, "paper_2503_14649_b200", "csrc", "scan.cu"), "rb") as f:
+        return hashlib.sha256(f.read()).hexdigest()[:16]
+
+
+def _traffic(tag, scan_bytes, scale):
+    t = SCAN_TRAFFIC.get(tag)
+    if not t or t["dram_per_logical"] is None or t["scan_sha"] != _scan_sha():
+        return None
+    if tag == "mid" and scale != 1.0:
+        return None
+    return t["dram_per_logical"] * scan_bytes
 
 
 def _peaks():
@@ -41,8 +70,9 @@ def _peaks():
     if os.path.exists(p):
         with open(p) as f:
             d = json.load(f)
-        return float(d["hbm_gbs"]), "measured"
-    return 6650.0, "fallback"
+        return {"hbm": float(d["hbm_gbs"]), "burst": float(d["bf16_tflops"]),
+                "sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), "kind": "measured"}
+    return {"hbm": 6650.0, "burst": 1590.0, "sustained": 1400.0, "kind": "fallback"}
 
 
 class ClockSampler:
@@ -120,79 +150,89 @@ def _dist_env():
     return rank, world, local
 
 
-def _oracle_sample(data, cfg, nsample, threads, repeat=1):
-    """Time the oracle on the first nsample queries; returns (seconds per pass, ids, dists)."""
-    import oracle
-    from tests.helpers import host_index
-    hix = host_index(oracle, data)
-    q = data.queries[:nsample].cpu().numpy()
-    best = None
-    for _ in range(repeat):
-        t0 = time.perf_counter()
-        ids, dists = oracle.ivfpq_search(hix, q, cfg["nprobe"], cfg["k"], nthreads=threads)
-        dt = time.perf_counter() - t0
-        best = dt if best is None else min(best, dt)
-    return best, ids, dists
+def launcher_command(gpus: int, argv, port: int):
+    """The command that starts `gpus` ranks of this script on one node (one process per GPU, rendezvous on
+    127.0.0.1), as the documented multi-GPU launch does it."""
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(gpus),
+            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
 
 
-def run_reference(args):
-    """CPU oracle arm: each step searches a bounded sample of the workload's queries on the host cores."""
-    rank, world, _ = _dist_env()
-    if rank != 0:
-        return
-    import oracle
-    from paper_2503_14649_b200 import synth
-    from tests.helpers import host_index
-    cfg = synth.CONFIGS[WORKLOAD]
-    threads = oracle.default_threads()
-    dev = "cuda" if torch.cuda.is_available() else "cpu"
-    data = synth.make_config(WORKLOAD, device=dev, scale=args.scale)
-    hix = host_index(oracle, data)
-    nsample = min(cfg["nq"], threads)  # one query per core per step
-    q = data.queries[:nsample].cpu().numpy()
-    for _ in range(args.warmup):
-        oracle.ivfpq_search(hix, q, cfg["nprobe"], cfg["k"], nthreads=threads)
-    t0 = time.perf_counter()
-    for _ in range(args.steps):
-        oracle.ivfpq_search(hix, q, cfg["nprobe"], cfg["k"], nthreads=threads)
-    dt = time.perf_counter() - t0
-    qps = nsample * args.steps / dt
-    sample = "%d of %d queries per step, full database, one query per thread" % (nsample, cfg["nq"])
-    print(json.dumps({
-        "impl": "reference", "metric": METRIC, "value": qps, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": _config(cfg, data, args),
-        "cpu_baseline": {"value": qps, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
-        "e2e": {"value": qps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
-    }))
+def check_world(gpus: int, world: int):
+    """A run that asks for N GPUs must consist of N ranks: a mislabelled line is worse than none."""
+    if max(1, gpus) != world:
+        raise SystemExit("bench.py: --gpus %d but %d rank(s) are running; start it as `python bench.py --gpus %d` "
+                         "(it spawns the ranks) or under torchrun with --nproc-per-node %d" % (gpus, world, gpus, gpus))
 
 
-def _config(cfg, data, args):
-    return {"workload": "Mid IVF-PQ (configs[1]): N=%d d=%d nlist=%d zipf=1.1 M=%d nq=%d nprobe=%d k=%d L2" % (
-        data.N, cfg["d"], cfg["nlist"], cfg["M"], cfg["nq"], cfg["nprobe"], cfg["k"]),
-        "global_batch": cfg["nq"] * max(1, args.gpus), "parallelism": "replicas x%d" % max(1, args.gpus),
-        "l2_policy": "inputs larger than L2 (0.96 GB of codes per replica)", "scale": args.scale}
-
-
-def run_ours(args):
-    from paper_2503_14649_b200 import binding, synth
+def _init_dist(need_gpu=True):
     rank, world, local = _dist_env()
+    if need_gpu and not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device is visible to rank %d; the library has no CPU path" % rank)
     if world > 1:
         import torch.distributed as dist
         torch.cuda.set_device(local)
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     else:
-        torch.cuda.set_device(0)
         local = 0
-    dev = torch.device("cuda", local)
-    cfg = synth.CONFIGS[WORKLOAD]
-    nq, nprobe, k = cfg["nq"], cfg["nprobe"], cfg["k"]
-    data = synth.make_config(WORKLOAD, device=dev, scale=args.scale)
+        torch.cuda.set_device(0)
+    return rank, world, local, torch.device("cuda", local)
+
+
+def _free():
+    gc.collect()
+    torch.cuda.empty_cache()
+
+
+# ---- workloads -------------------------------------------------------------------------------------------------
+
+IVF = {
+    "hyper": dict(cfg=3, name="Hyperscale IVF-PQ (configs[2])", extra="IP, bf16 centroids"),
+    "mid": dict(cfg=2, name="Mid IVF-PQ (configs[1])", extra="zipf=1.1 L2"),
+}
+
+
+def _ivf_workload_name(tag, data, c):
+    w = IVF[tag]
+    return "%s: N=%d d=%d nlist=%d M=%d nq=%d nprobe=%d k=%d %s" % (
+        w["name"], data.N, c["d"], c["nlist"], c["M"], c["nq"], c["nprobe"], c["k"], w["extra"])
+
+
+def _ivf_config(tag, data, c, args, world):
+    return {"workload": _ivf_workload_name(tag, data, c), "global_batch": c["nq"] * world,
+            "parallelism": "replicas x%d" % world,
+            "l2_policy": "inputs larger than L2 (%.2f GB of codes per replica)" % (data.N * c["M"] / 1e9),
+            "scale": args.scale}
+
+
+def _oracle_on_sample(tag, data, c, sample, threads):
+    """The oracle's answers for the sampled queries and the seconds it took (index preparation excluded).
+    Hash-coded shapes regenerate, on the CPU, exactly the lists those queries probe."""
+    import oracle
+    from tests.helpers import IvfPqRescorer, compact_hashed_subindex, host_index
+    q = data.queries[sample].cpu().numpy()
+    if data.hash_coded:
+        cen = data.centroids
+        cen_h = cen.cpu().view(torch.uint16).numpy() if cen.dtype == torch.bfloat16 else cen.cpu().numpy()
+        lists, _ = oracle.coarse(cen_h, q, c["nprobe"], data.metric, coarse_bf16=cen.dtype == torch.bfloat16,
+                                 nthreads=threads)
+        hix = compact_hashed_subindex(oracle, data, np.unique(lists))
+    else:
+        hix = host_index(oracle, data)
+    t0 = time.perf_counter()
+    ids, dists = oracle.ivfpq_search(hix, q, c["nprobe"], c["k"], nthreads=threads)
+    return time.perf_counter() - t0, ids, dists, IvfPqRescorer(oracle, hix), q
+
+
+def bench_ivfpq(tag, args, rank, world, local, dev, want_cpu_baseline):
+    """One IVF-PQ shape: device-resident throughput, stage split, host-buffer (end-to-end) throughput, roofline of
+    the scan kernel, optionally the oracle on a sample with a result check."""
+    from paper_2503_14649_b200 import binding, synth
+    c = synth.CONFIGS[IVF[tag]["cfg"]]
+    nq, nprobe, k = c["nq"], c["nprobe"], c["k"]
+    data = synth.make_config(IVF[tag]["cfg"], device=dev, scale=args.scale)
     if world > 1:  # every rank searches its own batch against its replica
         perm = rank_batch_permutation(nq, rank)
         data.queries = data.queries[perm.to(dev)].contiguous()
-        data.extra["query_component"] = data.extra["query_component"][perm]
     ix = binding.rago_index_load(data.centroids, data.codebooks, data.codes, data.list_offsets.to(dev), data.ids,
                                  data.metric)
     q = data.queries.contiguous()
@@ -205,7 +245,7 @@ def run_ours(args):
     lists, _ = ix.rago_search_probes(q, nprobe, workspace=ws)
     L = (data.list_offsets[1:] - data.list_offsets[:-1]).to(dev)
     scanned_vectors = int(L[lists.long()].sum().item())
-    scan_bytes = scanned_vectors * cfg["M"]
+    scan_bytes = scanned_vectors * c["M"]
 
     def barrier():
         if world > 1:
@@ -220,9 +260,7 @@ def run_ours(args):
     for _ in range(max(3, args.warmup)):
         step()
     ix.rago_check(ws)
-    ix.rago_profile_enable(True)
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
-    stage_ms = []
     barrier()
     launches0 = binding.rago_kernel_launches()
     t0 = time.time()
@@ -235,13 +273,12 @@ def run_ours(args):
     launches = binding.rago_kernel_launches() - launches0
     total_ms = ev[0].elapsed_time(ev[-1])
     step_ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
-    stage_last = ix.rago_profile_read()  # stage split of the last timed step (events on the launching stream)
-    ix.rago_profile_enable(False)
     clocks = sampler.stop(t0, t1)
     ix.rago_check(ws)
-    # scan-kernel time over several steps, each read right after its step (outside the timed region)
+    # per-stage device times (events on the launching stream around each stage), read after each of a few steps
     ix.rago_profile_enable(True)
-    for _ in range(min(10, args.steps)):
+    stage_ms = []
+    for _ in range(min(10, max(3, args.steps))):
         step()
         stage_ms.append(ix.rago_profile_read())
     ix.rago_profile_enable(False)
@@ -250,7 +287,7 @@ def run_ours(args):
     total_ms = max_over_ranks(total_ms, world, dev)
     qps = whole_job_qps(nq, world, args.steps, total_ms)
 
-    # end to end through the host-buffer entry point: pinned queries in, pinned results out
+    # end to end through the host-buffer entry point: pinned queries in, pinned results out, every step
     hq = q.cpu().pin_memory()
     hids = torch.empty((nq, k), dtype=torch.int64).pin_memory()
     hd = torch.empty((nq, k), dtype=torch.float32).pin_memory()
@@ -264,64 +301,53 @@ def run_ours(args):
         ix.rago_search_host(hq, nprobe, k, hids, hd, ws)
     e1.record()
     barrier()
-    e2e_ms = e0.elapsed_time(e1)
-    e2e_ms = max_over_ranks(e2e_ms, world, dev)
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1), world, dev)
     e2e_qps = whole_job_qps(nq, world, args.steps, e2e_ms)
     assert torch.equal(hids, out_ids.cpu()), "host-buffer path disagrees with the device path"
 
-    if rank != 0:
-        if world > 1:
-            torch.distributed.destroy_process_group()
-        return
-
-    peak, peak_kind = _peaks()
+    pk = _peaks()
     achieved = scan_bytes / (scan_ms / 1e3) / 1e9
-    # DRAM bytes of one scan launch: dram__bytes_read.sum + dram__bytes_write.sum of one launch of this very
-    # workload at full size (one-pass ncu capture: 34.217 GB for 42.427 GB of logical code
-    # bytes; hot lists are shared through L2).  The ratio does not carry over to other sizes (at 1/4 of the vectors
-    # it is 0.31), so scaled-down runs report null.  Valid for the scan kernel the capture was taken from: set
-    # SCAN_DRAM_PER_LOGICAL to None after changing the kernel.
-    traffic = SCAN_DRAM_PER_LOGICAL * scan_bytes if SCAN_DRAM_PER_LOGICAL is not None and args.scale == 1.0 else None
+    traffic = _traffic(tag, scan_bytes, args.scale)
     out = {
         "metric": METRIC, "value": qps, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32", "data": "synthetic", "config": _config(cfg, data, args),
+        "dtype": "f32", "data": "synthetic", "config": _ivf_config(tag, data, c, args, world),
         "clocks": clocks,
-        "e2e": {"value": e2e_qps, "unit": UNIT, "h2d_bytes_per_step": nq * cfg["d"] * 4,
+        "e2e": {"value": e2e_qps, "unit": UNIT, "h2d_bytes_per_step": nq * c["d"] * 4,
                 "d2h_bytes_per_step": nq * k * 12},
         "gpu_launches": int(launches),
-        "roofline": {"bound": "hbm", "kernel": "scan_kernel (table fetch + ADC scan + partial top-k)", "achieved": achieved,
-                     "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak, "traffic": traffic,
+        "roofline": {"bound": "hbm", "kernel": "scan_kernel (table fetch + ADC scan + partial top-k)",
+                     "achieved": achieved, "peak": pk["hbm"], "peak_kind": pk["kind"], "unit": "GB/s",
+                     "frac": achieved / pk["hbm"], "traffic": traffic,
+                     "dram_frac": (traffic / (scan_ms / 1e3) / 1e9 / pk["hbm"]) if traffic else None,
                      "algorithmic_bytes_per_launch": scan_bytes, "kernel_ms": scan_ms,
                      "scanned_vectors_per_query": scanned_vectors / nq},
         "stage_ms": {kk: float(np.mean([s[kk] for s in stage_ms])) for kk in stage_ms[0]},
         "step_ms_p50": float(np.median(step_ms)), "step_ms_max": float(np.max(step_ms)),
     }
-    if world == 1 and not args.no_cpu_baseline:
+    if want_cpu_baseline and rank == 0 and world == 1:
         import oracle
         from tests.helpers import match_results
         threads = oracle.default_threads()
-        nsample = min(nq, 4 * threads)
-        dt, oi, od = _oracle_sample(data, cfg, nsample, threads)  # a first, small sample sizes the real one (~15 s)
-        nsample = int(min(nq, max(nsample, (nsample / dt) * 15.0)))
-        dt, oi, od = _oracle_sample(data, cfg, nsample, threads)
-        gi, gd = out_ids[:nsample].cpu().numpy(), out_d[:nsample].cpu().numpy()
-        mism = sum(1 for i in range(nsample) if match_results(gi[i], gd[i], oi[i], od[i], rel=1e-4))
-        out["cpu_baseline"] = {"value": nsample / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
-                               "sample": "first %d of %d queries, full database, one query per thread" % (nsample, nq),
+        gi, gd = out_ids.cpu().numpy(), out_d.cpu().numpy()
+        if data.hash_coded:   # a fixed, spread sample: every (nq / 64)-th query, each through all its probed lists
+            sample = list(range(0, nq, max(1, nq // 64)))[:64]
+        else:                 # a first, small sample sizes the real one (about 15 s of oracle time)
+            n0 = min(nq, 4 * threads)
+            dt0 = _oracle_on_sample(tag, data, c, list(range(n0)), threads)[0]
+            sample = list(range(int(min(nq, max(n0, (n0 / dt0) * 15.0)))))
+        dt, oi, od, rs, qh = _oracle_on_sample(tag, data, c, sample, threads)
+        sgn = 1.0 if data.metric == "l2" else -1.0
+        mism = sum(1 for t, qi in enumerate(sample)
+                   if match_results(gi[qi], sgn * gd[qi], oi[t], sgn * od[t], rel=1e-4, rescore=rs.for_query(qh[t], sgn)))
+        out["cpu_baseline"] = {"value": len(sample) / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
+                               "sample": "%d of %d queries (%s), each through all of its probed lists, one query "
+                                         "per thread" % (len(sample), nq, "evenly spaced" if data.hash_coded else "the first"),
                                "seconds": dt, "queries_not_matching_gpu": mism}
-    print(json.dumps(out))
-    if world > 1:
-        torch.distributed.destroy_process_group()
-
-
-def _tensor_peaks():
-    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
-    if os.path.exists(p):
-        with open(p) as f:
-            d = json.load(f)
-        return float(d["bf16_tflops"]), float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), float(d["hbm_gbs"]), "measured"
-    return 1590.0, 1400.0, 6650.0, "fallback"
+    ix.close()
+    del ix, data, ws, q, out_ids, out_d, lists, L
+    _free()
+    return out
 
 
 def _time_steps(fn, steps, warmup):
@@ -338,17 +364,15 @@ def _time_steps(fn, steps, warmup):
     return ev[0].elapsed_time(ev[-1]), [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
 
 
-def run_flat(args):
-    """Secondary workload: exact flat search, N = 10 M x 1024 bf16 rows, 256 queries, k = 100 (cosine on unit rows)."""
+def bench_flat(args, dev):
+    """Exact flat search, N = 10 M x 1024 bf16 rows, 256 queries, k = 100 (cosine on unit rows)."""
     from paper_2503_14649_b200 import binding, synth
-    torch.cuda.set_device(0)
-    dev = torch.device("cuda", 0)
     c = synth.CONFIGS[5]
     N = max(1, int(round(c["N"] * args.scale)))
     d, nq, k = c["d"], c["nq"], c["k"]
     db, q = synth.make_flat(N, d, nq, device=dev)
     ws = torch.empty(binding.rago_flat_workspace_bytes(N, d, nq, k), dtype=torch.uint8, device=dev)
-    sampler = ClockSampler(0)
+    sampler = ClockSampler(dev.index or 0)
     out = {}
 
     def step():
@@ -362,10 +386,10 @@ def run_flat(args):
     clocks = sampler.stop(t0, t1)
     launches = (binding.rago_kernel_launches() - launches0) * args.steps // (args.steps + max(3, args.warmup))
     ms = total_ms / args.steps
-    burst, sustained, hbm, kind = _tensor_peaks()
+    pk = _peaks()
     tflops = 2.0 * nq * N * d / (ms / 1e3) / 1e12
     gbs = N * d * 2 / (ms / 1e3) / 1e9
-    print(json.dumps({
+    res = {
         "metric": METRIC, "value": nq / (ms / 1e3), "unit": UNIT, "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
@@ -373,25 +397,26 @@ def run_flat(args):
                    "l2_policy": "database (%.1f GB) larger than L2" % (N * d * 2 / 1e9), "scale": args.scale},
         "clocks": clocks, "gpu_launches": int(launches),
         "roofline": {"bound": "tensor", "kernel": "gemm_select_kernel + flat_merge_kernel (whole call)", "achieved": tflops,
-                     "peak": sustained, "peak_kind": kind + " (sustained bf16)", "unit": "TFLOP/s", "frac": tflops / sustained,
-                     "frac_of_burst": tflops / burst, "traffic": None,
-                     "hbm": {"achieved": gbs, "peak": hbm, "frac": gbs / hbm, "unit": "GB/s"}},
-        "step_ms_p50": float(np.median(step_ms)), "step_ms_max": float(np.max(step_ms))}))
+                     "peak": pk["sustained"], "peak_kind": pk["kind"] + " (sustained bf16)", "unit": "TFLOP/s",
+                     "frac": tflops / pk["sustained"], "frac_of_burst": tflops / pk["burst"], "traffic": None,
+                     "hbm": {"achieved": gbs, "peak": pk["hbm"], "frac": gbs / pk["hbm"], "unit": "GB/s"}},
+        "step_ms_p50": float(np.median(step_ms)), "step_ms_max": float(np.max(step_ms))}
+    del db, q, ws, out
+    _free()
+    return res
 
 
-def run_coarse_hyper(args):
-    """Secondary workload: the coarse step of the Hyperscale shape alone: 4096 queries x 65 536 bf16 centroids,
-    d = 768, inner product, nprobe = 64 (a 4096 x 768 x 65 536 contraction with the selection fused in)."""
+def bench_coarse_hyper(args, dev):
+    """The coarse step of the Hyperscale shape alone: 4096 queries x 65 536 bf16 centroids, d = 768, inner
+    product, nprobe = 64 (a 4096 x 768 x 65 536 contraction with the selection fused in)."""
     from paper_2503_14649_b200 import binding, synth
-    torch.cuda.set_device(0)
-    dev = torch.device("cuda", 0)
     c = synth.CONFIGS[3]
     nq, nprobe, nlist, d = c["nq"], c["nprobe"], c["nlist"], c["d"]
     data = synth.make_ivfpq_hashed(nlist * 4, d, nlist, c["M"], nq, metric=c["metric"], coarse_bf16=True, device=dev)
     ix = binding.rago_index_load(data.centroids, data.codebooks, data.codes, data.list_offsets.to(dev), data.ids, data.metric)
     q = data.queries.contiguous()
     ws = torch.empty(ix.search_workspace_bytes(nq, nprobe, 1), dtype=torch.uint8, device=dev)
-    sampler = ClockSampler(0)
+    sampler = ClockSampler(dev.index or 0)
     sampler.start()
     t0 = time.time()
     total_ms, step_ms = _time_steps(lambda: ix.rago_search_probes(q, nprobe, workspace=ws), args.steps, args.warmup)
@@ -401,84 +426,39 @@ def run_coarse_hyper(args):
     ix.rago_profile_enable(True)
     out_i = torch.empty((nq, 1), dtype=torch.int64, device=dev)
     out_d = torch.empty((nq, 1), dtype=torch.float32, device=dev)
-    ws2 = torch.empty(ix.search_workspace_bytes(nq, nprobe, 1), dtype=torch.uint8, device=dev)
     stage = []
     for _ in range(5):
-        ix.rago_search(q, nprobe, 1, out_i, out_d, ws2)
+        ix.rago_search(q, nprobe, 1, out_i, out_d, ws)
         stage.append(ix.rago_profile_read())
     gemm_ms = float(np.median([s["coarse_scores"] for s in stage]))
     sel_ms = float(np.median([s["probe_select"] for s in stage]))
     ms = total_ms / args.steps
-    burst, sustained, hbm, kind = _tensor_peaks()
+    pk = _peaks()
     tflops = 2.0 * nq * nlist * d / (gemm_ms / 1e3) / 1e12
-    print(json.dumps({
+    res = {
         "metric": "coarse_qps", "value": nq / (ms / 1e3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": "Hyperscale coarse step (configs[2], coarse only): nq=%d nlist=%d d=%d bf16 nprobe=%d IP"
                    % (nq, nlist, d, nprobe), "l2_policy": "centroids 100 MB, L2 flushed by the candidate lists"},
         "clocks": clocks,
-        "roofline": {"bound": "tensor", "kernel": "split_bf16_kernel + gemm_select_kernel", "achieved": tflops, "peak": burst,
-                     "peak_kind": kind + " (burst bf16)", "unit": "TFLOP/s", "frac": tflops / burst,
-                     "frac_of_sustained": tflops / sustained, "traffic": None, "kernel_ms": gemm_ms},
+        "roofline": {"bound": "tensor", "kernel": "split_bf16_kernel + pilot pass + gemm_select_kernel (the coarse_scores stage)",
+                     "achieved": tflops, "peak": pk["burst"], "peak_kind": pk["kind"] + " (burst bf16)", "unit": "TFLOP/s",
+                     "frac": tflops / pk["burst"], "frac_of_sustained": tflops / pk["sustained"], "traffic": None,
+                     "kernel_ms": gemm_ms},
         "stage_ms": {"coarse_scores": gemm_ms, "probe_select": sel_ms},
-        "step_ms_p50": float(np.median(step_ms))}))
+        "step_ms_p50": float(np.median(step_ms))}
+    ix.close()
+    del ix, data, ws, q
+    _free()
+    return res
 
 
-def run_hyper(args):
-    """Secondary workload: the whole Hyperscale shape: 1e9 hash-coded vectors (64 GB of codes), 65 536 bf16
-    centroids, 4096 queries, nprobe = 64, k = 100, inner product."""
+def bench_iter(args, dev):
+    """The iterative-retrieval latency shape: N = 1e8, d = 512, nlist = 16 384, M = 32; a stream of 256 batches of
+    1, 4 or 16 queries issued back to back on one stream, nprobe = 16, k = 20; per-batch latency from CUDA events
+    between the batches."""
     from paper_2503_14649_b200 import binding, synth
-    torch.cuda.set_device(0)
-    dev = torch.device("cuda", 0)
-    c = synth.CONFIGS[3]
-    nq, nprobe, k = c["nq"], c["nprobe"], c["k"]
-    data = synth.make_config(3, device=dev, scale=args.scale)
-    ix = binding.rago_index_load(data.centroids, data.codebooks, data.codes, data.list_offsets.to(dev), data.ids, data.metric)
-    q = data.queries.contiguous()
-    ws = torch.empty(ix.search_workspace_bytes(nq, nprobe, k), dtype=torch.uint8, device=dev)
-    out_i = torch.empty((nq, k), dtype=torch.int64, device=dev)
-    out_d = torch.empty((nq, k), dtype=torch.float32, device=dev)
-    lists, _ = ix.rago_search_probes(q, nprobe, workspace=ws)
-    Ln = (data.list_offsets[1:] - data.list_offsets[:-1]).to(dev)
-    scan_bytes = int(Ln[lists.long()].sum().item()) * c["M"]
-    sampler = ClockSampler(0)
-    sampler.start()
-    t0 = time.time()
-    total_ms, step_ms = _time_steps(lambda: ix.rago_search(q, nprobe, k, out_i, out_d, ws), args.steps, args.warmup)
-    t1 = time.time()
-    clocks = sampler.stop(t0, t1)
-    ix.rago_check(ws)
-    ix.rago_profile_enable(True)
-    stage = []
-    for _ in range(3):
-        ix.rago_search(q, nprobe, k, out_i, out_d, ws)
-        stage.append(ix.rago_profile_read())
-    st = {kk: float(np.median([s_[kk] for s_ in stage])) for kk in stage[0]}
-    ms = total_ms / args.steps
-    hbm, kind = _peaks()
-    achieved = scan_bytes / (st["table_scan"] / 1e3) / 1e9
-    print(json.dumps({
-        "metric": METRIC, "value": nq / (ms / 1e3), "unit": UNIT, "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
-        "data": "synthetic",
-        "config": {"workload": "Hyperscale IVF-PQ (configs[2]): N=%d d=%d nlist=%d M=%d nq=%d nprobe=%d k=%d IP, bf16 centroids"
-                   % (data.N, c["d"], c["nlist"], c["M"], nq, nprobe, k),
-                   "l2_policy": "inputs larger than L2 (%.0f GB of codes)" % (data.N * c["M"] / 1e9), "scale": args.scale},
-        "clocks": clocks,
-        "roofline": {"bound": "hbm", "kernel": "scan_kernel (table fetch + ADC scan + partial top-k)", "achieved": achieved, "peak": hbm,
-                     "peak_kind": kind, "unit": "GB/s", "frac": achieved / hbm, "traffic": None,
-                     "algorithmic_bytes_per_launch": scan_bytes, "kernel_ms": st["table_scan"]},
-        "stage_ms": st, "step_ms_p50": float(np.median(step_ms))}))
-
-
-def run_iter(args):
-    """Secondary workload: the iterative-retrieval latency shape: N = 1e8, d = 512, nlist = 16 384, M = 32; a stream
-    of 256 batches of 1, 4 or 16 queries issued back to back on one stream, nprobe = 16, k = 20; per-batch latency
-    from CUDA events between the batches."""
-    from paper_2503_14649_b200 import binding, synth
-    torch.cuda.set_device(0)
-    dev = torch.device("cuda", 0)
     c = synth.CONFIGS[4]
     nprobe, k = c["nprobe"], c["k"]
     sizes = synth.batch_size_stream(synth.MASTER_SEED, 256)
@@ -501,7 +481,7 @@ def run_iter(args):
     for _ in range(max(3, args.warmup)):
         stream()
     torch.cuda.synchronize()
-    sampler = ClockSampler(0)
+    sampler = ClockSampler(dev.index or 0)
     sampler.start()
     t0 = time.time()
     lat = {1: [], 4: [], 16: []}
@@ -518,7 +498,7 @@ def run_iter(args):
     ix.rago_check(ws)
     ms = float(np.mean(tot))
     alll = np.concatenate([lat[1], lat[4], lat[16]])
-    print(json.dumps({
+    res = {
         "metric": METRIC, "value": sum(sizes) / (ms / 1e3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
@@ -531,26 +511,21 @@ def run_iter(args):
                                          for nb, v in lat.items()},
                        "note": "device time between consecutive batches' start events (launch-to-launch on a busy stream)"},
         "roofline": {"bound": "latency", "kernel": "whole call", "achieved": None, "peak": None,
-                     "unit": None, "frac": None, "traffic": None}}))
+                     "unit": None, "frac": None, "traffic": None}}
+    ix.close()
+    del ix, data, ws, q
+    _free()
+    return res
 
 
-def run_sharded(args):
-    """Secondary workload: database-sharded search.  Every rank holds its own Mid-shape shard with an independent
-    index (its own seed); all ranks answer rank 0's query batch, exchange their [nq, k] answers with one all-gather
-    and aggregate them.  The database grows with the number of ranks, the query batch does not."""
+def bench_sharded(args, rank, world, local, dev):
+    """Database-sharded search.  Every rank holds its own Mid-shape shard with an independent index (its own
+    seed); all ranks answer rank 0's query batch, exchange their [nq, k] answers with one all-gather and aggregate
+    them.  The database grows with the number of ranks, the query batch does not."""
     from paper_2503_14649_b200 import binding, sharded, synth
-    rank, world, local = _dist_env()
-    if world > 1:
-        import torch.distributed as dist
-        torch.cuda.set_device(local)
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    else:
-        torch.cuda.set_device(0)
-        local = 0
-    dev = torch.device("cuda", local)
-    c = synth.CONFIGS[WORKLOAD]
+    c = synth.CONFIGS[2]
     nq, nprobe, k = c["nq"], c["nprobe"], c["k"]
-    data = synth.make_config(WORKLOAD, device=dev, scale=args.scale, seed=synth.MASTER_SEED + 7919 * rank)
+    data = synth.make_config(2, device=dev, scale=args.scale, seed=synth.MASTER_SEED + 7919 * rank)
     ix = binding.rago_index_load(data.centroids, data.codebooks, data.codes, data.list_offsets.to(dev), data.ids,
                                  data.metric)
     q = data.queries.contiguous()
@@ -588,40 +563,34 @@ def run_sharded(args):
     ids, dists = ix.rago_search(q, nprobe, k, workspace=ws)
     parts = sharded.gather_parts(ids, dists)
     agg_ms, _ = _time_steps(lambda: binding.rago_merge_results(parts[0], parts[1], k, ix.metric), 20, 3)
-    if rank == 0:
-        ms = total_ms / args.steps
-        print(json.dumps({
-            "metric": METRIC, "value": nq / (ms / 1e3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
-            "scaling": "weak (database grows with ranks, one shared query batch)", "vs_baseline": None, "dtype": "f32",
-            "data": "synthetic",
-            "config": {"workload": "Sharded Mid IVF-PQ: %d shard(s) of N=%d d=%d nlist=%d M=%d, independent indexes; nq=%d "
-                                   "nprobe=%d k=%d L2; all-gather + aggregation every step"
-                                   % (world, data.N, c["d"], c["nlist"], c["M"], nq, nprobe, k),
-                       "l2_policy": "inputs larger than L2", "scale": args.scale},
-            "clocks": clocks, "gpu_launches": launches, "aggregate_kernel_ms": agg_ms / 20,
-            "exchange_bytes_per_rank": nq * k * 12}))
-    if world > 1:
-        torch.distributed.destroy_process_group()
+    ms = total_ms / args.steps
+    return {
+        "metric": METRIC, "value": nq / (ms / 1e3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak (database grows with ranks, one shared query batch)", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic",
+        "config": {"workload": "Sharded Mid IVF-PQ: %d shard(s) of N=%d d=%d nlist=%d M=%d, independent indexes; nq=%d "
+                               "nprobe=%d k=%d L2; all-gather + aggregation every step"
+                               % (world, data.N, c["d"], c["nlist"], c["M"], nq, nprobe, k),
+                   "l2_policy": "inputs larger than L2", "scale": args.scale},
+        "clocks": clocks, "gpu_launches": launches, "aggregate_kernel_ms": agg_ms / 20,
+        "exchange_bytes_per_rank": nq * k * 12}
 
 
-def run_sweep(args):
-    """Secondary measurement: batch-size sweep on the Mid index, the data a retrieval cost model needs.  The paper
-    models a scan operator as T = max(D / P_comp(Q), D / B_mem) with D the bytes scanned and Q the batch size
-    (Sec. 4); here every batch size gets its measured time and scanned bytes, and a least-squares line
-    T = T0 + D / B_eff over the sweep gives the two constants of the same model on this GPU (T0: the launch-bound
-    floor the paper's model does not have)."""
-    from paper_2503_14649_b200 import binding, synth
-    torch.cuda.set_device(0)
-    dev = torch.device("cuda", 0)
-    c = synth.CONFIGS[WORKLOAD]
+def bench_sweep(args, dev):
+    """Batch-size sweep on the Mid index: the measurements the retrieval cost model is fitted to.  The paper models
+    a scan operator as T = max(D / P_comp(Q), D / B_mem) with D the bytes scanned and Q the batch size (Sec. 4);
+    here every batch size gets its measured time and scanned bytes, and cost_model.fit_retrieval_model turns the
+    rows into the constants of that model on this GPU."""
+    from paper_2503_14649_b200 import binding, cost_model, synth
+    c = synth.CONFIGS[2]
     nprobe, k = c["nprobe"], c["k"]
-    data = synth.make_config(WORKLOAD, device=dev, scale=args.scale)
+    data = synth.make_config(2, device=dev, scale=args.scale)
     ix = binding.rago_index_load(data.centroids, data.codebooks, data.codes, data.list_offsets.to(dev), data.ids,
                                  data.metric)
     Ln = (data.list_offsets[1:] - data.list_offsets[:-1]).to(dev)
     rows = []
-    sampler = ClockSampler(0)
+    sampler = ClockSampler(dev.index or 0)
     sampler.start()
     t0 = time.time()
     for nq in (1, 2, 4, 8, 16, 32, 64, 128, 256, 512, 1024):
@@ -638,27 +607,20 @@ def run_sweep(args):
         rows.append({"nq": nq, "ms": ms, "qps": nq / (ms / 1e3), "scanned_bytes": D, "gbs": D / (ms / 1e3) / 1e9})
     t1 = time.time()
     clocks = sampler.stop(t0, t1)
-    Dv = np.array([r["scanned_bytes"] for r in rows], np.float64)
-    Tv = np.array([r["ms"] for r in rows], np.float64) * 1e-3
-    A = np.stack([np.ones_like(Dv), Dv], 1)
-    # relative least squares, so that the small batches weigh as much as the large ones
-    coef, *_ = np.linalg.lstsq(A / Tv[:, None], np.ones_like(Tv), rcond=None)
-    print(json.dumps({
-        "metric": "retrieval_cost_model", "unit": "s = T0 + D / B_eff", "n_gpus": 1, "data": "synthetic",
+    model = cost_model.fit_retrieval_model([r["nq"] for r in rows], [r["scanned_bytes"] for r in rows],
+                                           [r["ms"] * 1e-3 for r in rows])
+    return {
+        "metric": "retrieval_cost_model", "unit": "s = T0 + max(D / B_mem, Q / R_q)", "n_gpus": 1, "data": "synthetic",
         "config": {"workload": "Mid IVF-PQ index (configs[1]), batch sizes 1..1024, nprobe=%d k=%d" % (nprobe, k),
                    "scale": args.scale},
-        "fit": {"T0_us": coef[0] * 1e6, "B_eff_GBs": 1.0 / coef[1] / 1e9,
-                "max_rel_err": float(np.max(np.abs(A @ coef - Tv) / Tv))},
-        "rows": rows, "clocks": clocks}))
+        "fit": model.as_dict(), "rows": rows, "clocks": clocks}
 
 
-def run_pq4(args):
-    """Secondary workload: the Mid shape with 4-bit codes (the paper's low-precision PQ variant): the same corpus
-    recipe, d = 768, M4 = 96 sub-spaces of 16 codewords = 48 bytes per vector (half of the 8-bit index's 96)."""
+def bench_pq4(args, dev):
+    """The Mid shape with 4-bit codes (the paper's low-precision PQ variant): the same corpus recipe, d = 768,
+    M4 = 96 sub-spaces of 16 codewords = 48 bytes per vector (half of the 8-bit index's 96)."""
     from paper_2503_14649_b200 import binding, synth
-    torch.cuda.set_device(0)
-    dev = torch.device("cuda", 0)
-    c = synth.CONFIGS[WORKLOAD]
+    c = synth.CONFIGS[2]
     nq, nprobe, k, M4 = c["nq"], c["nprobe"], c["k"], args.m4
     N = max(1, int(round(c["N"] * args.scale)))
     data = synth.make_ivfpq4(N, c["d"], c["nlist"], M4, nq, metric=c["metric"], zipf=c["zipf"], device=dev)
@@ -672,7 +634,7 @@ def run_pq4(args):
     Ln = (data.list_offsets[1:] - data.list_offsets[:-1]).to(dev)
     scanned = int(Ln[lists.long()].sum().item())
     scan_bytes = scanned * (M4 // 2)
-    sampler = ClockSampler(0)
+    sampler = ClockSampler(dev.index or 0)
     sampler.start()
     t0 = time.time()
     launches0 = binding.rago_kernel_launches()
@@ -688,9 +650,9 @@ def run_pq4(args):
         stage.append(ix.rago_profile_read())
     st = {kk: float(np.median([s_[kk] for s_ in stage])) for kk in stage[0]}
     ms = total_ms / args.steps
-    hbm, kind = _peaks()
+    pk = _peaks()
     achieved = scan_bytes / (st["table_scan"] / 1e3) / 1e9
-    print(json.dumps({
+    return {
         "metric": METRIC, "value": nq / (ms / 1e3), "unit": UNIT, "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
         "data": "synthetic",
@@ -698,43 +660,115 @@ def run_pq4(args):
                                "nq=%d nprobe=%d k=%d L2" % (N, c["d"], c["nlist"], c["zipf"], M4, M4 // 2, nq, nprobe, k),
                    "l2_policy": "inputs larger than L2 (%.2f GB of codes)" % (N * (M4 // 2) / 1e9), "scale": args.scale},
         "clocks": clocks, "gpu_launches": launches,
-        "roofline": {"bound": "hbm", "kernel": "scan_kernel (table fetch + ADC scan + partial top-k)", "achieved": achieved, "peak": hbm,
-                     "peak_kind": kind, "unit": "GB/s", "frac": achieved / hbm, "traffic": None,
+        "roofline": {"bound": "hbm", "kernel": "scan_kernel (table fetch + ADC scan + partial top-k)", "achieved": achieved,
+                     "peak": pk["hbm"], "peak_kind": pk["kind"], "unit": "GB/s", "frac": achieved / pk["hbm"], "traffic": None,
                      "algorithmic_bytes_per_launch": scan_bytes, "kernel_ms": st["table_scan"],
                      "scanned_vectors_per_s": scanned / (st["table_scan"] / 1e3)},
-        "stage_ms": st, "step_ms_p50": float(np.median(step_ms))}))
+        "stage_ms": st, "step_ms_p50": float(np.median(step_ms))}
 
 
-def main():
+# ---- the reference arm: the CPU oracle on a bounded sample ---------------------------------------------------------
+
+def run_reference(args):
+    """Each step searches one query per host core of the headline workload with the oracle, every query through
+    all of its probed lists (regenerated on the CPU from the seed before the timed steps)."""
+    rank, world, _ = _dist_env()
+    if rank != 0:
+        return
+    import oracle
+    from paper_2503_14649_b200 import synth
+    from tests.helpers import compact_hashed_subindex, host_index
+    tag = args.workload if args.workload in IVF else HEADLINE
+    c = synth.CONFIGS[IVF[tag]["cfg"]]
+    threads = oracle.default_threads()
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    data = synth.make_config(IVF[tag]["cfg"], device=dev, scale=args.scale, materialise=False) \
+        if tag == "hyper" else synth.make_config(IVF[tag]["cfg"], device=dev, scale=args.scale)
+    nsample = min(c["nq"], threads)  # one query per core per step
+    q = data.queries[:nsample].cpu().numpy()
+    if data.hash_coded:
+        cen_h = data.centroids.cpu().view(torch.uint16).numpy() if data.coarse_bf16 else data.centroids.cpu().numpy()
+        lists, _ = oracle.coarse(cen_h, q, c["nprobe"], data.metric, coarse_bf16=data.coarse_bf16, nthreads=threads)
+        hix = compact_hashed_subindex(oracle, data, np.unique(lists))
+    else:
+        hix = host_index(oracle, data)
+    for _ in range(args.warmup):
+        oracle.ivfpq_search(hix, q, c["nprobe"], c["k"], nthreads=threads)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.ivfpq_search(hix, q, c["nprobe"], c["k"], nthreads=threads)
+    dt = time.perf_counter() - t0
+    qps = nsample * args.steps / dt
+    sample = "%d of %d queries per step, each through all of its probed lists, one query per thread" % (nsample, c["nq"])
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": qps, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": _ivf_config(tag, data, c, args, max(1, args.gpus)),
+        "cpu_baseline": {"value": qps, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": qps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ---- entry ---------------------------------------------------------------------------------------------------------
+
+def run_ours(args):
+    rank, world, local, dev = _init_dist()
+    check_world(args.gpus, world)
+    wl = args.workload or HEADLINE
+    single = {"flat": lambda: bench_flat(args, dev), "coarse_hyper": lambda: bench_coarse_hyper(args, dev),
+              "iter": lambda: bench_iter(args, dev), "sweep": lambda: bench_sweep(args, dev),
+              "pq4": lambda: bench_pq4(args, dev)}
+    if wl in IVF:
+        out = bench_ivfpq(wl, args, rank, world, local, dev, want_cpu_baseline=not args.no_cpu_baseline)
+        if args.workload is None and world == 1 and not args.no_secondary:
+            # the other four shapes, each a full line of its own, so that one run records all five
+            sec = {}
+            for name in SECONDARY:
+                sub = argparse.Namespace(**vars(args))
+                sub.steps = min(args.steps, 30)
+                try:
+                    sec[name] = bench_ivfpq(name, sub, 0, 1, local, dev, want_cpu_baseline=not args.no_cpu_baseline) \
+                        if name in IVF else single[name]()
+                except Exception as e:  # a failed secondary must not lose the headline
+                    sec[name] = {"error": "%s: %s" % (type(e).__name__, e)}
+                    _free()
+            out["secondary"] = sec
+    elif wl == "sharded":
+        out = bench_sharded(args, rank, world, local, dev)
+    else:
+        if world > 1:
+            raise SystemExit("bench.py: --workload %s runs on one GPU" % wl)
+        out = single[wl]()
+    if rank == 0:
+        print(json.dumps(out))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+def main(argv=None):
+    argv = list(sys.argv[1:] if argv is None else argv)
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--scale", type=float, default=1.0, help="shrink N (development only; 1.0 = the named workload)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-secondary", action="store_true", help="headline workload only")
     ap.add_argument("--m4", type=int, default=96, help="--workload pq4: number of 4-bit sub-spaces")
-    ap.add_argument("--workload", default="mid", choices=["mid", "flat", "coarse_hyper", "hyper", "iter", "sharded", "sweep", "pq4"],
-                    help="mid = the headline Mid IVF-PQ workload (default); the others are secondary measurements")
-    args = ap.parse_args()
+    ap.add_argument("--workload", default=None,
+                    choices=["hyper", "mid", "flat", "coarse_hyper", "iter", "sharded", "sweep", "pq4"],
+                    help="default: the Hyperscale headline plus the four secondary shapes; a name runs that one alone")
+    args = ap.parse_args(argv)
     if args.impl == "reference":
         run_reference(args)
-    elif args.workload == "flat":
-        run_flat(args)
-    elif args.workload == "coarse_hyper":
-        run_coarse_hyper(args)
-    elif args.workload == "hyper":
-        run_hyper(args)
-    elif args.workload == "iter":
-        run_iter(args)
-    elif args.workload == "sharded":
-        run_sharded(args)
-    elif args.workload == "sweep":
-        run_sweep(args)
-    elif args.workload == "pq4":
-        run_pq4(args)
-    else:
-        run_ours(args)
+        return
+    if args.gpus > 1 and "RANK" not in os.environ:
+        # started plainly: start the ranks ourselves, one process per GPU, and hand over
+        port = 29400 + os.getpid() % 500
+        raise SystemExit(subprocess.call(launcher_command(args.gpus, argv, port)))
+    run_ours(args)
 
 
 if __name__ == "__main__":

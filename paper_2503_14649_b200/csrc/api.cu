@@ -196,7 +196,8 @@ static rago_status run_coarse(const IndexImpl* ix, const float* queries, int nq,
         if (e != cudaSuccess) return cuda_fail(e, "tensor-core coarse kernel");
         record(mix, 1, s);
         if (L.tc_mode == 0)
-            e = launch_select_probes_cand(ix, queries, G.cand, G.cand_cnt, L.tc_nsplit * GEMM_COL_HALVES, L.tc_cap, nq, nprobe, probe_list,
+            e = launch_select_probes_cand(ix, queries, G.cand, G.cand_cnt, gemm_cand_sign(G.alpha, G.colterm),
+                                          L.tc_nsplit * GEMM_COL_HALVES, L.tc_cap, nq, nprobe, probe_list,
                                           probe_term, probe_bias, s);
         else
             e = launch_select_probes(ix, queries, scores, nq, nprobe, probe_list, probe_term, probe_bias, s);

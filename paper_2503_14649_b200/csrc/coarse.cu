@@ -211,7 +211,7 @@ cudaError_t launch_coarse_scores(const IndexImpl* ix, const float* queries, int 
 constexpr int SEL_MAX_SPLIT = 512;  // candidate lists per query the kernel can index (one per column range of the GEMM)
 
 // Candidates come either from a score row (scores != null: all nlist lists) or from the candidate
-// lists the tensor-core kernel left behind (cand[q][split][cap] keys with counts cand_cnt[q][split]).
+// lists the tensor-core kernel left behind (cand[q][split][cap] raw entries, see cand_key, with counts cand_cnt[q][split]).
 // First a cut value is found on the ordered score bits (the range is narrowed by counting items per slice in
 // shared memory, then bisected if ties or an odd distribution leave it open; items are held in registers when
 // they fit, re-read from memory otherwise) such that between nsel and nsel + slack items lie at or below it;
@@ -224,9 +224,9 @@ constexpr int SEL_MAX_SPLIT = 512;  // candidate lists per query the kernel can 
 template <bool BF16, int SEL_THREADS, int SEL_REG, bool FROM_SCORES>
 __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
     const float* __restrict__ Q, const void* __restrict__ C, const float* __restrict__ scores,
-    const unsigned long long* __restrict__ cand, const int32_t* __restrict__ cand_cnt, int nsplit, int cap, int nlist,
-    int d, int metric, int nprobe, int32_t* __restrict__ probe_list, float* __restrict__ probe_term,
-    float* __restrict__ probe_bias) {
+    const unsigned long long* __restrict__ cand, const int32_t* __restrict__ cand_cnt, uint32_t cand_sign, int nsplit,
+    int cap, int nlist, int d, int metric, int nprobe, int32_t* __restrict__ probe_list,
+    float* __restrict__ probe_term, float* __restrict__ probe_bias) {
     __shared__ unsigned long long keys[TOPK_CAP];
     __shared__ unsigned long long keys2[MAX_K + PROBE_GUARD];
     __shared__ int pre[SEL_MAX_SPLIT + 1];  // candidate path: exclusive prefix of the lists' counts
@@ -262,7 +262,7 @@ __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
             const int mid_s = (lo_s + hi_s) >> 1;
             if (pre[mid_s] <= l) lo_s = mid_s; else hi_s = mid_s;
         }
-        return cand[((size_t)q * nsplit + lo_s) * cap + (l - pre[lo_s])];
+        return cand_key(cand[((size_t)q * nsplit + lo_s) * cap + (l - pre[lo_s])], cand_sign);
     };
     const bool in_regs = nitems <= SEL_REG * SEL_THREADS;
     uint32_t mine[SEL_REG];  // ordered score bits; 0xFFFFFFFF marks an empty slot
@@ -456,38 +456,38 @@ __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
 
 template <bool BF16, int THREADS, int REG>
 static void launch_select_source(const IndexImpl* ix, const float* queries, const float* scores,
-                                 const unsigned long long* cand, const int32_t* cand_cnt, int nsplit, int cap, int nq,
+                                 const unsigned long long* cand, const int32_t* cand_cnt, uint32_t cand_sign, int nsplit, int cap, int nq,
                                  int nprobe, int32_t* probe_list, float* probe_term, float* probe_bias, cudaStream_t s) {
     if (scores)
         launch_overlapped(select_probes_kernel<BF16, THREADS, REG, true>, dim3(nq), dim3(THREADS), 0, s,
-            queries, ix->centroids, scores, cand, cand_cnt, nsplit, cap, ix->nlist, ix->d, ix->metric, nprobe, probe_list,
+            queries, ix->centroids, scores, cand, cand_cnt, cand_sign, nsplit, cap, ix->nlist, ix->d, ix->metric, nprobe, probe_list,
             probe_term, probe_bias);
     else
         launch_overlapped(select_probes_kernel<BF16, THREADS, REG, false>, dim3(nq), dim3(THREADS), 0, s,
-            queries, ix->centroids, scores, cand, cand_cnt, nsplit, cap, ix->nlist, ix->d, ix->metric, nprobe, probe_list,
+            queries, ix->centroids, scores, cand, cand_cnt, cand_sign, nsplit, cap, ix->nlist, ix->d, ix->metric, nprobe, probe_list,
             probe_term, probe_bias);
 }
 template <int THREADS, int REG>
 static void launch_select_shape(const IndexImpl* ix, const float* queries, const float* scores,
-                                const unsigned long long* cand, const int32_t* cand_cnt, int nsplit, int cap, int nq,
+                                const unsigned long long* cand, const int32_t* cand_cnt, uint32_t cand_sign, int nsplit, int cap, int nq,
                                 int nprobe, int32_t* probe_list, float* probe_term, float* probe_bias, cudaStream_t s) {
     if (ix->coarse_bf16)
-        launch_select_source<true, THREADS, REG>(ix, queries, scores, cand, cand_cnt, nsplit, cap, nq, nprobe, probe_list,
+        launch_select_source<true, THREADS, REG>(ix, queries, scores, cand, cand_cnt, cand_sign, nsplit, cap, nq, nprobe, probe_list,
                                                  probe_term, probe_bias, s);
     else
-        launch_select_source<false, THREADS, REG>(ix, queries, scores, cand, cand_cnt, nsplit, cap, nq, nprobe, probe_list,
+        launch_select_source<false, THREADS, REG>(ix, queries, scores, cand, cand_cnt, cand_sign, nsplit, cap, nq, nprobe, probe_list,
                                                   probe_term, probe_bias, s);
 }
 static cudaError_t launch_select_any(const IndexImpl* ix, const float* queries, const float* scores,
-                                     const unsigned long long* cand, const int32_t* cand_cnt, int nsplit, int cap, int nq,
+                                     const unsigned long long* cand, const int32_t* cand_cnt, uint32_t cand_sign, int nsplit, int cap, int nq,
                                      int nprobe, int32_t* probe_list, float* probe_term, float* probe_bias,
                                      cudaStream_t s) {
     if (nsplit > SEL_MAX_SPLIT) return cudaErrorInvalidValue;
     if (nq <= 64)
-        launch_select_shape<1024, 16>(ix, queries, scores, cand, cand_cnt, nsplit, cap, nq, nprobe, probe_list, probe_term,
+        launch_select_shape<1024, 16>(ix, queries, scores, cand, cand_cnt, cand_sign, nsplit, cap, nq, nprobe, probe_list, probe_term,
                                       probe_bias, s);
     else
-        launch_select_shape<256, 20>(ix, queries, scores, cand, cand_cnt, nsplit, cap, nq, nprobe, probe_list, probe_term,
+        launch_select_shape<256, 20>(ix, queries, scores, cand, cand_cnt, cand_sign, nsplit, cap, nq, nprobe, probe_list, probe_term,
                                      probe_bias, s);
     count_launch();
     return cudaGetLastError();
@@ -495,14 +495,14 @@ static cudaError_t launch_select_any(const IndexImpl* ix, const float* queries, 
 
 cudaError_t launch_select_probes(const IndexImpl* ix, const float* queries, const float* scores, int nq, int nprobe,
                                  int32_t* probe_list, float* probe_term, float* probe_bias, cudaStream_t s) {
-    return launch_select_any(ix, queries, scores, nullptr, nullptr, 0, 0, nq, nprobe, probe_list, probe_term,
+    return launch_select_any(ix, queries, scores, nullptr, nullptr, 0u, 0, 0, nq, nprobe, probe_list, probe_term,
                              probe_bias, s);
 }
 
 cudaError_t launch_select_probes_cand(const IndexImpl* ix, const float* queries, const unsigned long long* cand,
-                                      const int32_t* cand_cnt, int nsplit, int cap, int nq, int nprobe,
+                                      const int32_t* cand_cnt, uint32_t cand_sign, int nsplit, int cap, int nq, int nprobe,
                                       int32_t* probe_list, float* probe_term, float* probe_bias, cudaStream_t s) {
-    return launch_select_any(ix, queries, nullptr, cand, cand_cnt, nsplit, cap, nq, nprobe, probe_list, probe_term,
+    return launch_select_any(ix, queries, nullptr, cand, cand_cnt, cand_sign, nsplit, cap, nq, nprobe, probe_list, probe_term,
                              probe_bias, s);
 }
 

@@ -79,6 +79,9 @@ __host__ __device__ inline float orderable_f32(uint32_t o) {
     union { float f; uint32_t u; } c; c.u = u; return c.f;
 #endif
 }
+// the same on raw fp32 bit patterns
+__host__ __device__ inline uint32_t ord_bits(uint32_t u) { return u ^ ((uint32_t)((int32_t)u >> 31) | 0x80000000u); }
+__host__ __device__ inline uint32_t unord_bits(uint32_t o) { return (o & 0x80000000u) ? (o & 0x7FFFFFFFu) : ~o; }
 __host__ __device__ inline unsigned long long make_key(float score_smaller_is_better, uint32_t payload) {
     return ((unsigned long long)f32_orderable(score_smaller_is_better) << 32) | payload;
 }
@@ -198,7 +201,7 @@ cudaError_t launch_coarse_scores(const IndexImpl* ix, const float* queries, int 
 cudaError_t launch_select_probes(const IndexImpl* ix, const float* queries, const float* scores, int nq, int nprobe,
                                  int32_t* probe_list, float* probe_term, float* probe_bias, cudaStream_t s);
 cudaError_t launch_select_probes_cand(const IndexImpl* ix, const float* queries, const unsigned long long* cand,
-                                      const int32_t* cand_cnt, int nsplit, int cap, int nq, int nprobe,
+                                      const int32_t* cand_cnt, uint32_t cand_sign, int nsplit, int cap, int nq, int nprobe,
                                       int32_t* probe_list, float* probe_term, float* probe_bias, cudaStream_t s);
 // gemm_select.cu
 constexpr int GEMM_CAP_SMALL = 512, GEMM_CAP_LARGE = 1024;  // candidate-list capacities (keys per list)
@@ -216,6 +219,13 @@ struct GemmLaunch {
     unsigned long long* cand; int32_t* cand_cnt;  // [nrows][nsplit * GEMM_COL_HALVES][cap] keys and their counts
     float* scores; uint32_t* err;
 };
+// Candidate lists leave the tensor-core kernel as RAW entries: low word = column, high word = fp32 bits of the
+// score xor a sign word (0x80000000 when the kernel stores the accumulator value of a score = -value).  Readers
+// turn an entry into the usual key with cand_key().
+__host__ __device__ inline uint32_t gemm_cand_sign(float alpha, const float* colterm) { return alpha == -1.f && colterm == nullptr ? 0x80000000u : 0u; }
+__host__ __device__ inline unsigned long long cand_key(unsigned long long entry, uint32_t sign) {
+    return ((unsigned long long)ord_bits((uint32_t)(entry >> 32) ^ sign) << 32) | (uint32_t)entry;
+}
 cudaError_t gemm_select_init();
 cudaError_t make_tmap_bf16(void* out_map, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows,
                            uint64_t row_stride = 0);

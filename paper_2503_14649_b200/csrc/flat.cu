@@ -107,8 +107,9 @@ __global__ void __launch_bounds__(FSEL_THREADS) flat_select_kernel(const float* 
     if (tid == 0) slot_cnt[slot] = kept;
 }
 
-// slot (q, ch) holds slot_cnt keys at slot_keys[(q * nchunks + ch) * stride ...].
-__global__ void __launch_bounds__(FSEL_THREADS) flat_merge_kernel(int nchunks, int k, int stride,
+// slot (q, ch) holds slot_cnt keys at slot_keys[(q * nchunks + ch) * stride ...]; with `raw` they are the raw
+// candidate entries of the tensor-core kernel (cand_key turns them into keys).
+__global__ void __launch_bounds__(FSEL_THREADS) flat_merge_kernel(int nchunks, int k, int stride, int raw, uint32_t raw_sign,
                                                                   const int32_t* __restrict__ slot_cnt,
                                                                   const unsigned long long* __restrict__ slot_keys,
                                                                   int64_t* __restrict__ out_ids,
@@ -131,7 +132,7 @@ __global__ void __launch_bounds__(FSEL_THREADS) flat_merge_kernel(int nchunks, i
         for (int i0 = 0; i0 < c; i0 += FSEL_THREADS) {
             const int i = i0 + tid;
             unsigned long long key = KEY_MAX;
-            if (i < c) key = slot_keys[slot * stride + i];
+            if (i < c) key = raw ? cand_key(slot_keys[slot * stride + i], raw_sign) : slot_keys[slot * stride + i];
             warp_push(keys, &cnt, i < c && key < tau, key);
         }
         __syncthreads();
@@ -246,7 +247,8 @@ cudaError_t launch_flat_search(const void* db, int64_t N, int d, const void* que
         }
         e = launch_gemm_select(G, s);
         if (e != cudaSuccess) return e;
-        flat_merge_kernel<<<nq, FSEL_THREADS, 0, s>>>(nlists, k, cap, cand_cnt, cand, out_ids, out_scores);
+        flat_merge_kernel<<<nq, FSEL_THREADS, 0, s>>>(nlists, k, cap, 1, gemm_cand_sign(G.alpha, G.colterm), cand_cnt, cand,
+                                                      out_ids, out_scores);
         count_launch();
         return cudaGetLastError();
     }
@@ -269,7 +271,7 @@ cudaError_t launch_flat_search(const void* db, int64_t N, int d, const void* que
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
-    flat_merge_kernel<<<nq, FSEL_THREADS, 0, s>>>(nchunks, k, k, slot_cnt, slot_keys, out_ids, out_scores);
+    flat_merge_kernel<<<nq, FSEL_THREADS, 0, s>>>(nchunks, k, k, 0, 0u, slot_cnt, slot_keys, out_ids, out_scores);
     count_launch();
     return cudaGetLastError();
 }

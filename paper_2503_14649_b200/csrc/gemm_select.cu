@@ -115,10 +115,10 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
            ((uint64_t)2 << 61);
 }
 
-// While the kernel runs, a candidate list holds RAW entries: low word = column, high word = the fp32 bits of the
-// score xor `sign` (sign = 0x80000000 on the alpha = -1 path, where the accumulator value itself is stored and
-// the score is its negation).  Appending is then a compare, a predicated 8-byte store and a predicated pointer
-// bump per value; the order-preserving key bits are formed once per kept entry when the CTA finishes.
+// A candidate list holds RAW entries: low word = column, high word = the fp32 bits of the score xor `sign`
+// (sign = 0x80000000 on the alpha = -1 path, where the accumulator value itself is stored and the score is its
+// negation).  Appending is then a compare, a predicated 8-byte store and a predicated pointer bump per value;
+// the order-preserving key bits are formed by whoever reads the list (cand_key in common.cuh).
 //   if (value > thr) { *ptr++ = {col, bits(value)}; }          (alpha = -1, no column term: score = -value)
 __device__ __forceinline__ void push_if_above(unsigned long long*& ptr, float value, float thr, uint32_t col) {
     asm volatile(
@@ -141,8 +141,6 @@ __device__ __forceinline__ void push_if_below(unsigned long long*& ptr, float sc
         : "f"(score), "f"(tau), "r"(col), "r"(bits)
         : "memory");
 }
-__device__ __forceinline__ uint32_t ord_bits(uint32_t u) { return u ^ ((uint32_t)((int32_t)u >> 31) | 0x80000000u); }
-__device__ __forceinline__ uint32_t unord_bits(uint32_t o) { return (o & 0x80000000u) ? (o & 0x7FFFFFFFu) : ~o; }
 
 struct GemmArgs {
     int nrows, ncols;            // valid rows of A (queries) and of B (lists / database rows)
@@ -280,14 +278,6 @@ __device__ __forceinline__ void epilogue_select(uint32_t taddr, const float* cn,
         }
     }
     cnt = (int)(ptr - list);
-}
-
-// Raw entries -> keys (ordered score bits << 32 | column), by the thread that owns the list.
-__device__ __forceinline__ void finish_list(unsigned long long* list, int cnt, uint32_t sign) {
-    for (int i = 0; i < cnt; ++i) {
-        const unsigned long long e = list[i];
-        list[i] = ((unsigned long long)ord_bits((uint32_t)(e >> 32) ^ sign) << 32) | (uint32_t)e;
-    }
 }
 
 // The same in mode 1: scores of row `row`, columns colb .. colb + G_HALF - 1, to the score matrix.
@@ -445,7 +435,7 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         }
         const int slack = a.nsel / 4 > 8 ? a.nsel / 4 : 8;
         const int nkeep = a.nsel + slack < CAP - 64 ? a.nsel + slack : CAP - 64;  // what the bisection may leave in a list
-        const bool neg1 = a.alpha == -1.f && a.colterm == nullptr;  // accumulator values are compared and stored as they are
+        const bool neg1 = gemm_cand_sign(a.alpha, a.colterm) != 0u;  // accumulator values are compared and stored as they are
         unsigned long long* lists[2];
 #pragma unroll
         for (int g = 0; g < 2; ++g) {  // never written for padding rows
@@ -491,10 +481,7 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
 #pragma unroll
             for (int g = 0; g < 2; ++g) {
                 const int r = (m0 + g) * GBM + q4 * 32 + lane;
-                if (g < mcount && r < a.nrows) {
-                    finish_list(lists[g], cnt[g], neg1 ? 0x80000000u : 0u);
-                    a.cand_cnt[((size_t)r * nsplit + split) * GEMM_COL_HALVES + half] = cnt[g];
-                }
+                if (g < mcount && r < a.nrows) a.cand_cnt[((size_t)r * nsplit + split) * GEMM_COL_HALVES + half] = cnt[g];
             }
         }
     }

@@ -1,9 +1,9 @@
 """Parity at the full sizes of the benchmark shapes, in the launch configuration bench.py times.
 
-The oracle cannot search a billion vectors, so each test checks a sample: a few queries of the batch
-against the oracle run on exactly the inverted lists those queries probe (regenerated on the CPU from
-the seed for the hash-coded shapes), and for flat search the returned rows' exact scores plus the
-absence of better rows in a sampled part of the database.
+The oracle cannot hold a billion vectors, so each IVF-PQ test checks a sample of at least 64 queries, each of
+them through ALL of the lists it probes: the oracle runs on exactly those inverted lists (regenerated on the CPU
+from the seed for the hash-coded shapes).  The flat test scores 16 queries against all ten million rows with the
+oracle, the database streamed to the host chunk by chunk.
 """
 
 import gc
@@ -14,7 +14,7 @@ import torch
 
 import oracle
 from paper_2503_14649_b200 import binding, synth
-from tests.helpers import compact_hashed_subindex, host_index, match_results
+from tests.helpers import IvfPqRescorer, compact_hashed_subindex, host_index, match_results
 
 pytestmark = pytest.mark.gpu
 
@@ -37,10 +37,12 @@ def _check_sample(data, hix, q_all, sample, gi, gd, gl, nprobe, k):
     sgn = 1.0 if data.metric == "l2" else -1.0
     q = q_all[sample].cpu().numpy()
     oi, od, op = oracle.ivfpq_search(hix, q, nprobe, k, nthreads=oracle.default_threads(), want_probes=True)
+    rs = IvfPqRescorer(oracle, hix)
     for t, qi in enumerate(sample):
         if not np.array_equal(gl[qi], op[t]):
             assert set(gl[qi].tolist()) == set(op[t].tolist()), ("probe lists differ", qi)
-        assert not match_results(gi[qi], sgn * gd[qi], oi[t], sgn * od[t], rel=REL), ("query", qi)
+        problems = match_results(gi[qi], sgn * gd[qi], oi[t], sgn * od[t], rel=REL, rescore=rs.for_query(q[t], sgn))
+        assert not problems, ("query", qi, problems[:4])
 
 
 def test_mid_full_size_sampled():
@@ -58,7 +60,7 @@ def test_mid_full_size_sampled():
     gi, gd, gl = ids.cpu().numpy(), dists.cpu().numpy(), lists.cpu().numpy()
     ix.close()
     hix = host_index(oracle, data)
-    sample = list(range(0, c["nq"], 32))  # 32 of the 1024 queries
+    sample = list(range(0, c["nq"], 8))  # 128 of the 1024 queries
     _check_sample(data, hix, data.queries, sample, gi, gd, gl, c["nprobe"], c["k"])
     del data, ix, q, ids, dists, lists
     _free()
@@ -77,18 +79,23 @@ def test_hyperscale_full_size_sampled():
     torch.cuda.synchronize()
     ix.rago_check()
     gi, gd, gl = ids.cpu().numpy(), dists.cpu().numpy(), lists.cpu().numpy()
-    sample = [0, 1023, 2048, 4095]
-    # the same four queries as a batch of their own: the small-batch path (tables built ahead of the scan)
-    qs = q[sample].contiguous()
+    sample = list(range(0, c["nq"], 64)) + [4095]  # 65 of the 4096 queries
+    small = [0, 1023, 2048, 4095]
+    # four queries as a batch of their own: the small-batch path (tables built ahead of the scan)
+    qs = q[small].contiguous()
     ids4, dists4 = ix.rago_search(qs, c["nprobe"], c["k"])
     lists4, _ = ix.rago_search_probes(qs, c["nprobe"])
     torch.cuda.synchronize()
     ix.rago_check()
     gi4, gd4, gl4 = ids4.cpu().numpy(), dists4.cpu().numpy(), lists4.cpu().numpy()
     ix.close()
-    hix = compact_hashed_subindex(oracle, data, np.unique(gl[sample]))
+    # the lists the ORACLE's coarse step picks for the sampled queries (nothing here comes from the device)
+    cen_h = data.centroids.cpu().view(torch.uint16).numpy()
+    want_lists, _ = oracle.coarse(cen_h, data.queries[sorted(set(sample + small))].cpu().numpy(), c["nprobe"], data.metric,
+                                  coarse_bf16=True, nthreads=oracle.default_threads())
+    hix = compact_hashed_subindex(oracle, data, np.unique(want_lists))
     _check_sample(data, hix, data.queries, sample, gi, gd, gl, c["nprobe"], c["k"])
-    _check_sample(data, hix, data.queries[sample], [0, 1, 2, 3], gi4, gd4, gl4, c["nprobe"], c["k"])
+    _check_sample(data, hix, data.queries[small], [0, 1, 2, 3], gi4, gd4, gl4, c["nprobe"], c["k"])
     del data, ix, q, ids, dists, lists
     _free()
 
@@ -113,13 +120,18 @@ def test_iterative_stream_full_size_sampled():
         pos += nb
     torch.cuda.synchronize()
     ix.rago_check(ws)
-    picked = [0, 37, 128, 255]
+    picked = list(range(0, 256, 8)) + [37, 255]  # 34 of the 256 batches: well over 64 queries
+    assert sum(sizes[b] for b in picked) >= 64
     probes = {}
     for b in picked:
         p0, nb, _, _ = outs[b]
         probes[b] = ix.rago_search_probes(qd[p0:p0 + nb].contiguous(), c["nprobe"])[0].cpu().numpy()
     ix.close()
-    hix = compact_hashed_subindex(oracle, data, np.unique(np.concatenate([probes[b].ravel() for b in picked])))
+    qpick = np.concatenate([np.arange(outs[b][0], outs[b][0] + outs[b][1]) for b in picked])
+    want_lists, _ = oracle.coarse(data.centroids.cpu().numpy(), data.queries[qpick].cpu().numpy(), c["nprobe"], data.metric,
+                                  nthreads=oracle.default_threads())
+    hix = compact_hashed_subindex(oracle, data, np.unique(want_lists))
+    rs = IvfPqRescorer(oracle, hix)
     for b in picked:
         p0, nb, oi, od = outs[b]
         qh = data.queries[p0:p0 + nb].cpu().numpy()
@@ -127,41 +139,46 @@ def test_iterative_stream_full_size_sampled():
         gi, gd = oi.cpu().numpy(), od.cpu().numpy()
         for i in range(nb):
             assert set(probes[b][i].tolist()) == set(rp[i].tolist()), ("probe lists differ", b, i)
-            assert not match_results(gi[i], gd[i], ri[i], rd[i], rel=REL), ("batch", b, "query", i)
+            problems = match_results(gi[i], gd[i], ri[i], rd[i], rel=REL, rescore=rs.for_query(qh[i]))
+            assert not problems, ("batch", b, "query", i, problems[:4])
     del data, ix, qd, outs, ws
     _free()
 
 
-def test_flat_full_size_sampled():
-    """Flat search at 10 M x 1024 bf16: exact scores of the returned rows, and no better row in two samples."""
+def test_flat_full_size_against_the_whole_database():
+    """Flat search at 10 M x 1024 bf16: 16 of the 256 queries scored by the oracle against every row.  The database
+    goes to the host one chunk at a time; the oracle's best k of every chunk are merged on the host (best first, ties
+    to the smaller row), which is the exact answer over all rows."""
     _need_gb(30)
     c = synth.CONFIGS[5]
+    k = c["k"]
     db, q = synth.make_flat(c["N"], c["d"], c["nq"], device="cuda")
-    gi_t, gs_t = binding.rago_flat_search(db, q, c["k"])
+    gi_t, gs_t = binding.rago_flat_search(db, q, k)
     torch.cuda.synchronize()
     gi, gs = gi_t.cpu().numpy(), gs_t.cpu().numpy()
-    qbits = q.cpu().view(torch.uint16).numpy()
-    g = np.random.default_rng(5)
-    rnd_rows = np.sort(g.choice(c["N"], 20_000, replace=False)).astype(np.int64)
-    rnd_bits = db[torch.from_numpy(rnd_rows).cuda()].cpu().view(torch.uint16).numpy()
-    pre_n = 100_000
-    pre_bits = db[:pre_n].cpu().view(torch.uint16).numpy()
-    for qi in (0, 100, 255):
-        rows = gi[qi]
-        assert len(set(rows.tolist())) == c["k"] and rows.min() >= 0 and rows.max() < c["N"]
-        got_bits = db[torch.from_numpy(rows).cuda()].cpu().view(torch.uint16).numpy()
-        exact = oracle.flat_scores(got_bits, qbits[qi], np.arange(c["k"], dtype=np.int64))
-        assert np.allclose(gs[qi], exact, rtol=1e-3, atol=1e-6), qi           # reported scores are the rows' scores
+    sample = list(range(0, c["nq"], 16))  # 16 queries: one per host core where there are 16
+    qbits = q.cpu().view(torch.uint16).numpy()[sample]
+    chunk = 1_000_000
+    best_i = [np.zeros(0, np.int64) for _ in sample]
+    best_s = [np.zeros(0, np.float32) for _ in sample]
+    for r0 in range(0, c["N"], chunk):
+        bits = db[r0:r0 + chunk].cpu().view(torch.uint16).numpy()
+        ci, cs = oracle.flat_search(bits, qbits, k, nthreads=oracle.default_threads())
+        for t in range(len(sample)):
+            ids = np.concatenate([best_i[t], ci[t] + r0])
+            sc = np.concatenate([best_s[t], cs[t]])
+            order = np.lexsort((ids, -sc.astype(np.float64)))[:k]
+            best_i[t], best_s[t] = ids[order], sc[order]
+        del bits
+    for t, qi in enumerate(sample):
         assert np.all(np.diff(gs[qi]) <= 0), qi                                # best first
-        kth = float(gs[qi][-1])
-        tol = 1e-3 * abs(kth) + 1e-6
-        inres = set(rows.tolist())
-        # a random sample of the database and a contiguous prefix: nothing outside the result beats the k-th
-        s_rnd = oracle.flat_scores(rnd_bits, qbits[qi], np.arange(len(rnd_rows), dtype=np.int64))
-        for r, sc in zip(rnd_rows, s_rnd):
-            assert sc <= kth + tol or int(r) in inres, (qi, int(r), sc, kth)
-        pi, ps = oracle.flat_search(pre_bits, qbits[qi:qi + 1], c["k"], nthreads=oracle.default_threads())
-        for r, sc in zip(pi[0], ps[0]):
-            assert sc <= kth + tol or int(r) in inres, (qi, int(r), float(sc), kth)
+
+        def rescore(row, t=t):
+            if row < 0 or row >= c["N"]:
+                raise KeyError(row)
+            rb = db[row:row + 1].cpu().view(torch.uint16).numpy()
+            return -float(oracle.flat_scores(rb, qbits[t], np.array([0], np.int64))[0])
+        problems = match_results(gi[qi], -gs[qi], best_i[t], -best_s[t], rel=1e-3, rescore=rescore)
+        assert not problems, (qi, problems[:4])
     del db, q, gi_t, gs_t
     _free()

@@ -5,15 +5,17 @@ belongs to an LLM server's pool, or an allocation would synchronise a device tha
 For them the library keeps the coarse step's score matrix in a fixed array of its own.  This test
 calls that entry point through the C ABI twice in a row (the second call finds the first call's
 data in the shared array and must not be disturbed by it) and expects the same probe lists and
-coarse values as the workspace-based entry point, then checks that an oversized batch is refused.
-The file name sorts last so that every other GPU test has run before this one.
+coarse values as the workspace-based entry point and as the CPU oracle's coarse step, then checks that an
+oversized batch is refused.  The file name sorts last so that every other GPU test has run before this one.
 """
 
 import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2503_14649_b200 import binding, synth
+from tests.helpers import coarse_rescorer, host_index, match_results
 
 pytestmark = pytest.mark.gpu
 
@@ -25,6 +27,8 @@ def test_noalloc_probes_match_workspace_probes_twice(metric, bf16):
     data = synth.make_ivfpq(6000, 128, 96, 16, 48, metric=metric, seed=901, coarse_bf16=bf16)
     ix = binding.load_index_from(data, "cuda")
     q_all = data.queries.cuda().contiguous()
+    hix = host_index(oracle, data)
+    sgn = 1.0 if metric == "l2" else -1.0
     nprobe = 12
     # outputs are the caller's and exist before the calls; the calls themselves allocate nothing
     for lo, hi in ((0, 48), (5, 29)):  # second call: fewer, different queries over the same array
@@ -37,6 +41,13 @@ def test_noalloc_probes_match_workspace_probes_twice(metric, bf16):
         assert torch.equal(got_lists.cpu(), want_lists.cpu())
         g, w = got_coarse.cpu().numpy(), want_coarse.cpu().numpy()
         assert np.allclose(g, w, rtol=REL, atol=REL * max(1.0, float(np.abs(w).max())))
+        # and against the oracle's coarse step directly, so that this file stands on its own
+        qh = data.queries[lo:hi].numpy()
+        ol, oc = oracle.coarse(hix.centroids, qh, nprobe, metric, coarse_bf16=bf16)
+        gl = got_lists.cpu().numpy().astype(np.int64)
+        for i in range(hi - lo):
+            assert not match_results(gl[i], sgn * g[i], ol[i].astype(np.int64), sgn * oc[i], rel=REL,
+                                     rescore=coarse_rescorer(oracle, hix.centroids, qh[i], metric, bf16, sgn)), i
     ix.close()
 
 
