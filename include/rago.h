@@ -214,6 +214,22 @@ rago_status rago_flat_workspace_bytes(int64_t N, int32_t d, int32_t nq, int32_t 
 rago_status rago_check(void* workspace, void* cuda_stream);
 
 /*
+ * Test hook for the failure path of rago_check (no counterpart in the paper: the library's kernels wait on
+ * copies and on the tensor pipe, every such wait is bounded, and this call lets a test see a bound expire
+ * without anything being wrong).  Launches one small kernel in which a wait on a barrier that nothing signals
+ * gives up after `max_polls` polls (1 .. 4096, each at most 4 microseconds) exactly as a wait inside a search
+ * kernel would: it records RAGO_ETIMEOUT in the first word of `workspace`, a second waiting warp is released by
+ * the abort flag, and with `with_tmem` != 0 the kernel holds and then releases the SM's tensor memory the way
+ * the tensor-core kernel does.  The kernel ends normally; the device stays usable.
+ *
+ *   workspace   dev, 256-byte aligned, at least 256 bytes.  After the call (asynchronous on cuda_stream)
+ *               rago_check(workspace, stream) returns RAGO_ETIMEOUT; words 8 and 9 of the workspace are 1 if
+ *               the first wait expired and if the second was released by the abort flag.  Any later search
+ *               call that is given this workspace clears the error word first.
+ */
+rago_status rago_selftest_wait_timeout(void* workspace, uint32_t max_polls, int32_t with_tmem, void* cuda_stream);
+
+/*
  * Which kernel computes the coarse scores: 0 = automatic (tensor cores for batches of more than 16
  * queries, the fp32 kernel for smaller ones), 1 = always the fp32 kernel, 2 = always tensor cores.
  * The tensor-core kernel multiplies bf16 operands; fp32 queries and centroids are split into three

@@ -27,7 +27,7 @@ STAGE_NAMES = ("coarse_scores", "probe_select", "plan", "table_scan", "merge")
 EXPORTS = ("rago_index_load", "rago_index_load_pq4", "rago_index_free", "rago_search_workspace_bytes", "rago_search",
            "rago_search_probes", "rago_search_probes_noalloc", "rago_search_host", "rago_host_staging_bytes", "rago_flat_search",
            "rago_flat_workspace_bytes", "rago_check", "rago_set_coarse_mode", "rago_profile_enable", "rago_profile_read",
-           "rago_merge_results", "rago_kernel_launches", "rago_last_error")
+           "rago_merge_results", "rago_selftest_wait_timeout", "rago_kernel_launches", "rago_last_error")
 
 
 class RagoError(RuntimeError):
@@ -59,6 +59,7 @@ def lib() -> ctypes.CDLL:
         L.rago_flat_workspace_bytes.argtypes = [i64, i32, i32, i32, ctypes.POINTER(sz)]
         L.rago_merge_results.argtypes = [vp, vp, i32, i64, i32, i32, i32, i32, vp, vp, vp]
         L.rago_check.argtypes = [vp, vp]
+        L.rago_selftest_wait_timeout.argtypes = [vp, ctypes.c_uint32, i32, vp]
         L.rago_set_coarse_mode.argtypes = [vp, i32]
         L.rago_profile_enable.argtypes = [vp, i32]
         L.rago_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
@@ -206,6 +207,16 @@ def rago_index_load_pq4(centroids, pq4_codebooks, packed_codes, list_offsets, id
     if pq4_codebooks.shape[1] != 16:
         raise ValueError("4-bit codebooks have 16 codewords per sub-space")
     return Index(centroids, pq4_codebooks, packed_codes, list_offsets, ids, metric)
+
+
+def rago_selftest_wait_timeout(workspace: torch.Tensor, max_polls: int, with_tmem: bool):
+    """Launch the bounded-wait self-test on `workspace` (see rago.h); follow with rago_check(workspace)."""
+    _check(lib().rago_selftest_wait_timeout(_ptr(workspace), int(max_polls), int(bool(with_tmem)), _stream()))
+
+
+def rago_check(workspace: torch.Tensor):
+    """rago_check on a bare workspace tensor (Index.rago_check does the same for an index's workspace)."""
+    _check(lib().rago_check(_ptr(workspace), _stream()))
 
 
 def rago_flat_workspace_bytes(N: int, d: int, nq: int, k: int) -> int:

@@ -491,6 +491,18 @@ rago_status rago_check(void* workspace, void* cuda_stream) {
     return RAGO_OK;
 }
 
+rago_status rago_selftest_wait_timeout(void* workspace, uint32_t max_polls, int32_t with_tmem, void* cuda_stream) {
+    if (!workspace) return fail(RAGO_EINVAL, "workspace is null");
+    if (!aligned(workspace, 256)) return fail(RAGO_EALIGN, "workspace needs 256-byte alignment");
+    if (max_polls < 1 || max_polls > 4096) return fail(RAGO_EINVAL, "max_polls = %u outside [1, 4096]", max_polls);
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    uint32_t* w = static_cast<uint32_t*>(workspace);
+    cudaError_t e = cudaMemsetAsync(workspace, 0, 256, s);
+    if (e == cudaSuccess) e = launch_selftest_wait(w, max_polls, with_tmem ? 1 : 0, w + 8, s);
+    if (e != cudaSuccess) return cuda_fail(e, "wait self-test");
+    return RAGO_OK;
+}
+
 rago_status rago_set_coarse_mode(rago_index* index, int32_t mode) {
     if (!index) return fail(RAGO_EINVAL, "index is null");
     if (mode < 0 || mode > 2) return fail(RAGO_EINVAL, "mode = %d: 0 auto, 1 fp32 pipes, 2 tensor cores", mode);

@@ -124,14 +124,16 @@ __device__ __forceinline__ bool mbar_try_wait_hint(uint32_t bar, uint32_t parity
         : "memory");
     return ok != 0;
 }
-// Bounded wait: each poll may park the thread for up to 4 us, and the wait gives up after 2^18
-// polls (about a second) or as soon as *abort_flag is set by another warp.  On give-up it raises the
+// Bounded wait: each poll may park the thread for up to 4 us, and the wait gives up after max_polls
+// polls (2^18: about a second) or as soon as *abort_flag is set by another warp.  On give-up it raises the
 // CTA abort flag and the global error word; callers keep their control flow (so CTA-wide barriers
 // still match) but the data is garbage.
+constexpr uint32_t MBAR_MAX_POLLS = 1u << 18;
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                          uint32_t* err_word, uint32_t backoff_ns = 0) {
+                                          uint32_t* err_word, uint32_t backoff_ns = 0,
+                                          uint32_t max_polls = MBAR_MAX_POLLS) {
     if (mbar_try_wait(bar, parity)) return true;
-    for (uint32_t it = 0; it < (1u << 18); ++it) {
+    for (uint32_t it = 0; it < max_polls; ++it) {
         if (mbar_try_wait_hint(bar, parity, 4000u)) return true;
         if (backoff_ns) __nanosleep(backoff_ns);  // single-lane roles: leave the issue slots to the working warps
         if ((it & 15) == 15 && *abort_flag) return false;
@@ -236,6 +238,7 @@ int gemm_cand_cap(int nsel);  // 0: nsel too large for the fused selection
 void gemm_grid(int nrows, int64_t ncols, int num_sms, int* mg, int* nsplit, int* mgroups);
 cudaError_t launch_gemm_select(const GemmLaunch& L, cudaStream_t s);
 cudaError_t launch_split_bf16(const float* x, size_t n, int parts, void* out, cudaStream_t s);
+cudaError_t launch_selftest_wait(uint32_t* err_word, uint32_t max_polls, int with_tmem, uint32_t* observed, cudaStream_t s);
 // scan.cu
 bool scan_supported(int M);
 cudaError_t scan_plan(const IndexImpl* ix, ScanPlan* plan);

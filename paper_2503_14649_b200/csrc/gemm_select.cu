@@ -676,6 +676,55 @@ cudaError_t gemm_select_init() {
     return e;
 }
 
+// ---- self-test of the bounded waits ---------------------------------------------------------------
+// One CTA, two warps, the roles of the kernels above in miniature.  Lane 0 of warp 0 waits, through the same
+// mbar_wait the kernels use, on a barrier that nothing ever arrives at, with a poll limit of the caller's choice:
+// the wait runs out, sets the CTA's abort flag and the error word.  Lane 0 of warp 1 waits on a second such
+// barrier with the full limit and must be released early by the abort flag (the hand-off that lets every role
+// of a kernel leave its loop after one of them timed out).  With with_tmem the CTA holds all 512 TMEM columns
+// meanwhile and gives them back before it exits, as gemm_select_kernel does after an abort.  Nothing traps,
+// faults or spins without a limit: the kernel ends normally.
+// observed[0] = 1 if the first wait gave up, observed[1] = 1 if the second was released by the abort flag.
+__global__ void __launch_bounds__(64, 1) selftest_wait_kernel(uint32_t* err_word, uint32_t max_polls, int with_tmem,
+                                                              uint32_t* observed) {
+    __shared__ unsigned long long bars[2];
+    __shared__ uint32_t tmem_slot;
+    __shared__ uint32_t abort_word;
+    volatile uint32_t* abort_flag = &abort_word;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) {
+        mbar_init(smem_u32(&bars[0]), 1);
+        mbar_init(smem_u32(&bars[1]), 1);
+        abort_word = 0;
+        fence_barrier_init();
+    }
+    if (with_tmem && warp == 0) tmem_alloc(smem_u32(&tmem_slot), G_TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (lane == 0) {
+        if (warp == 0) {
+            const bool ok = mbar_wait(smem_u32(&bars[0]), 0u, abort_flag, err_word, 0, max_polls);
+            observed[0] = ok ? 0u : 1u;
+        } else {
+            // given the first warp's limit of max_polls polls of at most 4 us, this one must not need its own
+            const bool ok = mbar_wait(smem_u32(&bars[1]), 0u, abort_flag, err_word, 0, MBAR_MAX_POLLS);
+            observed[1] = (!ok && *abort_flag) ? 1u : 0u;
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (with_tmem && warp == 0) {
+        tc_fence_after();
+        tmem_dealloc(tmem_slot, G_TMEM_COLS);
+    }
+}
+cudaError_t launch_selftest_wait(uint32_t* err_word, uint32_t max_polls, int with_tmem, uint32_t* observed, cudaStream_t s) {
+    selftest_wait_kernel<<<1, 64, 0, s>>>(err_word, max_polls, with_tmem, observed);
+    count_launch();
+    return cudaGetLastError();
+}
+
 // ---- fp32 -> stacked bf16 parts: out[p][i] = bf16 part p of x[i] ---------------------------------
 __global__ void split_bf16_kernel(const float* __restrict__ x, size_t n, int parts, __nv_bfloat16* __restrict__ out) {
     for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
