@@ -130,6 +130,17 @@ rago_status rago_search_workspace_bytes(const rago_index* index, int32_t nq, int
  * With a RAGO_BF16 coarse quantiser the query is rounded to bf16 (nearest-even) for the coarse
  * step only; tables are built from the fp32 query.  Ties are broken by storage position.
  * nq == 0 is a no-op.
+ *
+ * Accuracy of out_dists (fp32).  Candidates are RANKED by an expanded form of the score,
+ * ||q-c||^2 + (||r||^2 + 2<c,r>) - 2<q,r> for L2 and <q,c> + <q,r> for IP (c the list's centroid, r the
+ * decoded residual), whose table sum is exact in fixed point (per-query step at most max|entry| * M / 2^30);
+ * its absolute error is a few fp32 ulps of the LARGEST of its terms.  Reported L2 distances are accurate to
+ * about 1e-5 RELATIVE: a result whose value is below 1/32 of its largest term (a query that nearly coincides
+ * with a stored vector) is re-computed in the direct form sum_j ((q_j - c_j) - cw_j)^2 before it is written,
+ * and the k results are re-ordered by the corrected values.  Two candidates whose true distances differ by
+ * less than the ranking error may still swap places at the k-th position.  IP scores are sums of mixed
+ * sign: their error is absolute, a few ulps of max(|<q,c>|, |<q,r>|), not relative to the (possibly
+ * cancelling) result.
  */
 rago_status rago_search(const rago_index* index, const float* queries, int32_t nq, int32_t nprobe, int32_t k,
                         int64_t* out_ids, float* out_dists, void* workspace, size_t workspace_bytes,

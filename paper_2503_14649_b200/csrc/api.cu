@@ -410,7 +410,8 @@ rago_status rago_search(const rago_index* index, const float* queries, int32_t n
                     slot_keys, reinterpret_cast<uint32_t*>(ws + L.err), lut_img, lut_inv, s);
     if (e != cudaSuccess) return cuda_fail(e, "scan kernel");
     record(mix, 4, s);
-    e = launch_merge(ix, work_prefix, nq, nprobe, k, ix->plan.ctas, slot_cnt, slot_keys, qthresh, out_ids, out_dists, s);
+    e = launch_merge(ix, work_prefix, nq, nprobe, k, ix->plan.ctas, slot_cnt, slot_keys, qthresh, queries, probe_list, probe_term,
+                     out_ids, out_dists, s);
     if (e != cudaSuccess) return cuda_fail(e, "merge kernel");
     record(mix, 5, s);
     return RAGO_OK;

@@ -260,7 +260,8 @@ cudaError_t noalloc_prepare();  // with the index's device current: look up (and
 // merge.cu
 cudaError_t launch_merge(const IndexImpl* ix, const int64_t* work_prefix, int nq, int nprobe, int k, int ctas,
                          const int32_t* slot_cnt, const unsigned long long* slot_keys, const unsigned long long* qthresh,
-                         int64_t* out_ids, float* out_dists, cudaStream_t s);
+                         const float* queries, const int32_t* probe_list, const float* probe_bias, int64_t* out_ids,
+                         float* out_dists, cudaStream_t s);
 cudaError_t launch_fill_u64(unsigned long long* p, size_t n, unsigned long long v, cudaStream_t s);
 // flat.cu
 size_t flat_workspace_bytes(int64_t N, int d, int nq, int k);

@@ -1,8 +1,71 @@
 // Final top-k per query: merge the partial candidate lists the scan CTAs left behind, sort, map
 // storage positions to caller ids, and write results best-first.
+//
+// Squared-L2 results whose terms cancel are re-scored before they are written.  The scan ranks candidates with
+// the expanded form  bias + term + sum  =  ||q-c||^2 + (||r||^2 + 2<c,r>) - 2<q,r>,  whose rounding error is a
+// few ulps of its LARGEST term T: harmless for ranking, but for a query that almost coincides with a stored
+// vector the terms (tens to thousands) cancel to a distance of 1e-3 or less and the relative error of the sum
+// becomes large.  A winner whose value is below T / 32 (relative error of the expanded form possibly above
+// ~1e-5; T is known at this point from the list's bias and the vector's stored term) is therefore scored again
+// in the direct form  sum_j ((q_j - c_j) - cw_j)^2  (all terms non-negative: relative error about sqrt(d) ulps),
+// and the winners are re-ordered if any value changed.  On ordinary data no winner qualifies and the check costs
+// one 4-byte load per winner.
 #include "topk.cuh"
 
 namespace rago {
+
+struct RescoreArgs {
+    int enabled;                 // squared L2 only
+    const float* queries;        // [nq][d]
+    const void* centroids;       // [nlist][d] fp32 or bf16
+    int coarse_bf16;
+    const float* cbT;            // [256][M][dsub]: the library's own copy of the codebook, codeword index outermost
+    const uint8_t* codes;        // [N][M]
+    const int64_t* list_offsets; // [nlist + 1]
+    const int32_t* probe_list;   // [nq][nprobe]: a result lies in one of the lists its query probed
+    const float* probe_bias;     // [nq][nprobe]: ||q - c||^2 of those lists (the scan's per-list term)
+    const float* vterm;          // [N]: the scan's per-vector term
+    int nlist, d, M, dsub;
+};
+
+// ||q - (c_list + decoded codewords)||^2 of the vector at storage position pos, which lies in inverted list
+// `list`, by one warp (d a multiple of 4).  All of a lane's loads are independent of each other except the
+// codeword, which follows its code byte.
+__device__ __forceinline__ float direct_l2(const RescoreArgs& r, const float* qrow, uint32_t pos, int list, int lane) {
+    const uint8_t* code = r.codes + (size_t)pos * r.M;
+    float acc = 0.f;
+    for (int j = lane * 4; j < r.d; j += 128) {
+        const float4 qv = *reinterpret_cast<const float4*>(qrow + j);
+        float c[4], cw[4];
+        if (r.coarse_bf16) {
+            const uint2 raw = *reinterpret_cast<const uint2*>(static_cast<const __nv_bfloat16*>(r.centroids) + (size_t)list * r.d + j);
+            c[0] = __uint_as_float(raw.x << 16); c[1] = __uint_as_float(raw.x & 0xFFFF0000u);
+            c[2] = __uint_as_float(raw.y << 16); c[3] = __uint_as_float(raw.y & 0xFFFF0000u);
+        } else {
+            const float4 cv = *reinterpret_cast<const float4*>(static_cast<const float*>(r.centroids) + (size_t)list * r.d + j);
+            c[0] = cv.x; c[1] = cv.y; c[2] = cv.z; c[3] = cv.w;
+        }
+        if ((r.dsub & 3) == 0) {  // the four dimensions share a sub-space: one code byte, one 16-byte codeword load
+            const int m = j / r.dsub, t = j - m * r.dsub;
+            const float4 w = __ldg(reinterpret_cast<const float4*>(r.cbT + ((size_t)code[m] * r.M + m) * r.dsub + t));
+            cw[0] = w.x; cw[1] = w.y; cw[2] = w.z; cw[3] = w.w;
+        } else {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int jj = j + i, m = jj / r.dsub, t = jj - m * r.dsub;
+                cw[i] = __ldg(r.cbT + ((size_t)code[m] * r.M + m) * r.dsub + t);
+            }
+        }
+        const float qq[4] = {qv.x, qv.y, qv.z, qv.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float e = (qq[i] - c[i]) - cw[i];  // residual first, as the definition forms it
+            acc = fmaf(e, e, acc);
+        }
+    }
+    for (int o = 16; o; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    return acc;
+}
 
 // Slot numbering: CTA b working on query q writes slot q + b.  Along the CTAs' contiguous walk over the
 // batch that number strictly increases, so the slots of one query form one range (unused numbers in
@@ -18,15 +81,27 @@ template <int THREADS>
 __global__ void __launch_bounds__(THREADS) merge_kernel(
     const int64_t* __restrict__ work_prefix, const int64_t* __restrict__ ids, int npairs, int nprobe, int k, int ctas,
     int metric, const int32_t* __restrict__ slot_cnt, const unsigned long long* __restrict__ slot_keys,
-    const unsigned long long* __restrict__ qthresh,
+    const unsigned long long* __restrict__ qthresh, const RescoreArgs rs,
     int64_t* __restrict__ out_ids, float* __restrict__ out_dists) {
     __shared__ unsigned long long keys[TOPK_CAP];
     __shared__ int cnt;
+    __shared__ int p_list[MAX_K];          // re-scoring: the query's probed lists and their storage ranges
+    __shared__ uint32_t p_lo[MAX_K], p_hi[MAX_K];
+    __shared__ int redo[MAX_K], redo_list[MAX_K];  // winners to score again (index into keys) and their lists
+    __shared__ int nredo;
     const int q = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     auto sync = [] { __syncthreads(); };
     grid_dependency_wait();
     grid_dependents_may_launch();
-    if (tid == 0) cnt = 0;
+    if (tid == 0) { cnt = 0; nredo = 0; }
+    if (rs.enabled) {
+        for (int i = tid; i < nprobe; i += THREADS) {
+            const int l = rs.probe_list[(size_t)q * nprobe + i];
+            p_list[i] = l;
+            p_lo[i] = (uint32_t)rs.list_offsets[l];
+            p_hi[i] = (uint32_t)rs.list_offsets[l + 1];
+        }
+    }
     __syncthreads();
     const long long W = work_prefix[npairs];
     const long long u0 = work_prefix[(size_t)q * nprobe], u1 = work_prefix[(size_t)(q + 1) * nprobe];
@@ -109,7 +184,40 @@ __global__ void __launch_bounds__(THREADS) merge_kernel(
         }
     }
     __syncthreads();
-    const int kept = block_select(keys, &cnt, k, tid, THREADS, sync);
+    int kept = block_select(keys, &cnt, k, tid, THREADS, sync);
+    if (rs.enabled && kept > 0) {  // uniform
+        // which winners lost too many bits to cancellation: one thread per winner
+        for (int i = tid; i < kept; i += THREADS) {
+            const uint32_t pos = (uint32_t)(keys[i] & 0xFFFFFFFFull);
+            int p = 0;
+            while (p < nprobe && !(pos >= p_lo[p] && pos < p_hi[p])) ++p;
+            if (p == nprobe) continue;  // cannot happen: every candidate comes from a probed list
+            const float dist = orderable_f32((uint32_t)(keys[i] >> 32));
+            const float bias = rs.probe_bias[(size_t)q * nprobe + p], vt = rs.vterm[pos];
+            const float T = fmaxf(fmaxf(bias, fabsf(vt)), fabsf(dist - (bias + vt)));
+            if (dist < T * (1.f / 32.f)) {
+                const int at = atomicAdd(&nredo, 1);
+                redo[at] = i;
+                redo_list[at] = p_list[p];
+            }
+        }
+        __syncthreads();
+        const int nr = nredo;
+        if (nr > 0) {  // uniform
+            const float* qrow = rs.queries + (size_t)q * rs.d;
+            for (int e = warp; e < nr; e += THREADS / 32) {
+                const int i = redo[e];
+                const uint32_t pos = (uint32_t)(keys[i] & 0xFFFFFFFFull);
+                const float dist = direct_l2(rs, qrow, pos, redo_list[e], lane);
+                __syncwarp();
+                if (lane == 0) keys[i] = make_key(dist, pos);
+            }
+            __syncthreads();
+            if (tid == 0) cnt = kept;
+            __syncthreads();
+            kept = block_select(keys, &cnt, k, tid, THREADS, sync);  // order by the new values
+        }
+    }
     for (int i = tid; i < k; i += THREADS) {
         int64_t id = -1;
         float dist = metric == RAGO_L2 ? __int_as_float(0x7f800000) : __int_as_float(0xff800000);
@@ -126,13 +234,20 @@ __global__ void __launch_bounds__(THREADS) merge_kernel(
 
 cudaError_t launch_merge(const IndexImpl* ix, const int64_t* work_prefix, int nq, int nprobe, int k, int ctas,
                          const int32_t* slot_cnt, const unsigned long long* slot_keys, const unsigned long long* qthresh,
-                         int64_t* out_ids, float* out_dists, cudaStream_t s) {
+                         const float* queries, const int32_t* probe_list, const float* probe_bias, int64_t* out_ids,
+                         float* out_dists, cudaStream_t s) {
+    RescoreArgs rs;
+    rs.enabled = ix->metric == RAGO_L2 && ix->vterm != nullptr && ix->d % 4 == 0 ? 1 : 0;
+    rs.queries = queries; rs.centroids = ix->centroids; rs.coarse_bf16 = ix->coarse_bf16; rs.cbT = ix->cbT;
+    rs.codes = ix->codes; rs.list_offsets = ix->list_offsets; rs.probe_list = probe_list;
+    rs.probe_bias = probe_bias; rs.vterm = ix->vterm; rs.nlist = ix->nlist; rs.d = ix->d; rs.M = ix->M;
+    rs.dsub = ix->dsub;
     if (nq <= 64)
         launch_overlapped(merge_kernel<1024>, dim3(nq), dim3(1024), 0, s, work_prefix, ix->ids, nq * nprobe, nprobe, k, ctas,
-                          ix->metric, slot_cnt, slot_keys, qthresh, out_ids, out_dists);
+                          ix->metric, slot_cnt, slot_keys, qthresh, rs, out_ids, out_dists);
     else
         launch_overlapped(merge_kernel<256>, dim3(nq), dim3(256), 0, s, work_prefix, ix->ids, nq * nprobe, nprobe, k, ctas,
-                          ix->metric, slot_cnt, slot_keys, qthresh, out_ids, out_dists);
+                          ix->metric, slot_cnt, slot_keys, qthresh, rs, out_ids, out_dists);
     count_launch();
     return cudaGetLastError();
 }

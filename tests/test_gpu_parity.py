@@ -301,3 +301,24 @@ def test_batch_beyond_the_prebuilt_table_limit_builds_tables_in_the_scan(metric,
     fixed-point scale) instead of fetching an image built ahead."""
     data = synth.make_ivfpq(20_000, d, 64, M, 4200, metric=metric, seed=5)
     _compare(data, 4, 10, max_probe_mismatch=8)
+
+
+def test_near_duplicate_queries_get_relatively_accurate_l2_distances():
+    """Queries that almost coincide with a stored (decoded) vector: the true squared distance is about 1e-4 while
+    the terms of the expanded form the scan ranks with are of size 100 (centroid norms near 28 at d = 768), so
+    only a final score in the direct form meets a relative tolerance.  Distances are compared at 1e-4 relative
+    with the usual tiny floor, i.e. the nearest neighbour's 1e-4 must be right to 1e-8."""
+    data = synth.make_ivfpq(40_000, 768, 64, 96, 8, metric="l2", seed=515)
+    cen, cb = data.centroids.numpy().astype(np.float64), data.codebooks.numpy().astype(np.float64)
+    codes, off = data.codes.numpy(), data.list_offsets.numpy()
+    g = np.random.default_rng(7)
+    rows = g.choice(data.N, 24, replace=False)
+    q = np.empty((24, 768), np.float32)
+    for t, pos in enumerate(rows):
+        lst = int(np.searchsorted(off, pos, side="right") - 1)
+        decoded = cen[lst] + np.concatenate([cb[m, codes[pos, m]] for m in range(96)])
+        q[t] = (decoded + 1e-3 * synth.SIGMA * g.standard_normal(768)).astype(np.float32)
+    data.queries = torch.from_numpy(q)
+    gi, gd = _compare(data, 8, 10)
+    assert np.all(gd[:, 0] < 1e-3) and np.all(gd[:, 0] > 0)           # the near-duplicate itself, far below the terms
+    assert np.array_equal(gi[:, 0], data.ids.numpy()[rows])
