@@ -105,6 +105,42 @@ def ivfpq_search(ix: Index, queries, nprobe, k, nthreads=1, want_probes=False):
     return (ids, dists, probes) if want_probes else (ids, dists)
 
 
+def coarse_tree(centroids, level1, child_offsets, b1, queries, nprobe, metric, coarse_bf16=False, nthreads=1):
+    """Coarse step through a two-level quantiser (see rago_oracle.cpp): the best b1 level-1 nodes, then the best
+    nprobe of their children.  level1 has the storage type of `centroids`; children of node i are the consecutive
+    lists child_offsets[i] .. child_offsets[i + 1] - 1.  Lists come back best first, -1 where the chosen nodes
+    have fewer than nprobe children."""
+    dt = np.uint16 if coarse_bf16 else np.float32
+    cen, top = _c(centroids, dt), _c(level1, dt)
+    off = _c(child_offsets, np.int32)
+    q = _c(queries, np.float32)
+    nq, d = q.shape
+    lists = np.empty((nq, nprobe), np.int32)
+    scores = np.empty((nq, nprobe), np.float64)
+    rc = lib().oracle_coarse_tree(_p(cen), ctypes.c_int(bool(coarse_bf16)), d, cen.shape[0], _METRIC[metric], _p(top),
+                                  _p(off), top.shape[0], int(b1), _p(q), nq, nprobe, _p(lists), _p(scores), nthreads)
+    if rc:
+        raise ValueError("oracle_coarse_tree: bad arguments")
+    return lists, scores
+
+
+def ivfpq_search_tree(ix: Index, level1, child_offsets, b1, queries, nprobe, k, nthreads=1, want_probes=False):
+    """ivfpq_search with the probe lists chosen through the two-level quantiser."""
+    top = _c(level1, np.uint16 if ix.coarse_bf16 else np.float32)
+    off = _c(child_offsets, np.int32)
+    q = _c(queries, np.float32)
+    nq = q.shape[0]
+    ids = np.empty((nq, k), np.int64)
+    dists = np.empty((nq, k), np.float32)
+    probes = np.empty((nq, nprobe), np.int32) if want_probes else None
+    rc = lib().oracle_ivfpq_search_tree(*ix._head(), _p(ix.offsets), _p(ix.ids), ctypes.c_int64(ix.N), ix.d, ix.nlist,
+                                        ix.M, ix.metric, _p(top), _p(off), top.shape[0], int(b1), _p(q), nq, nprobe, k,
+                                        _p(ids), _p(dists), _p(probes), nthreads)
+    if rc:
+        raise ValueError("oracle_ivfpq_search_tree: bad arguments")
+    return (ids, dists, probes) if want_probes else (ids, dists)
+
+
 def adc_score(ix: Index, query, list_no, pos) -> float:
     q = _c(query, np.float32)
     out = ctypes.c_double()

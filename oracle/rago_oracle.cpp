@@ -28,6 +28,18 @@
 // list number / smaller id; missing results are id -1 with +inf (L2) or -inf
 // (inner product).
 //
+// Two-level coarse quantiser (functions with "tree" in their name).  The paper
+// indexes its database with a multi-level tree (Methodology, "Models and
+// database": three levels, balanced fan-out) and models a search as scanning
+// the levels top-down (Methodology, retrieval performance modelling: a sequence
+// of scan operations, one per level).  With two levels above the vectors that
+// is: score every level-1 centroid, keep the best b1 nodes, score the coarse
+// centroids that are their children, keep the best nprobe of those as the
+// probe lists; everything after that is unchanged.  Children of node i are the
+// consecutive lists child_offsets[i] .. child_offsets[i+1]-1.  Pins: with
+// b1 = all nodes the result equals the one-level search; a hand-worked
+// example; a numpy restatement.
+//
 // Parity pins (tests/test_oracle_pins.py): hand-worked 2-D and 4-D examples,
 // numpy brute force, decode-then-exact, lossless-PQ exhaustive search ==
 // exact kNN, bf16 rounding against a library conversion.  Nothing here is
@@ -147,17 +159,48 @@ struct Cand {
 };
 
 // Steps 1-4 for one query.
+struct Tree {
+    const void* level1;         // [n1][d], same storage type as the coarse centroids
+    const int32_t* child_offsets;  // [n1 + 1]
+    int n1, b1;
+};
+
+// Probe lists through a two-level coarse quantiser: the best b1 level-1 nodes by the coarse score
+// formula applied to the level-1 centroids, then the best nprobe of their children by the lists'
+// own coarse scores cs (ties: smaller node / smaller list number).  Fewer than nprobe children
+// among the chosen nodes leaves the tail of `probes` at -1.
+void tree_probes(const Index& ix, const Tree& tr, const float* q, const std::vector<double>& cs, int nprobe,
+                 std::vector<int>& probes) {
+    Index top = ix;
+    top.centroids = tr.level1;
+    top.nlist = tr.n1;
+    std::vector<double> s1;
+    coarse_scores(top, q, s1);
+    std::vector<int> nodes;
+    select_probes(top, s1, tr.b1, nodes);
+    std::vector<int> cand;
+    for (int node : nodes)
+        for (int l = tr.child_offsets[node]; l < tr.child_offsets[node + 1]; ++l) cand.push_back(l);
+    std::sort(cand.begin(), cand.end(), [&](int a, int b) { return better(ix.metric, cs[a], a, cs[b], b); });
+    probes.assign(nprobe, -1);
+    for (int p = 0; p < nprobe && p < int(cand.size()); ++p) probes[p] = cand[p];
+}
+
 void search_one(const Index& ix, const float* q, int nprobe, int k, int64_t* out_ids, float* out_dists,
-                int32_t* out_probes) {
+                int32_t* out_probes, const Tree* tree = nullptr) {
     std::vector<double> cs;
     coarse_scores(ix, q, cs);
     std::vector<int> probes;
-    select_probes(ix, cs, nprobe, probes);
+    if (tree)
+        tree_probes(ix, *tree, q, cs, nprobe, probes);
+    else
+        select_probes(ix, cs, nprobe, probes);
     std::vector<Cand> cands;
     std::vector<double> T;
     for (int p = 0; p < nprobe; ++p) {
         const int list = probes[p];
         if (out_probes) out_probes[p] = list;
+        if (list < 0) continue;  // two-level quantiser with fewer than nprobe children among the chosen nodes
         if (ix.offsets[list + 1] == ix.offsets[list]) continue;
         build_table(ix, q, list, T);
         const double bias = ix.metric == IP ? cs[list] : 0.0;
@@ -236,6 +279,43 @@ int oracle_ivfpq_search(const void* centroids, int coarse_bf16, const float* cod
     parallel_for(nq, nthreads, [&](int qi) {
         search_one(ix, queries + size_t(qi) * d, nprobe, k, out_ids + size_t(qi) * k, out_dists + size_t(qi) * k,
                    out_probes ? out_probes + size_t(qi) * nprobe : nullptr);
+    });
+    return 0;
+}
+
+// Coarse step through a two-level quantiser: best-first probe lists (-1 where the chosen nodes have too few
+// children) and their coarse scores.
+int oracle_coarse_tree(const void* centroids, int coarse_bf16, int d, int nlist, int metric, const void* level1,
+                       const int32_t* child_offsets, int n1, int b1, const float* queries, int nq, int nprobe,
+                       int32_t* out_lists, double* out_scores, int nthreads) {
+    if (d <= 0 || nlist <= 0 || nprobe <= 0 || nprobe > nlist || n1 <= 0 || b1 <= 0 || b1 > n1) return 1;
+    Index ix = make_index(centroids, coarse_bf16, nullptr, nullptr, nullptr, nullptr, 0, d, nlist, 1, metric);
+    Tree tr{level1, child_offsets, n1, b1};
+    parallel_for(nq, nthreads, [&](int qi) {
+        std::vector<double> cs;
+        coarse_scores(ix, queries + size_t(qi) * d, cs);
+        std::vector<int> probes;
+        tree_probes(ix, tr, queries + size_t(qi) * d, cs, nprobe, probes);
+        for (int p = 0; p < nprobe; ++p) {
+            out_lists[size_t(qi) * nprobe + p] = probes[p];
+            out_scores[size_t(qi) * nprobe + p] = probes[p] >= 0 ? cs[probes[p]] : 0.0;
+        }
+    });
+    return 0;
+}
+
+// Full IVF-PQ search whose probe lists come from the two-level quantiser.
+int oracle_ivfpq_search_tree(const void* centroids, int coarse_bf16, const float* codebooks, const uint8_t* codes,
+                             const int64_t* offsets, const int64_t* ids, int64_t N, int d, int nlist, int M, int metric,
+                             const void* level1, const int32_t* child_offsets, int n1, int b1, const float* queries,
+                             int nq, int nprobe, int k, int64_t* out_ids, float* out_dists, int32_t* out_probes,
+                             int nthreads) {
+    if (bad(N, d, nlist, M, metric) || nprobe <= 0 || nprobe > nlist || k <= 0 || n1 <= 0 || b1 <= 0 || b1 > n1) return 1;
+    Index ix = make_index(centroids, coarse_bf16, codebooks, codes, offsets, ids, N, d, nlist, M, metric);
+    Tree tr{level1, child_offsets, n1, b1};
+    parallel_for(nq, nthreads, [&](int qi) {
+        search_one(ix, queries + size_t(qi) * d, nprobe, k, out_ids + size_t(qi) * k, out_dists + size_t(qi) * k,
+                   out_probes ? out_probes + size_t(qi) * nprobe : nullptr, &tr);
     });
     return 0;
 }

@@ -288,9 +288,24 @@ def make_ivfpq_shards(S: int, N_per: int, d: int, nlist: int, M: int, nq: int, *
     return shards
 
 
+def make_coarse_tree(centroids: torch.Tensor, n1: int):
+    """A second quantiser level over existing coarse centroids: node i owns the consecutive lists
+    child_offsets[i] .. child_offsets[i+1]-1 (an even split of the list numbers) and its centroid is the mean of
+    theirs, stored in the centroids' dtype.  Returns (level1 [n1, d], child_offsets int32 [n1 + 1], CPU)."""
+    nlist = centroids.shape[0]
+    assert 1 <= n1 <= nlist
+    off = torch.tensor([(i * nlist) // n1 for i in range(n1 + 1)], dtype=torch.int32)
+    cen = centroids.float()
+    top = torch.stack([cen[int(off[i]):int(off[i + 1])].mean(0) for i in range(n1)])
+    return top.to(centroids.dtype).contiguous(), off
+
+
+TREE_SPREAD = 0.5  # std of a coarse centroid around its level-1 centre, when lists are drawn as a two-level hierarchy
+
+
 def make_ivfpq_hashed(N: int, d: int, nlist: int, M: int, nq: int, *, metric: str, seed: int = MASTER_SEED,
                       coarse_bf16: bool = False, device="cpu", materialise: bool = True,
-                      chunk: int = 1 << 22) -> IvfPqData:
+                      chunk: int = 1 << 22, tree_n1: Optional[int] = None) -> IvfPqData:
     """Index whose codes and ids are pure functions of (seed, position).
 
     Used for the shapes too large to encode from vectors: list lengths from
@@ -298,11 +313,20 @@ def make_ivfpq_hashed(N: int, d: int, nlist: int, M: int, nq: int, *, metric: st
     centroids ~ N(0,1), codewords ~ N(0, SIGMA^2); a query is a random
     centroid plus SIGMA * N(0,1).  With `materialise=False` only the small
     tensors are built (a host-side caller regenerates the lists it needs).
+
+    `tree_n1` draws the coarse centroids as a two-level hierarchy instead: tree_n1 level-1 centres
+    ~ N(0,1), every list's centroid = the centre of its node (lists are dealt to nodes in equal
+    consecutive runs) + TREE_SPREAD * N(0,1); extra["level1"] / extra["child_offsets"] then hold
+    the second quantiser level (level-1 centroid = mean of its children, in the centroids' dtype).
     """
     dev = torch.device(device)
     g = _generator(seed, dev)
     dsub = d // M
     centres = torch.randn((nlist, d), generator=g, device=dev, dtype=torch.float32)
+    if tree_n1:
+        top_centres = torch.randn((tree_n1, d), generator=g, device=dev, dtype=torch.float32)
+        node = (torch.arange(nlist, device=dev) * tree_n1) // nlist
+        centres = top_centres[node] + TREE_SPREAD * centres
     codebooks = SIGMA * torch.randn((M, 256, dsub), generator=g, device=dev, dtype=torch.float32)
     qc = torch.randint(0, nlist, (nq,), generator=g, device=dev)
     queries = centres[qc] + SIGMA * torch.randn((nq, d), generator=g, device=dev, dtype=torch.float32)
@@ -317,9 +341,12 @@ def make_ivfpq_hashed(N: int, d: int, nlist: int, M: int, nq: int, *, metric: st
             c = min(chunk, N - s)
             codes[s:s + c] = hash_codes(seed, s, c, M, dev)
             ids[s:s + c] = hash_ids(s, c, dev)
+    extra = {"query_component": qc.cpu()}
+    if tree_n1:
+        extra["level1"], extra["child_offsets"] = make_coarse_tree(centroids_q, tree_n1)
     return IvfPqData(N=N, d=d, nlist=nlist, M=M, metric=metric, centroids=centroids_q, codebooks=codebooks,
                      codes=codes, list_offsets=list_offsets, ids=ids, queries=queries, seed=seed, hash_coded=True,
-                     extra={"query_component": qc.cpu()})
+                     extra=extra)
 
 
 def make_flat(N: int, d: int, nq: int, *, seed: int = MASTER_SEED, device="cpu", chunk: int = 1 << 18):
@@ -365,7 +392,7 @@ def make_config(n: int, *, device="cpu", scale: float = 1.0, seed: int = MASTER_
     if c["kind"] == "hashed":
         return make_ivfpq_hashed(N, c["d"], c["nlist"], c["M"], c["nq"], metric=c["metric"], seed=seed,
                                  coarse_bf16=c["coarse_bf16"], device=device,
-                                 materialise=c.get("materialise", True))
+                                 materialise=c.get("materialise", True), tree_n1=c.get("tree_n1"))
     raise ValueError("config %d is not an IVF-PQ shape" % n)
 
 

@@ -375,3 +375,94 @@ def test_merge_results_invariants():
     # inner product: the same lists with the sign flipped rank the same way
     c = oracle.merge_results(ids, np.where(np.isinf(d), -np.inf, -d).astype(np.float32), k, "ip")
     assert np.array_equal(c[0], a[0])
+
+
+# ---- two-level coarse quantiser ------------------------------------------------------------------------------
+
+def _numpy_tree_probes(cen, top, off, b1, q, nprobe, metric):
+    """The definition again, in numpy: best b1 nodes, then the best nprobe of their children (ties: smaller index)."""
+    def score(rows):
+        rows = np.asarray(rows, np.float64)
+        return ((q[None, :] - rows) ** 2).sum(1) if metric == "l2" else rows @ q
+    s1 = score(top)
+    key1 = s1 if metric == "l2" else -s1
+    nodes = np.lexsort((np.arange(len(top)), key1))[:b1]
+    cand = np.concatenate([np.arange(off[n], off[n + 1]) for n in nodes])
+    s2 = score(cen[cand])
+    key2 = s2 if metric == "l2" else -s2
+    order = np.lexsort((cand, key2))[:nprobe]
+    out = np.full(nprobe, -1, np.int64)
+    out[:order.size] = cand[order]
+    return out
+
+
+def test_tree_coarse_matches_the_hand_worked_example():
+    g = json.load(open(os.path.join(GOLD, "handworked_tree.json")))
+    cen = np.array(g["centroids"], np.float32)
+    top = np.array(g["level1"], np.float32)
+    off = np.array(g["child_offsets"], np.int32)
+    for metric in ("l2", "ip"):
+        q = np.array([g[metric]["query"]], np.float32)
+        _, flat = oracle.coarse(cen, q, 4, metric)
+        assert sorted(flat[0].tolist()) == sorted(g[metric]["list_scores"])       # the per-list values themselves
+        for case in g[metric]["cases"]:
+            lists, scores = oracle.coarse_tree(cen, top, off, case["b1"], q, case["nprobe"], metric)
+            assert lists[0].tolist() == case["lists"], (metric, case)
+            for l, s in zip(lists[0], scores[0]):
+                if l >= 0:
+                    assert s == g[metric]["list_scores"][l]
+    lists, _ = oracle.coarse(cen, np.array([g["l2"]["query"]], np.float32), 2, "l2")
+    assert lists[0].tolist() == g["l2"]["flat_nprobe2"]                         # the tree with b1 = 1 differs from it
+
+
+@pytest.mark.parametrize("metric,bf16", [("l2", False), ("ip", False), ("l2", True), ("ip", True)])
+def test_tree_with_every_node_kept_is_the_one_level_search(metric, bf16):
+    data = synth.make_ivfpq(3000, 32, 48, 16, 9, metric=metric, seed=71, coarse_bf16=bf16)
+    top, off = synth.make_coarse_tree(data.centroids, 6)
+    hix = host_index(oracle, data)
+    top_h = top.view(torch.uint16).numpy() if bf16 else top.numpy()
+    q = data.queries.numpy()
+    want_l, want_s = oracle.coarse(hix.centroids, q, 7, metric, coarse_bf16=bf16)
+    got_l, got_s = oracle.coarse_tree(hix.centroids, top_h, off.numpy(), 6, q, 7, metric, coarse_bf16=bf16)
+    assert np.array_equal(want_l, got_l) and np.array_equal(want_s, got_s)
+    a = oracle.ivfpq_search(hix, q, 7, 12)
+    b = oracle.ivfpq_search_tree(hix, top_h, off.numpy(), 6, q, 7, 12)
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
+
+
+@pytest.mark.parametrize("metric", ["l2", "ip"])
+def test_tree_coarse_equals_its_numpy_restatement(metric):
+    data = synth.make_ivfpq_hashed(2000, 24, 60, 8, 11, metric=metric, seed=72, tree_n1=10)
+    cen = data.centroids.numpy()
+    top, off = data.extra["level1"].numpy(), data.extra["child_offsets"].numpy()
+    q = data.queries.numpy()
+    for b1, nprobe in ((1, 4), (3, 9), (10, 60), (2, 20)):
+        lists, _ = oracle.coarse_tree(cen, top, off, b1, q, nprobe, metric)
+        for i in range(q.shape[0]):
+            want = _numpy_tree_probes(cen.astype(np.float64), top, off, b1, q[i].astype(np.float64), nprobe, metric)
+            assert lists[i].tolist() == want.tolist(), (metric, b1, nprobe, i)
+    # narrowing the first level can only lose lists the one-level search would have probed, never invent new scores
+    flat_l, flat_s = oracle.coarse(cen, q, 9, metric)
+    tree_l, tree_s = oracle.coarse_tree(cen, top, off, 3, q, 9, metric)
+    sgn = 1.0 if metric == "l2" else -1.0
+    assert np.all(sgn * tree_s >= sgn * flat_s - 1e-12)
+
+
+def test_tree_search_scans_only_the_lists_the_tree_picks():
+    data = synth.make_ivfpq_hashed(4000, 32, 40, 16, 6, metric="l2", seed=73, tree_n1=8)
+    hix = host_index(oracle, data)
+    top, off = data.extra["level1"].numpy(), data.extra["child_offsets"].numpy()
+    q = data.queries.numpy()
+    ids, dists, probes = oracle.ivfpq_search_tree(hix, top, off, 2, q, 5, 10, want_probes=True)
+    want_probes, _ = oracle.coarse_tree(hix.centroids, top, off, 2, q, 5, "l2")
+    assert np.array_equal(probes, want_probes)
+    # the same answer as a one-level search over an index in which every other list is empty
+    for i in range(q.shape[0]):
+        keep = set(probes[i].tolist())
+        lens = np.diff(hix.offsets)
+        sel = np.concatenate([np.arange(hix.offsets[l], hix.offsets[l + 1]) for l in sorted(keep)])
+        new_off = np.zeros(hix.nlist + 1, np.int64)
+        new_off[1:] = np.cumsum([lens[l] if l in keep else 0 for l in range(hix.nlist)])
+        sub = oracle.Index(hix.centroids, hix.codebooks, hix.codes[sel], new_off, hix.ids[sel], "l2")
+        a = oracle.ivfpq_search(sub, q[i:i + 1], hix.nlist, 10)
+        assert np.array_equal(a[0][0], ids[i]) and np.array_equal(a[1][0], dists[i])
