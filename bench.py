@@ -454,16 +454,18 @@ def bench_coarse_hyper(args, dev):
     return res
 
 
-def bench_iter(args, dev):
-    """The iterative-retrieval latency shape: N = 1e8, d = 512, nlist = 16 384, M = 32; a stream of 256 batches of
-    1, 4 or 16 queries issued back to back on one stream, nprobe = 16, k = 20; per-batch latency from CUDA events
-    between the batches."""
+def _iter_stream(args, dev, tree):
+    """One measurement of the 256-batch stream; tree = (n1, b1) puts a second quantiser level above the coarse
+    centroids (the centroids are then drawn as a two-level hierarchy), None is the one-level index."""
     from paper_2503_14649_b200 import binding, synth
     c = synth.CONFIGS[4]
     nprobe, k = c["nprobe"], c["k"]
     sizes = synth.batch_size_stream(synth.MASTER_SEED, 256)
-    data = synth.make_config(4, device=dev, scale=args.scale, nq=sum(sizes))
+    over = {"tree_n1": tree[0]} if tree else {}
+    data = synth.make_config(4, device=dev, scale=args.scale, nq=sum(sizes), **over)
     ix = binding.rago_index_load(data.centroids, data.codebooks, data.codes, data.list_offsets.to(dev), data.ids, data.metric)
+    if tree:
+        ix.rago_index_set_coarse_tree(data.extra["level1"].to(dev), data.extra["child_offsets"].to(dev), tree[1])
     q = data.queries.contiguous()
     ws = torch.empty(ix.search_workspace_bytes(16, nprobe, k), dtype=torch.uint8, device=dev)
     out_i = torch.empty((16, k), dtype=torch.int64, device=dev)
@@ -496,26 +498,52 @@ def bench_iter(args, dev):
     t1 = time.time()
     clocks = sampler.stop(t0, t1)
     ix.rago_check(ws)
+    # stage split of a batch of one (events around every stage serialise the launches: shares, not a latency)
+    ix.rago_profile_enable(True)
+    st1 = []
+    for _ in range(20):
+        ix.rago_search(q[:1], nprobe, k, out_i[:1], out_d[:1], ws)
+        st1.append(ix.rago_profile_read())
+    ix.rago_profile_enable(False)
     ms = float(np.mean(tot))
     alll = np.concatenate([lat[1], lat[4], lat[16]])
-    res = {
-        "metric": METRIC, "value": sum(sizes) / (ms / 1e3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32", "data": "synthetic",
-        "config": {"workload": "Iterative-retrieval stream (configs[3]): N=%d d=%d nlist=%d M=%d, 256 batches of 1/4/16 "
-                   "queries back to back on one stream, nprobe=%d k=%d L2" % (data.N, c["d"], c["nlist"], c["M"], nprobe, k),
-                   "step": "one pass over the 256-batch stream (%d queries)" % sum(sizes), "scale": args.scale},
-        "clocks": clocks,
-        "latency_ms": {"p50": float(np.percentile(alll, 50)), "p99": float(np.percentile(alll, 99)),
-                       "by_batch_size": {str(nb): {"p50": float(np.percentile(v, 50)), "p99": float(np.percentile(v, 99))}
-                                         for nb, v in lat.items()},
-                       "note": "device time between consecutive batches' start events (launch-to-launch on a busy stream)"},
-        "roofline": {"bound": "latency", "kernel": "whole call", "achieved": None, "peak": None,
-                     "unit": None, "frac": None, "traffic": None}}
+    res = {"qps": sum(sizes) / (ms / 1e3), "ms_per_stream": ms, "clocks": clocks, "N": data.N, "queries": sum(sizes),
+           "latency_ms": {"p50": float(np.percentile(alll, 50)), "p99": float(np.percentile(alll, 99)),
+                          "by_batch_size": {str(nb): {"p50": float(np.percentile(v, 50)), "p99": float(np.percentile(v, 99))}
+                                            for nb, v in lat.items()},
+                          "note": "device time between consecutive batches' start events (launch-to-launch on a busy stream)"},
+           "stage_ms_batch_of_1": {kk: float(np.median([s_[kk] for s_ in st1])) for kk in st1[0]}}
     ix.close()
     del ix, data, ws, q
     _free()
     return res
+
+
+def bench_iter(args, dev):
+    """The iterative-retrieval latency shape: N = 1e8, d = 512, nlist = 16 384, M = 32; a stream of 256 batches of
+    1, 4 or 16 queries issued back to back on one stream, nprobe = 16, k = 20; per-batch latency from CUDA events
+    between the batches.  Measured twice: on the one-level index the shape names, and with a level of 128 nodes
+    above the coarse centroids (8 nodes kept), the paper's multi-level index in its smallest form."""
+    from paper_2503_14649_b200 import synth
+    c = synth.CONFIGS[4]
+    one = _iter_stream(args, dev, None)
+    two = _iter_stream(args, dev, (128, 8))
+    return {
+        "metric": METRIC, "value": one["qps"], "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": one["ms_per_stream"], "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "Iterative-retrieval stream (configs[3]): N=%d d=%d nlist=%d M=%d, 256 batches of 1/4/16 "
+                   "queries back to back on one stream, nprobe=%d k=%d L2" % (one["N"], c["d"], c["nlist"], c["M"],
+                                                                               c["nprobe"], c["k"]),
+                   "step": "one pass over the 256-batch stream (%d queries)" % one["queries"], "scale": args.scale},
+        "clocks": one["clocks"], "latency_ms": one["latency_ms"], "stage_ms_batch_of_1": one["stage_ms_batch_of_1"],
+        "two_level_coarse": {"n1": 128, "b1": 8, "value": two["qps"], "unit": UNIT, "ms_per_step": two["ms_per_stream"],
+                             "latency_ms": two["latency_ms"], "stage_ms_batch_of_1": two["stage_ms_batch_of_1"],
+                             "clocks": two["clocks"],
+                             "note": "same shape with hierarchical coarse centroids (synth tree_n1 = 128); results "
+                                     "follow the two-level definition, not the one-level one"},
+        "roofline": {"bound": "latency", "kernel": "whole call", "achieved": None, "peak": None,
+                     "unit": None, "frac": None, "traffic": None}}
 
 
 def bench_sharded(args, rank, world, local, dev):

@@ -106,6 +106,32 @@ rago_status rago_index_load_pq4(rago_index** out, const void* coarse_centroids, 
                                 const int64_t* ids, int64_t N, int32_t d, int32_t nlist, int32_t M4,
                                 rago_metric metric, void* cuda_stream);
 
+/*
+ * Put a second quantiser level above the coarse centroids, or remove it (n1 = 0).  The paper's index is a
+ * multi-level tree whose levels are scanned top-down, each level's best nodes deciding which nodes of the next
+ * are scored (Methodology: "Models and database", and the retrieval performance model: one scan operator per
+ * level).  With the level set, the coarse step of every search on this index scores the n1 level-1 centroids,
+ * keeps the best b1 nodes (same score as the coarse step: squared L2 distance or inner product, with the query
+ * rounded to bf16 for a RAGO_BF16 quantiser; ties to the smaller node number), and chooses the nprobe probe lists
+ * among the children of those nodes only.  Everything after the coarse step is unchanged.  The result is what
+ * the two-level definition gives, which differs from the one-level search whenever a good list hangs under a
+ * node that was not kept; b1 = n1 reproduces the one-level search.
+ *
+ *   level1_centroids  dev [n1][d], row-major, the index's coarse dtype, 16-byte aligned; borrowed until the
+ *                     level is removed or the index freed
+ *   child_offsets     dev [n1 + 1] int32, offsets[0] = 0, non-decreasing, offsets[n1] = nlist: node i owns the
+ *                     consecutive lists offsets[i] .. offsets[i + 1] - 1; borrowed likewise
+ *   n1, b1            1 <= b1 <= n1 <= nlist; b1 <= 64, n1 <= 4096, d a multiple of 4, d * 4 + n1 * 8 <= 48 KB,
+ *                     else RAGO_EUNSUPPORTED
+ *
+ * A search whose nprobe exceeds the number of lists the b1 smallest nodes own is refused with RAGO_EINVAL
+ * (the b1 kept nodes might not have nprobe children).  Workspace sizes change with the level: ask for them
+ * after this call.  Synchronises cuda_stream (it reads child_offsets to validate them).
+ * rago_search_probes_noalloc is not available while a level is set.
+ */
+rago_status rago_index_set_coarse_tree(rago_index* index, const void* level1_centroids, const int32_t* child_offsets,
+                                       int32_t n1, int32_t b1, void* cuda_stream);
+
 /* Release the handle and the arrays the library allocated for it (never the borrowed ones).
  * Synchronises the device first.  NULL is accepted. */
 rago_status rago_index_free(rago_index* index);

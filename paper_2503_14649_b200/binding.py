@@ -24,7 +24,7 @@ RAGO_F32, RAGO_BF16 = 0, 1
 NUM_STAGES = 5
 STAGE_NAMES = ("coarse_scores", "probe_select", "plan", "table_scan", "merge")
 
-EXPORTS = ("rago_index_load", "rago_index_load_pq4", "rago_index_free", "rago_search_workspace_bytes", "rago_search",
+EXPORTS = ("rago_index_load", "rago_index_load_pq4", "rago_index_set_coarse_tree", "rago_index_free", "rago_search_workspace_bytes", "rago_search",
            "rago_search_probes", "rago_search_probes_noalloc", "rago_search_host", "rago_host_staging_bytes", "rago_flat_search",
            "rago_flat_workspace_bytes", "rago_check", "rago_set_coarse_mode", "rago_profile_enable", "rago_profile_read",
            "rago_merge_results", "rago_selftest_wait_timeout", "rago_kernel_launches", "rago_last_error")
@@ -48,6 +48,7 @@ def lib() -> ctypes.CDLL:
         L.rago_index_load.argtypes = [ctypes.POINTER(vp), vp, ctypes.c_int, vp, vp, vp, vp, i64, i32, i32, i32,
                                       ctypes.c_int, vp]
         L.rago_index_load_pq4.argtypes = L.rago_index_load.argtypes
+        L.rago_index_set_coarse_tree.argtypes = [vp, vp, vp, i32, i32, vp]
         L.rago_index_free.argtypes = [vp]
         L.rago_search_workspace_bytes.argtypes = [vp, i32, i32, i32, ctypes.POINTER(sz)]
         L.rago_host_staging_bytes.argtypes = [vp, i32, i32, ctypes.POINTER(sz)]
@@ -188,6 +189,17 @@ class Index:
     def rago_set_coarse_mode(self, mode: int):
         _check(lib().rago_set_coarse_mode(self._h, int(mode)))
         self._ws = None  # workspace sizes depend on the mode
+
+    def rago_index_set_coarse_tree(self, level1: Optional[torch.Tensor], child_offsets: Optional[torch.Tensor], b1: int = 0):
+        """Set (or, with level1 = None, remove) the level above the coarse centroids; tensors are borrowed."""
+        if level1 is None:
+            _check(lib().rago_index_set_coarse_tree(self._h, None, None, 0, 0, _stream()))
+            self._tree = None
+        else:
+            _check(lib().rago_index_set_coarse_tree(self._h, _ptr(level1), _ptr(child_offsets), level1.shape[0], int(b1),
+                                                    _stream()))
+            self._tree = (level1, child_offsets)
+        self._ws = None  # workspace sizes depend on it
 
     def rago_profile_enable(self, enable: bool = True):
         _check(lib().rago_profile_enable(self._h, int(enable)))

@@ -1,4 +1,5 @@
 // C ABI of the retrieval library: argument checks, workspace layout, stage launches.
+#include <algorithm>
 #include <atomic>
 #include <cstdarg>
 #include <cstdio>
@@ -47,6 +48,7 @@ struct Layout {
     int pilot_cols;                 // 0: no pilot pass
     size_t nslots;
     int tc, tc_mode, tc_cap, tc_mg, tc_nsplit;  // coarse plan for this (nq, nprobe)
+    int tree_S, tree_cap;           // two-level coarse quantiser: CTAs per query and candidate slots per CTA (0: not used)
 };
 
 // Which coarse kernel a batch takes.  The tensor-core kernel pays off once a batch fills a good part of
@@ -71,7 +73,14 @@ static Layout make_layout(const IndexImpl* ix, int nq, int nprobe, int k) {
     L.probe_list = take(npairs * 4);
     L.probe_term = take(npairs * 4);
     L.probe_bias = take(npairs * 4);
-    L.tc = use_tensor_cores(ix, nq) ? 1 : 0;
+    L.tree_S = L.tree_cap = 0;
+    if (ix->tree_n1) {  // a few CTAs per query when the batch alone cannot fill the GPU
+        int S = (ix->num_sms + nq - 1) / (nq > 0 ? nq : 1);  // every CTA of a query repeats the first level: not too many
+        S = S < 1 ? 1 : (S > 32 ? 32 : S);
+        L.tree_S = S;
+        L.tree_cap = (ix->tree_max_cand + S - 1) / S;
+    }
+    L.tc = !ix->tree_n1 && use_tensor_cores(ix, nq) ? 1 : 0;
     L.tc_mode = 1; L.tc_cap = 0; L.tc_mg = 1; L.tc_nsplit = 1;
     L.qparts = L.cand = L.cand_cnt = L.pilot_scores = L.row_tau = 0;
     L.pilot_cols = 0;
@@ -95,7 +104,11 @@ static Layout make_layout(const IndexImpl* ix, int nq, int nprobe, int k) {
             }
         }
     }
-    L.scores = take((!L.tc || L.tc_mode == 1) ? (size_t)nq * ix->nlist * 4 : 0);
+    if (L.tree_S) {
+        L.cand = take((size_t)nq * L.tree_S * L.tree_cap * 8);
+        L.cand_cnt = take((size_t)nq * L.tree_S * 4);
+    }
+    L.scores = take(!L.tree_S && (!L.tc || L.tc_mode == 1) ? (size_t)nq * ix->nlist * 4 : 0);
     L.pair_tiles = take(npairs * 4);
     L.work_prefix = take((npairs + 1) * 8);
     L.qthresh = take((size_t)nq * 8);
@@ -129,6 +142,9 @@ static rago_status check_search_args(const IndexImpl* ix, int nq, int nprobe, in
     if (k < 1) return fail(RAGO_EINVAL, "k = %d must be at least 1", k);
     if (k > MAX_K) return fail(RAGO_EUNSUPPORTED, "k = %d exceeds %d", k, MAX_K);
     if ((long long)nq * nprobe > 0x7fffffffLL - 4096) return fail(RAGO_EUNSUPPORTED, "nq * nprobe too large");
+    if (ix->tree_n1 && nprobe > ix->tree_min_cand)
+        return fail(RAGO_EINVAL, "nprobe = %d, but %d level-1 nodes can have as few as %d lists between them", nprobe,
+                    ix->tree_b1, ix->tree_min_cand);
     return RAGO_OK;
 }
 
@@ -145,7 +161,15 @@ static rago_status run_coarse(const IndexImpl* ix, const float* queries, int nq,
     float* probe_bias = reinterpret_cast<float*>(ws + L.probe_bias);
     float* scores = reinterpret_cast<float*>(ws + L.scores);
     record(mix, 0, s);
-    if (L.tc) {
+    if (L.tree_S) {
+        unsigned long long* cand = reinterpret_cast<unsigned long long*>(ws + L.cand);
+        int32_t* cand_cnt = reinterpret_cast<int32_t*>(ws + L.cand_cnt);
+        e = launch_tree_candidates(ix, queries, nq, L.tree_S, L.tree_cap, cand, cand_cnt, s);
+        if (e != cudaSuccess) return cuda_fail(e, "two-level coarse kernel");
+        record(mix, 1, s);
+        e = launch_select_probes_cand(ix, queries, cand, cand_cnt, 0u, L.tree_S, L.tree_cap, nq, nprobe, probe_list,
+                                      probe_term, probe_bias, s);
+    } else if (L.tc) {
         // queries -> stacked bf16 parts, then the tensor-core kernel with the selection fused in
         const int parts = ix->cparts_n;
         e = launch_split_bf16(queries, (size_t)nq * ix->d, parts, ws + L.qparts, s);
@@ -489,6 +513,47 @@ rago_status rago_check(void* workspace, void* cuda_stream) {
     if (w == ERR_WAIT_TIMEOUT) return fail(RAGO_ETIMEOUT, "a bounded device-side wait expired");
     if (w == ERR_SMEM_LAYOUT) return fail(RAGO_ECUDA, "the scan kernel's shared-memory plan does not fit this device");
     if (w != ERR_NONE) return fail(RAGO_ECUDA, "device error word = %u", w);
+    return RAGO_OK;
+}
+
+rago_status rago_index_set_coarse_tree(rago_index* index, const void* level1_centroids, const int32_t* child_offsets,
+                                       int32_t n1, int32_t b1, void* cuda_stream) {
+    if (!index) return fail(RAGO_EINVAL, "index is null");
+    IndexImpl* ix = reinterpret_cast<IndexImpl*>(index);
+    rago_status st = check_device(ix);
+    if (st != RAGO_OK) return st;
+    if (n1 == 0) {  // back to the one-level quantiser
+        ix->tree_n1 = ix->tree_b1 = 0;
+        ix->tree_level1 = nullptr; ix->tree_child_offsets = nullptr;
+        return RAGO_OK;
+    }
+    if (!level1_centroids || !child_offsets) return fail(RAGO_EINVAL, "null pointer");
+    if (n1 < 1 || n1 > ix->nlist) return fail(RAGO_EINVAL, "n1 = %d outside [1, nlist = %d]", n1, ix->nlist);
+    if (b1 < 1 || b1 > n1) return fail(RAGO_EINVAL, "b1 = %d outside [1, n1 = %d]", b1, n1);
+    if (n1 > TREE_LIMIT_N1 || b1 > TREE_LIMIT_B1)
+        return fail(RAGO_EUNSUPPORTED, "n1 = %d / b1 = %d exceed %d / %d", n1, b1, TREE_LIMIT_N1, TREE_LIMIT_B1);
+    if (ix->d % 4 != 0) return fail(RAGO_EUNSUPPORTED, "d = %d must be a multiple of 4 for the two-level quantiser", ix->d);
+    if (!aligned(level1_centroids, 16) || !aligned(child_offsets, 4)) return fail(RAGO_EALIGN, "level-1 centroids need 16-byte alignment");
+    if ((size_t)ix->d * 4 + (size_t)n1 * 8 > 48 * 1024)
+        return fail(RAGO_EUNSUPPORTED, "d = %d with n1 = %d does not fit the kernel's shared memory", ix->d, n1);
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    std::vector<int32_t> off((size_t)n1 + 1);
+    cudaError_t e = cudaMemcpyAsync(off.data(), child_offsets, off.size() * 4, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return cuda_fail(e, "reading child_offsets");
+    if (off[0] != 0 || off[n1] != ix->nlist) return fail(RAGO_EINVAL, "child_offsets must start at 0 and end at nlist");
+    std::vector<int> cnt(n1);
+    for (int i = 0; i < n1; ++i) {
+        if (off[i + 1] < off[i]) return fail(RAGO_EINVAL, "child_offsets decrease at node %d", i);
+        cnt[i] = off[i + 1] - off[i];
+    }
+    std::sort(cnt.begin(), cnt.end());
+    long long mn = 0, mx = 0;
+    for (int i = 0; i < b1; ++i) { mn += cnt[i]; mx += cnt[n1 - 1 - i]; }
+    ix->tree_level1 = level1_centroids;
+    ix->tree_child_offsets = child_offsets;
+    ix->tree_n1 = n1; ix->tree_b1 = b1;
+    ix->tree_min_cand = (int)mn; ix->tree_max_cand = (int)mx;
     return RAGO_OK;
 }
 

@@ -207,6 +207,172 @@ cudaError_t launch_coarse_scores(const IndexImpl* ix, const float* queries, int 
     return cudaGetLastError();
 }
 
+// ---- two-level coarse quantiser: candidates of a query through the first level -------------------------------
+// The paper's index is a multi-level tree whose levels are scanned top-down (Methodology, "Models and database"
+// and the retrieval performance model).  With one level above the coarse centroids: score the n1 level-1
+// centroids, keep the best b1 nodes, and only the coarse centroids that are their children become candidates for
+// the nprobe selection.  Children of node i are the consecutive lists child_offsets[i] .. child_offsets[i+1]-1.
+//
+// grid (S, nq): the S CTAs of a query all score the whole first level (n1 rows, L2-resident) and reach the same
+// b1 nodes; then CTA s scores its share of the candidate slots (the children of the chosen nodes, in node-rank
+// order) and leaves them as raw candidate entries {list, score bits} in cand[q][s][cap] with count cand_cnt[q][s],
+// the format select_probes_kernel reads.  Level-1 scores use the direct form (sum (q-c)^2 or <q,c>), so that
+// near-ties between nodes are decided as the definition decides them up to fp32 rounding; candidate scores are
+// the ranking form of the one-level path (||c||^2 - 2<q,c> or -<q,c>).
+constexpr int TREE_THREADS = 512;
+constexpr int TREE_RPW = 4;        // rows a warp scores at a time (independent loads in flight)
+constexpr int TREE_MAX_B1 = 64;
+
+// Scores of TREE_RPW rows against the query in shared memory, by one warp: DIRECT: sum (q-c)^2 / <q,c> by metric;
+// else <q,c> only.  Rows past `nrows` repeat the last valid one.  out[u] valid in every lane.
+template <bool BF16, bool DIRECT>
+__device__ __forceinline__ void warp_score_rows(const float* qs, const void* C, const int (&row)[TREE_RPW], int d,
+                                                int metric, int lane, float (&out)[TREE_RPW]) {
+    float acc[TREE_RPW];
+#pragma unroll
+    for (int u = 0; u < TREE_RPW; ++u) acc[u] = 0.f;
+#pragma unroll 4
+    for (int j0 = lane * 4; j0 < d; j0 += 128) {  // unrolled: the loads of four steps are in flight together
+        float4 cv[TREE_RPW];
+#pragma unroll
+        for (int u = 0; u < TREE_RPW; ++u) {
+            if (BF16) {
+                const uint2 raw = *reinterpret_cast<const uint2*>(static_cast<const __nv_bfloat16*>(C) + (size_t)row[u] * d + j0);
+                cv[u].x = __uint_as_float(raw.x << 16); cv[u].y = __uint_as_float(raw.x & 0xFFFF0000u);
+                cv[u].z = __uint_as_float(raw.y << 16); cv[u].w = __uint_as_float(raw.y & 0xFFFF0000u);
+            } else {
+                cv[u] = *reinterpret_cast<const float4*>(static_cast<const float*>(C) + (size_t)row[u] * d + j0);
+            }
+        }
+        const float4 qv = *reinterpret_cast<const float4*>(qs + j0);
+#pragma unroll
+        for (int u = 0; u < TREE_RPW; ++u) {
+            if (DIRECT && metric == RAGO_L2) {
+                const float t0 = qv.x - cv[u].x, t1 = qv.y - cv[u].y, t2 = qv.z - cv[u].z, t3 = qv.w - cv[u].w;
+                acc[u] = fmaf(t0, t0, fmaf(t1, t1, fmaf(t2, t2, fmaf(t3, t3, acc[u]))));
+            } else {
+                acc[u] = fmaf(qv.x, cv[u].x, fmaf(qv.y, cv[u].y, fmaf(qv.z, cv[u].z, fmaf(qv.w, cv[u].w, acc[u]))));
+            }
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < TREE_RPW; ++u) {
+        for (int o = 16; o; o >>= 1) acc[u] += __shfl_xor_sync(0xffffffffu, acc[u], o);
+        out[u] = acc[u];
+    }
+}
+
+template <bool BF16>
+__global__ void __launch_bounds__(TREE_THREADS) tree_candidates_kernel(
+    const float* __restrict__ Q, const void* __restrict__ C1, const int32_t* __restrict__ child_offsets, int n1, int b1,
+    const void* __restrict__ C, const float* __restrict__ cnorm, int d, int metric, int cap,
+    unsigned long long* __restrict__ cand, int32_t* __restrict__ cand_cnt) {
+    extern __shared__ __align__(16) float tree_smem[];  // [d] query, [n1] level-1 keys as two words each
+    float* qs = tree_smem;
+    unsigned long long* k1 = reinterpret_cast<unsigned long long*>(tree_smem + ((d + 3) & ~3));  // (d * 4) % 16 == 0
+    __shared__ int sel_node[TREE_MAX_B1];     // chosen nodes, best first
+    __shared__ int sel_first[TREE_MAX_B1];    // first list of each chosen node
+    __shared__ int sel_pre[TREE_MAX_B1 + 1];  // candidate slots before each chosen node
+    const int q = blockIdx.y, s = blockIdx.x, S = gridDim.x;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    constexpr int NW = TREE_THREADS / 32;
+    grid_dependency_wait();
+    grid_dependents_may_launch();
+    for (int i = tid; i < d; i += TREE_THREADS) qs[i] = BF16 ? round_bf16(Q[(size_t)q * d + i]) : Q[(size_t)q * d + i];
+    __syncthreads();
+    // first level: every node, direct form
+    for (int r0 = warp * TREE_RPW; r0 < n1; r0 += NW * TREE_RPW) {
+        int row[TREE_RPW];
+#pragma unroll
+        for (int u = 0; u < TREE_RPW; ++u) row[u] = r0 + u < n1 ? r0 + u : n1 - 1;
+        float sc[TREE_RPW];
+        warp_score_rows<BF16, true>(qs, C1, row, d, metric, lane, sc);
+        if (lane == 0) {
+#pragma unroll
+            for (int u = 0; u < TREE_RPW; ++u)
+                if (r0 + u < n1) k1[r0 + u] = make_key(metric == RAGO_L2 ? sc[u] : -sc[u], (uint32_t)(r0 + u));
+        }
+    }
+    __syncthreads();
+    // the b1 best nodes, best first (ties: smaller node), by warp 0: b1 rounds of a minimum over the keys
+    if (warp == 0) {
+        unsigned long long last = 0ull;
+        bool first = true;
+        for (int r = 0; r < b1; ++r) {
+            unsigned long long best = KEY_MAX;
+            for (int i = lane; i < n1; i += 32) {
+                const unsigned long long k = k1[i];
+                if ((first || k > last) && k < best) best = k;  // keys are distinct: the node number is part of them
+            }
+            for (int o = 16; o; o >>= 1) {
+                const unsigned long long other = shfl_xor_u64(best, o);
+                best = other < best ? other : best;
+            }
+            last = best;
+            first = false;
+            if (lane == 0) sel_node[r] = (int)(best & 0xFFFFFFFFull);
+        }
+        __syncwarp();
+        // the chosen nodes' child ranges: all loads at once, then a running sum (b1 <= 64: two values per lane)
+        int cnt0 = 0, cnt1 = 0;
+        if (lane < b1) { const int n = sel_node[lane]; const int f = child_offsets[n]; sel_first[lane] = f; cnt0 = child_offsets[n + 1] - f; }
+        if (lane + 32 < b1) { const int n = sel_node[lane + 32]; const int f = child_offsets[n]; sel_first[lane + 32] = f; cnt1 = child_offsets[n + 1] - f; }
+        int inc0 = cnt0, inc1 = cnt1;
+        for (int o = 1; o < 32; o <<= 1) {
+            const int y0 = __shfl_up_sync(0xffffffffu, inc0, o), y1 = __shfl_up_sync(0xffffffffu, inc1, o);
+            if (lane >= o) { inc0 += y0; inc1 += y1; }
+        }
+        const int tot0 = __shfl_sync(0xffffffffu, inc0, 31);
+        if (lane < b1) sel_pre[lane] = inc0 - cnt0;
+        if (lane + 32 < b1) sel_pre[lane + 32] = tot0 + inc1 - cnt1;
+        if (lane == 31) sel_pre[b1] = tot0 + inc1;
+    }
+    __syncthreads();
+    // second level: this CTA's share of the candidate slots
+    const int total = sel_pre[b1];
+    const int c_begin = s * cap < total ? s * cap : total;
+    const int c_end = (s + 1) * cap < total ? (s + 1) * cap : total;
+    unsigned long long* out = cand + ((size_t)q * S + s) * cap;
+    auto list_of = [&](int slot) {
+        int r = 0;
+        while (r + 1 < b1 && sel_pre[r + 1] <= slot) ++r;
+        return sel_first[r] + (slot - sel_pre[r]);
+    };
+    for (int c0 = c_begin + warp * TREE_RPW; c0 < c_end; c0 += NW * TREE_RPW) {
+        int row[TREE_RPW];
+#pragma unroll
+        for (int u = 0; u < TREE_RPW; ++u) row[u] = list_of(c0 + u < c_end ? c0 + u : c_end - 1);
+        float dot[TREE_RPW];
+        warp_score_rows<BF16, false>(qs, C, row, d, metric, lane, dot);
+        if (lane == 0) {
+#pragma unroll
+            for (int u = 0; u < TREE_RPW; ++u) {
+                if (c0 + u < c_end) {
+                    const float sc = metric == RAGO_L2 ? fmaf(-2.f, dot[u], __ldg(cnorm + row[u])) : -dot[u];
+                    out[c0 + u - c_begin] = ((unsigned long long)__float_as_uint(sc) << 32) | (uint32_t)row[u];
+                }
+            }
+        }
+    }
+    if (tid == 0) cand_cnt[(size_t)q * S + s] = c_end - c_begin;
+}
+
+cudaError_t launch_tree_candidates(const IndexImpl* ix, const float* queries, int nq, int S, int cap,
+                                   unsigned long long* cand, int32_t* cand_cnt, cudaStream_t s) {
+    const size_t smem = (size_t)((ix->d + 3) & ~3) * 4 + (size_t)ix->tree_n1 * 8;
+    if (smem > 48 * 1024) return cudaErrorInvalidValue;
+    if (ix->coarse_bf16)
+        launch_overlapped(tree_candidates_kernel<true>, dim3(S, nq), dim3(TREE_THREADS), smem, s, queries, ix->tree_level1,
+                          ix->tree_child_offsets, ix->tree_n1, ix->tree_b1, ix->centroids, ix->cnorm, ix->d, ix->metric,
+                          cap, cand, cand_cnt);
+    else
+        launch_overlapped(tree_candidates_kernel<false>, dim3(S, nq), dim3(TREE_THREADS), smem, s, queries, ix->tree_level1,
+                          ix->tree_child_offsets, ix->tree_n1, ix->tree_b1, ix->centroids, ix->cnorm, ix->d, ix->metric,
+                          cap, cand, cand_cnt);
+    count_launch();
+    return cudaGetLastError();
+}
+
 // ---- per-query selection of the nprobe best lists ----------------------------------------------
 constexpr int SEL_MAX_SPLIT = 512;  // candidate lists per query the kernel can index (one per column range of the GEMM)
 

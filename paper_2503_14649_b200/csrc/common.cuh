@@ -54,6 +54,12 @@ struct IndexImpl {
     alignas(64) unsigned char tmap_b[128];  // CUtensorMap of the stacked centroid parts
     alignas(64) unsigned char tmap_b_pilot[128];  // the same, every pilot_stride-th centroid
     int pilot_stride;  // 0: no pilot pass for this index
+    // optional first quantiser level (borrowed; tree_n1 = 0: none).  Node i owns lists child_offsets[i] .. [i+1]-1.
+    const void* tree_level1;            // [tree_n1][d], the coarse dtype
+    const int32_t* tree_child_offsets;  // [tree_n1 + 1]
+    int tree_n1, tree_b1;
+    int tree_max_cand;                  // most candidates b1 nodes can have (sum of the b1 largest child counts)
+    int tree_min_cand;                  // fewest (sum of the b1 smallest): nprobe must not exceed it
     int device, num_sms;
     ScanPlan plan;
     int profile;
@@ -202,6 +208,9 @@ cudaError_t launch_centroid_norms(const void* centroids, int bf16, int nlist, in
 cudaError_t launch_coarse_scores(const IndexImpl* ix, const float* queries, int nq, float* scores, cudaStream_t s);
 cudaError_t launch_select_probes(const IndexImpl* ix, const float* queries, const float* scores, int nq, int nprobe,
                                  int32_t* probe_list, float* probe_term, float* probe_bias, cudaStream_t s);
+cudaError_t launch_tree_candidates(const IndexImpl* ix, const float* queries, int nq, int S, int cap,
+                                   unsigned long long* cand, int32_t* cand_cnt, cudaStream_t s);
+constexpr int TREE_LIMIT_B1 = 64, TREE_LIMIT_N1 = 4096;
 cudaError_t launch_select_probes_cand(const IndexImpl* ix, const float* queries, const unsigned long long* cand,
                                       const int32_t* cand_cnt, uint32_t cand_sign, int nsplit, int cap, int nq, int nprobe,
                                       int32_t* probe_list, float* probe_term, float* probe_bias, cudaStream_t s);

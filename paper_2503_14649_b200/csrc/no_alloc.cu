@@ -57,6 +57,7 @@ extern "C" rago_status rago_search_probes_noalloc(const rago_index* index, const
         return RAGO_EINVAL;
     }
     if (nprobe > MAX_K) { set_error("nprobe = %d exceeds %d", nprobe, MAX_K); return RAGO_EUNSUPPORTED; }
+    if (ix->tree_n1) { set_error("this entry point scores every list: not available while a two-level quantiser is set"); return RAGO_EUNSUPPORTED; }
     if (nq == 0) return RAGO_OK;
     if (!queries || !out_lists || !out_coarse) { set_error("null pointer"); return RAGO_EINVAL; }
     int dev = -1;

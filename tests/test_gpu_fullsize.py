@@ -145,6 +145,44 @@ def test_iterative_stream_full_size_sampled():
     _free()
 
 
+def test_iterative_stream_with_two_level_quantiser_full_size_sampled():
+    """The iterative-retrieval shape (1e8 vectors, 16 384 lists) with a level of 128 nodes above the coarse
+    centroids, 8 nodes kept: 64 single-query searches and 8 batches of 16 against the oracle's two-level search."""
+    _need_gb(12)
+    c = synth.CONFIGS[4]
+    data = synth.make_config(4, device="cuda", nq=192, tree_n1=128)
+    ix = binding.rago_index_load(data.centroids, data.codebooks, data.codes, data.list_offsets.cuda(), data.ids,
+                                 data.metric)
+    top, off = data.extra["level1"].cuda(), data.extra["child_offsets"].cuda()
+    ix.rago_index_set_coarse_tree(top, off, 8)
+    qd = data.queries.contiguous()
+    ws = torch.empty(ix.search_workspace_bytes(16, c["nprobe"], c["k"]), dtype=torch.uint8, device="cuda")
+    outs = []
+    batches = [(i, 1) for i in range(64)] + [(64 + 16 * j, 16) for j in range(8)]
+    for p0, nb in batches:
+        oi = torch.empty((nb, c["k"]), dtype=torch.int64, device="cuda")
+        od = torch.empty((nb, c["k"]), dtype=torch.float32, device="cuda")
+        ix.rago_search(qd[p0:p0 + nb], c["nprobe"], c["k"], oi, od, ws)
+        outs.append((oi, od))
+    torch.cuda.synchronize()
+    ix.rago_check(ws)
+    ix.close()
+    qh = data.queries.cpu().numpy()
+    top_h, off_h = data.extra["level1"].cpu().numpy(), data.extra["child_offsets"].cpu().numpy()
+    want_lists, _ = oracle.coarse_tree(data.centroids.cpu().numpy(), top_h, off_h, 8, qh, c["nprobe"], data.metric,
+                                       nthreads=oracle.default_threads())
+    hix = compact_hashed_subindex(oracle, data, np.unique(want_lists))
+    ri, rd = oracle.ivfpq_search_tree(hix, top_h, off_h, 8, qh, c["nprobe"], c["k"], nthreads=oracle.default_threads())
+    rs = IvfPqRescorer(oracle, hix)
+    for (p0, nb), (oi, od) in zip(batches, outs):
+        gi, gd = oi.cpu().numpy(), od.cpu().numpy()
+        for i in range(nb):
+            problems = match_results(gi[i], gd[i], ri[p0 + i], rd[p0 + i], rel=REL, rescore=rs.for_query(qh[p0 + i]))
+            assert not problems, ("query", p0 + i, problems[:4])
+    del data, ix, qd, outs, ws
+    _free()
+
+
 def test_flat_full_size_against_the_whole_database():
     """Flat search at 10 M x 1024 bf16: 16 of the 256 queries scored by the oracle against every row.  The database
     goes to the host one chunk at a time; the oracle's best k of every chunk are merged on the host (best first, ties
