@@ -537,21 +537,78 @@ __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
         ++round;
     }
     const uint32_t T = (uint32_t)hi;
-    // collect the items at or below the cut (a tie group larger than the buffer is cut arbitrarily)
+    // A tie group at the cut that would not fit the buffer (thousands of lists with bit-identical scores): which
+    // of the tied items are kept must not depend on the order in which warps reach the buffer, and no item
+    // below the cut may lose its place to a tied one.  The cut is then refined on the payload (list number) among
+    // the items that score exactly T, by the same counting bisection: items below T are all kept, tied ones up to
+    // payload P, so that at most nsel + slack are collected and they include the nsel smallest keys.
+    uint32_t P = 0xFFFFFFFFu;
+    if (c_hi > (uint32_t)TOPK_CAP) {  // uniform
+        auto payload_of = [&](int l, int j) -> uint32_t {
+            (void)j;
+            if constexpr (FROM_SCORES) return (uint32_t)l;
+            else return (uint32_t)(item(l) & 0xFFFFFFFFull);
+        };
+        auto count_cta = [&](uint32_t c) -> uint32_t {  // sum of c over the CTA, same value in every thread
+            c = __reduce_add_sync(0xffffffffu, c);
+            const int slot = round % 3;
+            if (lane == 0 && c) atomicAdd(&s_round[slot], c);
+            if (tid == 0) s_round[(slot + 1) % 3] = 0u;
+            __syncthreads();
+            ++round;
+            return s_round[slot];
+        };
+        uint32_t less = 0;
+        if (in_regs) {
+#pragma unroll
+            for (int j = 0; j < SEL_REG; ++j) less += mine[j] < T ? 1u : 0u;
+        } else {
+            for (int l = tid; l < nitems; l += SEL_THREADS) {
+                const unsigned long long k = item(l);
+                less += (k != KEY_MAX && (uint32_t)(k >> 32) < T) ? 1u : 0u;
+            }
+        }
+        less = count_cta(less);
+        const uint32_t need = (uint32_t)nsel - less;  // >= 1: fewer than nsel items lie below T
+        long long plo = -1, phi = 0xFFFFFFFFll;       // #(tied, payload <= plo) < need <= #(tied, payload <= phi)
+        uint32_t pc_hi = c_hi - less;
+        while (phi - plo > 1 && pc_hi > need + (uint32_t)slack) {  // uniform
+            const uint32_t mid = (uint32_t)(plo + (phi - plo) / 2);
+            uint32_t c = 0;
+            if (in_regs) {
+#pragma unroll
+                for (int j = 0; j < SEL_REG; ++j) {
+                    const int l = tid + j * SEL_THREADS;
+                    if (mine[j] == T && l < nitems && payload_of(l, j) <= mid) ++c;
+                }
+            } else {
+                for (int l = tid; l < nitems; l += SEL_THREADS) {
+                    const unsigned long long k = item(l);
+                    if (k != KEY_MAX && (uint32_t)(k >> 32) == T && (uint32_t)k <= mid) ++c;
+                }
+            }
+            c = count_cta(c);
+            if (c < need) plo = mid; else { phi = mid; pc_hi = c; }
+        }
+        P = (uint32_t)phi;
+    }
+    // collect the items below the cut, and those at the cut up to payload P
     if (in_regs) {
 #pragma unroll
         for (int j = 0; j < SEL_REG; ++j) {
-            const bool take = mine[j] != 0xFFFFFFFFu && mine[j] <= T;
+            bool take = mine[j] != 0xFFFFFFFFu && mine[j] <= T;
             unsigned long long key = KEY_MAX;
             if (FROM_SCORES) key = ((unsigned long long)mine[j] << 32) | (uint32_t)(tid + j * SEL_THREADS);
             else if (take) key = item(tid + j * SEL_THREADS);
+            if (take && mine[j] == T && (uint32_t)key > P) take = false;
             warp_push(keys, &cnt, take, key);
         }
     } else {
         for (int l0 = 0; l0 < nitems; l0 += SEL_THREADS) {
             const int l = l0 + tid;
             const unsigned long long k = l < nitems ? item(l) : KEY_MAX;
-            warp_push(keys, &cnt, k != KEY_MAX && (uint32_t)(k >> 32) <= T, k);
+            const uint32_t o = (uint32_t)(k >> 32);
+            warp_push(keys, &cnt, k != KEY_MAX && (o < T || (o == T && (uint32_t)k <= P)), k);
         }
     }
     __syncthreads();

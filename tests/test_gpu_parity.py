@@ -322,3 +322,35 @@ def test_near_duplicate_queries_get_relatively_accurate_l2_distances():
     gi, gd = _compare(data, 8, 10)
     assert np.all(gd[:, 0] < 1e-3) and np.all(gd[:, 0] > 0)           # the near-duplicate itself, far below the terms
     assert np.array_equal(gi[:, 0], data.ids.numpy()[rows])
+
+
+@pytest.mark.parametrize("mode", [1, 2])
+def test_thousands_of_identical_centroids_do_not_displace_a_closer_list(mode):
+    """2500 coarse centroids are the same vector, so their scores tie bit for bit and the tie group is larger than
+    the selection buffer; one further list is strictly closer to each query.  The closer list must always be
+    probed first, and the fp32-pipe path fills the rest with the smallest list numbers, as the oracle does."""
+    data = synth.make_ivfpq(2000, 32, 3000, 16, 4, metric="l2", seed=90)
+    g = torch.Generator().manual_seed(5)
+    data.centroids[:2500] = data.centroids[0]
+    data.queries = data.centroids[0][None, :] + 0.05 * torch.randn((4, 32), generator=g)
+    for i in range(4):
+        data.centroids[2700 + i] = data.queries[i]
+    hix = host_index(oracle, data)
+    q = data.queries.numpy()
+    ol, oc = oracle.coarse(hix.centroids, q, 16, "l2")
+    for i in range(4):
+        assert ol[i].tolist() == [2700 + i] + list(range(15))           # what the definition gives
+    ix = binding.load_index_from(data, "cuda")
+    ix.rago_set_coarse_mode(mode)
+    for _ in range(3):                                                     # the same answer every time
+        gl, gc = ix.rago_search_probes(data.queries.cuda().contiguous(), 16)
+        torch.cuda.synchronize()
+        ix.rago_check()
+        gl, gc = gl.cpu().numpy(), gc.cpu().numpy()
+        for i in range(4):
+            assert gl[i][0] == 2700 + i and gc[i][0] < 1e-9
+            assert np.all(gl[i][1:] < 2500) and len(set(gl[i].tolist())) == 16
+            assert np.allclose(gc[i][1:], oc[i][1:], rtol=REL)
+            if mode == 1:
+                assert gl[i].tolist() == ol[i].tolist()
+    ix.close()
