@@ -46,8 +46,8 @@ SECONDARY = ("mid", "flat", "coarse_hyper", "iter")
 # of codes; the capture-size rule) and carries over to the full size because the lists are uniform and no list is
 # shared through L2 at either size; "mid" was captured at full size and is not scaled to other sizes.
 SCAN_TRAFFIC = {
-    "hyper": {"scan_sha": None, "dram_per_logical": None},
-    "mid": {"scan_sha": None, "dram_per_logical": None},
+    "hyper": {"scan_sha": "e8b5e3b88fc72587", "dram_per_logical": (15969621504 + 10022144) / 16004289600},   # 0.9985
+    "mid": {"scan_sha": "e8b5e3b88fc72587", "dram_per_logical": (35089437184 + 7926784) / 42427363200},      # 0.8272
 }
 
 

@@ -251,6 +251,16 @@ rago_status rago_flat_workspace_bytes(int64_t N, int32_t d, int32_t nq, int32_t 
 rago_status rago_check(void* workspace, void* cuda_stream);
 
 /*
+ * Test hook (no counterpart in the paper).  The tensor-core kernel has two main loops: one row tile of 128
+ * queries per CTA, or two row tiles that share every tile of the other operand.  The library picks by the
+ * size of that operand (sharing pays when it streams from HBM, i.e. for flat search over gigabytes); this
+ * call forces the choice process-wide so that tests reach both loops on small inputs: 0 = by size (default),
+ * 1 = never share, 2 = share whenever a batch has more than 128 queries.  Workspace sizes depend on it: set it
+ * before asking for them.  Not thread-safe against running searches.
+ */
+rago_status rago_debug_set_gemm_pairing(int32_t mode);
+
+/*
  * Test hook for the failure path of rago_check (no counterpart in the paper: the library's kernels wait on
  * copies and on the tensor pipe, every such wait is bounded, and this call lets a test see a bound expire
  * without anything being wrong).  Launches one small kernel in which a wait on a barrier that nothing signals

@@ -27,7 +27,7 @@ STAGE_NAMES = ("coarse_scores", "probe_select", "plan", "table_scan", "merge")
 EXPORTS = ("rago_index_load", "rago_index_load_pq4", "rago_index_set_coarse_tree", "rago_index_free", "rago_search_workspace_bytes", "rago_search",
            "rago_search_probes", "rago_search_probes_noalloc", "rago_search_host", "rago_host_staging_bytes", "rago_flat_search",
            "rago_flat_workspace_bytes", "rago_check", "rago_set_coarse_mode", "rago_profile_enable", "rago_profile_read",
-           "rago_merge_results", "rago_selftest_wait_timeout", "rago_kernel_launches", "rago_last_error")
+           "rago_merge_results", "rago_selftest_wait_timeout", "rago_debug_set_gemm_pairing", "rago_kernel_launches", "rago_last_error")
 
 
 class RagoError(RuntimeError):
@@ -61,6 +61,7 @@ def lib() -> ctypes.CDLL:
         L.rago_merge_results.argtypes = [vp, vp, i32, i64, i32, i32, i32, i32, vp, vp, vp]
         L.rago_check.argtypes = [vp, vp]
         L.rago_selftest_wait_timeout.argtypes = [vp, ctypes.c_uint32, i32, vp]
+        L.rago_debug_set_gemm_pairing.argtypes = [i32]
         L.rago_set_coarse_mode.argtypes = [vp, i32]
         L.rago_profile_enable.argtypes = [vp, i32]
         L.rago_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
@@ -219,6 +220,11 @@ def rago_index_load_pq4(centroids, pq4_codebooks, packed_codes, list_offsets, id
     if pq4_codebooks.shape[1] != 16:
         raise ValueError("4-bit codebooks have 16 codewords per sub-space")
     return Index(centroids, pq4_codebooks, packed_codes, list_offsets, ids, metric)
+
+
+def rago_debug_set_gemm_pairing(mode: int):
+    """0: the library chooses the tensor-core main loop by operand size, 1: one row tile per CTA, 2: paired row tiles."""
+    _check(lib().rago_debug_set_gemm_pairing(int(mode)))
 
 
 def rago_selftest_wait_timeout(workspace: torch.Tensor, max_polls: int, with_tmem: bool):

@@ -88,7 +88,7 @@ static Layout make_layout(const IndexImpl* ix, int nq, int nprobe, int k) {
         int nsel = nprobe + PROBE_GUARD;
         if (nsel > ix->nlist) nsel = ix->nlist;
         int mgroups = 1;
-        gemm_grid(nq, ix->nlist, ix->num_sms, &L.tc_mg, &L.tc_nsplit, &mgroups);
+        gemm_grid(nq, ix->nlist, ix->d * ix->cparts_n, ix->num_sms, &L.tc_mg, &L.tc_nsplit, &mgroups);
         L.tc_cap = gemm_cand_cap(nsel);
         L.tc_mode = L.tc_cap ? 0 : 1;
         L.qparts = take((size_t)ix->cparts_n * nq * ix->d * 2);
@@ -206,7 +206,7 @@ static rago_status run_coarse(const IndexImpl* ix, const float* queries, int nq,
             int mgroups = 1;
             P.tmap_b = ix->tmap_b_pilot;
             P.ncols = L.pilot_cols; P.b_part_rows = L.pilot_cols;
-            gemm_grid(nq, L.pilot_cols, ix->num_sms, &P.mg, &P.nsplit, &mgroups);
+            gemm_grid(nq, L.pilot_cols, ix->d * ix->cparts_n, ix->num_sms, &P.mg, &P.nsplit, &mgroups);
             P.colterm_stride = ix->pilot_stride;
             P.mode = 1;
             P.scores = reinterpret_cast<float*>(ws + L.pilot_scores);
@@ -554,6 +554,12 @@ rago_status rago_index_set_coarse_tree(rago_index* index, const void* level1_cen
     ix->tree_child_offsets = child_offsets;
     ix->tree_n1 = n1; ix->tree_b1 = b1;
     ix->tree_min_cand = (int)mn; ix->tree_max_cand = (int)mx;
+    return RAGO_OK;
+}
+
+rago_status rago_debug_set_gemm_pairing(int32_t mode) {
+    if (mode < 0 || mode > 2) return fail(RAGO_EINVAL, "mode = %d: 0 by operand size, 1 never, 2 always", mode);
+    gemm_set_pairing(mode);
     return RAGO_OK;
 }
 

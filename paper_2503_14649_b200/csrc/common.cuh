@@ -244,7 +244,8 @@ cudaError_t make_tmap_bf16(void* out_map, const void* ptr, uint64_t rows, uint64
 inline int gemm_pilot_stride(int64_t ncols) { const int64_t s = (ncols + 32767) / 32768; return s > 16 ? (int)s : 16; }
 cudaError_t launch_row_tau(const float* scores, int nrows, int n, int nsel, float* row_tau, cudaStream_t s);
 int gemm_cand_cap(int nsel);  // 0: nsel too large for the fused selection
-void gemm_grid(int nrows, int64_t ncols, int num_sms, int* mg, int* nsplit, int* mgroups);
+void gemm_grid(int nrows, int64_t ncols, int d, int num_sms, int* mg, int* nsplit, int* mgroups);
+void gemm_set_pairing(int mode);
 cudaError_t launch_gemm_select(const GemmLaunch& L, cudaStream_t s);
 cudaError_t launch_split_bf16(const float* x, size_t n, int parts, void* out, cudaStream_t s);
 cudaError_t launch_selftest_wait(uint32_t* err_word, uint32_t max_polls, int with_tmem, uint32_t* observed, cudaStream_t s);

@@ -180,7 +180,7 @@ static int flat_pilot_cols(int64_t N, int k) {
 size_t flat_workspace_bytes(int64_t N, int d, int nq, int k) {
     if (flat_on_tensor_cores(d, k)) {
         int mg, nsplit, mgroups;
-        gemm_grid(nq > 0 ? nq : 1, N > 0 ? N : 1, sm_count(), &mg, &nsplit, &mgroups);
+        gemm_grid(nq > 0 ? nq : 1, N > 0 ? N : 1, d, sm_count(), &mg, &nsplit, &mgroups);
         const size_t nlists = (size_t)nsplit * GEMM_COL_HALVES;
         return 256 + align_up((size_t)nq * nlists * gemm_cand_cap(k) * 8, 256) + align_up((size_t)nq * nlists * 4, 256) +
                align_up((size_t)nq * flat_pilot_cols(N, k) * 4, 256) + align_up((size_t)nq * 4, 256);
@@ -199,7 +199,7 @@ cudaError_t launch_flat_search(const void* db, int64_t N, int d, const void* que
         cudaError_t e = gemm_select_init();
         if (e != cudaSuccess) return e;
         int mg, nsplit, mgroups;
-        gemm_grid(nq, N, sm_count(), &mg, &nsplit, &mgroups);
+        gemm_grid(nq, N, d, sm_count(), &mg, &nsplit, &mgroups);
         const int cap = gemm_cand_cap(k);
         const int nlists = nsplit * GEMM_COL_HALVES;
         uint8_t* w = static_cast<uint8_t*>(workspace) + 256;
@@ -238,7 +238,7 @@ cudaError_t launch_flat_search(const void* db, int64_t N, int d, const void* que
             int pg = 1;
             P.tmap_b = tmap_p;
             P.ncols = np; P.b_part_rows = np;
-            gemm_grid(nq, np, sm_count(), &P.mg, &P.nsplit, &pg);
+            gemm_grid(nq, np, d, sm_count(), &P.mg, &P.nsplit, &pg);
             P.mode = 1; P.scores = pilot_scores;
             e = launch_gemm_select(P, s);
             if (e == cudaSuccess) e = launch_row_tau(pilot_scores, nq, np, G.nsel, row_tau, s);

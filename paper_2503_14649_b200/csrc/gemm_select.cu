@@ -534,13 +534,22 @@ cudaError_t make_tmap_bf16(void* out_map, const void* ptr, uint64_t rows, uint64
 
 int gemm_cand_cap(int nsel) { return nsel <= GEMM_CAP_SMALL - 128 ? GEMM_CAP_SMALL : (nsel <= GEMM_CAP_LARGE - 64 ? GEMM_CAP_LARGE : 0); }
 
-void gemm_grid(int nrows, int64_t ncols, int num_sms, int* mg, int* nsplit, int* mgroups) {
+// Grid shape.  mg = 2 pairs two row tiles on every B tile (the PAIR main loop: a third less operand traffic, but
+// the epilogue no longer overlaps the MMAs); it pays when B streams from HBM and is considered only for a B operand
+// well beyond the L2 (measured: flat search over 20 GB -8%, but the Hyperscale coarse step, whose 100 MB of
+// centroids stay in L2, +13%).  Among the shapes considered the one with the fewest tile-units per CTA wins.
+constexpr int64_t GEMM_PAIR_MIN_B_BYTES = 512ll << 20;
+static int g_pairing = 0;  // 0: by the size of B, 1: never pair, 2: pair whenever there are two row tiles
+void gemm_set_pairing(int mode) { g_pairing = mode; }
+void gemm_grid(int nrows, int64_t ncols, int d, int num_sms, int* mg, int* nsplit, int* mgroups) {
     const int mtiles = (nrows + GBM - 1) / GBM;
     const int64_t ntiles = (ncols + GBN - 1) / GBN;
+    const bool may_pair = g_pairing == 2 || (g_pairing == 0 && ncols * (int64_t)d * 2 >= GEMM_PAIR_MIN_B_BYTES);
     int best_mg = 1, best_split = 1;
     int64_t best_units = -1;
-    for (int g = 1; g <= 2; ++g) {
+    for (int g = 1; g <= (may_pair ? 2 : 1); ++g) {
         if (g > mtiles) break;
+        if (g_pairing == 2 && g == 1 && mtiles >= 2) continue;
         const int groups = (mtiles + g - 1) / g;
         int64_t split = num_sms / groups;
         if (split < 1) split = 1;

@@ -46,23 +46,39 @@ TC_CASES = [
 ]
 
 
-@pytest.mark.parametrize("case", TC_CASES, ids=lambda c: "d%d_nl%d_nq%d_np%d_%s%s" % (c[1], c[2], c[4], c[5], c[6],
-                                                                                        "_bf16" if c[7] else ""))
-def test_tensor_core_probes_match_oracle(case):
+@pytest.fixture(params=[1, 2], ids=["one_row_tile", "paired_row_tiles"])
+def pairing(request):
+    """Both main loops of the tensor-core kernel: batches of more than 128 queries take the forced one."""
+    binding.rago_debug_set_gemm_pairing(request.param)
+    yield request.param
+    binding.rago_debug_set_gemm_pairing(0)
+
+
+# every case under the one-row-tile loop, and those with more than 128 queries under the paired loop as well
+TC_RUNS = [(c, 1) for c in TC_CASES] + [(c, 2) for c in TC_CASES if c[4] > 128]
+
+
+@pytest.mark.parametrize("case,pair", TC_RUNS, ids=lambda v: ("d%d_nl%d_nq%d_np%d_%s%s" % (v[1], v[2], v[4], v[5], v[6],
+                         "_bf16" if v[7] else "")) if isinstance(v, tuple) else ("paired" if v == 2 else "single"))
+def test_tensor_core_probes_match_oracle(case, pair):
     N, d, nlist, M, nq, nprobe, metric, bf16 = case
-    data = synth.make_ivfpq(N, d, nlist, M, nq, metric=metric, seed=300 + nlist + nq, coarse_bf16=bf16)
-    _probe_parity(data, nprobe, mode=2)
+    binding.rago_debug_set_gemm_pairing(pair)
+    try:
+        data = synth.make_ivfpq(N, d, nlist, M, nq, metric=metric, seed=300 + nlist + nq, coarse_bf16=bf16)
+        _probe_parity(data, nprobe, mode=2)
+    finally:
+        binding.rago_debug_set_gemm_pairing(0)
 
 
 @pytest.mark.parametrize("metric,bf16", [("l2", False), ("ip", True)])
-def test_long_rows_exercise_list_compaction(metric, bf16):
+def test_long_rows_exercise_list_compaction(metric, bf16, pairing):
     """16 384 lists, 600 queries: a CTA sees several column tiles of a row, so candidate lists fill up and
     are compacted while the GEMM runs."""
     data = synth.make_ivfpq(4000, 64, 16384, 16, 600, metric=metric, seed=77, coarse_bf16=bf16)
     _probe_parity(data, 32, mode=2)
 
 
-def test_large_nprobe_uses_the_wide_lists_and_the_score_matrix():
+def test_large_nprobe_uses_the_wide_lists_and_the_score_matrix(pairing):
     data = synth.make_ivfpq(3000, 64, 8192, 16, 150, metric="l2", seed=78)
     _probe_parity(data, 300, mode=2)    # nsel = 308: 1024-key lists
     _probe_parity(data, 1000, mode=2)   # nsel = 1008: score-matrix epilogue

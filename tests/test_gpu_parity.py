@@ -151,12 +151,26 @@ def test_results_do_not_depend_on_run():
     ix.close()
 
 
-@pytest.mark.parametrize("N,d,nq,k", [(5000, 64, 7, 10), (70_000, 128, 33, 100), (3, 64, 2, 5),
-                                      (200_000, 64, 200, 100),   # two row tiles, lists compacted while streaming
-                                      (300_000, 64, 40, 50),     # large enough for the pilot-threshold pass
-                                      (40_000, 64, 9, 300),      # wide candidate lists
-                                      (30_000, 64, 5, 1000)])    # k above the fused selection: fp32-pipe fallback
-def test_flat_search_matches_oracle(N, d, nq, k):
+FLAT_CASES = [(5000, 64, 7, 10), (70_000, 128, 33, 100), (3, 64, 2, 5),
+              (200_000, 64, 200, 100),   # two row tiles, lists compacted while streaming
+              (300_000, 64, 40, 50),     # large enough for the pilot-threshold pass
+              (300_000, 64, 300, 100),   # three row tiles (a pair and a single) behind pilot thresholds
+              (40_000, 64, 9, 300),      # wide candidate lists
+              (30_000, 64, 5, 1000)]     # k above the fused selection: fp32-pipe fallback
+# every case with one row tile per CTA; batches of more than 128 queries also with paired row tiles
+FLAT_RUNS = [c + (1,) for c in FLAT_CASES] + [c + (2,) for c in FLAT_CASES if c[2] > 128]
+
+
+@pytest.mark.parametrize("N,d,nq,k,pairing", FLAT_RUNS)
+def test_flat_search_matches_oracle(N, d, nq, k, pairing):
+    binding.rago_debug_set_gemm_pairing(pairing)
+    try:
+        _flat_case(N, d, nq, k)
+    finally:
+        binding.rago_debug_set_gemm_pairing(0)
+
+
+def _flat_case(N, d, nq, k):
     db, q = synth.make_flat(N, d, nq, seed=N)
     gi, gs = binding.rago_flat_search(db.cuda(), q.cuda(), k)
     torch.cuda.synchronize()
