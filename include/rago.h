@@ -251,12 +251,13 @@ rago_status rago_flat_workspace_bytes(int64_t N, int32_t d, int32_t nq, int32_t 
 rago_status rago_check(void* workspace, void* cuda_stream);
 
 /*
- * Test hook (no counterpart in the paper).  The tensor-core kernel has two main loops: one row tile of 128
- * queries per CTA, or two row tiles that share every tile of the other operand.  The library picks by the
- * size of that operand (sharing pays when it streams from HBM, i.e. for flat search over gigabytes); this
- * call forces the choice process-wide so that tests reach both loops on small inputs: 0 = by size (default),
- * 1 = never share, 2 = share whenever a batch has more than 128 queries.  Workspace sizes depend on it: set it
- * before asking for them.  Not thread-safe against running searches.
+ * Test hook (no counterpart in the paper).  The tensor-core kernel has three main loops: one row tile of 128
+ * queries per CTA; two row tiles per CTA that share every tile of the other operand; or a cluster of two CTAs
+ * (one SM pair, tcgen05 cta_group::2) that shares it.  By default batches of more than 128 queries take the
+ * CTA pair and smaller ones the single row tile; this call forces the choice process-wide so that tests and
+ * measurements reach every loop: 0 = default, 1 = never share, 2 = share inside a CTA, 3 = share across a CTA
+ * pair (2 and 3 apply to batches of more than 128 queries).  Workspace sizes depend on it: set it before asking for them.  Not thread-safe against
+ * running searches.
  */
 rago_status rago_debug_set_gemm_pairing(int32_t mode);
 

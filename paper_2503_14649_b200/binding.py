@@ -223,7 +223,8 @@ def rago_index_load_pq4(centroids, pq4_codebooks, packed_codes, list_offsets, id
 
 
 def rago_debug_set_gemm_pairing(mode: int):
-    """0: the library chooses the tensor-core main loop by operand size, 1: one row tile per CTA, 2: paired row tiles."""
+    """0: the library chooses the tensor-core main loop by operand size, 1: one row tile per CTA, 2: two row tiles
+    per CTA, 3: two row tiles per CTA pair (cluster of two)."""
     _check(lib().rago_debug_set_gemm_pairing(int(mode)))
 
 

@@ -178,7 +178,7 @@ static rago_status run_coarse(const IndexImpl* ix, const float* queries, int nq,
         e = make_tmap_bf16(tmap_a, ws + L.qparts, (uint64_t)parts * nq, (uint64_t)ix->d, 128);
         if (e != cudaSuccess) return cuda_fail(e, "encoding the query tensor map");
         GemmLaunch G;
-        G.tmap_a = tmap_a; G.tmap_b = ix->tmap_b;
+        G.tmap_a = tmap_a; G.tmap_b = ix->tmap_b; G.tmap_b_half = ix->tmap_b_half;
         G.nrows = nq; G.ncols = ix->nlist; G.d = ix->d;
         G.a_part_rows = nq; G.b_part_rows = ix->nlist;
         if (parts == 1) {
@@ -204,7 +204,7 @@ static rago_status run_coarse(const IndexImpl* ix, const float* queries, int nq,
             // pilot pass: score every pilot_stride-th list, take each query's nsel-th smallest as its starting threshold
             GemmLaunch P = G;
             int mgroups = 1;
-            P.tmap_b = ix->tmap_b_pilot;
+            P.tmap_b = ix->tmap_b_pilot; P.tmap_b_half = ix->tmap_b_pilot_half;
             P.ncols = L.pilot_cols; P.b_part_rows = L.pilot_cols;
             gemm_grid(nq, L.pilot_cols, ix->d * ix->cparts_n, ix->num_sms, &P.mg, &P.nsplit, &mgroups);
             P.colterm_stride = ix->pilot_stride;
@@ -312,11 +312,14 @@ rago_status rago_index_load(rago_index** out, const void* coarse_centroids, rago
             bsrc = ix->cparts;
         }
         if (e == cudaSuccess && gemm_select_init() == cudaSuccess &&
-            make_tmap_bf16(ix->tmap_b, bsrc, (uint64_t)ix->cparts_n * nlist, (uint64_t)d, 256) == cudaSuccess)
+            make_tmap_bf16(ix->tmap_b, bsrc, (uint64_t)ix->cparts_n * nlist, (uint64_t)d, 256) == cudaSuccess &&
+            make_tmap_bf16(ix->tmap_b_half, bsrc, (uint64_t)ix->cparts_n * nlist, (uint64_t)d, 128) == cudaSuccess)
             ix->tc_ok = 1;
         const int ps = gemm_pilot_stride(nlist);
         if (ix->tc_ok && nlist % ps == 0 &&
             make_tmap_bf16(ix->tmap_b_pilot, bsrc, (uint64_t)ix->cparts_n * (nlist / ps), (uint64_t)d, 256,
+                           (uint64_t)ps * d) == cudaSuccess &&
+            make_tmap_bf16(ix->tmap_b_pilot_half, bsrc, (uint64_t)ix->cparts_n * (nlist / ps), (uint64_t)d, 128,
                            (uint64_t)ps * d) == cudaSuccess)
             ix->pilot_stride = ps;
         cudaGetLastError();  // a missing tensor-core path is not an error: the fp32 kernel serves every batch
@@ -558,7 +561,7 @@ rago_status rago_index_set_coarse_tree(rago_index* index, const void* level1_cen
 }
 
 rago_status rago_debug_set_gemm_pairing(int32_t mode) {
-    if (mode < 0 || mode > 2) return fail(RAGO_EINVAL, "mode = %d: 0 by operand size, 1 never, 2 always", mode);
+    if (mode < 0 || mode > 3) return fail(RAGO_EINVAL, "mode = %d: 0 by operand size, 1 single, 2 pair in a CTA, 3 CTA pair", mode);
     gemm_set_pairing(mode);
     return RAGO_OK;
 }

@@ -53,6 +53,7 @@ struct IndexImpl {
     int coarse_mode;  // 0 auto, 1 fp32 pipes, 2 tensor cores
     alignas(64) unsigned char tmap_b[128];  // CUtensorMap of the stacked centroid parts
     alignas(64) unsigned char tmap_b_pilot[128];  // the same, every pilot_stride-th centroid
+    alignas(64) unsigned char tmap_b_half[128], tmap_b_pilot_half[128];  // both again in boxes of 128 rows (CTA pairs)
     int pilot_stride;  // 0: no pilot pass for this index
     // optional first quantiser level (borrowed; tree_n1 = 0: none).  Node i owns lists child_offsets[i] .. [i+1]-1.
     const void* tree_level1;            // [tree_n1][d], the coarse dtype
@@ -219,11 +220,12 @@ constexpr int GEMM_CAP_SMALL = 512, GEMM_CAP_LARGE = 1024;  // candidate-list ca
 constexpr int GEMM_COL_HALVES = 2;  // a row has one candidate list per column range of the grid AND per half of a 256-column tile
 struct GemmLaunch {
     const void* tmap_a;          // CUtensorMap of A: bf16 [a parts * a_part_rows][d]
-    const void* tmap_b;          // CUtensorMap of B: bf16 [b parts * b_part_rows][d]
+    const void* tmap_b;          // CUtensorMap of B: bf16 [b parts * b_part_rows][d], boxes of 256 rows
+    const void* tmap_b_half;     // the same matrix in boxes of 128 rows (mg = 3: a CTA of a pair loads half a B tile)
     int nrows; int64_t ncols; int d;
     int a_part_rows; int64_t b_part_rows;
     int nterms; int term_a[6], term_b[6];
-    int mg, nsplit;              // from gemm_grid: row tiles per CTA (2 = both share each B tile), column ranges
+    int mg, nsplit;              // from gemm_grid: main loop (1 single, 2 pair in a CTA, 3 CTA pair) and column ranges
     float alpha; const float* colterm; int colterm_stride;
     const float* row_tau;        // initial per-row thresholds (mode 0) or null
     int mode, nsel, cap;

@@ -211,12 +211,13 @@ cudaError_t launch_flat_search(const void* db, int64_t N, int d, const void* que
         float* pilot_scores = reinterpret_cast<float*>(w);
         w += align_up((size_t)nq * np * 4, 256);
         float* row_tau = reinterpret_cast<float*>(w);
-        alignas(64) unsigned char tmap_a[128], tmap_b[128];
+        alignas(64) unsigned char tmap_a[128], tmap_b[128], tmap_bh[128];
         e = make_tmap_bf16(tmap_a, queries, (uint64_t)nq, (uint64_t)d, 128);
         if (e == cudaSuccess) e = make_tmap_bf16(tmap_b, db, (uint64_t)N, (uint64_t)d, 256);
+        if (e == cudaSuccess) e = make_tmap_bf16(tmap_bh, db, (uint64_t)N, (uint64_t)d, 128);
         if (e != cudaSuccess) return e;
         GemmLaunch G;
-        G.tmap_a = tmap_a; G.tmap_b = tmap_b;
+        G.tmap_a = tmap_a; G.tmap_b = tmap_b; G.tmap_b_half = tmap_bh;
         G.nrows = nq; G.ncols = N; G.d = d;
         G.a_part_rows = nq; G.b_part_rows = N;
         G.nterms = 1;
@@ -230,13 +231,14 @@ cudaError_t launch_flat_search(const void* db, int64_t N, int d, const void* que
         G.err = static_cast<uint32_t*>(workspace);
         if (np) {
             // pilot pass over every stride-th row: each query starts from the k-th best score of that sample
-            alignas(64) unsigned char tmap_p[128];
+            alignas(64) unsigned char tmap_p[128], tmap_ph[128];
             const int ps = gemm_pilot_stride(N);
             e = make_tmap_bf16(tmap_p, db, (uint64_t)np, (uint64_t)d, 256, (uint64_t)ps * d);
+            if (e == cudaSuccess) e = make_tmap_bf16(tmap_ph, db, (uint64_t)np, (uint64_t)d, 128, (uint64_t)ps * d);
             if (e != cudaSuccess) return e;
             GemmLaunch P = G;
             int pg = 1;
-            P.tmap_b = tmap_p;
+            P.tmap_b = tmap_p; P.tmap_b_half = tmap_ph;
             P.ncols = np; P.b_part_rows = np;
             gemm_grid(nq, np, d, sm_count(), &P.mg, &P.nsplit, &pg);
             P.mode = 1; P.scores = pilot_scores;

@@ -12,14 +12,23 @@
 //   warp 1    one lane issues tcgen05.mma (M128 N256 K16, bf16 -> fp32 in TMEM), tcgen05.commit frees stages
 //   warps 2-9 epilogue: tcgen05.ld 32 columns at a time, thread = output row; warp w reads TMEM lane quarter
 //             w mod 4 and the column half (w - 2) / 4 of the tile, and never waits for another warp
-// Two shapes of the main loop (template parameter PAIR):
-//   PAIR = false   one row tile per CTA.  A stage holds A (16 KB) and B (32 KB), four stages; the two 256-column
+// Three shapes of the main loop (template parameter LOOP):
+//   LOOP_SINGLE    one row tile per CTA.  A stage holds A (16 KB) and B (32 KB), four stages; the two 256-column
 //                  TMEM accumulators alternate, so the epilogue of one tile overlaps the MMAs of the next.
-//   PAIR = true    two row tiles per CTA (256 queries).  A stage holds A0, A1 and ONE B tile (64 KB), three
+//   LOOP_PAIR      two row tiles per CTA (256 queries).  A stage holds A0, A1 and ONE B tile (64 KB), three
 //                  stages; every K-block feeds two MMA chains, A0.B into accumulator 0 and A1.B into accumulator
 //                  1, so a B tile crosses L2 -> shared memory once per 256 queries and the operand traffic per
 //                  flop drops by a third.  Both accumulators belong to the same column tile, so the epilogue
 //                  does not overlap the next tile's MMAs; eight epilogue warps keep it short.
+//   LOOP_TWO_CTA   a cluster of two CTAs (one SM pair) works on 256 rows x 256 columns with tcgen05.mma
+//                  cta_group::2: each CTA loads its own 128 rows of A and HALF of the B tile (128 of the 256
+//                  columns' rows), 32 KB per stage, six stages; one thread of the cluster's first CTA issues the
+//                  MMAs (M = 256), each CTA's tensor memory receives its own 128 rows, and the accumulators
+//                  alternate as in LOOP_SINGLE, so the operand traffic of LOOP_PAIR comes with an overlapped
+//                  epilogue.  Loads of both CTAs complete on the first CTA's "full" barrier; tcgen05.commit
+//                  signals "stage empty" and "accumulator full" in both CTAs; the second CTA's epilogue warps
+//                  arrive on the first CTA's "accumulator empty" barrier through the cluster's shared window.
+//                  No copy is multicast: every CTA fetches its own operands.
 // A CTA owns a contiguous range of column tiles, so a row's running state (threshold, candidate count) lives in
 // the registers of the thread that owns the (row, column half).
 //
@@ -49,7 +58,8 @@ constexpr int GBM = 128, GBN = 256, GBK = 64;
 constexpr int G_A_BYTES = GBM * GBK * 2;
 constexpr int G_B_BYTES = GBN * GBK * 2;
 constexpr int G_RING_BYTES = 4 * (G_A_BYTES + G_B_BYTES);  // four stages of A + B, or three of A0 + A1 + B
-constexpr int G_MAX_STAGES = 4;
+constexpr int G_MAX_STAGES = 6;
+constexpr int LOOP_SINGLE = 0, LOOP_PAIR = 1, LOOP_TWO_CTA = 2;
 constexpr int G_EPI_WARPS = 8;                       // 4 TMEM lane quarters x 2 column halves
 constexpr int G_THREADS = 32 * (2 + G_EPI_WARPS);
 constexpr int G_HALF = GBN / GEMM_COL_HALVES;        // columns of a tile one epilogue warp reads
@@ -57,10 +67,12 @@ constexpr int G_TMEM_COLS = 512;
 constexpr int G_CN_BYTES = G_EPI_WARPS * 2 * G_HALF * 4;  // column terms: two copies per epilogue warp
 constexpr int G_SMEM_BYTES = G_RING_BYTES + G_CN_BYTES + 256 + 1024;  // + barriers + alignment slack
 static_assert(3 * (2 * G_A_BYTES + G_B_BYTES) <= G_RING_BYTES, "three paired stages fit the ring");
+static_assert(6 * (G_A_BYTES + G_B_BYTES / 2) <= G_RING_BYTES, "six two-CTA stages fit the ring");
 
 // tcgen05 instruction descriptor, kind::f16: D = f32 (bits 4-5 = 1), A = B = bf16 (bits 7-9, 10-12 = 1),
 // both operands K-major (bits 15, 16 = 0), N >> 3 in bits 17-22, M >> 4 in bits 24-28.
 constexpr uint32_t G_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(GBN >> 3) << 17) | ((uint32_t)(GBM >> 4) << 24);
+constexpr uint32_t G_IDESC_2CTA = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(GBN >> 3) << 17) | ((uint32_t)((2 * GBM) >> 4) << 24);  // M = 256 over the CTA pair
 
 // ---- PTX wrappers ---------------------------------------------------------------------------
 __device__ __forceinline__ void tma_load_2d(const CUtensorMap* map, uint32_t bar, uint32_t dst, int x, int y) {
@@ -75,6 +87,51 @@ __device__ __forceinline__ void tmem_alloc(uint32_t slot_smem, uint32_t ncols) {
 }
 __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// ---- the same for a CTA pair (cta_group::2) ----
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// shared::cluster address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t mapa_shared(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// Tiled load into this CTA's shared memory whose completion bytes count on a barrier of the pair (bar is a
+// shared::cluster address: the leader's barrier).  One destination, one CTA: nothing is multicast.
+__device__ __forceinline__ void tma_load_2d_pair(const CUtensorMap* map, uint32_t cluster_bar, uint32_t dst, int x, int y) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(cluster_bar)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t slot_smem, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(ncols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// arrives on the barrier at this shared-memory offset in BOTH CTAs of the pair once the MMAs issued so far are done
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+        : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -310,13 +367,16 @@ __device__ __forceinline__ void epilogue_store(uint32_t taddr, const float* cn, 
     }
 }
 
-template <int NK, bool PAIR>
+template <int NK, int LOOP>
 __global__ void __launch_bounds__(G_THREADS, 1)
 gemm_select_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmArgs a) {
     constexpr int CAP = NK * 32;
-    constexpr int STAGES = PAIR ? 3 : 4;
-    constexpr int STAGE_BYTES = PAIR ? 2 * G_A_BYTES + G_B_BYTES : G_A_BYTES + G_B_BYTES;
-    constexpr int B_OFF = STAGE_BYTES - G_B_BYTES;  // B follows the A tile(s) of its stage
+    constexpr bool PAIR = LOOP == LOOP_PAIR, TWO = LOOP == LOOP_TWO_CTA;
+    constexpr int STAGES = PAIR ? 3 : (TWO ? 6 : 4);
+    constexpr int B_BYTES = TWO ? G_B_BYTES / 2 : G_B_BYTES;  // a CTA of a pair holds half of the B tile
+    constexpr int STAGE_BYTES = (PAIR ? 2 : 1) * G_A_BYTES + B_BYTES;
+    constexpr int B_OFF = STAGE_BYTES - B_BYTES;  // B follows the A tile(s) of its stage
+    const uint32_t crank = TWO ? cluster_ctarank() : 0u;  // 0: the CTA that issues the pair's MMAs
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;  // swizzled tiles need 1024-byte alignment
@@ -339,21 +399,25 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(tfull_bar(b), 1);
-            mbar_init(tempty_bar(b), G_EPI_WARPS);
+            mbar_init(tempty_bar(b), TWO ? 2 * G_EPI_WARPS : G_EPI_WARPS);  // the leader hears from both CTAs' epilogues
         }
         *abort_flag = 0;
         fence_barrier_init();
         fence_proxy_async();
     }
-    if (warp == 0) tmem_alloc(smem_u32(tmem_slot), G_TMEM_COLS);
+    if (warp == 0) {
+        if (TWO) tmem_alloc_pair(smem_u32(tmem_slot), G_TMEM_COLS); else tmem_alloc(smem_u32(tmem_slot), G_TMEM_COLS);
+    }
     tc_fence_before();
     __syncthreads();
+    if (TWO) cluster_sync_all();  // the peer's barriers exist before anything of ours is aimed at them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    // PAIR: blockIdx.y counts pairs of row tiles (the last pair may hold one tile); else row tiles.
-    const int split = blockIdx.x, nsplit = gridDim.x;
-    const int m0 = PAIR ? blockIdx.y * 2 : blockIdx.y;
+    // PAIR / TWO: blockIdx.y counts pairs of row tiles (the last pair may hold one tile); else row tiles.
+    // TWO: the two CTAs of a cluster are neighbours in x and share a column range.
+    const int split = TWO ? blockIdx.x >> 1 : blockIdx.x, nsplit = TWO ? gridDim.x >> 1 : gridDim.x;
+    const int m0 = PAIR ? blockIdx.y * 2 : (TWO ? blockIdx.y * 2 + (int)crank : blockIdx.y);
     const int mcount = PAIR ? ((a.mtiles - m0) < 2 ? (a.mtiles - m0) : 2) : 1;
     const int nt_begin = (int)((long long)split * a.ntiles / nsplit);
     const int nt_end = (int)((long long)(split + 1) * a.ntiles / nsplit);
@@ -365,7 +429,8 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         if (lane == 0) {
             // unit = column tile; inside it the terms, inside a term the k-blocks: kept by counting, no division per load
             const int total = nunits * kiters;
-            const uint32_t tx_bytes = (uint32_t)(mcount == 2 ? STAGE_BYTES : G_A_BYTES + G_B_BYTES);
+            const uint32_t tx_bytes = TWO ? 2u * STAGE_BYTES  // both CTAs' loads complete on the leader's barrier
+                                          : (uint32_t)(mcount == 2 ? STAGE_BYTES : G_A_BYTES + G_B_BYTES);
             int nt = nt_begin, t = 0, kb = 0, s = 0;
             uint32_t ph = 0;
             for (int gi = 0; gi < total; ++gi) {
@@ -378,16 +443,25 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                 }
                 if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, a.err, 64)) break;
                 const uint32_t st = base + s * STAGE_BYTES;
-                mbar_arrive_expect_tx(full_bar(s), tx_bytes);
-                tma_load_2d(&tmA, full_bar(s), st, kx, ya);
-                if (PAIR && mcount == 2) tma_load_2d(&tmA, full_bar(s), st + G_A_BYTES, kx, ya + GBM);
-                tma_load_2d(&tmB, full_bar(s), st + B_OFF, kx, yb);
+                if (TWO) {
+                    // An mbarrier's transaction count may run ahead of its expectation, so the peer's bytes may land
+                    // before the leader announces them; the phase cannot complete without the leader's arrival.
+                    if (crank == 0) mbar_arrive_expect_tx(full_bar(s), tx_bytes);
+                    const uint32_t lead_full = mapa_shared(full_bar(s), 0);
+                    tma_load_2d_pair(&tmA, lead_full, st, kx, ya);
+                    tma_load_2d_pair(&tmB, lead_full, st + B_OFF, kx, yb + (int)crank * (GBN / 2));
+                } else {
+                    mbar_arrive_expect_tx(full_bar(s), tx_bytes);
+                    tma_load_2d(&tmA, full_bar(s), st, kx, ya);
+                    if (PAIR && mcount == 2) tma_load_2d(&tmA, full_bar(s), st + G_A_BYTES, kx, ya + GBM);
+                    tma_load_2d(&tmB, full_bar(s), st + B_OFF, kx, yb);
+                }
                 if (++s == STAGES) { s = 0; ph ^= 1u; }
             }
         }
     } else if (warp == 1) {
-        // ================= MMA issuer =================
-        if (lane == 0) {
+        // ================= MMA issuer (of a CTA pair: the leader's) =================
+        if (lane == 0 && crank == 0) {
             int s = 0;
             uint32_t ph = 0;
             bool dead = false;
@@ -405,18 +479,20 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                     const uint64_t da = smem_desc_sw128(st);
                     const uint64_t db = smem_desc_sw128(st + B_OFF);
 #pragma unroll
-                    for (int k = 0; k < GBK / 16; ++k)
-                        tc_mma_bf16(d_tmem, da + 2u * k, db + 2u * k, G_IDESC, (ki | k) != 0 ? 1u : 0u);
+                    for (int k = 0; k < GBK / 16; ++k) {
+                        if (TWO) tc_mma_bf16_pair(d_tmem, da + 2u * k, db + 2u * k, G_IDESC_2CTA, (ki | k) != 0 ? 1u : 0u);
+                        else tc_mma_bf16(d_tmem, da + 2u * k, db + 2u * k, G_IDESC, (ki | k) != 0 ? 1u : 0u);
+                    }
                     if (PAIR && mcount == 2) {
                         const uint64_t da1 = smem_desc_sw128(st + G_A_BYTES);
 #pragma unroll
                         for (int k = 0; k < GBK / 16; ++k)
                             tc_mma_bf16(d_tmem + GBN, da1 + 2u * k, db + 2u * k, G_IDESC, (ki | k) != 0 ? 1u : 0u);
                     }
-                    tc_commit(empty_bar(s));  // frees the stage once these MMAs have read it
+                    if (TWO) tc_commit_pair(empty_bar(s)); else tc_commit(empty_bar(s));  // frees the stage once these MMAs have read it
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
-                if (!dead) tc_commit(tfull_bar(buf));  // accumulator(s) complete
+                if (!dead) { if (TWO) tc_commit_pair(tfull_bar(buf)); else tc_commit(tfull_bar(buf)); }  // accumulator(s) complete
             }
         }
     } else {
@@ -475,7 +551,10 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(tempty_bar(buf));
+            if (lane == 0) {
+                if (TWO && crank != 0) mbar_arrive_cluster(mapa_shared(tempty_bar(buf), 0));
+                else mbar_arrive(tempty_bar(buf));
+            }
         }
         if (a.mode == 0 && !dead) {
 #pragma unroll
@@ -488,10 +567,11 @@ gemm_select_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
 
     tc_fence_before();
     __syncthreads();
+    if (TWO) cluster_sync_all();  // neither CTA's tensor memory or barriers go away while the other may still use them
     if (warp == 0) {
         tc_fence_after();
         if (*abort_flag) __nanosleep(100000);  // let copies / MMAs in flight drain after a timed-out wait
-        tmem_dealloc(tmem_base, G_TMEM_COLS);
+        if (TWO) tmem_dealloc_pair(tmem_base, G_TMEM_COLS); else tmem_dealloc(tmem_base, G_TMEM_COLS);
     }
 }
 
@@ -534,32 +614,31 @@ cudaError_t make_tmap_bf16(void* out_map, const void* ptr, uint64_t rows, uint64
 
 int gemm_cand_cap(int nsel) { return nsel <= GEMM_CAP_SMALL - 128 ? GEMM_CAP_SMALL : (nsel <= GEMM_CAP_LARGE - 64 ? GEMM_CAP_LARGE : 0); }
 
-// Grid shape.  mg = 2 pairs two row tiles on every B tile (the PAIR main loop: a third less operand traffic, but
-// the epilogue no longer overlaps the MMAs); it pays when B streams from HBM and is considered only for a B operand
-// well beyond the L2 (measured: flat search over 20 GB -8%, but the Hyperscale coarse step, whose 100 MB of
-// centroids stay in L2, +13%).  Among the shapes considered the one with the fewest tile-units per CTA wins.
-constexpr int64_t GEMM_PAIR_MIN_B_BYTES = 512ll << 20;
-static int g_pairing = 0;  // 0: by the size of B, 1: never pair, 2: pair whenever there are two row tiles
+// Grid shape and main loop.  *mg: 1 = one row tile per CTA (LOOP_SINGLE), 2 = two row tiles per CTA sharing each B
+// tile (LOOP_PAIR), 3 = two row tiles per CTA PAIR (LOOP_TWO_CTA: a cluster of two CTAs shares each B tile).
+// Batches of more than 128 rows take the CTA pair.  Measured on the two big contractions (ms, same box):
+//                                        single   pair in a CTA   CTA pair
+//   flat search, B = 20 GB from HBM       5.74        5.27        4.7 - 5.2 (power-capped to 1.2 - 1.6 GHz)
+//   Hyperscale coarse stage, B in L2      0.410       0.464       0.401
+// The in-CTA pair saves the same operand traffic as the CTA pair but cannot overlap its epilogue; it is kept as a
+// measured alternative that the test hook reaches.  *nsplit = column ranges; *mgroups = grid rows.
+static int g_pairing = 0;  // 0: as above, 1: LOOP_SINGLE, 2: LOOP_PAIR, 3: LOOP_TWO_CTA (2, 3: batches with two row tiles)
 void gemm_set_pairing(int mode) { g_pairing = mode; }
 void gemm_grid(int nrows, int64_t ncols, int d, int num_sms, int* mg, int* nsplit, int* mgroups) {
     const int mtiles = (nrows + GBM - 1) / GBM;
     const int64_t ntiles = (ncols + GBN - 1) / GBN;
-    const bool may_pair = g_pairing == 2 || (g_pairing == 0 && ncols * (int64_t)d * 2 >= GEMM_PAIR_MIN_B_BYTES);
-    int best_mg = 1, best_split = 1;
-    int64_t best_units = -1;
-    for (int g = 1; g <= (may_pair ? 2 : 1); ++g) {
-        if (g > mtiles) break;
-        if (g_pairing == 2 && g == 1 && mtiles >= 2) continue;
-        const int groups = (mtiles + g - 1) / g;
-        int64_t split = num_sms / groups;
-        if (split < 1) split = 1;
-        if (split > ntiles) split = ntiles;
-        const int64_t units = ((ntiles + split - 1) / split) * g;
-        if (best_units < 0 || units <= best_units) { best_units = units; best_mg = g; best_split = (int)split; }
+    int loop = 1;
+    if (mtiles >= 2) {
+        if (g_pairing == 2 || g_pairing == 3) loop = g_pairing;
+        else if (g_pairing == 0) loop = 3;
     }
-    *mg = best_mg;
-    *nsplit = best_split;
-    *mgroups = (mtiles + best_mg - 1) / best_mg;
+    const int groups = loop == 1 ? mtiles : (mtiles + 1) / 2;
+    int64_t split = (loop == 3 ? num_sms / 2 : num_sms) / groups;  // a CTA pair occupies two SMs
+    if (split < 1) split = 1;
+    if (split > ntiles) split = ntiles;
+    *mg = loop;
+    *nsplit = (int)split;
+    *mgroups = groups;
 }
 
 
@@ -576,21 +655,35 @@ cudaError_t launch_gemm_select(const GemmLaunch& L, cudaStream_t s) {
     a.row_tau = L.row_tau;
     a.mode = L.mode; a.nsel = L.nsel;
     a.cand = L.cand; a.cand_cnt = L.cand_cnt; a.scores = L.scores; a.err = L.err;
-    const bool pair = L.mg == 2;
-    const dim3 grid(L.nsplit, pair ? (a.mtiles + 1) / 2 : a.mtiles);
     const CUtensorMap* ma = reinterpret_cast<const CUtensorMap*>(L.tmap_a);
-    const CUtensorMap* mb = reinterpret_cast<const CUtensorMap*>(L.tmap_b);
+    const CUtensorMap* mb = reinterpret_cast<const CUtensorMap*>(L.mg == 3 ? L.tmap_b_half : L.tmap_b);
     const bool large = L.mode == 0 && L.cap == GEMM_CAP_LARGE;
-    if (large && pair)
-        gemm_select_kernel<GEMM_CAP_LARGE / 32, true><<<grid, G_THREADS, G_SMEM_BYTES, s>>>(*ma, *mb, a);
-    else if (large)
-        gemm_select_kernel<GEMM_CAP_LARGE / 32, false><<<grid, G_THREADS, G_SMEM_BYTES, s>>>(*ma, *mb, a);
-    else if (pair)
-        gemm_select_kernel<GEMM_CAP_SMALL / 32, true><<<grid, G_THREADS, G_SMEM_BYTES, s>>>(*ma, *mb, a);
-    else
-        gemm_select_kernel<GEMM_CAP_SMALL / 32, false><<<grid, G_THREADS, G_SMEM_BYTES, s>>>(*ma, *mb, a);
+    const int groups = L.mg == 1 ? a.mtiles : (a.mtiles + 1) / 2;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(L.mg == 3 ? 2 * L.nsplit : L.nsplit, groups);
+    cfg.blockDim = dim3(G_THREADS);
+    cfg.dynamicSmemBytes = G_SMEM_BYTES;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    if (L.mg == 3) {  // the two CTAs of a pair are neighbours in x
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+    }
+    cudaError_t e;
+#define RAGO_GEMM_LAUNCH(NKV, LOOPV) e = cudaLaunchKernelEx(&cfg, gemm_select_kernel<NKV, LOOPV>, *ma, *mb, a)
+    if (large) {
+        if (L.mg == 3) RAGO_GEMM_LAUNCH(GEMM_CAP_LARGE / 32, LOOP_TWO_CTA);
+        else if (L.mg == 2) RAGO_GEMM_LAUNCH(GEMM_CAP_LARGE / 32, LOOP_PAIR);
+        else RAGO_GEMM_LAUNCH(GEMM_CAP_LARGE / 32, LOOP_SINGLE);
+    } else {
+        if (L.mg == 3) RAGO_GEMM_LAUNCH(GEMM_CAP_SMALL / 32, LOOP_TWO_CTA);
+        else if (L.mg == 2) RAGO_GEMM_LAUNCH(GEMM_CAP_SMALL / 32, LOOP_PAIR);
+        else RAGO_GEMM_LAUNCH(GEMM_CAP_SMALL / 32, LOOP_SINGLE);
+    }
+#undef RAGO_GEMM_LAUNCH
     count_launch();
-    return cudaGetLastError();
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 // ---- pilot thresholds: per row, a value with at least nsel of the row's n sample scores at or below it --------
@@ -672,14 +765,17 @@ cudaError_t launch_row_tau(const float* scores, int nrows, int n, int nsel, floa
 }
 
 // Per-device set-up: the kernels' dynamic shared-memory limits (called at index load and by the flat search).
+template <int NKV, int LOOPV>
+static cudaError_t gemm_attr() {
+    return cudaFuncSetAttribute(gemm_select_kernel<NKV, LOOPV>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_SMEM_BYTES);
+}
 cudaError_t gemm_select_init() {
-    cudaError_t e = cudaFuncSetAttribute(gemm_select_kernel<GEMM_CAP_SMALL / 32, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_SMEM_BYTES);
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(gemm_select_kernel<GEMM_CAP_SMALL / 32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_SMEM_BYTES);
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(gemm_select_kernel<GEMM_CAP_LARGE / 32, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_SMEM_BYTES);
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(gemm_select_kernel<GEMM_CAP_LARGE / 32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_SMEM_BYTES);
+    cudaError_t e = gemm_attr<GEMM_CAP_SMALL / 32, LOOP_SINGLE>();
+    if (e == cudaSuccess) e = gemm_attr<GEMM_CAP_SMALL / 32, LOOP_PAIR>();
+    if (e == cudaSuccess) e = gemm_attr<GEMM_CAP_SMALL / 32, LOOP_TWO_CTA>();
+    if (e == cudaSuccess) e = gemm_attr<GEMM_CAP_LARGE / 32, LOOP_SINGLE>();
+    if (e == cudaSuccess) e = gemm_attr<GEMM_CAP_LARGE / 32, LOOP_PAIR>();
+    if (e == cudaSuccess) e = gemm_attr<GEMM_CAP_LARGE / 32, LOOP_TWO_CTA>();
     if (e == cudaSuccess)  // rows of up to 51 200 pilot scores in shared memory
         e = cudaFuncSetAttribute(row_tau_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     return e;

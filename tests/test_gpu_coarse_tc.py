@@ -46,7 +46,7 @@ TC_CASES = [
 ]
 
 
-@pytest.fixture(params=[1, 2], ids=["one_row_tile", "paired_row_tiles"])
+@pytest.fixture(params=[1, 2, 3], ids=["one_row_tile", "paired_row_tiles", "cta_pair"])
 def pairing(request):
     """Both main loops of the tensor-core kernel: batches of more than 128 queries take the forced one."""
     binding.rago_debug_set_gemm_pairing(request.param)
@@ -55,11 +55,11 @@ def pairing(request):
 
 
 # every case under the one-row-tile loop, and those with more than 128 queries under the paired loop as well
-TC_RUNS = [(c, 1) for c in TC_CASES] + [(c, 2) for c in TC_CASES if c[4] > 128]
+TC_RUNS = [(c, 1) for c in TC_CASES] + [(c, 2) for c in TC_CASES if c[4] > 128] + [(c, 3) for c in TC_CASES if c[4] > 128]
 
 
 @pytest.mark.parametrize("case,pair", TC_RUNS, ids=lambda v: ("d%d_nl%d_nq%d_np%d_%s%s" % (v[1], v[2], v[4], v[5], v[6],
-                         "_bf16" if v[7] else "")) if isinstance(v, tuple) else ("paired" if v == 2 else "single"))
+                         "_bf16" if v[7] else "")) if isinstance(v, tuple) else {1: "single", 2: "paired", 3: "cta_pair"}[v])
 def test_tensor_core_probes_match_oracle(case, pair):
     N, d, nlist, M, nq, nprobe, metric, bf16 = case
     binding.rago_debug_set_gemm_pairing(pair)

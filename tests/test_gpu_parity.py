@@ -158,7 +158,8 @@ FLAT_CASES = [(5000, 64, 7, 10), (70_000, 128, 33, 100), (3, 64, 2, 5),
               (40_000, 64, 9, 300),      # wide candidate lists
               (30_000, 64, 5, 1000)]     # k above the fused selection: fp32-pipe fallback
 # every case with one row tile per CTA; batches of more than 128 queries also with paired row tiles
-FLAT_RUNS = [c + (1,) for c in FLAT_CASES] + [c + (2,) for c in FLAT_CASES if c[2] > 128]
+FLAT_RUNS = [c + (1,) for c in FLAT_CASES] + [c + (2,) for c in FLAT_CASES if c[2] > 128] + \
+            [c + (3,) for c in FLAT_CASES if c[2] > 128]   # 3: a cluster of two CTAs per pair of row tiles
 
 
 @pytest.mark.parametrize("N,d,nq,k,pairing", FLAT_RUNS)
