@@ -40,14 +40,14 @@ HEADLINE = "hyper"
 SECONDARY = ("mid", "flat", "coarse_hyper", "iter")
 
 # DRAM bytes per logical (algorithmic) code byte of one scan_kernel launch, from ncu one-pass captures of
-# dram__bytes_read.sum + dram__bytes_write.sum (profiles/scan_kernel_dram_traffic.md).  A figure is only valid for
+# dram__bytes_read.sum + dram__bytes_write.sum (profiles/scan_kernel_hyperscale_sixteenth_scale.md, profiles/scan_kernel_mid_quarter_scale.md).  A figure is only valid for
 # the kernel source it was captured from: each entry names the SHA-256 of csrc/scan.cu (first 16 hex digits) and a
 # run whose scan.cu hashes differently reports traffic = null.  "hyper" was captured at 1/16 of the vectors (4 GB
 # of codes; the capture-size rule) and carries over to the full size because the lists are uniform and no list is
 # shared through L2 at either size; "mid" was captured at full size and is not scaled to other sizes.
 SCAN_TRAFFIC = {
-    "hyper": {"scan_sha": "e8b5e3b88fc72587", "dram_per_logical": (15969621504 + 10022144) / 16004289600},   # 0.9985
-    "mid": {"scan_sha": "e8b5e3b88fc72587", "dram_per_logical": (35089437184 + 7926784) / 42427363200},      # 0.8272
+    "hyper": {"scan_sha": "e8b5e3b88fc72587", "dram_per_logical": (15969510400 + 10154496) / 16004289600},   # 0.9985
+    "mid": {"scan_sha": "e8b5e3b88fc72587", "dram_per_logical": (34599481856 + 8223488) / 42427363200},      # 0.8157
 }
 
 

@@ -369,3 +369,51 @@ def test_thousands_of_identical_centroids_do_not_displace_a_closer_list(mode):
             if mode == 1:
                 assert gl[i].tolist() == ol[i].tolist()
     ix.close()
+
+
+# ---- 64-byte codes (the Hyperscale code size) on shapes that stress list boundaries and ties ----
+
+CODES64_CASES = [
+    # N, d, nlist, nq, nprobe, k, metric, bf16, zipf, hashed
+    (60_000, 128, 40, 9, 6, 10, "l2", False, None, False),      # ragged lists (lengths not multiples of 8)
+    (60_000, 256, 64, 33, 64, 100, "ip", True, None, True),     # every list probed, bf16 quantiser, k = 100
+    (300, 64, 50, 5, 20, 160, "l2", False, None, False),        # lists of a handful of vectors, padding in the results
+    (400_000, 768, 96, 20, 24, 100, "l2", False, 1.1, False),   # long skewed lists: many tiles per pair
+    (250_000, 64, 7, 1, 7, 50, "ip", False, None, True),        # one query whose lists are spread over all CTAs
+]
+
+
+@pytest.mark.parametrize("case", CODES64_CASES, ids=lambda c: "N%d_d%d_nl%d_nq%d_np%d_k%d_%s" % (c[0], c[1], c[2], c[3], c[4], c[5], c[6]))
+def test_64_byte_codes(case):
+    N, d, nlist, nq, nprobe, k, metric, bf16, zipf, hashed = case
+    if hashed:
+        data = synth.make_ivfpq_hashed(N, d, nlist, 64, nq, metric=metric, seed=600 + nlist, coarse_bf16=bf16)
+    else:
+        data = synth.make_ivfpq(N, d, nlist, 64, nq, metric=metric, seed=600 + nlist, coarse_bf16=bf16, zipf=zipf)
+    _compare(data, nprobe, k, max_probe_mismatch=1)
+
+
+def test_thousands_of_identical_vectors_still_give_k_distinct_results():
+    """Every vector of the probed lists has the same code, so all scores tie: the buffer cuts and the merge must
+    still return k distinct vectors of the right score, run after run."""
+    data = synth.make_ivfpq(50_000, 64, 8, 64, 3, metric="l2", seed=77)
+    data.codes[:] = data.codes[0]
+    ix = binding.load_index_from(data, "cuda")
+    q = data.queries.cuda().contiguous()
+    first = None
+    for _ in range(3):
+        ids, dists = ix.rago_search(q, 4, 100)
+        torch.cuda.synchronize()
+        ix.rago_check()
+        ids, dists = ids.cpu().numpy(), dists.cpu().numpy()
+        for i in range(3):
+            assert len(set(ids[i].tolist())) == 100 and ids[i].min() >= 0
+            assert np.all(np.diff(dists[i]) >= 0)
+        first = dists if first is None else first
+        assert np.array_equal(first, dists)
+    hix = host_index(oracle, data)
+    oi, od = oracle.ivfpq_search(hix, data.queries.numpy(), 4, 100)
+    rs = IvfPqRescorer(oracle, hix)
+    for i in range(3):
+        assert not match_results(ids[i], dists[i], oi[i], od[i], rel=REL, rescore=rs.for_query(data.queries[i].numpy())), i
+    ix.close()
