@@ -68,15 +68,16 @@ class RetrievalModel:
 
 def fit_retrieval_model(Q: Sequence[float], D: Sequence[float], T: Sequence[float]) -> RetrievalModel:
     """Relative least squares of T = T0 + D / B_mem over the rows (small batches weigh as much as large ones);
-    R_q is then the tightest per-query rate no row contradicts (inf when the bandwidth leg explains every row)."""
+    R_q is then the per-query rate of the rows the bandwidth leg cannot explain (those whose bytes account for less
+    than half of their time beyond T0), inf when there are none."""
     Qv, Dv, Tv = (np.asarray(x, np.float64) for x in (Q, D, T))
     A = np.stack([np.ones_like(Dv), Dv], 1)
     coef, *_ = np.linalg.lstsq(A / Tv[:, None], np.ones_like(Tv), rcond=None)
     T0 = max(float(coef[0]), 0.0)
     B = 1.0 / max(float(coef[1]), 1e-30)
-    resid = Tv - T0 - Dv / B                       # time the bandwidth leg leaves unexplained
-    slow = resid > 0.1 * Tv
-    R_q = float(np.min(Qv[slow] / (Tv[slow] - T0))) if slow.any() else float("inf")
+    over = Tv - T0                                  # time beyond the floor
+    slow = (over > 0) & (Dv / B < 0.5 * over)       # rows whose bytes explain less than half of it
+    R_q = float(np.min(Qv[slow] / over[slow])) if slow.any() else float("inf")
     m = RetrievalModel(T0, B, R_q)
     m.max_rel_err = float(np.max(np.abs(np.array([m.time(q, d) for q, d in zip(Qv, Dv)]) - Tv) / Tv))
     return m
