@@ -47,6 +47,8 @@
 // A warp works on RGW row groups of 32 (virtual) rows per tile, unrolled, so that several independent
 // chains code word -> address -> table entry are in flight per warp; with R lanes per vector one
 // epilogue (term, bias, key, push) serves R row groups.
+#include <type_traits>
+
 #include "topk.cuh"
 
 namespace rago {
@@ -60,11 +62,10 @@ __device__ __forceinline__ void l2_prefetch(const void* g, uint32_t bytes) {
 constexpr int SMEM_OPTIN = 227 * 1024;          // dynamic shared memory asked for (the sm_100 per-block limit)
 constexpr uint32_t SMEM_BASE_EXPECTED = 1024;   // shared-window address of dynamic shared memory when the kernel has no static part
 constexpr int CTRL_BYTES = 1024;
-constexpr uint32_t LUT_WINDOW = 0x10000;        // banked tables start here (absolute shared address)
 
 struct TileDesc {
     int32_t pair;      // index into probe_list (query * nprobe + rank)
-    int32_t list;      // inverted list number
+    float term;        // the pair's (query, list) term of the score
     uint32_t pos0;     // storage position of the tile's first vector
     int32_t nvec;      // vectors in this tile
     int32_t newpair;   // bit 0: first tile of this pair inside this CTA; bit 1: cut the candidate buffer before this tile
@@ -113,6 +114,9 @@ struct Cfg {
     static constexpr int TILE_BYTES = TILE_VROWS * MV;
     static constexpr int VT_BYTES = (TV + 4) * 4;       // staged per-vector terms (start rounded down to 16 bytes)
     static constexpr int KCAP = LUT_BYTES <= 65536 ? 2 * TOPK_CAP : TOPK_CAP;  // keys of the CTA's candidate buffer
+    // Banked tables start at this absolute shared address (a multiple of 64 KB).  Two tiles of more than 48 KB do not
+    // fit above a table at 64 KB, so configurations with such tiles keep their tiles below a table at 128 KB.
+    static constexpr uint32_t LUT_WINDOW = (NBANK == 1 && TILE_BYTES > 48 * 1024) ? 0x20000u : 0x10000u;
     static_assert(WV % G == 0, "virtual rows are whole blocks");
     static_assert(TILE_VROWS % R == 0, "tile must hold whole vectors");
     static_assert(RGW % (R < RGW ? R : RGW) == 0, "row groups are taken min(R, RGW) at a time");
@@ -155,15 +159,15 @@ struct SmemPlan {
 };
 
 template <class C>
-__host__ __device__ inline SmemPlan plan_smem(uint32_t base, uint32_t dyn_bytes, int d, int stages) {
+__host__ __device__ inline SmemPlan plan_smem(uint32_t base, uint32_t dyn_bytes, int d, int stages, bool need_vt) {
     SmemPlan p;
     p.ok = 1;
     const uint32_t end = base + dyn_bytes;
     uint32_t lo_cur, lo_end, hi_cur;
     if (C::BANKED) {
-        p.lut = LUT_WINDOW;
-        if (base > LUT_WINDOW) p.ok = 0;
-        lo_cur = base; lo_end = LUT_WINDOW; hi_cur = LUT_WINDOW + C::LUT_BYTES;
+        p.lut = C::LUT_WINDOW;
+        if (base > C::LUT_WINDOW) p.ok = 0;
+        lo_cur = base; lo_end = C::LUT_WINDOW; hi_cur = C::LUT_WINDOW + C::LUT_BYTES;
     } else {
         p.lut = (base + 127u) & ~127u;
         lo_cur = lo_end = 0; hi_cur = p.lut + C::LUT_BYTES;
@@ -177,11 +181,12 @@ __host__ __device__ inline SmemPlan plan_smem(uint32_t base, uint32_t dyn_bytes,
         p.ok = 0;
         return base;
     };
-    p.ctrl = take(CTRL_BYTES, 16);
-    p.keys = take(C::KCAP * 8, 16);
-    p.rT = take((uint32_t)d * 4, 16);
-    for (int s = 0; s < MAX_STAGES; ++s) p.vt[s] = s < stages ? take(C::VT_BYTES, 16) : base;
+    // largest pieces first, each below the table if it fits there, else above it
     for (int s = 0; s < MAX_STAGES; ++s) p.tile[s] = s < stages ? take(C::TILE_BYTES, 128) : base;
+    p.keys = take(C::KCAP * 8, 16);
+    for (int s = 0; s < MAX_STAGES; ++s) p.vt[s] = (s < stages && need_vt) ? take(C::VT_BYTES, 16) : base;
+    p.rT = take((uint32_t)d * 4, 16);
+    p.ctrl = take(CTRL_BYTES, 16);
     return p;
 }
 
@@ -280,12 +285,14 @@ __device__ __forceinline__ void quantise_table(uint32_t lut, int ctid, float sca
 
 // Code words of one virtual row, all loaded before the first look-up (look-up addresses depend on them,
 // so loading block by block would expose the shared-memory latency once per block).
-template <class C, int G, int BLK>
+// wa[il] is the lane's address of word (il ^ a(L)) of its row in the tile's first row group of this warp; OFF is
+// the byte offset of the row group being read, a compile-time constant that ends up in the load's immediate.
+template <class C, int G, int BLK, int OFF>
 struct LoadWords {
-    __device__ __forceinline__ static void run(uint32_t rowaddr, const uint32_t (&xo)[G], uint32_t (&x)[C::NBLK][G]) {
+    __device__ __forceinline__ static void run(const uint32_t (&wa)[G], uint32_t (&x)[C::NBLK][G]) {
 #pragma unroll
-        for (int il = 0; il < G; ++il) x[BLK][il] = lds_u32_imm<BLK * G * 4>(rowaddr + xo[il]);
-        if constexpr (BLK + 1 < C::NBLK) LoadWords<C, G, BLK + 1>::run(rowaddr, xo, x);
+        for (int il = 0; il < G; ++il) x[BLK][il] = lds_u32_imm<OFF + BLK * G * 4>(wa[il]);
+        if constexpr (BLK + 1 < C::NBLK) LoadWords<C, G, BLK + 1, OFF>::run(wa, x);
     }
 };
 
@@ -334,7 +341,7 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int S = a.stages;
     const uint32_t base = smem_u32(smem);
-    const SmemPlan P = plan_smem<C>(base, a.dyn_bytes, a.d, S);
+    const SmemPlan P = plan_smem<C>(base, a.dyn_bytes, a.d, S, a.vterm != nullptr);
     if (!P.ok) {  // uniform: every thread sees the same plan
         if (tid == 0) atomicExch(a.err, (uint32_t)ERR_SMEM_LAYOUT);
         return;
@@ -377,7 +384,7 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
             if (a.work_prefix[mid] <= u_begin) lo = mid; else hi = mid;
         }
         int cache_base = lo;  // lane i caches pair cache_base + i
-        int c_list = 0; long long c_off = 0, c_len = 0, c_ws = 0, c_we = 0;
+        int c_list = 0; long long c_off = 0, c_len = 0, c_ws = 0, c_we = 0; float c_term = 0.f;
         auto fill = [&]() {
             const int p = cache_base + lane;
             if (p < a.npairs) {
@@ -386,8 +393,9 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
                 c_len = a.list_offsets[c_list + 1] - c_off;
                 c_ws = a.work_prefix[p];
                 c_we = a.work_prefix[p + 1];
+                c_term = a.probe_term[p];
             } else {
-                c_list = 0; c_off = 0; c_len = 0; c_ws = c_we = W;
+                c_list = 0; c_off = 0; c_len = 0; c_ws = c_we = W; c_term = 0.f;
             }
         };
         fill();
@@ -411,7 +419,7 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
             const long long ws = __shfl_sync(0xffffffffu, c_ws, cur);
             const long long off = __shfl_sync(0xffffffffu, c_off, cur);
             const long long len = __shfl_sync(0xffffffffu, c_len, cur);
-            const int list = __shfl_sync(0xffffffffu, c_list, cur);
+            const float term = __shfl_sync(0xffffffffu, c_term, cur);
             if (round > 0) dead = !mbar_wait(smem_u32(&ctrl->empty[st]), (round - 1) & 1, abort_flag, a.err);
             if (dead) break;
             if (lane == 0) {
@@ -422,7 +430,7 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
                 const uint32_t pos0 = (uint32_t)(off + v0);
                 TileDesc& D = ctrl->desc[st];
                 D.pair = cache_base + cur;
-                D.list = list;
+                D.term = term;
                 D.pos0 = pos0;
                 D.nvec = (int32_t)nvec;
                 // everything tiles n-S+1 .. n can still push must fit behind what is in the buffer now
@@ -481,7 +489,7 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
     uint32_t xo[G], cc[G][2], lo[G][4], sel[4];
 #pragma unroll
     for (int il = 0; il < G; ++il) {
-        xo[il] = 4u * (uint32_t)(il ^ xa);
+        xo[il] = (uint32_t)(warp * C::RGW * 32 + lane) * C::MV + 4u * (uint32_t)(il ^ xa);  // offset in a tile of the lane's word il of the warp's first row group
 #pragma unroll
         for (int t = 0; t < 4; ++t)
             lo[il][t] = C::BANKED ? 0u : 4u * (uint32_t)(colbase + 4 * (il ^ xa) + (t ^ xb));
@@ -648,8 +656,7 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
                 begin_query(q);
                 if (dead) break;
             }
-            const float term = a.probe_term[D.pair];
-            bias = ip ? -term : term;
+            bias = ip ? -D.term : D.term;
         }
         if (D.newpair & 2) {  // the producer saw the buffer filling up: keep the best k (or a few more), lower the threshold
             csync();
@@ -670,23 +677,31 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
         // the vector's sum, so lane slice g finishes row group g and one epilogue serves MERGE row groups.
         constexpr int MERGE = R < C::RGW ? R : C::RGW;
         bool released = false;
+        uint32_t wa[G];  // this lane's word addresses in the warp's first row group of the tile
 #pragma unroll
-        for (int rg = 0; rg < C::RGW; rg += MERGE) {
+        for (int il = 0; il < G; ++il) wa[il] = tile_base + xo[il];
+        // One pass: MERGE row groups and their shared epilogue.  RG is a type carrying the first row group's index,
+        // so that every shared-memory offset below is a compile-time constant.  Returns false when the tile ended.
+        auto pass = [&](auto RG) -> bool {
+            constexpr int rg = decltype(RG)::value;
             const int vr0 = (warp * C::RGW + rg) * 32;
-            if (vr0 >= nvr) break;
+            if (vr0 >= nvr) return false;
             int mine = 0;
-#pragma unroll
-            for (int g = 0; g < MERGE; ++g) {
-                const uint32_t rowaddr = tile_base + (uint32_t)(vr0 + g * 32 + lane) * C::MV;
+            auto group = [&](auto GI) {
+                constexpr int g = decltype(GI)::value;
                 int acc[4] = {0, 0, 0, 0};
                 uint32_t x[C::NBLK][G];
-                LoadWords<C, G, 0>::run(rowaddr, xo, x);
+                LoadWords<C, G, 0, (rg + g) * 32 * C::MV>::run(wa, x);
                 ScanBlocks<C, G, 0>::run(x, cc, sel, lo, P.lut, acc);
                 int si = (acc[0] + acc[1]) + (acc[2] + acc[3]);
                 if (R >= 2) si += __shfl_xor_sync(0xffffffffu, si, 1);
                 if (R >= 4) si += __shfl_xor_sync(0xffffffffu, si, 2);
                 if (MERGE == 1 || sr == g) mine = si;
-            }
+            };
+            group(std::integral_constant<int, 0>{});
+            if constexpr (MERGE >= 2) group(std::integral_constant<int, 1>{});
+            if constexpr (MERGE >= 3) group(std::integral_constant<int, 2>{});
+            if constexpr (MERGE >= 4) group(std::integral_constant<int, 3>{});
             const int vr = vr0 + (MERGE == 1 ? 0 : sr * 32) + lane;  // the virtual row whose vector this lane finishes
             const float s = (float)mine * inv_scale;
             // per-vector term of the L2 expansion (0 for inner product); rows past the tile's end read
@@ -694,7 +709,7 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
             const float vt = a.vterm != nullptr ? lds_f32(vt_base + (uint32_t)(vr / R) * 4u) : 0.f;
             // In the last pass over the tile that was this warp's last read of the stage: hand the stage back
             // before the rest of the epilogue, so that the refill starts that much earlier (M = 96: -1%).
-            if (rg + MERGE >= C::RGW) {  // compile-time under the unrolled loop
+            if constexpr (rg + MERGE >= C::RGW) {
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&ctrl->empty[st]));
                 released = true;
@@ -703,7 +718,13 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
             const unsigned long long key = make_key(score, D.pos0 + (uint32_t)(vr / R));
             const bool owner = MERGE == 1 ? sr == 0 : sr < MERGE;
             warp_push(keys, &ctrl->cnt, vr < nvr && owner && key < tau, key, C::KCAP);
-        }
+            return true;
+        };
+        static_assert(C::RGW / MERGE <= 4, "passes are written out below");
+        bool more = pass(std::integral_constant<int, 0>{});
+        if constexpr (C::RGW > MERGE) more = more && pass(std::integral_constant<int, MERGE>{});
+        if constexpr (C::RGW > 2 * MERGE) more = more && pass(std::integral_constant<int, 2 * MERGE>{});
+        if constexpr (C::RGW > 3 * MERGE) more = more && pass(std::integral_constant<int, 3 * MERGE>{});
         if (!released) {  // a warp that left the loop early: no rows of this tile are its own
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ctrl->empty[st]));
@@ -717,13 +738,13 @@ struct Variant {
     int M;
     void (*kernel)(const ScanArgs);
     int threads, tile_vecs;
-    int (*stages_for)(int d);
+    int (*stages_for)(int d, bool need_vt);
     int lut_bytes, lut_banked, lut_copies, lut_copy_off, lut_stride;
 };
 template <class C>
-static int stages_for(int d) {
+static int stages_for(int d, bool need_vt) {
     for (int s = C::SMAX; s >= 2; --s)
-        if (plan_smem<C>(SMEM_BASE_EXPECTED, SMEM_OPTIN, d, s).ok) return s;
+        if (plan_smem<C>(SMEM_BASE_EXPECTED, SMEM_OPTIN, d, s, need_vt).ok) return s;
     return 0;
 }
 #define RAGO_VARIANT(WV, G, R, NCW, RGW) \
@@ -732,30 +753,35 @@ static int stages_for(int d) {
       Cfg<WV, G, R, NCW, RGW>::BANKED ? 1 : 0, Cfg<WV, G, R, NCW, RGW>::COPIES, Cfg<WV, G, R, NCW, RGW>::COPY_OFF, \
       Cfg<WV, G, R, NCW, RGW>::LSTRIDE }
 // Warps x unrolled row groups per warp were chosen by measurement: independent row groups in flight inside a warp
-// hide the look-up latency better than more warps do (M = 64: 16 x 2 -> 12 x 4 gave +30%).
+// hide the look-up latency better than more warps do (M = 64: 16 x 2 -> 12 x 4 gave +30%).  Where a code size has
+// two entries the first one whose shared-memory plan fits the index (dimension, metric) is taken.
 static const Variant kVariants[] = {
     RAGO_VARIANT(4, 4, 1, 16, 2),   // M = 16
     RAGO_VARIANT(8, 8, 1, 10, 3),   // M = 32
     RAGO_VARIANT(12, 4, 1, 8, 2),   // M = 48
-    RAGO_VARIANT(8, 8, 2, 12, 4),   // M = 64
+    RAGO_VARIANT(8, 8, 2, 15, 4),   // M = 64: 15 + 1 warps fill the four schedulers evenly; two 60 KB tiles below the table
+    RAGO_VARIANT(8, 8, 2, 12, 4),   // M = 64 where those do not fit (per-vector terms, d > 768)
     RAGO_VARIANT(20, 4, 1, 8, 1),   // M = 80
     RAGO_VARIANT(24, 8, 1, 12, 1),  // M = 96
     RAGO_VARIANT(8, 8, 4, 12, 3),   // M = 128
 };
 
-static const Variant* find_variant(int M) {
+static const Variant* find_variant(int M, int d, bool need_vt) {
     for (const Variant& v : kVariants)
-        if (v.M == M) return &v;
+        if (v.M == M && v.stages_for(d, need_vt) >= 2) return &v;
     return nullptr;
 }
 
-bool scan_supported(int M) { return find_variant(M) != nullptr; }
+bool scan_supported(int M) {
+    for (const Variant& v : kVariants)
+        if (v.M == M) return true;
+    return false;
+}
 
 cudaError_t scan_plan(const IndexImpl* ix, ScanPlan* plan) {
-    const Variant* v = find_variant(ix->M);
+    const Variant* v = find_variant(ix->M, ix->d, ix->metric != RAGO_IP);
     if (!v) return cudaErrorInvalidValue;
-    const int stages = v->stages_for(ix->d);
-    if (stages < 2) return cudaErrorInvalidValue;
+    const int stages = v->stages_for(ix->d, ix->metric != RAGO_IP);
     plan->tile_vecs = v->tile_vecs;
     plan->stages = stages;
     plan->ctas = ix->num_sms;
@@ -769,7 +795,7 @@ cudaError_t launch_scan(const IndexImpl* ix, const ScanPlan& plan, const float* 
                         const float* probe_term, const int64_t* work_prefix, int nq, int nprobe, int k,
                         unsigned long long* qthresh, int32_t* slot_cnt, unsigned long long* slot_keys,
                         uint32_t* err_word, const uint8_t* lut_img, const float* lut_inv, cudaStream_t s) {
-    const Variant* v = find_variant(ix->M);
+    const Variant* v = find_variant(ix->M, ix->d, ix->metric != RAGO_IP);
     if (!v) return cudaErrorInvalidValue;
     ScanArgs a;
     a.codes = ix->codes; a.list_offsets = ix->list_offsets; a.probe_list = probe_list; a.probe_term = probe_term;
