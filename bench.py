@@ -120,6 +120,18 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def _per_clock(achieved_gbs, clocks, dev):
+    """The same rate per SM clock: the step runs under the board's power cap, so the sampled median SM clock says how
+    much of a lower rate is the clock's and how much the kernel's.  bytes / clock / SM, and the rate that figure
+    gives at the maximum SM clock."""
+    mhz, mx = clocks.get("sm_mhz"), clocks.get("sm_max_mhz")
+    if not mhz or not mx:
+        return {}
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    per = achieved_gbs * 1e9 / (sms * mhz * 1e6)
+    return {"bytes_per_clk_per_sm": per, "achieved_at_max_sm_clock": per * sms * mx * 1e6 / 1e9, "sm_mhz": mhz}
+
+
 def rank_batch_permutation(nq: int, rank: int) -> torch.Tensor:
     """Which of the workload's queries, in which order, rank `rank` searches: a seeded permutation, so every
     replica works on its own batch and any rank's batch can be rebuilt elsewhere (CPU generator: the same on
@@ -321,7 +333,8 @@ def bench_ivfpq(tag, args, rank, world, local, dev, want_cpu_baseline):
                      "frac": achieved / pk["hbm"], "traffic": traffic,
                      "dram_frac": (traffic / (scan_ms / 1e3) / 1e9 / pk["hbm"]) if traffic else None,
                      "algorithmic_bytes_per_launch": scan_bytes, "kernel_ms": scan_ms,
-                     "scanned_vectors_per_query": scanned_vectors / nq},
+                     "scanned_vectors_per_query": scanned_vectors / nq,
+                     **_per_clock(achieved, clocks, dev)},
         "stage_ms": {kk: float(np.mean([s[kk] for s in stage_ms])) for kk in stage_ms[0]},
         "step_ms_p50": float(np.median(step_ms)), "step_ms_max": float(np.max(step_ms)),
     }

@@ -101,11 +101,16 @@ __global__ void __launch_bounds__(256) coarse_scores_kernel(const float* __restr
 }
 
 // ---- score matrix for tiny batches (the latency-bound iterative-retrieval shape) -------------------
-// For up to CS_MAXQ queries: a warp streams CS_CPW centroid rows at a time (16-byte loads) and keeps one partial sum
-// per (row, query), so the centroid table is read exactly once per batch however few queries there are.
+// For up to CS_MAXQ queries: a warp takes CS_CPW centroid rows at a time and keeps one partial sum per (row, query),
+// so the centroid table is read exactly once per batch however few queries there are.  The launch is latency-bound
+// (a few rows per warp).  NQ (1, 4 or 16) bounds the batch at compile time: the partial sums and their reduction
+// shrink with it, and the registers that frees go to loads in flight: with up to 4 queries a warp asks for
+// CS_CPW x 512 values per round before it multiplies any of them; with 16 it takes 128 values of each row per round
+// and has the next round's in flight while it multiplies (the sums alone take 64 registers).  The grid is sized so
+// that most warps have a single step.
 constexpr int CS_MAXQ = 16;
-constexpr int CS_CPW = 4;  // centroids per warp per step
-template <bool BF16>
+constexpr int CS_CPW = 4;    // centroids per warp per step
+template <bool BF16, int NQ>
 __global__ void __launch_bounds__(256) coarse_small_kernel(const float* __restrict__ Q, const void* __restrict__ C,
                                                            const float* __restrict__ cnorm, int nq, int nlist, int d,
                                                            int metric, float* __restrict__ scores) {
@@ -116,56 +121,77 @@ __global__ void __launch_bounds__(256) coarse_small_kernel(const float* __restri
     __syncthreads();
     const int lane = threadIdx.x & 31;
     const int warps = (gridDim.x * blockDim.x) >> 5;
-    // A warp takes CS_CPW consecutive centroids at a time: each query value read from shared memory serves CS_CPW
-    // rows, and the next slice of the rows is already in flight while the current one is multiplied.
     for (int c0 = ((blockIdx.x * blockDim.x + threadIdx.x) >> 5) * CS_CPW; c0 < nlist; c0 += warps * CS_CPW) {
-        float acc[CS_CPW][CS_MAXQ];
+        float acc[CS_CPW][NQ];
         float cn[CS_CPW];
 #pragma unroll
         for (int u = 0; u < CS_CPW; ++u) {
             cn[u] = metric == RAGO_L2 ? __ldg(cnorm + (c0 + u < nlist ? c0 + u : nlist - 1)) : 0.f;
 #pragma unroll
-            for (int qi = 0; qi < CS_MAXQ; ++qi) acc[u][qi] = 0.f;
+            for (int qi = 0; qi < NQ; ++qi) acc[u][qi] = 0.f;
         }
-        auto load_rows = [&](float4 (&cv)[CS_CPW], int j0) {
+        constexpr int CHUNK = NQ <= 4 ? 4 : 1;  // 16-byte (fp32) / 8-byte (bf16) loads per lane and row in one round
+        auto load_rows = [&](float4 (&cv)[CS_CPW][CHUNK], int jb) {
 #pragma unroll
             for (int u = 0; u < CS_CPW; ++u) {
                 const int c = c0 + u < nlist ? c0 + u : nlist - 1;  // rows past the end repeat the last one, unused
-                if (BF16) {
-                    const uint2 raw = *reinterpret_cast<const uint2*>(static_cast<const __nv_bfloat16*>(C) + (size_t)c * d + j0);
-                    cv[u].x = __uint_as_float(raw.x << 16); cv[u].y = __uint_as_float(raw.x & 0xFFFF0000u);
-                    cv[u].z = __uint_as_float(raw.y << 16); cv[u].w = __uint_as_float(raw.y & 0xFFFF0000u);
-                } else {
-                    cv[u] = *reinterpret_cast<const float4*>(static_cast<const float*>(C) + (size_t)c * d + j0);
+#pragma unroll
+                for (int h = 0; h < CHUNK; ++h) {
+                    const int j0 = jb + h * 128 + lane * 4;
+                    if (j0 < d) {
+                        if (BF16) {
+                            const uint2 raw = *reinterpret_cast<const uint2*>(static_cast<const __nv_bfloat16*>(C) + (size_t)c * d + j0);
+                            cv[u][h].x = __uint_as_float(raw.x << 16); cv[u][h].y = __uint_as_float(raw.x & 0xFFFF0000u);
+                            cv[u][h].z = __uint_as_float(raw.y << 16); cv[u][h].w = __uint_as_float(raw.y & 0xFFFF0000u);
+                        } else {
+                            cv[u][h] = *reinterpret_cast<const float4*>(static_cast<const float*>(C) + (size_t)c * d + j0);
+                        }
+                    } else {
+                        cv[u][h] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
                 }
             }
         };
-        float4 cv[CS_CPW], nx[CS_CPW];
-        if (lane * 4 < d) load_rows(cv, lane * 4);
-        for (int j0 = lane * 4; j0 < d; j0 += 128) {
-            const bool more = j0 + 128 < d;
-            if (more) load_rows(nx, j0 + 128);
+        float4 cv[CS_CPW][CHUNK], nx[CS_CPW][CHUNK];
+        load_rows(cv, 0);
+        for (int jb = 0; jb < d; jb += 128 * CHUNK) {
+            const bool more = jb + 128 * CHUNK < d;
+            if constexpr (CHUNK == 1) {  // next round's values in flight during this round's arithmetic
+                if (more) load_rows(nx, jb + 128 * CHUNK);
+            }
 #pragma unroll
-            for (int qi = 0; qi < CS_MAXQ; ++qi) {
-                if (qi < nq) {  // uniform
-                    const float4 qv = *reinterpret_cast<const float4*>(qs + qi * d + j0);
+            for (int h = 0; h < CHUNK; ++h) {
+                const int j0 = jb + h * 128 + lane * 4;
+                if (j0 < d) {
 #pragma unroll
-                    for (int u = 0; u < CS_CPW; ++u)
-                        acc[u][qi] = fmaf(qv.x, cv[u].x, fmaf(qv.y, cv[u].y, fmaf(qv.z, cv[u].z, fmaf(qv.w, cv[u].w, acc[u][qi]))));
+                    for (int qi = 0; qi < NQ; ++qi) {
+                        if (qi < nq) {  // uniform
+                            const float4 qv = *reinterpret_cast<const float4*>(qs + qi * d + j0);
+#pragma unroll
+                            for (int u = 0; u < CS_CPW; ++u)
+                                acc[u][qi] = fmaf(qv.x, cv[u][h].x, fmaf(qv.y, cv[u][h].y, fmaf(qv.z, cv[u][h].z, fmaf(qv.w, cv[u][h].w, acc[u][qi]))));
+                        }
+                    }
                 }
             }
             if (more) {
+                if constexpr (CHUNK == 1) {
 #pragma unroll
-                for (int u = 0; u < CS_CPW; ++u) cv[u] = nx[u];
+                    for (int u = 0; u < CS_CPW; ++u) cv[u][0] = nx[u][0];
+                } else {
+                    load_rows(cv, jb + 128 * CHUNK);
+                }
             }
         }
-        // Sum over the lanes, all CS_MAXQ queries of a row at once: at each halving a lane keeps the half of its
-        // values that its lane-number bit selects and hands over the other half, so 16 + 1 exchanges do the work of
-        // 16 x 5, and the total of query 8 b4 + 4 b3 + 2 b2 + b1 (lane bits) ends in the lanes with bit 0 clear.
+        // Sum over the lanes, all NQ queries of a row at once: at each halving a lane keeps the half of its values
+        // that its lane-number bit selects and hands over the other half (NQ - 1 exchanges instead of 5 NQ), then
+        // the single value left is summed over the remaining lane bits.  The total of the query whose number is
+        // the leading log2(NQ) lane bits ends in the lanes whose other bits are clear.
 #pragma unroll
         for (int u = 0; u < CS_CPW; ++u) {
+            int o = 16;
 #pragma unroll
-            for (int half = CS_MAXQ / 2, o = 16; half >= 1; half >>= 1, o >>= 1) {
+            for (int half = NQ / 2; half >= 1; half >>= 1, o >>= 1) {
                 const bool upper = (lane & o) != 0;
 #pragma unroll
                 for (int i = 0; i < half; ++i) {
@@ -174,25 +200,39 @@ __global__ void __launch_bounds__(256) coarse_small_kernel(const float* __restri
                     acc[u][i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
                 }
             }
-            const float v = acc[u][0] + __shfl_xor_sync(0xffffffffu, acc[u][0], 1);
-            const int qi = (lane >> 1) & 15;  // bits 4..1 of the lane, most significant first: 8 b4 + 4 b3 + 2 b2 + b1
-            if ((lane & 1) == 0 && qi < nq && c0 + u < nlist)
+            float v = acc[u][0];
+#pragma unroll
+            for (; o >= 1; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+            constexpr int REST = 32 / NQ;  // lanes that end up with the same query's total
+            const int qi = NQ == 1 ? 0 : (lane / REST);
+            if ((lane & (REST - 1)) == 0 && qi < nq && c0 + u < nlist)
                 scores[(size_t)qi * nlist + c0 + u] = metric == RAGO_L2 ? fmaf(-2.f, v, cn[u]) : -v;
         }
     }
+}
+
+template <bool BF16>
+static void launch_coarse_small(const IndexImpl* ix, const float* queries, int nq, float* scores, int blocks, size_t qbytes,
+                                cudaStream_t s) {
+    if (nq == 1)
+        launch_overlapped(coarse_small_kernel<BF16, 1>, dim3(blocks), dim3(256), qbytes, s, queries, ix->centroids, ix->cnorm,
+                          nq, ix->nlist, ix->d, ix->metric, scores);
+    else if (nq <= 4)
+        launch_overlapped(coarse_small_kernel<BF16, 4>, dim3(blocks), dim3(256), qbytes, s, queries, ix->centroids, ix->cnorm,
+                          nq, ix->nlist, ix->d, ix->metric, scores);
+    else
+        launch_overlapped(coarse_small_kernel<BF16, CS_MAXQ>, dim3(blocks), dim3(256), qbytes, s, queries, ix->centroids,
+                          ix->cnorm, nq, ix->nlist, ix->d, ix->metric, scores);
 }
 
 cudaError_t launch_coarse_scores(const IndexImpl* ix, const float* queries, int nq, float* scores, cudaStream_t s) {
     const size_t qbytes = (size_t)nq * ix->d * 4;
     if (nq <= CS_MAXQ && qbytes <= 48 * 1024) {
         const int want = (ix->nlist + 8 * CS_CPW - 1) / (8 * CS_CPW);  // 8 warps per CTA, CS_CPW rows per warp step
-        const int blocks = want < ix->num_sms * 2 ? want : ix->num_sms * 2;
-        if (ix->coarse_bf16)
-            launch_overlapped(coarse_small_kernel<true>, dim3(blocks), dim3(256), qbytes, s, queries, ix->centroids, ix->cnorm,
-                              nq, ix->nlist, ix->d, ix->metric, scores);
-        else
-            launch_overlapped(coarse_small_kernel<false>, dim3(blocks), dim3(256), qbytes, s, queries, ix->centroids, ix->cnorm,
-                              nq, ix->nlist, ix->d, ix->metric, scores);
+        const int cap = ix->num_sms * (nq <= 4 ? 4 : 2);
+        const int blocks = want < cap ? want : cap;
+        if (ix->coarse_bf16) launch_coarse_small<true>(ix, queries, nq, scores, blocks, qbytes, s);
+        else launch_coarse_small<false>(ix, queries, nq, scores, blocks, qbytes, s);
         count_launch();
         return cudaGetLastError();
     }

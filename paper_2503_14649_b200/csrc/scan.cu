@@ -185,7 +185,9 @@ __host__ __device__ inline SmemPlan plan_smem(uint32_t base, uint32_t dyn_bytes,
     for (int s = 0; s < MAX_STAGES; ++s) p.tile[s] = s < stages ? take(C::TILE_BYTES, 128) : base;
     p.keys = take(C::KCAP * 8, 16);
     for (int s = 0; s < MAX_STAGES; ++s) p.vt[s] = (s < stages && need_vt) ? take(C::VT_BYTES, 16) : base;
-    p.rT = take((uint32_t)d * 4, 16);
+    // The scaled, transposed query is only alive while a table is built, when the candidate buffer is empty: it
+    // shares the buffer's space when it fits there.
+    p.rT = (uint32_t)d * 4 <= (uint32_t)C::KCAP * 8 ? p.keys : take((uint32_t)d * 4, 16);
     p.ctrl = take(CTRL_BYTES, 16);
     return p;
 }
@@ -760,7 +762,7 @@ static const Variant kVariants[] = {
     RAGO_VARIANT(8, 8, 1, 10, 3),   // M = 32
     RAGO_VARIANT(12, 4, 1, 8, 2),   // M = 48
     RAGO_VARIANT(8, 8, 2, 15, 4),   // M = 64: 15 + 1 warps fill the four schedulers evenly; two 60 KB tiles below the table
-    RAGO_VARIANT(8, 8, 2, 12, 4),   // M = 64 where those do not fit (per-vector terms, d > 768)
+    RAGO_VARIANT(8, 8, 2, 12, 4),   // M = 64 where those do not fit
     RAGO_VARIANT(20, 4, 1, 8, 1),   // M = 80
     RAGO_VARIANT(24, 8, 1, 12, 1),  // M = 96
     RAGO_VARIANT(8, 8, 4, 12, 3),   // M = 128

@@ -78,6 +78,23 @@ def test_small_cases_match_oracle(case):
     _compare(data, nprobe, k)
 
 
+LARGE_BATCH_CASES = [
+    # N, d, nlist, M, nprobe, k, metric: batches above the limit up to which lookup tables are built by a kernel of
+    # their own; beyond it every scan CTA builds the table of each query it meets
+    (2500, 64, 8, 16, 2, 5, "l2"),
+    (2500, 128, 8, 64, 2, 5, "ip"),     # dsub = 2: the generic table builder
+    (2500, 512, 8, 64, 2, 5, "l2"),     # dsub = 8
+    (2500, 384, 8, 96, 2, 5, "l2"),     # dsub = 4
+]
+
+
+@pytest.mark.parametrize("case", LARGE_BATCH_CASES, ids=lambda c: "d%d_M%d_%s" % (c[1], c[3], c[6]))
+def test_batch_above_the_prebuilt_table_limit(case):
+    N, d, nlist, M, nprobe, k, metric = case
+    data = synth.make_ivfpq(N, d, nlist, M, 4200, metric=metric, seed=300 + d + M)
+    _compare(data, nprobe, k, max_probe_mismatch=8)
+
+
 def test_empty_lists_and_short_lists():
     data = synth.make_ivfpq(900, 64, 16, 16, 8, metric="l2", seed=5)
     # empty every other list by moving its vectors to the next one
