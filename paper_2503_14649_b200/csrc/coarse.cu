@@ -426,8 +426,10 @@ constexpr int SEL_MAX_SPLIT = 512;  // candidate lists per query the kernel can 
 // batches (latency), a small one when there are enough queries to fill the GPU.
 // FROM_SCORES: the items are a row of the score matrix (else the candidate lists the GEMM left).  The two sources
 // are separate instantiations because the kernel body runs once per CTA, largely unrolled: its size is what a
-// small batch pays for, in instruction fetches.
-template <bool BF16, int SEL_THREADS, int SEL_REG, bool FROM_SCORES>
+// small batch pays for, in instruction fetches.  For the same reason ALL_REGS (the launcher knows that every item
+// fits the registers: a score row of at most SEL_REG x SEL_THREADS lists) leaves out the re-reading variants of
+// every phase, and the refinement of an oversized tie group always re-reads its items, as one compact loop.
+template <bool BF16, int SEL_THREADS, int SEL_REG, bool FROM_SCORES, bool ALL_REGS>
 __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
     const float* __restrict__ Q, const void* __restrict__ C, const float* __restrict__ scores,
     const unsigned long long* __restrict__ cand, const int32_t* __restrict__ cand_cnt, uint32_t cand_sign, int nsplit,
@@ -470,7 +472,7 @@ __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
         }
         return cand_key(cand[((size_t)q * nsplit + lo_s) * cap + (l - pre[lo_s])], cand_sign);
     };
-    const bool in_regs = nitems <= SEL_REG * SEL_THREADS;
+    const bool in_regs = ALL_REGS || nitems <= SEL_REG * SEL_THREADS;
     uint32_t mine[SEL_REG];  // ordered score bits; 0xFFFFFFFF marks an empty slot
     uint32_t mn = 0xFFFFFFFFu, mx = 0u, nvalid = 0;
     if (in_regs) {
@@ -584,11 +586,6 @@ __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
     // payload P, so that at most nsel + slack are collected and they include the nsel smallest keys.
     uint32_t P = 0xFFFFFFFFu;
     if (c_hi > (uint32_t)TOPK_CAP) {  // uniform
-        auto payload_of = [&](int l, int j) -> uint32_t {
-            (void)j;
-            if constexpr (FROM_SCORES) return (uint32_t)l;
-            else return (uint32_t)(item(l) & 0xFFFFFFFFull);
-        };
         auto count_cta = [&](uint32_t c) -> uint32_t {  // sum of c over the CTA, same value in every thread
             c = __reduce_add_sync(0xffffffffu, c);
             const int slot = round % 3;
@@ -599,14 +596,9 @@ __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
             return s_round[slot];
         };
         uint32_t less = 0;
-        if (in_regs) {
-#pragma unroll
-            for (int j = 0; j < SEL_REG; ++j) less += mine[j] < T ? 1u : 0u;
-        } else {
-            for (int l = tid; l < nitems; l += SEL_THREADS) {
-                const unsigned long long k = item(l);
-                less += (k != KEY_MAX && (uint32_t)(k >> 32) < T) ? 1u : 0u;
-            }
+        for (int l = tid; l < nitems; l += SEL_THREADS) {
+            const unsigned long long k = item(l);
+            less += (k != KEY_MAX && (uint32_t)(k >> 32) < T) ? 1u : 0u;
         }
         less = count_cta(less);
         const uint32_t need = (uint32_t)nsel - less;  // >= 1: fewer than nsel items lie below T
@@ -615,17 +607,9 @@ __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
         while (phi - plo > 1 && pc_hi > need + (uint32_t)slack) {  // uniform
             const uint32_t mid = (uint32_t)(plo + (phi - plo) / 2);
             uint32_t c = 0;
-            if (in_regs) {
-#pragma unroll
-                for (int j = 0; j < SEL_REG; ++j) {
-                    const int l = tid + j * SEL_THREADS;
-                    if (mine[j] == T && l < nitems && payload_of(l, j) <= mid) ++c;
-                }
-            } else {
-                for (int l = tid; l < nitems; l += SEL_THREADS) {
-                    const unsigned long long k = item(l);
-                    if (k != KEY_MAX && (uint32_t)(k >> 32) == T && (uint32_t)k <= mid) ++c;
-                }
+            for (int l = tid; l < nitems; l += SEL_THREADS) {
+                const unsigned long long k = item(l);
+                if (k != KEY_MAX && (uint32_t)(k >> 32) == T && (uint32_t)k <= mid) ++c;
             }
             c = count_cta(c);
             if (c < need) plo = mid; else { phi = mid; pc_hi = c; }
@@ -721,12 +705,16 @@ template <bool BF16, int THREADS, int REG>
 static void launch_select_source(const IndexImpl* ix, const float* queries, const float* scores,
                                  const unsigned long long* cand, const int32_t* cand_cnt, uint32_t cand_sign, int nsplit, int cap, int nq,
                                  int nprobe, int32_t* probe_list, float* probe_term, float* probe_bias, cudaStream_t s) {
-    if (scores)
-        launch_overlapped(select_probes_kernel<BF16, THREADS, REG, true>, dim3(nq), dim3(THREADS), 0, s,
+    if (scores && ix->nlist <= THREADS * REG)
+        launch_overlapped(select_probes_kernel<BF16, THREADS, REG, true, true>, dim3(nq), dim3(THREADS), 0, s,
+            queries, ix->centroids, scores, cand, cand_cnt, cand_sign, nsplit, cap, ix->nlist, ix->d, ix->metric, nprobe, probe_list,
+            probe_term, probe_bias);
+    else if (scores)
+        launch_overlapped(select_probes_kernel<BF16, THREADS, REG, true, false>, dim3(nq), dim3(THREADS), 0, s,
             queries, ix->centroids, scores, cand, cand_cnt, cand_sign, nsplit, cap, ix->nlist, ix->d, ix->metric, nprobe, probe_list,
             probe_term, probe_bias);
     else
-        launch_overlapped(select_probes_kernel<BF16, THREADS, REG, false>, dim3(nq), dim3(THREADS), 0, s,
+        launch_overlapped(select_probes_kernel<BF16, THREADS, REG, false, false>, dim3(nq), dim3(THREADS), 0, s,
             queries, ix->centroids, scores, cand, cand_cnt, cand_sign, nsplit, cap, ix->nlist, ix->d, ix->metric, nprobe, probe_list,
             probe_term, probe_bias);
 }

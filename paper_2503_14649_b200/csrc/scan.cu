@@ -755,12 +755,14 @@ static int stages_for(int d, bool need_vt) {
       Cfg<WV, G, R, NCW, RGW>::BANKED ? 1 : 0, Cfg<WV, G, R, NCW, RGW>::COPIES, Cfg<WV, G, R, NCW, RGW>::COPY_OFF, \
       Cfg<WV, G, R, NCW, RGW>::LSTRIDE }
 // Warps x unrolled row groups per warp were chosen by measurement: independent row groups in flight inside a warp
-// hide the look-up latency better than more warps do (M = 64: 16 x 2 -> 12 x 4 gave +30%).  Where a code size has
-// two entries the first one whose shared-memory plan fits the index (dimension, metric) is taken.
+// hide the look-up latency better than more warps do (M = 64: 16 x 2 -> 12 x 4 gave +30%), and 15 consumer warps
+// (four warps on every scheduler, the producer included) beat 12, 14 and 16 wherever their tiles fit (M = 32: +3%,
+// M = 48: +6%, M = 64: +4.5%).  Where a code size has two entries the first one whose shared-memory plan fits the
+// index (dimension, metric) is taken.
 static const Variant kVariants[] = {
     RAGO_VARIANT(4, 4, 1, 16, 2),   // M = 16
-    RAGO_VARIANT(8, 8, 1, 10, 3),   // M = 32
-    RAGO_VARIANT(12, 4, 1, 8, 2),   // M = 48
+    RAGO_VARIANT(8, 8, 1, 15, 2),   // M = 32
+    RAGO_VARIANT(12, 4, 1, 15, 1),  // M = 48 (two table copies: 128 KB, a 2 048-key buffer, tiles of at most 512 vectors)
     RAGO_VARIANT(8, 8, 2, 15, 4),   // M = 64: 15 + 1 warps fill the four schedulers evenly; two 60 KB tiles below the table
     RAGO_VARIANT(8, 8, 2, 12, 4),   // M = 64 where those do not fit
     RAGO_VARIANT(20, 4, 1, 8, 1),   // M = 80
