@@ -687,10 +687,13 @@ cudaError_t launch_gemm_select(const GemmLaunch& L, cudaStream_t s) {
 }
 
 // ---- pilot thresholds: per row, a value with at least nsel of the row's n sample scores at or below it --------
-// One CTA per row: the row is read once into shared memory (as ordered score bits), then bisected between its
-// minimum and maximum with CTA-wide counts; the search stops as soon as the count lies in
-// [nsel, nsel + nsel/4] and returns the next representable value above the cut, so that "score < tau" keeps
-// ties of the cut itself.
+// One CTA per row: the row is read once (as ordered score bits), then bisected between its minimum and maximum
+// with CTA-wide counts; the search stops as soon as the count lies in [nsel, nsel + nsel/4] and returns the next
+// representable value above the cut, so that "score < tau" keeps ties of the cut itself.
+// A row that fits the registers and gives every warp enough values is not bisected CTA-wide: each of the W warps
+// bisects its own share for a value with at least ceil(nsel / W) of its values at or below it (warp-wide counts,
+// no barrier), and the row's threshold is the largest of the W values: at least nsel sample scores lie at or below
+// it, which is all a threshold has to guarantee; it is a little looser than the sample's exact nsel-th smallest.
 constexpr int RT_THREADS = 256;
 constexpr int RT_REG = 16;  // values a thread keeps in registers (rows of up to RT_REG * RT_THREADS scores)
 template <bool IN_REGS>
@@ -719,6 +722,36 @@ __global__ void __launch_bounds__(RT_THREADS) row_tau_kernel(const float* __rest
     }
     mn = __reduce_min_sync(0xffffffffu, mn);
     mx = __reduce_max_sync(0xffffffffu, mx);
+    if (IN_REGS) {
+        constexpr int W = RT_THREADS / 32;
+        const int m = (nsel + W - 1) / W;
+        // values are dealt out round-robin by thread: the last warp holds the fewest
+        const int fewest = (n / RT_THREADS) * 32 + (n % RT_THREADS > RT_THREADS - 32 ? n % RT_THREADS - (RT_THREADS - 32) : 0);
+        if (fewest >= m) {  // uniform
+            uint32_t nv = 0;
+#pragma unroll
+            for (int j = 0; j < RT_REG; ++j) nv += tid + j * RT_THREADS < n ? 1u : 0u;
+            uint32_t c_hi = __reduce_add_sync(0xffffffffu, nv);
+            long long lo = (long long)mn - 1, hi = mx;  // #(<= lo) < m <= #(<= hi), within the warp
+            const uint32_t want_max = (uint32_t)(m + m / 4);
+            while (hi - lo > 1 && c_hi > want_max) {  // uniform within the warp
+                const uint32_t mid = (uint32_t)(lo + (hi - lo) / 2);
+                uint32_t c = 0;
+#pragma unroll
+                for (int j = 0; j < RT_REG; ++j) c += mine[j] <= mid ? 1u : 0u;  // padding holds the largest pattern
+                c = __reduce_add_sync(0xffffffffu, c);
+                if (c < (uint32_t)m) lo = mid; else { hi = mid; c_hi = c; }
+            }
+            if (lane == 0) red[0][warp] = (uint32_t)hi;
+            __syncthreads();
+            if (tid == 0) {
+                uint32_t T = red[0][0];
+                for (int w = 1; w < W; ++w) T = red[0][w] > T ? red[0][w] : T;
+                row_tau[row] = T == 0xFFFFFFFFu ? orderable_f32(T) : orderable_f32(T + 1u);
+            }
+            return;
+        }
+    }
     if (lane == 0) { red[0][warp] = mn; red[1][warp] = mx; }
     __syncthreads();
     mn = red[0][0]; mx = red[1][0];
