@@ -7,7 +7,7 @@
 #include <new>
 #include <vector>
 
-#include "common.cuh"
+#include "plan.cuh"
 
 namespace rago {
 
@@ -152,8 +152,9 @@ static void record(IndexImpl* ix, int i, cudaStream_t s) {
     if (ix->profile) cudaEventRecord(ix->ev[i], s);
 }
 
+// fp (may be null): the selection kernel also plans the scan and builds the lookup tables (small batches).
 static rago_status run_coarse(const IndexImpl* ix, const float* queries, int nq, int nprobe, uint8_t* ws,
-                              const Layout& L, cudaStream_t s) {
+                              const Layout& L, const FusedPlan* fp, cudaStream_t s) {
     IndexImpl* mix = const_cast<IndexImpl*>(ix);
     cudaError_t e;
     int32_t* probe_list = reinterpret_cast<int32_t*>(ws + L.probe_list);
@@ -168,7 +169,7 @@ static rago_status run_coarse(const IndexImpl* ix, const float* queries, int nq,
         if (e != cudaSuccess) return cuda_fail(e, "two-level coarse kernel");
         record(mix, 1, s);
         e = launch_select_probes_cand(ix, queries, cand, cand_cnt, 0u, L.tree_S, L.tree_cap, nq, nprobe, probe_list,
-                                      probe_term, probe_bias, s);
+                                      probe_term, probe_bias, fp, s);
     } else if (L.tc) {
         // queries -> stacked bf16 parts, then the tensor-core kernel with the selection fused in
         const int parts = ix->cparts_n;
@@ -222,14 +223,14 @@ static rago_status run_coarse(const IndexImpl* ix, const float* queries, int nq,
         if (L.tc_mode == 0)
             e = launch_select_probes_cand(ix, queries, G.cand, G.cand_cnt, gemm_cand_sign(G.alpha, G.colterm),
                                           L.tc_nsplit * GEMM_COL_HALVES, L.tc_cap, nq, nprobe, probe_list,
-                                          probe_term, probe_bias, s);
+                                          probe_term, probe_bias, fp, s);
         else
-            e = launch_select_probes(ix, queries, scores, nq, nprobe, probe_list, probe_term, probe_bias, s);
+            e = launch_select_probes(ix, queries, scores, nq, nprobe, probe_list, probe_term, probe_bias, fp, s);
     } else {
         e = launch_coarse_scores(ix, queries, nq, scores, s);
         if (e != cudaSuccess) return cuda_fail(e, "coarse score kernel");
         record(mix, 1, s);
-        e = launch_select_probes(ix, queries, scores, nq, nprobe, probe_list, probe_term, probe_bias, s);
+        e = launch_select_probes(ix, queries, scores, nq, nprobe, probe_list, probe_term, probe_bias, fp, s);
     }
     if (e != cudaSuccess) return cuda_fail(e, "probe selection kernel");
     record(mix, 2, s);
@@ -385,7 +386,7 @@ rago_status rago_search_probes(const rago_index* index, const float* queries, in
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     cudaError_t e = cudaMemsetAsync(ws + L.err, 0, 256, s);
     if (e != cudaSuccess) return cuda_fail(e, "clearing the error word");
-    st = run_coarse(ix, queries, nq, nprobe, ws, L, s);
+    st = run_coarse(ix, queries, nq, nprobe, ws, L, nullptr, s);
     if (st != RAGO_OK) return st;
     const size_t bytes = (size_t)nq * nprobe * 4;
     e = cudaMemcpyAsync(out_lists, ws + L.probe_list, bytes, cudaMemcpyDeviceToDevice, s);
@@ -415,23 +416,29 @@ rago_status rago_search(const rago_index* index, const float* queries, int32_t n
 
     cudaError_t e = cudaMemsetAsync(ws + L.err, 0, 256, s);
     if (e != cudaSuccess) return cuda_fail(e, "clearing the error word");
-    st = run_coarse(ix, queries, nq, nprobe, ws, L, s);
-    if (st != RAGO_OK) return st;
-
     int32_t* probe_list = reinterpret_cast<int32_t*>(ws + L.probe_list);
     float* probe_term = reinterpret_cast<float*>(ws + L.probe_bias);  // what the scan adds per (query, list)
     int64_t* work_prefix = reinterpret_cast<int64_t*>(ws + L.work_prefix);
     unsigned long long* qthresh = reinterpret_cast<unsigned long long*>(ws + L.qthresh);
     int32_t* slot_cnt = reinterpret_cast<int32_t*>(ws + L.slot_cnt);
     unsigned long long* slot_keys = reinterpret_cast<unsigned long long*>(ws + L.slot_keys);
-
-    // small batches: the lookup tables are built ahead of the scan, by CTAs of the planning launch
+    // small batches: the lookup tables are built ahead of the scan
     uint8_t* lut_img = L.prebuilt ? ws + L.lut_img : nullptr;
     float* lut_inv = L.prebuilt ? reinterpret_cast<float*>(ws + L.lut_inv) : nullptr;
-    e = launch_plan_work(ix, probe_list, npairs, ix->plan.tile_vecs, reinterpret_cast<int32_t*>(ws + L.pair_tiles),
-                         work_prefix, qthresh, nq, slot_cnt, (int)L.nslots, queries, lut_img, lut_inv,
-                         L.prebuilt ? reinterpret_cast<float*>(ws + L.lut_scale) : nullptr, s);
-    if (e != cudaSuccess) return cuda_fail(e, "work planning");
+
+    // Batches of at most 64 queries: the selection launch also builds the tables and plans the scan (its last CTA
+    // to finish), one launch less on the latency-bound path.  The ticket word lies in the block cleared above.
+    FusedPlan fp;
+    const bool fused = fused_plan_args(ix, nq, npairs, queries, lut_img, lut_inv, work_prefix, qthresh, slot_cnt,
+                                       (int)L.nslots, reinterpret_cast<uint32_t*>(ws + L.err) + ERR_TICKET_WORD, &fp);
+    st = run_coarse(ix, queries, nq, nprobe, ws, L, fused ? &fp : nullptr, s);
+    if (st != RAGO_OK) return st;
+    if (!fused) {
+        e = launch_plan_work(ix, probe_list, npairs, ix->plan.tile_vecs, reinterpret_cast<int32_t*>(ws + L.pair_tiles),
+                             work_prefix, qthresh, nq, slot_cnt, (int)L.nslots, queries, lut_img, lut_inv,
+                             L.prebuilt ? reinterpret_cast<float*>(ws + L.lut_scale) : nullptr, s);
+        if (e != cudaSuccess) return cuda_fail(e, "work planning");
+    }
     record(mix, 3, s);
     e = launch_scan(ix, ix->plan, queries, probe_list, probe_term, work_prefix, nq, nprobe, k, qthresh, slot_cnt,
                     slot_keys, reinterpret_cast<uint32_t*>(ws + L.err), lut_img, lut_inv, s);

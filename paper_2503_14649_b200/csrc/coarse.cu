@@ -4,6 +4,9 @@
 // The nprobe + PROBE_GUARD best lists by that score are re-scored exactly (sum of (q-c)^2, or <q,c>)
 // before the final cut, so the probe order follows the plain definition up to fp32 rounding.
 // With a bf16 coarse quantiser the query is rounded to bf16 first (coarse step only).
+#include <cstring>
+
+#include "plan.cuh"
 #include "topk.cuh"
 
 namespace rago {
@@ -434,7 +437,8 @@ __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
     const float* __restrict__ Q, const void* __restrict__ C, const float* __restrict__ scores,
     const unsigned long long* __restrict__ cand, const int32_t* __restrict__ cand_cnt, uint32_t cand_sign, int nsplit,
     int cap, int nlist, int d, int metric, int nprobe, int32_t* __restrict__ probe_list,
-    float* __restrict__ probe_term, float* __restrict__ probe_bias) {
+    float* __restrict__ probe_term, float* __restrict__ probe_bias, const FusedPlan fp) {
+    extern __shared__ float fp_smem[];  // fused planning only: the table builders' d + M floats
     __shared__ unsigned long long keys[TOPK_CAP];
     __shared__ unsigned long long keys2[MAX_K + PROBE_GUARD];
     __shared__ int pre[SEL_MAX_SPLIT + 1];  // candidate path: exclusive prefix of the lists' counts
@@ -448,6 +452,13 @@ __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
     auto sync = [] { __syncthreads(); };
     grid_dependency_wait();
     grid_dependents_may_launch();
+    if constexpr (SEL_THREADS == PFX_THREADS) {
+        if (fp.enabled && q >= fp.nq) {  // uniform: this CTA builds a part of a lookup table (queries only: no ordering needed)
+            const int b = q - fp.nq;
+            build_table_part(fp.tables, b / fp.table_parts, b % fp.table_parts, fp.table_parts, fp_smem);
+            return;
+        }
+    }
     int nsel = nprobe + PROBE_GUARD;
     if (nsel > nlist) nsel = nlist;
     if (tid == 0) { cnt = 0; s_mn = 0xFFFFFFFFu; s_mx = 0u; s_nv = 0u; s_round[0] = s_round[1] = s_round[2] = 0u; }
@@ -699,62 +710,89 @@ __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
             if (lane == 0) probe_bias[(size_t)q * nprobe + i] = acc;
         }
     }
+    // Fused planning: the CTA that finishes its query last (a ticket, nothing waits) plans the scan of the batch.
+    if constexpr (SEL_THREADS == PFX_THREADS) {
+        if (fp.enabled) {  // uniform
+            __shared__ int s_last;
+            __shared__ long long plan_sums[32];
+            __threadfence();  // this query's probe lists before the ticket
+            __syncthreads();
+            if (tid == 0) s_last = atomicAdd(fp.ticket, 1u) == (uint32_t)(fp.nq - 1) ? 1 : 0;
+            __syncthreads();
+            if (s_last) {
+                __threadfence();  // the other queries' probe lists after their tickets
+                plan_pairs_cta(probe_list, fp.offsets, fp.nq * nprobe, fp.tile_vecs, fp.prefix, fp.qthresh, fp.nq,
+                               fp.slot_cnt, fp.nslots, plan_sums);
+                if (tid == 0) *fp.ticket = 0u;
+            }
+        }
+    }
 }
 
 template <bool BF16, int THREADS, int REG>
 static void launch_select_source(const IndexImpl* ix, const float* queries, const float* scores,
                                  const unsigned long long* cand, const int32_t* cand_cnt, uint32_t cand_sign, int nsplit, int cap, int nq,
-                                 int nprobe, int32_t* probe_list, float* probe_term, float* probe_bias, cudaStream_t s) {
+                                 int nprobe, int32_t* probe_list, float* probe_term, float* probe_bias, const FusedPlan& fp, cudaStream_t s) {
+    const dim3 grid(fp.enabled ? nq * (1 + fp.table_parts) : nq);
+    const size_t smem = fp.enabled ? (size_t)(ix->d + ix->M) * 4 : 0;
     if (scores && ix->nlist <= THREADS * REG)
-        launch_overlapped(select_probes_kernel<BF16, THREADS, REG, true, true>, dim3(nq), dim3(THREADS), 0, s,
+        launch_overlapped(select_probes_kernel<BF16, THREADS, REG, true, true>, grid, dim3(THREADS), smem, s,
             queries, ix->centroids, scores, cand, cand_cnt, cand_sign, nsplit, cap, ix->nlist, ix->d, ix->metric, nprobe, probe_list,
-            probe_term, probe_bias);
+            probe_term, probe_bias, fp);
     else if (scores)
-        launch_overlapped(select_probes_kernel<BF16, THREADS, REG, true, false>, dim3(nq), dim3(THREADS), 0, s,
+        launch_overlapped(select_probes_kernel<BF16, THREADS, REG, true, false>, grid, dim3(THREADS), smem, s,
             queries, ix->centroids, scores, cand, cand_cnt, cand_sign, nsplit, cap, ix->nlist, ix->d, ix->metric, nprobe, probe_list,
-            probe_term, probe_bias);
+            probe_term, probe_bias, fp);
     else
-        launch_overlapped(select_probes_kernel<BF16, THREADS, REG, false, false>, dim3(nq), dim3(THREADS), 0, s,
+        launch_overlapped(select_probes_kernel<BF16, THREADS, REG, false, false>, grid, dim3(THREADS), smem, s,
             queries, ix->centroids, scores, cand, cand_cnt, cand_sign, nsplit, cap, ix->nlist, ix->d, ix->metric, nprobe, probe_list,
-            probe_term, probe_bias);
+            probe_term, probe_bias, fp);
 }
 template <int THREADS, int REG>
 static void launch_select_shape(const IndexImpl* ix, const float* queries, const float* scores,
                                 const unsigned long long* cand, const int32_t* cand_cnt, uint32_t cand_sign, int nsplit, int cap, int nq,
-                                int nprobe, int32_t* probe_list, float* probe_term, float* probe_bias, cudaStream_t s) {
+                                int nprobe, int32_t* probe_list, float* probe_term, float* probe_bias, const FusedPlan& fp,
+                                cudaStream_t s) {
     if (ix->coarse_bf16)
         launch_select_source<true, THREADS, REG>(ix, queries, scores, cand, cand_cnt, cand_sign, nsplit, cap, nq, nprobe, probe_list,
-                                                 probe_term, probe_bias, s);
+                                                 probe_term, probe_bias, fp, s);
     else
         launch_select_source<false, THREADS, REG>(ix, queries, scores, cand, cand_cnt, cand_sign, nsplit, cap, nq, nprobe, probe_list,
-                                                  probe_term, probe_bias, s);
+                                                  probe_term, probe_bias, fp, s);
 }
+// fp (may be null): the kernel also plans the scan of the batch and builds its lookup tables (batches of at most 64
+// queries, which run the 1024-thread shape).
 static cudaError_t launch_select_any(const IndexImpl* ix, const float* queries, const float* scores,
                                      const unsigned long long* cand, const int32_t* cand_cnt, uint32_t cand_sign, int nsplit, int cap, int nq,
                                      int nprobe, int32_t* probe_list, float* probe_term, float* probe_bias,
-                                     cudaStream_t s) {
+                                     const FusedPlan* fp, cudaStream_t s) {
     if (nsplit > SEL_MAX_SPLIT) return cudaErrorInvalidValue;
+    FusedPlan off;
+    std::memset(&off, 0, sizeof(off));
+    if (fp && fp->enabled && nq > 64) return cudaErrorInvalidValue;
     if (nq <= 64)
         launch_select_shape<1024, 16>(ix, queries, scores, cand, cand_cnt, cand_sign, nsplit, cap, nq, nprobe, probe_list, probe_term,
-                                      probe_bias, s);
+                                      probe_bias, fp ? *fp : off, s);
     else
         launch_select_shape<256, 20>(ix, queries, scores, cand, cand_cnt, cand_sign, nsplit, cap, nq, nprobe, probe_list, probe_term,
-                                     probe_bias, s);
+                                     probe_bias, off, s);
     count_launch();
     return cudaGetLastError();
 }
 
 cudaError_t launch_select_probes(const IndexImpl* ix, const float* queries, const float* scores, int nq, int nprobe,
-                                 int32_t* probe_list, float* probe_term, float* probe_bias, cudaStream_t s) {
+                                 int32_t* probe_list, float* probe_term, float* probe_bias, const FusedPlan* fp,
+                                 cudaStream_t s) {
     return launch_select_any(ix, queries, scores, nullptr, nullptr, 0u, 0, 0, nq, nprobe, probe_list, probe_term,
-                             probe_bias, s);
+                             probe_bias, fp, s);
 }
 
 cudaError_t launch_select_probes_cand(const IndexImpl* ix, const float* queries, const unsigned long long* cand,
                                       const int32_t* cand_cnt, uint32_t cand_sign, int nsplit, int cap, int nq, int nprobe,
-                                      int32_t* probe_list, float* probe_term, float* probe_bias, cudaStream_t s) {
+                                      int32_t* probe_list, float* probe_term, float* probe_bias, const FusedPlan* fp,
+                                      cudaStream_t s) {
     return launch_select_any(ix, queries, nullptr, cand, cand_cnt, cand_sign, nsplit, cap, nq, nprobe, probe_list, probe_term,
-                             probe_bias, s);
+                             probe_bias, fp, s);
 }
 
 }  // namespace rago

@@ -17,6 +17,7 @@ constexpr unsigned long long KEY_MAX = 0xFFFFFFFFFFFFFFFFull;
 
 // Device-side error word (first word of every workspace).
 enum : uint32_t { ERR_NONE = 0, ERR_WAIT_TIMEOUT = 1, ERR_SMEM_LAYOUT = 2 };
+constexpr int ERR_TICKET_WORD = 16;  // word of the 256-byte error block (cleared by every call) that small batches use as a ticket counter
 
 // Launch shape of the table-build + scan kernel for one index (fixed at index load).
 struct ScanPlan {
@@ -207,14 +208,9 @@ void set_error(const char* fmt, ...);
 // coarse.cu
 cudaError_t launch_centroid_norms(const void* centroids, int bf16, int nlist, int d, float* cnorm, cudaStream_t s);
 cudaError_t launch_coarse_scores(const IndexImpl* ix, const float* queries, int nq, float* scores, cudaStream_t s);
-cudaError_t launch_select_probes(const IndexImpl* ix, const float* queries, const float* scores, int nq, int nprobe,
-                                 int32_t* probe_list, float* probe_term, float* probe_bias, cudaStream_t s);
 cudaError_t launch_tree_candidates(const IndexImpl* ix, const float* queries, int nq, int S, int cap,
                                    unsigned long long* cand, int32_t* cand_cnt, cudaStream_t s);
 constexpr int TREE_LIMIT_B1 = 64, TREE_LIMIT_N1 = 4096;
-cudaError_t launch_select_probes_cand(const IndexImpl* ix, const float* queries, const unsigned long long* cand,
-                                      const int32_t* cand_cnt, uint32_t cand_sign, int nsplit, int cap, int nq, int nprobe,
-                                      int32_t* probe_list, float* probe_term, float* probe_bias, cudaStream_t s);
 // gemm_select.cu
 constexpr int GEMM_CAP_SMALL = 512, GEMM_CAP_LARGE = 1024;  // candidate-list capacities (keys per list)
 constexpr int GEMM_COL_HALVES = 2;  // a row has one candidate list per column range of the grid AND per half of a 256-column tile

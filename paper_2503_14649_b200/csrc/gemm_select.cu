@@ -49,6 +49,7 @@
 // Every wait is bounded (common.cuh); on a timeout the roles leave their loops, the error word is
 // set, TMEM is still released.
 #include <cuda.h>
+#include <cstring>
 
 #include "topk.cuh"
 
@@ -597,6 +598,20 @@ static EncodeTiledFn encode_fn() {
 cudaError_t make_tmap_bf16(void* out_map, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows,
                            uint64_t row_stride) {
     if (row_stride == 0) row_stride = cols;
+    // A map is a pure function of these five values.  A search loop asks for the same few maps call after call
+    // (the query operand in the caller's workspace, the flat database): the last ones each thread asked for are
+    // kept, so a repeated call encodes nothing.
+    struct Slot { const void* ptr; uint64_t rows, cols, stride; uint32_t box; bool used; alignas(64) unsigned char map[128]; };
+    constexpr int NSLOT = 8;
+    static thread_local Slot slots[NSLOT];
+    static thread_local int next_slot = 0;
+    for (int i = 0; i < NSLOT; ++i) {
+        const Slot& c = slots[i];
+        if (c.used && c.ptr == ptr && c.rows == rows && c.cols == cols && c.stride == row_stride && c.box == box_rows) {
+            std::memcpy(out_map, c.map, 128);
+            return cudaSuccess;
+        }
+    }
     EncodeTiledFn fn = encode_fn();
     if (!fn) return cudaErrorNotSupported;
     if (rows == 0 || cols == 0 || (row_stride * 2) % 16 != 0 || row_stride < cols ||
@@ -606,10 +621,16 @@ cudaError_t make_tmap_bf16(void* out_map, const void* ptr, uint64_t rows, uint64
     const cuuint64_t strides[1] = {row_stride * 2};
     const cuuint32_t box[2] = {GBK, box_rows};
     const cuuint32_t estr[2] = {1, 1};
-    CUresult r = fn(static_cast<CUtensorMap*>(out_map), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr),
+    Slot& c = slots[next_slot];
+    c.used = false;
+    CUresult r = fn(reinterpret_cast<CUtensorMap*>(c.map), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr),
                     dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+    if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+    c.ptr = ptr; c.rows = rows; c.cols = cols; c.stride = row_stride; c.box = box_rows; c.used = true;
+    next_slot = (next_slot + 1) % NSLOT;
+    std::memcpy(out_map, c.map, 128);
+    return cudaSuccess;
 }
 
 int gemm_cand_cap(int nsel) { return nsel <= GEMM_CAP_SMALL - 128 ? GEMM_CAP_SMALL : (nsel <= GEMM_CAP_LARGE - 64 ? GEMM_CAP_LARGE : 0); }

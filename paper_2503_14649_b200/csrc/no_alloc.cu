@@ -3,7 +3,7 @@
 // keeps in the caller's workspace, lives here in a fixed array that is part of the library image.
 #include <mutex>
 
-#include "common.cuh"
+#include "plan.cuh"
 
 namespace rago {
 
@@ -86,7 +86,7 @@ extern "C" rago_status rago_search_probes_noalloc(const rago_index* index, const
     // reads, and the bias block is write-only here.
     e = launch_coarse_scores(ix, queries, nq, scores, s);
     if (e == cudaSuccess)
-        e = launch_select_probes(ix, queries, scores, nq, nprobe, out_lists, out_coarse, bias, s);
+        e = launch_select_probes(ix, queries, scores, nq, nprobe, out_lists, out_coarse, bias, nullptr, s);
     if (e != cudaSuccess) { set_error("coarse kernels: %s", cudaGetErrorString(e)); return RAGO_ECUDA; }
     return RAGO_OK;
 }

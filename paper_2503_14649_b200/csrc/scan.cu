@@ -50,6 +50,7 @@
 #include <type_traits>
 
 #include "topk.cuh"
+#include "plan.cuh"
 
 namespace rago {
 
@@ -843,55 +844,6 @@ cudaError_t launch_codeword_norms(const float* codebooks, int M, int dsub, float
 }
 
 constexpr int BT_THREADS = 256;
-struct TableArgs {
-    const float* queries; const float* cbT; const float* cwmax;
-    int d, dsub, M, metric, lut_bytes, banked, copies, copy_off, lstride;
-    uint8_t* lut_img; float* lut_inv;
-};
-// Part `part` of `parts` of query q's table, by all threads of the CTA.  sm: d + M floats of shared memory.
-__device__ __forceinline__ void build_table_part(const TableArgs& t, int q, int part, int parts, float* sm) {
-    const int d = t.d, dsub = t.dsub, M = t.M, tid = threadIdx.x, nthreads = blockDim.x;
-    float* rT = sm;       // the scaled query with the sub-space index innermost
-    float* bnd = sm + d;  // bound of the entries of every sub-space
-    const float lut_scale = t.metric == RAGO_IP ? -1.f : -2.f;
-    const float* qrow = t.queries + (size_t)q * d;
-    for (int j = tid; j < d; j += nthreads) rT[(j % dsub) * M + j / dsub] = lut_scale * qrow[j];
-    for (int m = tid; m < M; m += nthreads) {
-        float n2 = 0.f;
-        for (int u = 0; u < dsub; ++u) { const float v = qrow[m * dsub + u]; n2 = fmaf(v, v, n2); }
-        bnd[m] = 2.0002f * sqrtf(n2) * t.cwmax[m];  // |s| <= 2, and a margin for the rounding of the norms
-    }
-    __syncthreads();
-    float mx = 0.f;
-    for (int m = 0; m < M; ++m) mx = fmaxf(mx, bnd[m]);
-    int ex = 0;
-    if (mx > 0.f && mx < 3.0e38f) frexpf(mx * (float)M, &ex);  // mx * M < 2^ex
-    ex = ex < -90 ? -90 : (ex > 120 ? 120 : ex);
-    const float scale = ldexpf(1.f, 30 - ex);
-    if (part == 0 && tid == 0) t.lut_inv[q] = ldexpf(1.f, ex - 30);
-    uint8_t* img = t.lut_img + (size_t)q * t.lut_bytes;
-    auto off = [&](int j, int col) -> uint32_t {
-        return t.banked ? (uint32_t)(col / 64) * 65536u + (uint32_t)j * 256u + (uint32_t)(col % 64) * 4u
-                        : ((uint32_t)j * t.lstride + (uint32_t)col) * 4u;
-    };
-    const int total = KSUB * M;
-    const int per = (total + parts - 1) / parts;
-    const int e1 = (part + 1) * per < total ? (part + 1) * per : total;
-    // entry e = (code value j, sub-space m), m fastest; (j, m) follow e by counting, not by dividing per entry
-    const int step_j = nthreads / M, step_m = nthreads - step_j * M;
-    int e = part * per + tid;
-    int j = e / M, m = e - j * M;
-    for (; e < e1; e += nthreads) {
-        float acc = 0.f;
-        for (int u = 0; u < dsub; ++u) acc = fmaf(rT[u * M + m], __ldg(t.cbT + (size_t)e * dsub + u), acc);
-        const int v = __float2int_rn(acc * scale);
-        *reinterpret_cast<int*>(img + off(j, m)) = v;
-        if (t.copies == 2) *reinterpret_cast<int*>(img + off(j, t.copy_off + m)) = v;
-        j += step_j;
-        m += step_m;
-        if (m >= M) { m -= M; ++j; }
-    }
-}
 __global__ void __launch_bounds__(BT_THREADS) build_tables_kernel(const TableArgs t) {
     extern __shared__ float bt_smem[];
     build_table_part(t, blockIdx.y, blockIdx.x, gridDim.x, bt_smem);
@@ -1123,9 +1075,6 @@ __global__ void __launch_bounds__(PT_THREADS) pair_tiles_kernel(const int32_t* _
     if (threadIdx.x == PT_THREADS - 1) block_sums[blockIdx.x] = before + v;
 }
 
-constexpr int PFX_THREADS = 1024;
-constexpr int PLAN_PER_THREAD = 4;       // pairs per thread of the single-CTA planning kernel
-constexpr int PLAN_SMALL_MAX = PFX_THREADS * PLAN_PER_THREAD;
 // In-place exclusive scan of n totals by one CTA; the grand total goes to *total_out.
 __global__ void __launch_bounds__(PFX_THREADS) scan_totals_kernel(long long* __restrict__ sums, int n,
                                                                   int64_t* __restrict__ total_out) {
@@ -1187,46 +1136,28 @@ __global__ void __launch_bounds__(PFX_THREADS) plan_small_kernel(const int32_t* 
         return;
     }
     __shared__ long long warp_sums[32];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    // thread t owns pairs PLAN_PER_THREAD * t .. + PLAN_PER_THREAD - 1
-    long long mine[PLAN_PER_THREAD];
-    long long v = 0;
-#pragma unroll
-    for (int j = 0; j < PLAN_PER_THREAD; ++j) {
-        const int p = tid * PLAN_PER_THREAD + j;
-        mine[j] = 0;
-        if (p < npairs) {
-            const int l = probe_list[p];
-            mine[j] = (offsets[l + 1] - offsets[l] + tile_vecs - 1) / tile_vecs;
-        }
-        v += mine[j];
-    }
-    long long incl = v;
-    for (int o = 1; o < 32; o <<= 1) {
-        const long long y = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += y;
-    }
-    if (lane == 31) warp_sums[warp] = incl;
-    __syncthreads();
-    if (warp == 0) {
-        long long w = warp_sums[lane];
-        for (int o = 1; o < 32; o <<= 1) {
-            const long long y = __shfl_up_sync(0xffffffffu, w, o);
-            if (lane >= o) w += y;
-        }
-        warp_sums[lane] = w;
-    }
-    __syncthreads();
-    long long before = (warp ? warp_sums[warp - 1] : 0) + incl - v;
-#pragma unroll
-    for (int j = 0; j < PLAN_PER_THREAD; ++j) {
-        const int p = tid * PLAN_PER_THREAD + j;
-        if (p < npairs) prefix[p] = before;
-        before += mine[j];
-        if (p == npairs - 1) prefix[npairs] = before;
-    }
-    for (int i = tid; i < nq; i += PFX_THREADS) qthresh[i] = KEY_MAX;
-    for (int i = tid; i < nslots; i += PFX_THREADS) slot_cnt[i] = 0;
+    plan_pairs_cta(probe_list, offsets, npairs, tile_vecs, prefix, qthresh, nq, slot_cnt, nslots, warp_sums);
+}
+
+// Small batches whose probe selection plans the scan itself (see FusedPlan): what that kernel needs, or false when
+// the batch does not qualify (tables not prebuilt, too many pairs for one CTA, more than 64 queries).
+bool fused_plan_args(const IndexImpl* ix, int nq, int npairs, const float* queries, uint8_t* lut_img, float* lut_inv,
+                     int64_t* work_prefix, unsigned long long* qthresh, int32_t* slot_cnt, int nslots, uint32_t* ticket,
+                     FusedPlan* fp) {
+    fp->enabled = 0;
+    if (!lut_img || npairs > PLAN_SMALL_MAX || nq > 64) return false;
+    fp->enabled = 1;
+    fp->nq = nq;
+    fp->ticket = ticket;
+    fp->offsets = ix->list_offsets;
+    fp->tile_vecs = ix->plan.tile_vecs;
+    fp->prefix = work_prefix;
+    fp->qthresh = qthresh;
+    fp->slot_cnt = slot_cnt;
+    fp->nslots = nslots;
+    fp->tables = table_args(ix, queries, lut_img, lut_inv);
+    fp->table_parts = table_parts(ix, nq);
+    return true;
 }
 
 cudaError_t launch_plan_work(const IndexImpl* ix, const int32_t* probe_list, int npairs, int tile_vecs,
