@@ -131,7 +131,7 @@ __global__ void __launch_bounds__(THREADS) merge_kernel(
         __syncthreads();
         if (m < k) {
             if (cnt >= k) {
-                block_select(keys, &cnt, k, tid, THREADS, sync);
+                block_select_short(keys, &cnt, k, tid, THREADS, sync);
                 tau = keys[k - 1];
             }
             const int rem = k - m, total_b = nslots * rem;  // at most (scan CTAs + 1) * MAX_K entries
@@ -184,7 +184,7 @@ __global__ void __launch_bounds__(THREADS) merge_kernel(
         }
     }
     __syncthreads();
-    int kept = block_select(keys, &cnt, k, tid, THREADS, sync);
+    int kept = block_select_short(keys, &cnt, k, tid, THREADS, sync);
     if (rs.enabled && kept > 0) {  // uniform
         // which winners lost too many bits to cancellation: one thread per winner
         for (int i = tid; i < kept; i += THREADS) {
@@ -215,7 +215,7 @@ __global__ void __launch_bounds__(THREADS) merge_kernel(
             __syncthreads();
             if (tid == 0) cnt = kept;
             __syncthreads();
-            kept = block_select(keys, &cnt, k, tid, THREADS, sync);  // order by the new values
+            kept = block_select_short(keys, &cnt, k, tid, THREADS, sync);  // order by the new values
         }
     }
     for (int i = tid; i < k; i += THREADS) {
@@ -225,6 +225,164 @@ __global__ void __launch_bounds__(THREADS) merge_kernel(
             const unsigned long long key = keys[i];
             id = ids[(uint32_t)(key & 0xFFFFFFFFull)];
             const float sc = orderable_f32((uint32_t)(key >> 32));
+            dist = metric == RAGO_L2 ? sc : -sc;
+        }
+        out_ids[(size_t)q * k + i] = id;
+        out_dists[(size_t)q * k + i] = dist;
+    }
+}
+
+// Small batches (latency): the same result by a shorter chain of dependent memory accesses.  A query's slots are
+// consecutive in memory, so the CTA's 1024 threads fetch ALL of their keys (at most KPT each) and the slot counts in
+// one round trip, keep them in registers, find a cut with between k and k + k/4 + 8 keys at or below it by a counting
+// bisection on the 64-bit keys (distinct, so it always ends), and only the keys up to the cut go to shared memory to
+// be sorted.  The ids of the winners are fetched together with the values the cancellation check needs.
+template <int KPT>
+__global__ void __launch_bounds__(1024) merge_small_kernel(
+    const int64_t* __restrict__ work_prefix, const int64_t* __restrict__ ids, int npairs, int nprobe, int k, int ctas,
+    int metric, const int32_t* __restrict__ slot_cnt, const unsigned long long* __restrict__ slot_keys,
+    const unsigned long long* __restrict__ qthresh, const RescoreArgs rs,
+    int64_t* __restrict__ out_ids, float* __restrict__ out_dists) {
+    constexpr int THREADS = 1024, BUF = 2 * MAX_K;
+    __shared__ unsigned long long keys[BUF];
+    __shared__ int cnt;
+    __shared__ unsigned long long s_mn, s_mx;
+    __shared__ uint32_t s_nv, s_round[3];
+    __shared__ int p_list[MAX_K];
+    __shared__ uint32_t p_lo[MAX_K], p_hi[MAX_K];
+    __shared__ int redo[MAX_K], redo_list[MAX_K];
+    __shared__ int nredo;
+    const int q = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    auto sync = [] { __syncthreads(); };
+    grid_dependency_wait();
+    grid_dependents_may_launch();
+    if (tid == 0) { cnt = 0; nredo = 0; s_mn = KEY_MAX; s_mx = 0ull; s_nv = 0u; s_round[0] = s_round[1] = s_round[2] = 0u; }
+    const long long W = work_prefix[npairs];
+    const long long u0 = work_prefix[(size_t)q * nprobe], u1 = work_prefix[(size_t)(q + 1) * nprobe];
+    unsigned long long tau = qthresh[q];
+    if (tau != KEY_MAX) ++tau;  // the threshold key itself is a result
+    if (rs.enabled) {
+        for (int i = tid; i < nprobe; i += THREADS) {
+            const int l = rs.probe_list[(size_t)q * nprobe + i];
+            p_list[i] = l;
+            p_lo[i] = (uint32_t)rs.list_offsets[l];
+            p_hi[i] = (uint32_t)rs.list_offsets[l + 1];
+        }
+    }
+    unsigned long long mine[KPT];
+#pragma unroll
+    for (int j = 0; j < KPT; ++j) mine[j] = KEY_MAX;
+    if (u1 > u0) {
+        const long long s0 = (long long)q + cta_of_unit(u0, W, ctas);
+        const int nslots = (int)((long long)q + cta_of_unit(u1 - 1, W, ctas) - s0) + 1;
+        const int total = nslots * k;  // at most KPT * THREADS: the launcher checked (ctas + 1) * k
+        const unsigned long long* src = slot_keys + (size_t)s0 * k;
+        const int32_t* csrc = slot_cnt + s0;
+#pragma unroll
+        for (int j = 0; j < KPT; ++j) {
+            const int e = tid + j * THREADS;
+            if (e < total) {
+                const int sl = e / k, i = e - sl * k;
+                const int c = csrc[sl];
+                const unsigned long long key = src[e];  // entries past a slot's count are stale, never out of bounds
+                if (i < c && key < tau) mine[j] = key;
+            }
+        }
+    }
+    unsigned long long mn = KEY_MAX, mx = 0ull;
+    uint32_t nv = 0;
+#pragma unroll
+    for (int j = 0; j < KPT; ++j)
+        if (mine[j] != KEY_MAX) { mn = mine[j] < mn ? mine[j] : mn; mx = mine[j] > mx ? mine[j] : mx; ++nv; }
+    __syncthreads();  // the shared words are initialised
+    nv = __reduce_add_sync(0xffffffffu, nv);
+    if (nv) {  // uniform within the warp
+        for (int o = 16; o; o >>= 1) {
+            const unsigned long long a = shfl_xor_u64(mn, o), b = shfl_xor_u64(mx, o);
+            mn = a < mn ? a : mn; mx = b > mx ? b : mx;
+        }
+        if (lane == 0) { atomicMin(&s_mn, mn); atomicMax(&s_mx, mx); atomicAdd(&s_nv, nv); }
+    }
+    __syncthreads();
+    mn = s_mn; mx = s_mx;
+    const uint32_t nvalid = s_nv;
+    const uint32_t want_max = (uint32_t)(k + (k >> 2) + 8);  // <= BUF
+    unsigned long long T = mx;  // keys up to T are collected
+    if (nvalid > want_max) {    // uniform.  k >= 2 here would not be needed: count(<= mn) = 1 <= k always
+        unsigned long long lo = mn, hi = mx;  // #(key <= lo) <= k  and  #(key <= hi) >= k; lo itself is always kept
+        uint32_t c_hi = nvalid;
+        int round = 0;
+        if (k > 1) {
+            while (hi - lo > 1 && c_hi > want_max) {  // uniform
+                const unsigned long long mid = lo + (hi - lo) / 2;
+                uint32_t c = 0;
+#pragma unroll
+                for (int j = 0; j < KPT; ++j) c += mine[j] <= mid ? 1u : 0u;  // mid < mx < the empty-slot pattern
+                c = __reduce_add_sync(0xffffffffu, c);
+                const int slot = round % 3;
+                if (lane == 0 && c) atomicAdd(&s_round[slot], c);
+                if (tid == 0) s_round[(slot + 1) % 3] = 0u;  // next round's word; its last readers passed two barriers ago
+                __syncthreads();
+                c = s_round[slot];
+                if (c < (uint32_t)k) lo = mid; else { hi = mid; c_hi = c; }
+                ++round;
+            }
+            T = hi;
+        } else {
+            T = mn;
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < KPT; ++j) warp_push(keys, &cnt, mine[j] <= T && mine[j] != KEY_MAX, mine[j], BUF);
+    __syncthreads();
+    int kept = block_select_short(keys, &cnt, k, tid, THREADS, sync, BUF);
+    // winners: id, and whether too many bits were lost to cancellation (one thread per winner, loads side by side)
+    int64_t my_id = -1;
+    unsigned long long my_key = KEY_MAX;
+    if (tid < kept) {
+        my_key = keys[tid];
+        const uint32_t pos = (uint32_t)(my_key & 0xFFFFFFFFull);
+        my_id = ids[pos];
+        if (rs.enabled) {
+            int p = 0;
+            while (p < nprobe && !(pos >= p_lo[p] && pos < p_hi[p])) ++p;
+            if (p < nprobe) {  // always: every candidate comes from a probed list
+                const float dist = orderable_f32((uint32_t)(my_key >> 32));
+                const float bias = rs.probe_bias[(size_t)q * nprobe + p], vt = rs.vterm[pos];
+                const float Tm = fmaxf(fmaxf(bias, fabsf(vt)), fabsf(dist - (bias + vt)));
+                if (dist < Tm * (1.f / 32.f)) {
+                    const int at = atomicAdd(&nredo, 1);
+                    redo[at] = tid;
+                    redo_list[at] = p_list[p];
+                }
+            }
+        }
+    }
+    if (rs.enabled && kept > 0) {  // uniform
+        __syncthreads();
+        const int nr = nredo;
+        if (nr > 0) {  // uniform
+            const float* qrow = rs.queries + (size_t)q * rs.d;
+            for (int e = warp; e < nr; e += THREADS / 32) {
+                const int i = redo[e];
+                const uint32_t pos = (uint32_t)(keys[i] & 0xFFFFFFFFull);
+                const float dist = direct_l2(rs, qrow, pos, redo_list[e], lane);
+                __syncwarp();
+                if (lane == 0) keys[i] = make_key(dist, pos);
+            }
+            __syncthreads();
+            if (tid == 0) cnt = kept;
+            __syncthreads();
+            kept = block_select_short(keys, &cnt, k, tid, THREADS, sync, BUF);  // order by the new values
+            if (tid < kept) { my_key = keys[tid]; my_id = ids[(uint32_t)(my_key & 0xFFFFFFFFull)]; }
+        }
+    }
+    for (int i = tid; i < k; i += THREADS) {  // k <= MAX_K = THREADS: one round
+        float dist = metric == RAGO_L2 ? __int_as_float(0x7f800000) : __int_as_float(0xff800000);
+        int64_t id = -1;
+        if (i < kept) {
+            id = my_id;
+            const float sc = orderable_f32((uint32_t)(my_key >> 32));
             dist = metric == RAGO_L2 ? sc : -sc;
         }
         out_ids[(size_t)q * k + i] = id;
@@ -242,7 +400,14 @@ cudaError_t launch_merge(const IndexImpl* ix, const int64_t* work_prefix, int nq
     rs.codes = ix->codes; rs.list_offsets = ix->list_offsets; rs.probe_list = probe_list;
     rs.probe_bias = probe_bias; rs.vterm = ix->vterm; rs.nlist = ix->nlist; rs.d = ix->d; rs.M = ix->M;
     rs.dsub = ix->dsub;
-    if (nq <= 64)
+    const long long worst = (long long)(ctas + 1) * k;  // keys of one query's slots, at most
+    if (nq <= 64 && worst <= 4 * 1024)
+        launch_overlapped(merge_small_kernel<4>, dim3(nq), dim3(1024), 0, s, work_prefix, ix->ids, nq * nprobe, nprobe, k, ctas,
+                          ix->metric, slot_cnt, slot_keys, qthresh, rs, out_ids, out_dists);
+    else if (nq <= 64 && worst <= 16 * 1024)
+        launch_overlapped(merge_small_kernel<16>, dim3(nq), dim3(1024), 0, s, work_prefix, ix->ids, nq * nprobe, nprobe, k, ctas,
+                          ix->metric, slot_cnt, slot_keys, qthresh, rs, out_ids, out_dists);
+    else if (nq <= 64)
         launch_overlapped(merge_kernel<1024>, dim3(nq), dim3(1024), 0, s, work_prefix, ix->ids, nq * nprobe, nprobe, k, ctas,
                           ix->metric, slot_cnt, slot_keys, qthresh, rs, out_ids, out_dists);
     else

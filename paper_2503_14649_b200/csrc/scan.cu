@@ -590,7 +590,7 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
             kept = ctrl->cnt;
         }
         if (kept > 1) {  // the slot is left in ascending order, which the merge relies on
-            kept = block_select(keys, &ctrl->cnt, k, ctid, NCT, csync, C::KCAP);
+            kept = block_select_short(keys, &ctrl->cnt, k, ctid, NCT, csync, C::KCAP);  // few keys: one warp, one barrier
             if (dead) return;
         }
         if (kept == k && ctid == 0) atomicMin(&a.qthresh[cur_q], keys[k - 1]);
