@@ -444,6 +444,8 @@ __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
     __shared__ int pre[SEL_MAX_SPLIT + 1];  // candidate path: exclusive prefix of the lists' counts
     __shared__ uint32_t hist[256];           // items per slice of the score range
     __shared__ uint32_t s_mn, s_mx, s_nv;    // CTA-wide minimum, maximum, count of the ordered score bits
+    __shared__ uint32_t s_cut_cnt;           // items at or below that cut
+    __shared__ uint32_t s_wmin[33];          // the warps' minima; [32]: the cut taken from them
     __shared__ uint32_t s_round[3];          // bisection counts, one word per round in rotation
     __shared__ uint32_t s_bin[3];            // slice holding the cut, items of the range up to and including / before it
     __shared__ int cnt;
@@ -461,7 +463,7 @@ __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
     }
     int nsel = nprobe + PROBE_GUARD;
     if (nsel > nlist) nsel = nlist;
-    if (tid == 0) { cnt = 0; s_mn = 0xFFFFFFFFu; s_mx = 0u; s_nv = 0u; s_round[0] = s_round[1] = s_round[2] = 0u; }
+    if (tid == 0) { cnt = 0; s_mn = 0xFFFFFFFFu; s_mx = 0u; s_nv = 0u; s_cut_cnt = 0u; s_round[0] = s_round[1] = s_round[2] = 0u; }
     for (int i = tid; i < 256; i += SEL_THREADS) hist[i] = 0u;
     const float* srow = FROM_SCORES ? scores + (size_t)q * nlist : nullptr;
     if (!FROM_SCORES) {  // the valid entries of the query's lists, numbered consecutively
@@ -509,8 +511,20 @@ __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
     mn = __reduce_min_sync(0xffffffffu, mn);
     mx = __reduce_max_sync(0xffffffffu, mx);
     nvalid = __reduce_add_sync(0xffffffffu, nvalid);
-    if (lane == 0) { atomicMin(&s_mn, mn); atomicMax(&s_mx, mx); atomicAdd(&s_nv, nvalid); }
+    if (lane == 0) { atomicMin(&s_mn, mn); atomicMax(&s_mx, mx); atomicAdd(&s_nv, nvalid); s_wmin[warp] = mn; }
     __syncthreads();
+    // Few lists wanted (nsel <= 32) out of many: the nsel-th smallest of the warps' minima has at least nsel items
+    // at or below it, one per warp, and on scores in no particular order only a few dozen in all.  It replaces the
+    // slice counts and the bisection below as the cut, for one small sort by one warp.
+    uint32_t warp_cut = 0xFFFFFFFFu;
+    if (SEL_THREADS == 1024 && in_regs && nsel <= 32) {  // uniform
+        if (warp == 0) {
+            const uint32_t sorted = warp_sort_u32(s_wmin[lane], lane);
+            if (lane == nsel - 1) s_wmin[32] = sorted;
+        }
+        __syncthreads();
+        warp_cut = s_wmin[32];  // 0xFFFFFFFF: fewer than nsel warps hold an item
+    }
     mn = s_mn; mx = s_mx; nvalid = s_nv;
     if ((int)nvalid < nsel) nsel = (int)nvalid;  // cannot happen for a well-formed candidate set; stay safe
     int slack = nsel / 4 > 8 ? nsel / 4 : 8;
@@ -520,6 +534,17 @@ __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
     // nsel + slack items at or below hi; ties and odd distributions are finished by the bisection below.
     long long lo = (long long)mn - 1, hi = mx;  // invariant: #(score <= lo) < nsel <= #(score <= hi)
     uint32_t c_hi = nvalid, below = 0;          // below = #(score <= lo)
+    if (warp_cut != 0xFFFFFFFFu) {  // uniform; in_regs holds
+        uint32_t c = 0;
+#pragma unroll
+        for (int j = 0; j < SEL_REG; ++j) c += mine[j] <= warp_cut ? 1u : 0u;  // warp_cut < the empty-slot pattern
+        c = __reduce_add_sync(0xffffffffu, c);
+        if (lane == 0 && c) atomicAdd(&s_cut_cnt, c);
+        __syncthreads();
+        hi = warp_cut;
+        c_hi = s_cut_cnt;  // >= nsel
+        if (nsel + slack < WARP_SORT_MAX) slack = WARP_SORT_MAX - nsel;  // what one warp sorts is as good as fewer
+    }
     for (int pass = 0; pass < 3 && hi - lo > 1 && c_hi > (uint32_t)(nsel + slack); ++pass) {  // uniform
         const uint32_t first = (uint32_t)(lo + 1), range = (uint32_t)(hi - lo - 1);
         const int shift = range < 256u ? 0 : 24 - __clz(range);  // (range >> shift) < 256
@@ -629,6 +654,10 @@ __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
     }
     // collect the items below the cut, and those at the cut up to payload P
     if (in_regs) {
+        bool any = false;  // most warps hold nothing at or below the cut: one vote instead of SEL_REG
+#pragma unroll
+        for (int j = 0; j < SEL_REG; ++j) any = any || (mine[j] != 0xFFFFFFFFu && mine[j] <= T);
+        if (__any_sync(0xffffffffu, any)) {
 #pragma unroll
         for (int j = 0; j < SEL_REG; ++j) {
             bool take = mine[j] != 0xFFFFFFFFu && mine[j] <= T;
@@ -637,6 +666,7 @@ __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
             else if (take) key = item(tid + j * SEL_THREADS);
             if (take && mine[j] == T && (uint32_t)key > P) take = false;
             warp_push(keys, &cnt, take, key);
+        }
         }
     } else {
         for (int l0 = 0; l0 < nitems; l0 += SEL_THREADS) {
@@ -710,20 +740,44 @@ __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
             if (lane == 0) probe_bias[(size_t)q * nprobe + i] = acc;
         }
     }
-    // Fused planning: the CTA that finishes its query last (a ticket, nothing waits) plans the scan of the batch.
+    // Fused planning.  A single query plans from what it still holds in shared memory: no ticket, no fence, no
+    // re-read.  With more queries the CTA that finishes its query last (a ticket, nothing waits) plans for the batch.
     if constexpr (SEL_THREADS == PFX_THREADS) {
         if (fp.enabled) {  // uniform
             __shared__ int s_last;
             __shared__ long long plan_sums[32];
-            __threadfence();  // this query's probe lists before the ticket
-            __syncthreads();
-            if (tid == 0) s_last = atomicAdd(fp.ticket, 1u) == (uint32_t)(fp.nq - 1) ? 1 : 0;
-            __syncthreads();
-            if (s_last) {
-                __threadfence();  // the other queries' probe lists after their tickets
-                plan_pairs_cta(probe_list, fp.offsets, fp.nq * nprobe, fp.tile_vecs, fp.prefix, fp.qthresh, fp.nq,
-                               fp.slot_cnt, fp.nslots, plan_sums);
-                if (tid == 0) *fp.ticket = 0u;
+            if (fp.nq == 1) {
+                long long v = 0;  // tiles of pair tid (nprobe <= MAX_K = SEL_THREADS)
+                if (tid < nprobe) {
+                    const uint32_t l = (uint32_t)(keys[tid] & 0xFFFFFFFFull);
+                    v = (fp.offsets[l + 1] - fp.offsets[l] + fp.tile_vecs - 1) / fp.tile_vecs;
+                }
+                fp.qthresh[0] = KEY_MAX;  // every thread the same value; the stores leave with the loads above
+                for (int i = tid; i < fp.nslots; i += SEL_THREADS) fp.slot_cnt[i] = 0;
+                long long incl = v;
+                for (int o = 1; o < 32; o <<= 1) {
+                    const long long y = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (lane >= o) incl += y;
+                }
+                if (lane == 31) plan_sums[warp] = incl;
+                __syncthreads();
+                long long before = incl - v;
+                for (int w = 0; w < warp; ++w) before += plan_sums[w];  // few warps hold pairs: short for small nprobe
+                if (tid < nprobe) fp.prefix[tid] = before;
+                if (tid == nprobe - 1) fp.prefix[nprobe] = before + v;
+            } else {
+                __syncthreads();  // this query's probe lists are written ...
+                if (tid == 0) {
+                    __threadfence();  // ... and ordered before the ticket (the barrier makes the fence cover them all)
+                    s_last = atomicAdd(fp.ticket, 1u) == (uint32_t)(fp.nq - 1) ? 1 : 0;
+                    __threadfence();
+                }
+                __syncthreads();
+                if (s_last) {
+                    plan_pairs_cta(probe_list, fp.offsets, fp.nq * nprobe, fp.tile_vecs, fp.prefix, fp.qthresh, fp.nq,
+                                   fp.slot_cnt, fp.nslots, plan_sums);
+                    if (tid == 0) *fp.ticket = 0u;
+                }
             }
         }
     }

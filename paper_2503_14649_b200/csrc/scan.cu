@@ -194,6 +194,7 @@ __host__ __device__ inline SmemPlan plan_smem(uint32_t base, uint32_t dyn_bytes,
 }
 
 // Control block.
+constexpr int WARP_CUT_MAX = 1024;  // buffer cuts of at most this many keys are bisected by one warp
 struct Ctrl {
     unsigned long long full[MAX_STAGES];
     unsigned long long empty[MAX_STAGES];
@@ -371,23 +372,48 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
     // kernels before it wrote.
     grid_dependency_wait();
     grid_dependents_may_launch();
+    // A batch of a few queries is latency-bound, and most of a CTA's start-up would be a chain of dependent reads
+    // (total, binary search for the first pair, the pair's list, the list's offset) before its first tile can be
+    // asked for.  With at most 32 pairs lane i of every warp reads pair i's first unit beside the total, so the
+    // first pair follows from one vote; the producer warp reads the rest of every pair's description in the same
+    // round trip (the offsets in a second one), and the consumers know their first query without the producer.
+    const bool few_pairs = a.npairs <= 32;
+    const long long pw = few_pairs ? a.work_prefix[lane < a.npairs ? lane : a.npairs] : 0;  // >= npairs: the total
+    int c_list = 0; long long c_off = 0, c_len = 0, c_ws = 0, c_we = 0; float c_term = 0.f;  // producer: lane i's cached pair
+    if (few_pairs && warp == NCW && lane < a.npairs) {
+        c_list = a.probe_list[lane];
+        c_term = a.probe_term[lane];
+        c_we = a.work_prefix[lane + 1];
+        c_off = a.list_offsets[c_list];
+        c_len = a.list_offsets[c_list + 1] - c_off;
+    }
     // This CTA's share of the work units (tiles).
     const long long W = a.work_prefix[a.npairs];
     const long long u_begin = (long long)blockIdx.x * W / gridDim.x;
     const long long u_end = (long long)(blockIdx.x + 1) * W / gridDim.x;
     const int T = (int)(u_end - u_begin);
     if (T <= 0) return;
+    // few pairs: the pair whose range contains u_begin = the largest p with work_prefix[p] <= u_begin
+    const int first_pair = few_pairs ? __popc(__ballot_sync(0xffffffffu, pw <= u_begin)) - 1 : -1;
 
     if (warp == NCW) {
         // ================= producer warp =================
         // first pair whose range contains u_begin: largest p with work_prefix[p] <= u_begin
         int lo = 0, hi = a.npairs;  // invariant: work_prefix[lo] <= u_begin < work_prefix[hi]
-        while (hi - lo > 1) {
-            const int mid = (lo + hi) >> 1;
-            if (a.work_prefix[mid] <= u_begin) lo = mid; else hi = mid;
+        while (!few_pairs && hi - lo > 1) {  // 32 probes per step, evenly spaced: lane i looks at lo + (i + 1) * step
+            const int step = (hi - lo + 31) / 32;
+            const int pp = lo + (lane + 1) * step;
+            const bool le = pp < hi && a.work_prefix[pp] <= u_begin;
+            const int c = __popc(__ballot_sync(0xffffffffu, le));  // the prefix is monotone: the first c probes pass
+            const int nhi = lo + (c + 1) * step;
+            lo += c * step;
+            hi = nhi < hi ? nhi : hi;
         }
-        int cache_base = lo;  // lane i caches pair cache_base + i
-        int c_list = 0; long long c_off = 0, c_len = 0, c_ws = 0, c_we = 0; float c_term = 0.f;
+        int cache_base = few_pairs ? 0 : lo;  // lane i caches pair cache_base + i
+        if (few_pairs) {
+            c_ws = pw;
+            if (lane >= a.npairs) { c_ws = c_we = W; }
+        }
         auto fill = [&]() {
             const int p = cache_base + lane;
             if (p < a.npairs) {
@@ -401,8 +427,8 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
                 c_list = 0; c_off = 0; c_len = 0; c_ws = c_we = W; c_term = 0.f;
             }
         };
-        fill();
-        int cur = 0;
+        if (!few_pairs) fill();
+        int cur = few_pairs ? first_pair : 0;
         long long u = u_begin;
         bool dead = false;
         int issued = 0;
@@ -536,6 +562,55 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
                 mx = o > mx ? o : mx;
             }
         }
+        if (n <= WARP_CUT_MAX) {  // uniform
+            // A short buffer (the close of a query in a small batch, mostly): one warp bisects alone, re-reading the
+            // score words from shared memory in every round, with no barrier per round; the others wait once.
+            if (warp == 0) {
+                const uint32_t* kw = reinterpret_cast<const uint32_t*>(keys);  // score word of key i: kw[2 i + 1]
+                uint32_t lmn = 0xFFFFFFFFu, wmx = 0u;  // this lane's smallest score word, the largest of all
+                for (int i = lane; i < n; i += 32) {
+                    const uint32_t o = kw[2 * i + 1];
+                    lmn = o < lmn ? o : lmn;
+                    wmx = o > wmx ? o : wmx;
+                }
+                const uint32_t wmn = __reduce_min_sync(0xffffffffu, lmn);
+                wmx = __reduce_max_sync(0xffffffffu, wmx);
+                long long lo = (long long)wmn - 1, hi = wmx;  // #(score <= lo) < k <= #(score <= hi)
+                uint32_t c_hi = (uint32_t)n;
+                uint32_t want_max = (uint32_t)(k + (k >> 2) + 8);
+                if (want_max < (uint32_t)WARP_SORT_MAX) want_max = WARP_SORT_MAX;  // what one warp sorts afterwards
+                if (k <= 32 && n >= 32) {
+                    // The k-th smallest of the 32 lanes' minima has at least k keys at or below it, and on keys in
+                    // no particular order only about 1.5 k: usually the cut is found in this one step.
+                    const uint32_t t0 = __shfl_sync(0xffffffffu, warp_sort_u32(lmn, lane), k - 1);
+                    uint32_t c = 0;
+                    for (int i = lane; i < n; i += 32) c += kw[2 * i + 1] <= t0 ? 1u : 0u;
+                    hi = t0;
+                    c_hi = __reduce_add_sync(0xffffffffu, c);
+                }
+                while (hi - lo > 1 && c_hi > want_max) {
+                    const uint32_t mid = (uint32_t)(lo + (hi - lo) / 2);
+                    uint32_t c = 0;
+                    for (int i = lane; i < n; i += 32) c += kw[2 * i + 1] <= mid ? 1u : 0u;
+                    c = __reduce_add_sync(0xffffffffu, c);
+                    if (c < (uint32_t)k) lo = mid; else { hi = mid; c_hi = c; }
+                }
+                if (lane == 0) ctrl->redu[0][0] = (uint32_t)hi;
+            }
+            csync();  // every thread holds its keys in registers; the cut value is known
+            if (dead) return;
+            const uint32_t T = ctrl->redu[0][0];
+            if (ctid == 0) ctrl->cnt = 0;
+            csync();
+            if (dead) return;
+#pragma unroll
+            for (int j = 0; j < KPT; ++j)
+                warp_push(keys, &ctrl->cnt, mine[j] != KEY_MAX && (uint32_t)(mine[j] >> 32) <= T, mine[j], C::KCAP);
+            const unsigned long long bound = ((unsigned long long)T << 32) | 0xFFFFFFFFull;  // >= the k-th best key
+            if (bound < tau) tau = bound;
+            if (ctid == 0) atomicMin(&a.qthresh[cur_q], bound);
+            return;
+        }
         mn = __reduce_min_sync(0xffffffffu, mn);
         mx = __reduce_max_sync(0xffffffffu, mx);
         if (lane == 0) { ctrl->redu[0][warp] = mn; ctrl->redu[1][warp] = mx; }
@@ -582,7 +657,47 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
         csync();
         if (dead) return;
         int kept = ctrl->cnt;
-        if (kept > 2 * k + 64) {  // a long buffer: bisect down to about k keys first, then sort only those
+        if (k <= 32 && kept > 32 && kept <= WARP_CUT_MAX) {  // uniform
+            // A short buffer and a small k (the close of a query in a latency-bound batch): warp 0 alone finds a cut
+            // and compacts the buffer in place, with no barrier and no atomic in between.  The cut is the k-th
+            // smallest of the 32 lanes' minima: at least k keys lie at or below it, about 1.5 k on keys in no
+            // particular order.
+            if (warp == 0) {
+                const uint32_t* kw = reinterpret_cast<const uint32_t*>(keys);  // score word of key i: kw[2 i + 1]
+                uint32_t lmn = 0xFFFFFFFFu;
+#pragma unroll 4
+                for (int i = lane; i < kept; i += 32) {
+                    const uint32_t o = kw[2 * i + 1];
+                    lmn = o < lmn ? o : lmn;
+                }
+                const uint32_t t0 = __shfl_sync(0xffffffffu, warp_sort_u32(lmn, lane), k - 1);
+                const uint32_t lt_mask = (1u << lane) - 1u;
+                int base = 0;
+                for (int i0 = 0; i0 < kept; i0 += 128) {  // four rows of 32 keys at a time: their loads overlap
+                    unsigned long long key[4];
+                    uint32_t m[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int i = i0 + 32 * u + lane;
+                        key[u] = i < kept ? keys[i] : KEY_MAX;
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u)
+                        m[u] = __ballot_sync(0xffffffffu, i0 + 32 * u + lane < kept && (uint32_t)(key[u] >> 32) <= t0);
+                    __syncwarp();  // a key moves to a position at or before its own, and these 128 have been read
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        if ((m[u] >> lane) & 1u) keys[base + __popc(m[u] & lt_mask)] = key[u];
+                        base += __popc(m[u]);
+                    }
+                }
+                if (lane == 0) ctrl->cnt = base;
+            }
+            csync();
+            if (dead) return;
+            kept = ctrl->cnt;
+        }
+        if (kept > WARP_SORT_MAX && kept > k + (k >> 2) + 8) {  // bisect down to about k keys first, then sort only those
             cut_buffer();
             if (dead) return;
             csync();
@@ -642,9 +757,12 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
         csync();
     };
 
+    // few pairs: the first query is known without the producer, so its table is fetched while the first tile is
+    // still on its way (the tile loop finds cur_q set and goes straight to the scan)
+    if (few_pairs) begin_query(first_pair / a.nprobe);
     int cst = 0;            // n % S and the parity of n / S, kept by counting
     uint32_t cparity = 0;
-    for (int n = 0; n < T; ++n) {
+    for (int n = 0; n < T && !dead; ++n) {
         const int st = cst;
         const uint32_t parity = cparity;
         if (++cst == S) { cst = 0; cparity ^= 1u; }

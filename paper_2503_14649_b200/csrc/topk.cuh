@@ -84,6 +84,20 @@ __device__ __forceinline__ void warp_bitonic_sort(unsigned long long* keys, int 
     __syncwarp();
 }
 constexpr int WARP_SORT_MAX = 64;
+// Ascending sort of one 32-bit value per lane across the warp (bitonic network on shuffles); lane L returns the
+// L-th smallest.
+__device__ __forceinline__ uint32_t warp_sort_u32(uint32_t v, int lane) {
+#pragma unroll
+    for (int size = 2; size <= 32; size <<= 1) {
+#pragma unroll
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            const uint32_t o = __shfl_xor_sync(0xffffffffu, v, stride);
+            const bool keep_min = ((lane & stride) == 0) == ((lane & size) == 0);
+            v = keep_min == (v < o) ? v : o;
+        }
+    }
+    return v;
+}
 
 // block_select for short buffers: when at most WARP_SORT_MAX keys are buffered, warp 0 sorts them alone while the
 // other warps wait at one barrier.  Same contract as block_select.
