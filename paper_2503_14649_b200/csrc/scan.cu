@@ -543,13 +543,88 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
     const float lut_scale = ip ? -1.f : -2.f;
     float inv_scale = 1.f;  // fp32 value of one unit of the current query's integer table
 
-    // Cut the candidate buffer (more than k keys, count stable, called by all consumer threads after a csync):
+    // Cut the candidate buffer (more than k keys, count stable, called by all consumer threads after a csync and
+    // followed by another before the buffer or its count is used again):
     // every thread takes its share of the keys into registers, the CTA bisects on the ordered score bits for a
     // value T with between k and k + k/4 keys at or below it (one barrier per step instead of the ~66 of a full
     // sort), and the keys up to T are pushed back.  All keys of the k best are kept; T bounds the k-th best.
     auto cut_buffer = [&]() {
         constexpr int KPT = (C::KCAP + NCT - 1) / NCT;
         const int n = ctrl->cnt < C::KCAP ? ctrl->cnt : C::KCAP;
+        if (n <= WARP_CUT_MAX) {  // uniform
+            // A short buffer (small batches, mostly): warp 0 alone finds the cut and compacts the buffer in place,
+            // with no barrier and no atomic on the way; the others wait once.  For k <= 32 the cut is the k-th
+            // smallest of the 32 lanes' minima: at least k keys lie at or below it, about 1.5 k on keys in no
+            // particular order.  Otherwise (or if ties leave too many) it is bisected, the score words re-read from
+            // shared memory in every round.
+            if (warp == 0) {
+                const uint32_t* kw = reinterpret_cast<const uint32_t*>(keys);  // score word of key i: kw[2 i + 1]
+                uint32_t lmn = 0xFFFFFFFFu, wmx = 0u;  // this lane's smallest score word, the largest of all
+#pragma unroll 4
+                for (int i = lane; i < n; i += 32) {
+                    const uint32_t o = kw[2 * i + 1];
+                    lmn = o < lmn ? o : lmn;
+                    wmx = o > wmx ? o : wmx;
+                }
+                const uint32_t wmn = __reduce_min_sync(0xffffffffu, lmn);
+                wmx = __reduce_max_sync(0xffffffffu, wmx);
+                long long lo = (long long)wmn - 1, hi = wmx;  // #(score <= lo) < k <= #(score <= hi)
+                uint32_t want_max = (uint32_t)(k + (k >> 2) + 8);
+                if (want_max < (uint32_t)WARP_SORT_MAX) want_max = WARP_SORT_MAX;  // what one warp sorts afterwards
+                const bool quick = k <= 32 && n >= 32;
+                uint32_t c_hi = (uint32_t)n;
+                if (quick) {  // the count at the quick cut comes out of the compaction
+                    hi = __shfl_sync(0xffffffffu, warp_sort_u32(lmn, lane), k - 1);
+                    c_hi = 0;
+                }
+                const uint32_t lt_mask = (1u << lane) - 1u;
+                int nn = n;
+                for (int attempt = 0; attempt < 2; ++attempt) {
+                    while (hi - lo > 1 && c_hi > want_max) {
+                        const uint32_t mid = (uint32_t)(lo + (hi - lo) / 2);
+                        uint32_t c = 0;
+#pragma unroll 4
+                        for (int i = lane; i < nn; i += 32) c += kw[2 * i + 1] <= mid ? 1u : 0u;
+                        c = __reduce_add_sync(0xffffffffu, c);
+                        if (c < (uint32_t)k) lo = mid; else { hi = mid; c_hi = c; }
+                    }
+                    const uint32_t Tw = (uint32_t)hi;
+                    int base = 0;
+                    for (int i0 = 0; i0 < nn; i0 += 128) {  // four rows of 32 keys at a time: their loads overlap
+                        unsigned long long key[4];
+                        uint32_t m[4];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const int i = i0 + 32 * u + lane;
+                            key[u] = i < nn ? keys[i] : KEY_MAX;
+                        }
+#pragma unroll
+                        for (int u = 0; u < 4; ++u)
+                            m[u] = __ballot_sync(0xffffffffu, i0 + 32 * u + lane < nn && (uint32_t)(key[u] >> 32) <= Tw);
+                        __syncwarp();  // a key moves to a position at or before its own, and these 128 have been read
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            if ((m[u] >> lane) & 1u) keys[base + __popc(m[u] & lt_mask)] = key[u];
+                            base += __popc(m[u]);
+                        }
+                    }
+                    __syncwarp();
+                    nn = base;
+                    c_hi = (uint32_t)base;
+                    if (!quick || attempt == 1 || c_hi <= want_max) break;
+                }
+                if (lane == 0) { ctrl->redu[0][1] = (uint32_t)nn; ctrl->redu[0][0] = (uint32_t)hi; }
+            }
+            csync();
+            if (dead) return;
+            // the count changes only now that every thread has taken this branch on the old one; nobody reads or
+            // adds to it before the barrier the callers follow this call with
+            if (ctid == 0) ctrl->cnt = (int)ctrl->redu[0][1];
+            const unsigned long long bound = ((unsigned long long)ctrl->redu[0][0] << 32) | 0xFFFFFFFFull;  // >= the k-th best key
+            if (bound < tau) tau = bound;
+            if (ctid == 0) atomicMin(&a.qthresh[cur_q], bound);
+            return;
+        }
         unsigned long long mine[KPT];
         uint32_t mn = 0xFFFFFFFFu, mx = 0u;
 #pragma unroll
@@ -561,55 +636,6 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
                 mn = o < mn ? o : mn;
                 mx = o > mx ? o : mx;
             }
-        }
-        if (n <= WARP_CUT_MAX) {  // uniform
-            // A short buffer (the close of a query in a small batch, mostly): one warp bisects alone, re-reading the
-            // score words from shared memory in every round, with no barrier per round; the others wait once.
-            if (warp == 0) {
-                const uint32_t* kw = reinterpret_cast<const uint32_t*>(keys);  // score word of key i: kw[2 i + 1]
-                uint32_t lmn = 0xFFFFFFFFu, wmx = 0u;  // this lane's smallest score word, the largest of all
-                for (int i = lane; i < n; i += 32) {
-                    const uint32_t o = kw[2 * i + 1];
-                    lmn = o < lmn ? o : lmn;
-                    wmx = o > wmx ? o : wmx;
-                }
-                const uint32_t wmn = __reduce_min_sync(0xffffffffu, lmn);
-                wmx = __reduce_max_sync(0xffffffffu, wmx);
-                long long lo = (long long)wmn - 1, hi = wmx;  // #(score <= lo) < k <= #(score <= hi)
-                uint32_t c_hi = (uint32_t)n;
-                uint32_t want_max = (uint32_t)(k + (k >> 2) + 8);
-                if (want_max < (uint32_t)WARP_SORT_MAX) want_max = WARP_SORT_MAX;  // what one warp sorts afterwards
-                if (k <= 32 && n >= 32) {
-                    // The k-th smallest of the 32 lanes' minima has at least k keys at or below it, and on keys in
-                    // no particular order only about 1.5 k: usually the cut is found in this one step.
-                    const uint32_t t0 = __shfl_sync(0xffffffffu, warp_sort_u32(lmn, lane), k - 1);
-                    uint32_t c = 0;
-                    for (int i = lane; i < n; i += 32) c += kw[2 * i + 1] <= t0 ? 1u : 0u;
-                    hi = t0;
-                    c_hi = __reduce_add_sync(0xffffffffu, c);
-                }
-                while (hi - lo > 1 && c_hi > want_max) {
-                    const uint32_t mid = (uint32_t)(lo + (hi - lo) / 2);
-                    uint32_t c = 0;
-                    for (int i = lane; i < n; i += 32) c += kw[2 * i + 1] <= mid ? 1u : 0u;
-                    c = __reduce_add_sync(0xffffffffu, c);
-                    if (c < (uint32_t)k) lo = mid; else { hi = mid; c_hi = c; }
-                }
-                if (lane == 0) ctrl->redu[0][0] = (uint32_t)hi;
-            }
-            csync();  // every thread holds its keys in registers; the cut value is known
-            if (dead) return;
-            const uint32_t T = ctrl->redu[0][0];
-            if (ctid == 0) ctrl->cnt = 0;
-            csync();
-            if (dead) return;
-#pragma unroll
-            for (int j = 0; j < KPT; ++j)
-                warp_push(keys, &ctrl->cnt, mine[j] != KEY_MAX && (uint32_t)(mine[j] >> 32) <= T, mine[j], C::KCAP);
-            const unsigned long long bound = ((unsigned long long)T << 32) | 0xFFFFFFFFull;  // >= the k-th best key
-            if (bound < tau) tau = bound;
-            if (ctid == 0) atomicMin(&a.qthresh[cur_q], bound);
-            return;
         }
         mn = __reduce_min_sync(0xffffffffu, mn);
         mx = __reduce_max_sync(0xffffffffu, mx);
@@ -657,46 +683,6 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
         csync();
         if (dead) return;
         int kept = ctrl->cnt;
-        if (k <= 32 && kept > 32 && kept <= WARP_CUT_MAX) {  // uniform
-            // A short buffer and a small k (the close of a query in a latency-bound batch): warp 0 alone finds a cut
-            // and compacts the buffer in place, with no barrier and no atomic in between.  The cut is the k-th
-            // smallest of the 32 lanes' minima: at least k keys lie at or below it, about 1.5 k on keys in no
-            // particular order.
-            if (warp == 0) {
-                const uint32_t* kw = reinterpret_cast<const uint32_t*>(keys);  // score word of key i: kw[2 i + 1]
-                uint32_t lmn = 0xFFFFFFFFu;
-#pragma unroll 4
-                for (int i = lane; i < kept; i += 32) {
-                    const uint32_t o = kw[2 * i + 1];
-                    lmn = o < lmn ? o : lmn;
-                }
-                const uint32_t t0 = __shfl_sync(0xffffffffu, warp_sort_u32(lmn, lane), k - 1);
-                const uint32_t lt_mask = (1u << lane) - 1u;
-                int base = 0;
-                for (int i0 = 0; i0 < kept; i0 += 128) {  // four rows of 32 keys at a time: their loads overlap
-                    unsigned long long key[4];
-                    uint32_t m[4];
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const int i = i0 + 32 * u + lane;
-                        key[u] = i < kept ? keys[i] : KEY_MAX;
-                    }
-#pragma unroll
-                    for (int u = 0; u < 4; ++u)
-                        m[u] = __ballot_sync(0xffffffffu, i0 + 32 * u + lane < kept && (uint32_t)(key[u] >> 32) <= t0);
-                    __syncwarp();  // a key moves to a position at or before its own, and these 128 have been read
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        if ((m[u] >> lane) & 1u) keys[base + __popc(m[u] & lt_mask)] = key[u];
-                        base += __popc(m[u]);
-                    }
-                }
-                if (lane == 0) ctrl->cnt = base;
-            }
-            csync();
-            if (dead) return;
-            kept = ctrl->cnt;
-        }
         if (kept > WARP_SORT_MAX && kept > k + (k >> 2) + 8) {  // bisect down to about k keys first, then sort only those
             cut_buffer();
             if (dead) return;
@@ -716,8 +702,12 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
     };
 
     // Table of a query: entry (j, m) = lut_scale * <q_m, codeword j of sub-space m>.
+    // Small k: once the first tiles of a query have put a hundred-odd keys into the buffer it is cut at once (cheap at
+    // that length), so that the tiles that follow are pushed against a threshold instead of in full.
+    bool early = false;
     auto begin_query = [&](int q) {
         cur_q = q;
+        early = k <= 32;
         if (a.lut_img != nullptr) {  // the table was built ahead of the scan: fetch its shared-memory image
             const uint4* src = reinterpret_cast<const uint4*>(a.lut_img + (size_t)q * C::LUT_BYTES);
             uint4* dst = reinterpret_cast<uint4*>(smem + (P.lut - base));
@@ -849,6 +839,17 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
         if (!released) {  // a warp that left the loop early: no rows of this tile are its own
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ctrl->empty[st]));
+        }
+        if (early && n + 1 < T) {  // uniform; after the CTA's last tile the close of the query does the same work
+            csync();
+            if (dead) break;
+            if (ctrl->cnt > 2 * WARP_SORT_MAX) {  // uniform: nothing is pushed between the two barriers
+                cut_buffer();
+                early = false;
+            }
+            if (dead) break;
+            csync();
+            if (dead) break;
         }
     }
     if (!dead && cur_q >= 0) finalize();
