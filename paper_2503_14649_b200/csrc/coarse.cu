@@ -105,12 +105,13 @@ __global__ void __launch_bounds__(256) coarse_scores_kernel(const float* __restr
 
 // ---- score matrix for tiny batches (the latency-bound iterative-retrieval shape) -------------------
 // For up to CS_MAXQ queries: a warp takes CS_CPW centroid rows at a time and keeps one partial sum per (row, query),
-// so the centroid table is read exactly once per batch however few queries there are.  The launch is latency-bound
-// (a few rows per warp).  NQ (1, 4 or 16) bounds the batch at compile time: the partial sums and their reduction
-// shrink with it, and the registers that frees go to loads in flight: with up to 4 queries a warp asks for
-// CS_CPW x 512 values per round before it multiplies any of them; with 16 it takes 128 values of each row per round
-// and has the next round's in flight while it multiplies (the sums alone take 64 registers).  The grid is sized so
-// that most warps have a single step.
+// so the centroid table is read exactly once per batch however few queries there are.  The launch is bound by the
+// latency of the table's reads (a few rows per warp, and between two searches the scan pushes much of the table out
+// of L2), so a warp asks for CS_CPW x 512 values before it multiplies any of them: 8 KB in flight per warp.  NQ
+// (1, 4 or 16) bounds the batch at compile time: the partial sums and their reduction shrink with it; 16 queries are
+// multiplied in two groups of 8 against the same registers, because 64 sums beside 64 row values do not fit (with
+// half as many values in flight and the next round prefetched the same launch took twice as long).  The grid is
+// sized so that most warps have a single step.
 constexpr int CS_MAXQ = 16;
 constexpr int CS_CPW = 4;    // centroids per warp per step
 template <bool BF16, int NQ>
@@ -120,21 +121,33 @@ __global__ void __launch_bounds__(256) coarse_small_kernel(const float* __restri
     extern __shared__ __align__(16) float qs[];  // [nq][d], rounded to bf16 values for a bf16 index
     grid_dependency_wait();
     grid_dependents_may_launch();
-    for (int i = threadIdx.x; i < nq * d; i += blockDim.x) qs[i] = BF16 ? round_bf16(Q[i]) : Q[i];
+    {   // d is a multiple of 4 and Q 16-byte aligned; eight 16-byte loads in flight per thread
+        const int n4 = (nq * d) >> 2;
+        const float4* Q4 = reinterpret_cast<const float4*>(Q);
+        float4* qs4 = reinterpret_cast<float4*>(qs);
+        for (int i0 = threadIdx.x; i0 < n4; i0 += 8 * 256) {
+            float4 v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) v[u] = i0 + u * 256 < n4 ? __ldg(Q4 + i0 + u * 256) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                if (BF16) { v[u].x = round_bf16(v[u].x); v[u].y = round_bf16(v[u].y); v[u].z = round_bf16(v[u].z); v[u].w = round_bf16(v[u].w); }
+                if (i0 + u * 256 < n4) qs4[i0 + u * 256] = v[u];
+            }
+        }
+    }
     __syncthreads();
     const int lane = threadIdx.x & 31;
     const int warps = (gridDim.x * blockDim.x) >> 5;
+    constexpr int QG = NQ <= 4 ? NQ : 8;   // queries multiplied against the rows held in registers at a time
+    constexpr int NGROUPS = NQ / QG;
+    constexpr int CHUNK = 4;               // 16-byte (fp32) / 8-byte (bf16) loads per lane and row in one round: 512 values
     for (int c0 = ((blockIdx.x * blockDim.x + threadIdx.x) >> 5) * CS_CPW; c0 < nlist; c0 += warps * CS_CPW) {
-        float acc[CS_CPW][NQ];
         float cn[CS_CPW];
 #pragma unroll
-        for (int u = 0; u < CS_CPW; ++u) {
-            cn[u] = metric == RAGO_L2 ? __ldg(cnorm + (c0 + u < nlist ? c0 + u : nlist - 1)) : 0.f;
-#pragma unroll
-            for (int qi = 0; qi < NQ; ++qi) acc[u][qi] = 0.f;
-        }
-        constexpr int CHUNK = NQ <= 4 ? 4 : 1;  // 16-byte (fp32) / 8-byte (bf16) loads per lane and row in one round
-        auto load_rows = [&](float4 (&cv)[CS_CPW][CHUNK], int jb) {
+        for (int u = 0; u < CS_CPW; ++u) cn[u] = metric == RAGO_L2 ? __ldg(cnorm + (c0 + u < nlist ? c0 + u : nlist - 1)) : 0.f;
+        float4 cv[CS_CPW][CHUNK];
+        auto load_rows = [&](int jb) {
 #pragma unroll
             for (int u = 0; u < CS_CPW; ++u) {
                 const int c = c0 + u < nlist ? c0 + u : nlist - 1;  // rows past the end repeat the last one, unused
@@ -155,61 +168,59 @@ __global__ void __launch_bounds__(256) coarse_small_kernel(const float* __restri
                 }
             }
         };
-        float4 cv[CS_CPW][CHUNK], nx[CS_CPW][CHUNK];
-        load_rows(cv, 0);
-        for (int jb = 0; jb < d; jb += 128 * CHUNK) {
-            const bool more = jb + 128 * CHUNK < d;
-            if constexpr (CHUNK == 1) {  // next round's values in flight during this round's arithmetic
-                if (more) load_rows(nx, jb + 128 * CHUNK);
-            }
 #pragma unroll
-            for (int h = 0; h < CHUNK; ++h) {
-                const int j0 = jb + h * 128 + lane * 4;
-                if (j0 < d) {
+        for (int g = 0; g < NGROUPS; ++g) {
+            if (g * QG >= nq) break;  // uniform
+            float acc[CS_CPW][QG];
 #pragma unroll
-                    for (int qi = 0; qi < NQ; ++qi) {
-                        if (qi < nq) {  // uniform
-                            const float4 qv = *reinterpret_cast<const float4*>(qs + qi * d + j0);
+            for (int u = 0; u < CS_CPW; ++u)
 #pragma unroll
-                            for (int u = 0; u < CS_CPW; ++u)
-                                acc[u][qi] = fmaf(qv.x, cv[u][h].x, fmaf(qv.y, cv[u][h].y, fmaf(qv.z, cv[u][h].z, fmaf(qv.w, cv[u][h].w, acc[u][qi]))));
+                for (int qi = 0; qi < QG; ++qi) acc[u][qi] = 0.f;
+            for (int jb = 0; jb < d; jb += 128 * CHUNK) {
+                // the rows of a block of 512 values stay in registers for every group of queries; a longer row is
+                // read again for the second group (from the caches)
+                if (g == 0 || d > 128 * CHUNK) load_rows(jb);
+#pragma unroll
+                for (int h = 0; h < CHUNK; ++h) {
+                    const int j0 = jb + h * 128 + lane * 4;
+                    if (j0 < d) {
+#pragma unroll
+                        for (int qi = 0; qi < QG; ++qi) {
+                            if (g * QG + qi < nq) {  // uniform
+                                const float4 qv = *reinterpret_cast<const float4*>(qs + (g * QG + qi) * d + j0);
+#pragma unroll
+                                for (int u = 0; u < CS_CPW; ++u)
+                                    acc[u][qi] = fmaf(qv.x, cv[u][h].x, fmaf(qv.y, cv[u][h].y, fmaf(qv.z, cv[u][h].z, fmaf(qv.w, cv[u][h].w, acc[u][qi]))));
+                            }
                         }
                     }
                 }
             }
-            if (more) {
-                if constexpr (CHUNK == 1) {
+            // Sum over the lanes, all QG queries of a row at once: at each halving a lane keeps the half of its values
+            // that its lane-number bit selects and hands over the other half (QG - 1 exchanges instead of 5 QG), then
+            // the single value left is summed over the remaining lane bits.  The total of the query whose number is
+            // the leading log2(QG) lane bits ends in the lanes whose other bits are clear.
 #pragma unroll
-                    for (int u = 0; u < CS_CPW; ++u) cv[u][0] = nx[u][0];
-                } else {
-                    load_rows(cv, jb + 128 * CHUNK);
+            for (int u = 0; u < CS_CPW; ++u) {
+                int o = 16;
+#pragma unroll
+                for (int half = QG / 2; half >= 1; half >>= 1, o >>= 1) {
+                    const bool upper = (lane & o) != 0;
+#pragma unroll
+                    for (int i = 0; i < half; ++i) {
+                        const float keep = upper ? acc[u][i + half] : acc[u][i];
+                        const float send = upper ? acc[u][i] : acc[u][i + half];
+                        acc[u][i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+                    }
                 }
+                float v = acc[u][0];
+#pragma unroll
+                for (; o >= 1; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                constexpr int REST = 32 / QG;  // lanes that end up with the same query's total
+                const int qi = g * QG + (QG == 1 ? 0 : (lane / REST));
+                if ((lane & (REST - 1)) == 0 && qi < nq && c0 + u < nlist)
+                    scores[(size_t)qi * nlist + c0 + u] = metric == RAGO_L2 ? fmaf(-2.f, v, cn[u]) : -v;
             }
-        }
-        // Sum over the lanes, all NQ queries of a row at once: at each halving a lane keeps the half of its values
-        // that its lane-number bit selects and hands over the other half (NQ - 1 exchanges instead of 5 NQ), then
-        // the single value left is summed over the remaining lane bits.  The total of the query whose number is
-        // the leading log2(NQ) lane bits ends in the lanes whose other bits are clear.
-#pragma unroll
-        for (int u = 0; u < CS_CPW; ++u) {
-            int o = 16;
-#pragma unroll
-            for (int half = NQ / 2; half >= 1; half >>= 1, o >>= 1) {
-                const bool upper = (lane & o) != 0;
-#pragma unroll
-                for (int i = 0; i < half; ++i) {
-                    const float keep = upper ? acc[u][i + half] : acc[u][i];
-                    const float send = upper ? acc[u][i] : acc[u][i + half];
-                    acc[u][i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
-                }
-            }
-            float v = acc[u][0];
-#pragma unroll
-            for (; o >= 1; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-            constexpr int REST = 32 / NQ;  // lanes that end up with the same query's total
-            const int qi = NQ == 1 ? 0 : (lane / REST);
-            if ((lane & (REST - 1)) == 0 && qi < nq && c0 + u < nlist)
-                scores[(size_t)qi * nlist + c0 + u] = metric == RAGO_L2 ? fmaf(-2.f, v, cn[u]) : -v;
         }
     }
 }
