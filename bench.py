@@ -508,6 +508,23 @@ def _iter_stream(args, dev, tree):
         for b, nb in enumerate(sizes):
             lat[nb].append(ev[b].elapsed_time(ev[b + 1]))
         tot.append(ev[0].elapsed_time(ev[-1]))
+    # the same call with nothing between the calls: 240 searches of one batch size back to back, time per call
+    b2b = {}
+    for nb in (1, 4, 16):
+        qs = [q[i * nb:(i + 1) * nb] for i in range(12)] * 20
+        oi, od = out_i[:nb], out_d[:nb]
+        best = None
+        for _ in range(3):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record()
+            for x in qs:
+                ix.rago_search(x, nprobe, k, oi, od, ws)
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / len(qs)
+            best = ms if best is None else min(best, ms)
+        b2b[str(nb)] = best
     t1 = time.time()
     clocks = sampler.stop(t0, t1)
     ix.rago_check(ws)
@@ -524,7 +541,10 @@ def _iter_stream(args, dev, tree):
            "latency_ms": {"p50": float(np.percentile(alll, 50)), "p99": float(np.percentile(alll, 99)),
                           "by_batch_size": {str(nb): {"p50": float(np.percentile(v, 50)), "p99": float(np.percentile(v, 99))}
                                             for nb, v in lat.items()},
-                          "note": "device time between consecutive batches' start events (launch-to-launch on a busy stream)"},
+                          "note": "device time between consecutive batches' start events (launch-to-launch on a busy stream)",
+                          "back_to_back_ms_per_call": b2b,
+                          "back_to_back_note": "240 calls of one batch size with nothing between them (no event per call), "
+                                               "device time / 240, best of 3"},
            "stage_ms_batch_of_1": {kk: float(np.median([s_[kk] for s_ in st1])) for kk in st1[0]}}
     ix.close()
     del ix, data, ws, q

@@ -194,7 +194,8 @@ __host__ __device__ inline SmemPlan plan_smem(uint32_t base, uint32_t dyn_bytes,
 }
 
 // Control block.
-constexpr int WARP_CUT_MAX = 1024;  // buffer cuts of at most this many keys are bisected by one warp
+constexpr int WARP_CUT_MAX = 1024;  // buffer cuts of at most this many keys, for k of at most WARP_CUT_K, are made by one warp
+constexpr int WARP_CUT_K = 32;      // (a larger k needs bisection rounds, which the whole CTA does faster)
 struct Ctrl {
     unsigned long long full[MAX_STAGES];
     unsigned long long empty[MAX_STAGES];
@@ -551,8 +552,8 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
     auto cut_buffer = [&]() {
         constexpr int KPT = (C::KCAP + NCT - 1) / NCT;
         const int n = ctrl->cnt < C::KCAP ? ctrl->cnt : C::KCAP;
-        if (n <= WARP_CUT_MAX) {  // uniform
-            // A short buffer (small batches, mostly): warp 0 alone finds the cut and compacts the buffer in place,
+        if (n <= WARP_CUT_MAX && k <= WARP_CUT_K) {  // uniform
+            // A short buffer and a small k (small batches, mostly): warp 0 alone finds the cut and compacts the buffer in place,
             // with no barrier and no atomic on the way; the others wait once.  For k <= 32 the cut is the k-th
             // smallest of the 32 lanes' minima: at least k keys lie at or below it, about 1.5 k on keys in no
             // particular order.  Otherwise (or if ties leave too many) it is bisected, the score words re-read from
@@ -683,7 +684,9 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
         csync();
         if (dead) return;
         int kept = ctrl->cnt;
-        if (kept > WARP_SORT_MAX && kept > k + (k >> 2) + 8) {  // bisect down to about k keys first, then sort only those
+        // a long buffer: bisect down to about k keys first, then sort only those.  A cut pays when it makes the sort
+        // smaller: for small k down to what one warp sorts, otherwise below the next power of two.
+        if (k <= 32 ? kept > WARP_SORT_MAX : kept > 2 * k + 64) {
             cut_buffer();
             if (dead) return;
             csync();
@@ -769,10 +772,16 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
             }
             bias = ip ? -D.term : D.term;
         }
-        if (D.newpair & 2) {  // the producer saw the buffer filling up: keep the best k (or a few more), lower the threshold
+        // the producer saw the buffer filling up, or (small k) this is the query's second tile in this CTA: keep the
+        // best k (or a few more), lower the threshold.  One site for both, so that the cut is in the loop once.
+        const bool full_cut = (D.newpair & 2) != 0;
+        if (full_cut || (early && !(D.newpair & 1))) {
             csync();
             if (dead) break;
-            if (ctrl->cnt > k) cut_buffer();
+            if (ctrl->cnt > (full_cut ? k : 2 * WARP_SORT_MAX)) {  // uniform: nothing is pushed between the two barriers
+                cut_buffer();
+                early = false;
+            }
             if (dead) break;
             const unsigned long long g = *reinterpret_cast<volatile unsigned long long*>(&a.qthresh[cur_q]);
             if (g < tau) tau = g;
@@ -839,17 +848,6 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
         if (!released) {  // a warp that left the loop early: no rows of this tile are its own
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ctrl->empty[st]));
-        }
-        if (early && n + 1 < T) {  // uniform; after the CTA's last tile the close of the query does the same work
-            csync();
-            if (dead) break;
-            if (ctrl->cnt > 2 * WARP_SORT_MAX) {  // uniform: nothing is pushed between the two barriers
-                cut_buffer();
-                early = false;
-            }
-            if (dead) break;
-            csync();
-            if (dead) break;
         }
     }
     if (!dead && cur_q >= 0) finalize();
