@@ -46,8 +46,8 @@ SECONDARY = ("mid", "flat", "coarse_hyper", "iter")
 # of codes; the capture-size rule) and carries over to the full size because the lists are uniform and no list is
 # shared through L2 at either size; "mid" was captured at full size and is not scaled to other sizes.
 SCAN_TRAFFIC = {
-    "hyper": {"scan_sha": "9ad01f6c9bf14f47", "dram_per_logical": (15967243776 + 10723328) / 16004289600},   # 0.9984
-    "mid": {"scan_sha": "9ad01f6c9bf14f47", "dram_per_logical": (34641810688 + 7572992) / 42427363200},      # 0.8167
+    "hyper": {"scan_sha": "beb728b04673be65", "dram_per_logical": (15968936960 + 11397376) / 16004289600},   # 0.9985
+    "mid": {"scan_sha": "beb728b04673be65", "dram_per_logical": (34410413312 + 7730688) / 42427363200},      # 0.8112
 }
 
 
