@@ -716,20 +716,10 @@ __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
         if (lane == 0) keys2[i] = make_key(metric == RAGO_L2 ? acc : -acc, l);
     }
     __syncthreads();
-    int n2 = 2;
-    while (n2 < kept) n2 <<= 1;
-    if (kept <= WARP_SORT_MAX) {  // the usual case: one warp orders the few survivors
-        if (warp == 0) {
-            for (int i = lane; i < n2; i += 32) keys[i] = i < kept ? keys2[i] : KEY_MAX;
-            __syncwarp();
-            warp_bitonic_sort(keys, n2, lane);
-        }
-        __syncthreads();
-    } else {
-        for (int i = tid; i < n2; i += SEL_THREADS) keys[i] = i < kept ? keys2[i] : KEY_MAX;
-        __syncthreads();
-        block_bitonic_sort(keys, n2, tid, SEL_THREADS, sync);
-    }
+    for (int i = tid; i < kept; i += SEL_THREADS) keys[i] = keys2[i];
+    if (tid == 0) cnt = kept;
+    __syncthreads();
+    block_select_short(keys, &cnt, kept, tid, SEL_THREADS, sync);  // the usual case: a few survivors, ranked
     for (int i = tid; i < nprobe; i += SEL_THREADS) {
         const unsigned long long key = keys[i];
         const float sc = orderable_f32((uint32_t)(key >> 32));

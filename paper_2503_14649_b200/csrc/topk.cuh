@@ -99,8 +99,11 @@ __device__ __forceinline__ uint32_t warp_sort_u32(uint32_t v, int lane) {
     return v;
 }
 
-// block_select for short buffers: when at most WARP_SORT_MAX keys are buffered, warp 0 sorts them alone while the
-// other warps wait at one barrier.  Same contract as block_select.
+// block_select for short buffers: at most WARP_SORT_MAX keys.  With at least eight warps the keys are ranked, not
+// sorted: warp w counts, for each of its few keys, how many of the (distinct) keys are smaller (two votes), keeps
+// key and rank in registers across one barrier and then stores the key at its rank: two barriers and a few dozen
+// instructions per warp, where a bitonic network on shuffles is several hundred dependent ones in a single warp.
+// Same contract as block_select.
 template <class Sync>
 __device__ __forceinline__ int block_select_short(unsigned long long* keys, int* cnt, int k, int tid, int nthreads,
                                                   Sync sync, int cap = TOPK_CAP) {
@@ -108,6 +111,34 @@ __device__ __forceinline__ int block_select_short(unsigned long long* keys, int*
     if (n > cap) n = cap;
     if (n > WARP_SORT_MAX) return block_select(keys, cnt, k, tid, nthreads, sync, cap);
     const int kept = n < k ? n : k;
+    if (nthreads >= 256) {  // uniform
+        constexpr int PER_WARP = WARP_SORT_MAX / 8;
+        const int warp = tid >> 5, lane = tid & 31, nwarps = nthreads >> 5;
+        const unsigned long long a = lane < n ? keys[lane] : KEY_MAX;
+        const unsigned long long b = lane + 32 < n ? keys[lane + 32] : KEY_MAX;
+        unsigned long long mine[PER_WARP];
+        int rank[PER_WARP];
+#pragma unroll
+        for (int t = 0; t < PER_WARP; ++t) {
+            const int i = warp + t * nwarps;
+            rank[t] = -1;
+            mine[t] = 0ull;
+            if (i < n) {  // uniform within the warp
+                const unsigned long long x = keys[i];
+                rank[t] = __popc(__ballot_sync(0xffffffffu, a < x)) + __popc(__ballot_sync(0xffffffffu, b < x));
+                mine[t] = x;
+            }
+        }
+        sync();  // every key has been read
+        if (lane == 0) {
+#pragma unroll
+            for (int t = 0; t < PER_WARP; ++t)
+                if (rank[t] >= 0 && rank[t] < kept) keys[rank[t]] = mine[t];
+        }
+        if (tid == 0) *cnt = kept;
+        sync();
+        return kept;
+    }
     if (tid < 32) {
         int n2 = 2;
         while (n2 < n) n2 <<= 1;
