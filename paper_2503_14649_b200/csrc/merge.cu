@@ -306,7 +306,8 @@ __global__ void __launch_bounds__(1024) merge_small_kernel(
     __syncthreads();
     mn = s_mn; mx = s_mx;
     const uint32_t nvalid = s_nv;
-    const uint32_t want_max = (uint32_t)(k + (k >> 2) + 8);  // <= BUF
+    uint32_t want_max = (uint32_t)(k + (k >> 2) + 8);  // <= BUF
+    if (want_max < (uint32_t)WARP_SORT_MAX) want_max = WARP_SORT_MAX;  // as many as the short selection ranks in one go
     unsigned long long T = mx;  // keys up to T are collected
     if (nvalid > want_max) {    // uniform.  k >= 2 here would not be needed: count(<= mn) = 1 <= k always
         unsigned long long lo = mn, hi = mx;  // #(key <= lo) <= k  and  #(key <= hi) >= k; lo itself is always kept
