@@ -154,7 +154,7 @@ static void record(IndexImpl* ix, int i, cudaStream_t s) {
 
 // fp (may be null): the selection kernel also plans the scan and builds the lookup tables (small batches).
 static rago_status run_coarse(const IndexImpl* ix, const float* queries, int nq, int nprobe, uint8_t* ws,
-                              const Layout& L, const FusedPlan* fp, cudaStream_t s) {
+                              const Layout& L, const FusedPlan* fp, bool kernel_clears, cudaStream_t s) {
     IndexImpl* mix = const_cast<IndexImpl*>(ix);
     cudaError_t e;
     int32_t* probe_list = reinterpret_cast<int32_t*>(ws + L.probe_list);
@@ -227,7 +227,7 @@ static rago_status run_coarse(const IndexImpl* ix, const float* queries, int nq,
         else
             e = launch_select_probes(ix, queries, scores, nq, nprobe, probe_list, probe_term, probe_bias, fp, s);
     } else {
-        e = launch_coarse_scores(ix, queries, nq, scores, s);
+        e = launch_coarse_scores(ix, queries, nq, scores, kernel_clears ? reinterpret_cast<uint32_t*>(ws + L.err) : nullptr, s);
         if (e != cudaSuccess) return cuda_fail(e, "coarse score kernel");
         record(mix, 1, s);
         e = launch_select_probes(ix, queries, scores, nq, nprobe, probe_list, probe_term, probe_bias, fp, s);
@@ -386,7 +386,7 @@ rago_status rago_search_probes(const rago_index* index, const float* queries, in
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     cudaError_t e = cudaMemsetAsync(ws + L.err, 0, 256, s);
     if (e != cudaSuccess) return cuda_fail(e, "clearing the error word");
-    st = run_coarse(ix, queries, nq, nprobe, ws, L, nullptr, s);
+    st = run_coarse(ix, queries, nq, nprobe, ws, L, nullptr, false, s);
     if (st != RAGO_OK) return st;
     const size_t bytes = (size_t)nq * nprobe * 4;
     e = cudaMemcpyAsync(out_lists, ws + L.probe_list, bytes, cudaMemcpyDeviceToDevice, s);
@@ -414,7 +414,10 @@ rago_status rago_search(const rago_index* index, const float* queries, int32_t n
     IndexImpl* mix = const_cast<IndexImpl*>(ix);
     const int npairs = nq * nprobe;
 
-    cudaError_t e = cudaMemsetAsync(ws + L.err, 0, 256, s);
+    // The error block is cleared first: by the tiny-batch coarse kernel itself when that is the first kernel of the
+    // search (a memset between two searches would keep their launches from overlapping), else by a memset.
+    const bool kernel_clears = !L.tree_S && !L.tc && coarse_small_applies(ix, nq);
+    cudaError_t e = kernel_clears ? cudaSuccess : cudaMemsetAsync(ws + L.err, 0, 256, s);
     if (e != cudaSuccess) return cuda_fail(e, "clearing the error word");
     int32_t* probe_list = reinterpret_cast<int32_t*>(ws + L.probe_list);
     float* probe_term = reinterpret_cast<float*>(ws + L.probe_bias);  // what the scan adds per (query, list)
@@ -431,7 +434,7 @@ rago_status rago_search(const rago_index* index, const float* queries, int32_t n
     FusedPlan fp;
     const bool fused = fused_plan_args(ix, nq, npairs, queries, lut_img, lut_inv, work_prefix, qthresh, slot_cnt,
                                        (int)L.nslots, reinterpret_cast<uint32_t*>(ws + L.err) + ERR_TICKET_WORD, &fp);
-    st = run_coarse(ix, queries, nq, nprobe, ws, L, fused ? &fp : nullptr, s);
+    st = run_coarse(ix, queries, nq, nprobe, ws, L, fused ? &fp : nullptr, kernel_clears, s);
     if (st != RAGO_OK) return st;
     if (!fused) {
         e = launch_plan_work(ix, probe_list, npairs, ix->plan.tile_vecs, reinterpret_cast<int32_t*>(ws + L.pair_tiles),

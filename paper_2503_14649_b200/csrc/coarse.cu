@@ -117,10 +117,13 @@ constexpr int CS_CPW = 4;    // centroids per warp per step
 template <bool BF16, int NQ>
 __global__ void __launch_bounds__(256) coarse_small_kernel(const float* __restrict__ Q, const void* __restrict__ C,
                                                            const float* __restrict__ cnorm, int nq, int nlist, int d,
-                                                           int metric, float* __restrict__ scores) {
+                                                           int metric, float* __restrict__ scores, uint32_t* __restrict__ clear_block) {
     extern __shared__ __align__(16) float qs[];  // [nq][d], rounded to bf16 values for a bf16 index
     grid_dependency_wait();
     grid_dependents_may_launch();
+    // first kernel of a search: the workspace's 256-byte error block (error word, ticket) starts at zero; doing it
+    // here instead of in a memset of its own keeps two searches on one stream overlapping their launches
+    if (clear_block != nullptr && blockIdx.x == 0 && threadIdx.x < 64) clear_block[threadIdx.x] = 0u;
     {   // d is a multiple of 4 and Q 16-byte aligned; eight 16-byte loads in flight per thread
         const int n4 = (nq * d) >> 2;
         const float4* Q4 = reinterpret_cast<const float4*>(Q);
@@ -227,29 +230,35 @@ __global__ void __launch_bounds__(256) coarse_small_kernel(const float* __restri
 
 template <bool BF16>
 static void launch_coarse_small(const IndexImpl* ix, const float* queries, int nq, float* scores, int blocks, size_t qbytes,
-                                cudaStream_t s) {
+                                uint32_t* clear_block, cudaStream_t s) {
     if (nq == 1)
         launch_overlapped(coarse_small_kernel<BF16, 1>, dim3(blocks), dim3(256), qbytes, s, queries, ix->centroids, ix->cnorm,
-                          nq, ix->nlist, ix->d, ix->metric, scores);
+                          nq, ix->nlist, ix->d, ix->metric, scores, clear_block);
     else if (nq <= 4)
         launch_overlapped(coarse_small_kernel<BF16, 4>, dim3(blocks), dim3(256), qbytes, s, queries, ix->centroids, ix->cnorm,
-                          nq, ix->nlist, ix->d, ix->metric, scores);
+                          nq, ix->nlist, ix->d, ix->metric, scores, clear_block);
     else
         launch_overlapped(coarse_small_kernel<BF16, CS_MAXQ>, dim3(blocks), dim3(256), qbytes, s, queries, ix->centroids,
-                          ix->cnorm, nq, ix->nlist, ix->d, ix->metric, scores);
+                          ix->cnorm, nq, ix->nlist, ix->d, ix->metric, scores, clear_block);
 }
 
-cudaError_t launch_coarse_scores(const IndexImpl* ix, const float* queries, int nq, float* scores, cudaStream_t s) {
+bool coarse_small_applies(const IndexImpl* ix, int nq) { return nq <= CS_MAXQ && (size_t)nq * ix->d * 4 <= 48 * 1024; }
+
+// clear_block (may be null): 64 words the tiny-batch kernel zeroes before anything else of the search runs; only
+// valid when coarse_small_applies().
+cudaError_t launch_coarse_scores(const IndexImpl* ix, const float* queries, int nq, float* scores, uint32_t* clear_block,
+                                 cudaStream_t s) {
     const size_t qbytes = (size_t)nq * ix->d * 4;
-    if (nq <= CS_MAXQ && qbytes <= 48 * 1024) {
+    if (coarse_small_applies(ix, nq)) {
         const int want = (ix->nlist + 8 * CS_CPW - 1) / (8 * CS_CPW);  // 8 warps per CTA, CS_CPW rows per warp step
         const int cap = ix->num_sms * (nq <= 4 ? 4 : 2);
         const int blocks = want < cap ? want : cap;
-        if (ix->coarse_bf16) launch_coarse_small<true>(ix, queries, nq, scores, blocks, qbytes, s);
-        else launch_coarse_small<false>(ix, queries, nq, scores, blocks, qbytes, s);
+        if (ix->coarse_bf16) launch_coarse_small<true>(ix, queries, nq, scores, blocks, qbytes, clear_block, s);
+        else launch_coarse_small<false>(ix, queries, nq, scores, blocks, qbytes, clear_block, s);
         count_launch();
         return cudaGetLastError();
     }
+    if (clear_block != nullptr) return cudaErrorInvalidValue;
     dim3 grid((ix->nlist + BN - 1) / BN, (nq + BM - 1) / BM);
     if (ix->coarse_bf16)
         coarse_scores_kernel<true><<<grid, 256, 0, s>>>(queries, ix->centroids, ix->cnorm, nq, ix->nlist, ix->d,

@@ -207,7 +207,9 @@ void set_error(const char* fmt, ...);
 
 // coarse.cu
 cudaError_t launch_centroid_norms(const void* centroids, int bf16, int nlist, int d, float* cnorm, cudaStream_t s);
-cudaError_t launch_coarse_scores(const IndexImpl* ix, const float* queries, int nq, float* scores, cudaStream_t s);
+bool coarse_small_applies(const IndexImpl* ix, int nq);
+cudaError_t launch_coarse_scores(const IndexImpl* ix, const float* queries, int nq, float* scores, uint32_t* clear_block,
+                                 cudaStream_t s);
 cudaError_t launch_tree_candidates(const IndexImpl* ix, const float* queries, int nq, int S, int cap,
                                    unsigned long long* cand, int32_t* cand_cnt, cudaStream_t s);
 constexpr int TREE_LIMIT_B1 = 64, TREE_LIMIT_N1 = 4096;

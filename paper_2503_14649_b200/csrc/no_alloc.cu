@@ -84,7 +84,7 @@ extern "C" rago_status rago_search_probes_noalloc(const rago_index* index, const
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     // Nothing in the array has to start at zero: the first kernel writes every score the second one
     // reads, and the bias block is write-only here.
-    e = launch_coarse_scores(ix, queries, nq, scores, s);
+    e = launch_coarse_scores(ix, queries, nq, scores, nullptr, s);
     if (e == cudaSuccess)
         e = launch_select_probes(ix, queries, scores, nq, nprobe, out_lists, out_coarse, bias, nullptr, s);
     if (e != cudaSuccess) { set_error("coarse kernels: %s", cudaGetErrorString(e)); return RAGO_ECUDA; }
