@@ -165,7 +165,8 @@ static rago_status run_coarse(const IndexImpl* ix, const float* queries, int nq,
     if (L.tree_S) {
         unsigned long long* cand = reinterpret_cast<unsigned long long*>(ws + L.cand);
         int32_t* cand_cnt = reinterpret_cast<int32_t*>(ws + L.cand_cnt);
-        e = launch_tree_candidates(ix, queries, nq, L.tree_S, L.tree_cap, cand, cand_cnt, s);
+        e = launch_tree_candidates(ix, queries, nq, L.tree_S, L.tree_cap, cand, cand_cnt,
+                                   kernel_clears ? reinterpret_cast<uint32_t*>(ws + L.err) : nullptr, s);
         if (e != cudaSuccess) return cuda_fail(e, "two-level coarse kernel");
         record(mix, 1, s);
         e = launch_select_probes_cand(ix, queries, cand, cand_cnt, 0u, L.tree_S, L.tree_cap, nq, nprobe, probe_list,
@@ -414,9 +415,9 @@ rago_status rago_search(const rago_index* index, const float* queries, int32_t n
     IndexImpl* mix = const_cast<IndexImpl*>(ix);
     const int npairs = nq * nprobe;
 
-    // The error block is cleared first: by the tiny-batch coarse kernel itself when that is the first kernel of the
-    // search (a memset between two searches would keep their launches from overlapping), else by a memset.
-    const bool kernel_clears = !L.tree_S && !L.tc && coarse_small_applies(ix, nq);
+    // The error block is cleared first: by the tiny-batch coarse kernel or the two-level kernel itself when that is the first kernel
+    // of the search (a memset between two searches would keep their launches from overlapping), else by a memset.
+    const bool kernel_clears = L.tree_S ? true : (!L.tc && coarse_small_applies(ix, nq));
     cudaError_t e = kernel_clears ? cudaSuccess : cudaMemsetAsync(ws + L.err, 0, 256, s);
     if (e != cudaSuccess) return cuda_fail(e, "clearing the error word");
     int32_t* probe_list = reinterpret_cast<int32_t*>(ws + L.probe_list);

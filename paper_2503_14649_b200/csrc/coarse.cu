@@ -329,7 +329,7 @@ template <bool BF16>
 __global__ void __launch_bounds__(TREE_THREADS) tree_candidates_kernel(
     const float* __restrict__ Q, const void* __restrict__ C1, const int32_t* __restrict__ child_offsets, int n1, int b1,
     const void* __restrict__ C, const float* __restrict__ cnorm, int d, int metric, int cap,
-    unsigned long long* __restrict__ cand, int32_t* __restrict__ cand_cnt) {
+    unsigned long long* __restrict__ cand, int32_t* __restrict__ cand_cnt, uint32_t* __restrict__ clear_block) {
     extern __shared__ __align__(16) float tree_smem[];  // [d] query, [n1] level-1 keys as two words each
     float* qs = tree_smem;
     unsigned long long* k1 = reinterpret_cast<unsigned long long*>(tree_smem + ((d + 3) & ~3));  // (d * 4) % 16 == 0
@@ -341,6 +341,8 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_candidates_kernel(
     constexpr int NW = TREE_THREADS / 32;
     grid_dependency_wait();
     grid_dependents_may_launch();
+    // first kernel of a search: the workspace's error block starts at zero (see coarse_small_kernel)
+    if (clear_block != nullptr && blockIdx.x == 0 && blockIdx.y == 0 && tid < 64) clear_block[tid] = 0u;
     for (int i = tid; i < d; i += TREE_THREADS) qs[i] = BF16 ? round_bf16(Q[(size_t)q * d + i]) : Q[(size_t)q * d + i];
     __syncthreads();
     // first level: every node, direct form
@@ -421,17 +423,17 @@ __global__ void __launch_bounds__(TREE_THREADS) tree_candidates_kernel(
 }
 
 cudaError_t launch_tree_candidates(const IndexImpl* ix, const float* queries, int nq, int S, int cap,
-                                   unsigned long long* cand, int32_t* cand_cnt, cudaStream_t s) {
+                                   unsigned long long* cand, int32_t* cand_cnt, uint32_t* clear_block, cudaStream_t s) {
     const size_t smem = (size_t)((ix->d + 3) & ~3) * 4 + (size_t)ix->tree_n1 * 8;
     if (smem > 48 * 1024) return cudaErrorInvalidValue;
     if (ix->coarse_bf16)
         launch_overlapped(tree_candidates_kernel<true>, dim3(S, nq), dim3(TREE_THREADS), smem, s, queries, ix->tree_level1,
                           ix->tree_child_offsets, ix->tree_n1, ix->tree_b1, ix->centroids, ix->cnorm, ix->d, ix->metric,
-                          cap, cand, cand_cnt);
+                          cap, cand, cand_cnt, clear_block);
     else
         launch_overlapped(tree_candidates_kernel<false>, dim3(S, nq), dim3(TREE_THREADS), smem, s, queries, ix->tree_level1,
                           ix->tree_child_offsets, ix->tree_n1, ix->tree_b1, ix->centroids, ix->cnorm, ix->d, ix->metric,
-                          cap, cand, cand_cnt);
+                          cap, cand, cand_cnt, clear_block);
     count_launch();
     return cudaGetLastError();
 }

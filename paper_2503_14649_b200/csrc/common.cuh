@@ -211,7 +211,7 @@ bool coarse_small_applies(const IndexImpl* ix, int nq);
 cudaError_t launch_coarse_scores(const IndexImpl* ix, const float* queries, int nq, float* scores, uint32_t* clear_block,
                                  cudaStream_t s);
 cudaError_t launch_tree_candidates(const IndexImpl* ix, const float* queries, int nq, int S, int cap,
-                                   unsigned long long* cand, int32_t* cand_cnt, cudaStream_t s);
+                                   unsigned long long* cand, int32_t* cand_cnt, uint32_t* clear_block, cudaStream_t s);
 constexpr int TREE_LIMIT_B1 = 64, TREE_LIMIT_N1 = 4096;
 // gemm_select.cu
 constexpr int GEMM_CAP_SMALL = 512, GEMM_CAP_LARGE = 1024;  // candidate-list capacities (keys per list)
