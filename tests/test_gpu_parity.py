@@ -155,6 +155,23 @@ def test_iterative_small_batches_back_to_back():
     ix.close()
 
 
+SMALL_BATCH_PATHS = [
+    # nq, nprobe, k, metric: batch sizes on both sides of the fused selection + plan (<= 64 queries), of the tiny-batch
+    # coarse kernel (<= 16) and of its query groups (8), k on both sides of the one-warp cut (<= 32) and of the two
+    # register shapes of the small-batch merge ((CTAs + 1) k <= 4 096 / 16 384) and beyond them
+    (1, 40, 33, "l2"), (2, 16, 20, "l2"), (3, 4, 1, "ip"), (8, 16, 27, "ip"), (9, 16, 28, "l2"), (17, 8, 100, "ip"),
+    (33, 16, 150, "l2"), (64, 32, 27, "l2"), (65, 16, 20, "ip"),
+]
+
+
+@pytest.mark.parametrize("nq,nprobe,k,metric", SMALL_BATCH_PATHS)
+def test_small_batch_paths(nq, nprobe, k, metric):
+    """The latency path's kernels change shape with the batch size and k (fused planning, one-warp cuts, ranked
+    short buffers, the small-batch merge): every combination must give the oracle's answer."""
+    data = synth.make_ivfpq(60_000, 128, 96, 32, nq, metric=metric, seed=500 + nq + k, zipf=1.05)
+    _compare(data, nprobe, k, max_probe_mismatch=1)
+
+
 def test_results_do_not_depend_on_run():
     """The shared per-query threshold makes scheduling vary between runs; results must not."""
     data = synth.make_ivfpq(120_000, 192, 64, 96, 32, metric="l2", seed=8, zipf=1.1)
