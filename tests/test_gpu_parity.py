@@ -427,7 +427,8 @@ def test_64_byte_codes(case):
     _compare(data, nprobe, k, max_probe_mismatch=1)
 
 
-def test_thousands_of_identical_vectors_still_give_k_distinct_results():
+@pytest.mark.parametrize("k", [100, 10])  # the CTA-wide cut / the one-warp cut of small k
+def test_thousands_of_identical_vectors_still_give_k_distinct_results(k):
     """Every vector of the probed lists has the same code, so all scores tie: the buffer cuts and the merge must
     still return k distinct vectors of the right score, run after run."""
     data = synth.make_ivfpq(50_000, 64, 8, 64, 3, metric="l2", seed=77)
@@ -436,17 +437,17 @@ def test_thousands_of_identical_vectors_still_give_k_distinct_results():
     q = data.queries.cuda().contiguous()
     first = None
     for _ in range(3):
-        ids, dists = ix.rago_search(q, 4, 100)
+        ids, dists = ix.rago_search(q, 4, k)
         torch.cuda.synchronize()
         ix.rago_check()
         ids, dists = ids.cpu().numpy(), dists.cpu().numpy()
         for i in range(3):
-            assert len(set(ids[i].tolist())) == 100 and ids[i].min() >= 0
+            assert len(set(ids[i].tolist())) == k and ids[i].min() >= 0
             assert np.all(np.diff(dists[i]) >= 0)
         first = dists if first is None else first
         assert np.array_equal(first, dists)
     hix = host_index(oracle, data)
-    oi, od = oracle.ivfpq_search(hix, data.queries.numpy(), 4, 100)
+    oi, od = oracle.ivfpq_search(hix, data.queries.numpy(), 4, k)
     rs = IvfPqRescorer(oracle, hix)
     for i in range(3):
         assert not match_results(ids[i], dists[i], oi[i], od[i], rel=REL, rescore=rs.for_query(data.queries[i].numpy())), i
