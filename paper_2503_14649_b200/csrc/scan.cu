@@ -91,6 +91,8 @@ struct ScanArgs {
     const uint8_t* lut_img;  // [nq][LUT_BYTES] tables built ahead of the scan (small batches), or null
     const float* lut_inv;    // [nq] fp32 value of one integer unit of each such table
     int32_t npairs, nprobe, d, dsub, metric, k, stages;
+    int32_t stream_once;     // the batch is small: code tiles are fetched with an evict-first hint, so that the centroid
+                             // table the next search's coarse step reads stays in L2
     uint32_t dyn_bytes;
 };
 
@@ -430,6 +432,7 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
         };
         if (!few_pairs) fill();
         int cur = few_pairs ? first_pair : 0;
+        const uint64_t once_policy = l2_policy_evict_first();
         long long u = u_begin;
         bool dead = false;
         int issued = 0;
@@ -475,8 +478,13 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
                 const uint32_t vbytes = a.vterm ? (((pos0 & 3u) + (uint32_t)nvec) * 4u + 15u) & ~15u : 0u;
                 const uint32_t bar = smem_u32(&ctrl->full[st]);
                 mbar_arrive_expect_tx(bar, bytes + vbytes);
-                bulk_g2s(P.tile[st], a.codes + (size_t)pos0 * C::M, bytes, bar);
-                if (vbytes) bulk_g2s(P.vt[st], a.vterm + (pos0 & ~3u), vbytes, bar);
+                if (a.stream_once) {  // small batch: the codes are read once and should leave L2 first
+                    bulk_g2s_hint(P.tile[st], a.codes + (size_t)pos0 * C::M, bytes, bar, once_policy);
+                    if (vbytes) bulk_g2s_hint(P.vt[st], a.vterm + (pos0 & ~3u), vbytes, bar, once_policy);
+                } else {
+                    bulk_g2s(P.tile[st], a.codes + (size_t)pos0 * C::M, bytes, bar);
+                    if (vbytes) bulk_g2s(P.vt[st], a.vterm + (pos0 & ~3u), vbytes, bar);
+                }
                 // pull the tiles a few steps ahead in this list into L2, so that their copies find them there
                 for (int ahead = (t_in_pair == 0 ? 1 : SCAN_PF); ahead <= SCAN_PF; ++ahead) {
                     const long long vp = v0 + (long long)ahead * C::TV;
@@ -927,6 +935,7 @@ cudaError_t launch_scan(const IndexImpl* ix, const ScanPlan& plan, const float* 
     a.lut_img = lut_img; a.lut_inv = lut_inv;
     a.npairs = nq * nprobe; a.nprobe = nprobe; a.d = ix->d; a.dsub = ix->dsub;
     a.metric = ix->metric; a.k = k; a.stages = plan.stages; a.dyn_bytes = (uint32_t)plan.smem_bytes;
+    a.stream_once = nq <= 64 ? 1 : 0;
     const cudaError_t e = launch_overlapped(v->kernel, dim3(plan.ctas), dim3(v->threads), plan.smem_bytes, s, a);
     count_launch();
     return e != cudaSuccess ? e : cudaGetLastError();
