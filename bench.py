@@ -46,8 +46,8 @@ SECONDARY = ("mid", "flat", "coarse_hyper", "iter")
 # of codes; the capture-size rule) and carries over to the full size because the lists are uniform and no list is
 # shared through L2 at either size; "mid" was captured at full size and is not scaled to other sizes.
 SCAN_TRAFFIC = {
-    "hyper": {"scan_sha": "beb728b04673be65", "dram_per_logical": (15968936960 + 11397376) / 16004289600},   # 0.9985
-    "mid": {"scan_sha": "beb728b04673be65", "dram_per_logical": (34410413312 + 7730688) / 42427363200},      # 0.8112
+    "hyper": {"scan_sha": "9b3c1451afed23ae", "dram_per_logical": (15971139328 + 11699456) / 16004289600},   # 0.9987
+    "mid": {"scan_sha": "9b3c1451afed23ae", "dram_per_logical": (33890812160 + 7975936) / 42427363200},      # 0.7990
 }
 
 
