@@ -84,6 +84,7 @@ __device__ __forceinline__ void warp_bitonic_sort(unsigned long long* keys, int 
     __syncwarp();
 }
 constexpr int WARP_SORT_MAX = 64;
+constexpr int RANK_MAX = 256;      // block_select_short ranks up to this many keys (buffers of at least twice as many)
 // Ascending sort of one 32-bit value per lane across the warp (bitonic network on shuffles); lane L returns the
 // L-th smallest.
 __device__ __forceinline__ uint32_t warp_sort_u32(uint32_t v, int lane) {
@@ -109,8 +110,30 @@ __device__ __forceinline__ int block_select_short(unsigned long long* keys, int*
                                                   Sync sync, int cap = TOPK_CAP) {
     int n = *cnt;
     if (n > cap) n = cap;
-    if (n > WARP_SORT_MAX) return block_select(keys, cnt, k, tid, nthreads, sync, cap);
     const int kept = n < k ? n : k;
+    if (n > WARP_SORT_MAX) {
+        if (n > RANK_MAX || cap < 2 * RANK_MAX || nthreads < 256) return block_select(keys, cnt, k, tid, nthreads, sync, cap);
+        // Up to RANK_MAX keys are ranked too: a lane holds every 32nd key in registers, a warp takes the keys one
+        // after the other, counts the smaller ones with one compare per register and a warp-wide sum, and stores
+        // the key at its rank in the free part of the buffer; three barriers where the bitonic network has dozens.
+        const int warp = tid >> 5, lane = tid & 31, nwarps = nthreads >> 5;
+        unsigned long long a[RANK_MAX / 32];
+#pragma unroll
+        for (int j = 0; j < RANK_MAX / 32; ++j) a[j] = lane + 32 * j < n ? keys[lane + 32 * j] : KEY_MAX;
+        for (int i = warp; i < n; i += nwarps) {  // uniform within the warp
+            const unsigned long long x = keys[i];
+            uint32_t c = 0;
+#pragma unroll
+            for (int j = 0; j < RANK_MAX / 32; ++j) c += a[j] < x ? 1u : 0u;
+            c = __reduce_add_sync(0xffffffffu, c);
+            if (lane == 0 && (int)c < kept) keys[RANK_MAX + c] = x;  // keys [0, n) are only read here
+        }
+        sync();
+        for (int i = tid; i < kept; i += nthreads) keys[i] = keys[RANK_MAX + i];
+        if (tid == 0) *cnt = kept;
+        sync();
+        return kept;
+    }
     if (nthreads >= 256) {  // uniform
         constexpr int PER_WARP = WARP_SORT_MAX / 8;
         const int warp = tid >> 5, lane = tid & 31, nwarps = nthreads >> 5;
