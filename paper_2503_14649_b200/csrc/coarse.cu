@@ -489,9 +489,12 @@ __global__ void __launch_bounds__(SEL_THREADS) select_probes_kernel(
     for (int i = tid; i < 256; i += SEL_THREADS) hist[i] = 0u;
     const float* srow = FROM_SCORES ? scores + (size_t)q * nlist : nullptr;
     if (!FROM_SCORES) {  // the valid entries of the query's lists, numbered consecutively
+        // the counts are fetched side by side (one thread reading them in turn paid a global round trip per list)
+        for (int sp = tid; sp < nsplit; sp += SEL_THREADS) pre[sp + 1] = cand_cnt[(size_t)q * nsplit + sp];
+        __syncthreads();
         if (tid == 0) {
             int acc = 0;
-            for (int sp = 0; sp < nsplit; ++sp) { pre[sp] = acc; acc += cand_cnt[(size_t)q * nsplit + sp]; }
+            for (int sp = 0; sp < nsplit; ++sp) { const int c = pre[sp + 1]; pre[sp] = acc; acc += c; }
             pre[nsplit] = acc;
         }
     }
