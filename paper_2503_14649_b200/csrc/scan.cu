@@ -202,6 +202,7 @@ struct Ctrl {
     unsigned long long full[MAX_STAGES];
     unsigned long long empty[MAX_STAGES];
     unsigned long long cbar;  // consumer barrier
+    unsigned long long lutbar;  // a prebuilt table has landed
     TileDesc desc[MAX_STAGES];
     int cnt;
     uint32_t abort_flag;
@@ -364,6 +365,7 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
             mbar_init(smem_u32(&ctrl->empty[s]), NCW);
         }
         mbar_init(smem_u32(&ctrl->cbar), NCW);
+        mbar_init(smem_u32(&ctrl->lutbar), 1);
         ctrl->cnt = 0;
         ctrl->abort_flag = 0;
         fence_barrier_init();
@@ -508,7 +510,7 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
 
     // ================= consumer warps =================
     const int ctid = tid;  // 0 .. NCT-1
-    uint32_t cphase = 0;
+    uint32_t cphase = 0, lphase = 0;
     bool dead = false;
     auto csync = [&]() {
         if (dead) return;
@@ -720,13 +722,24 @@ __global__ void __launch_bounds__(Cfg<WV, G, R, NCW_, RGW_>::THREADS, 1) scan_ke
         cur_q = q;
         early = k <= 32;
         if (a.lut_img != nullptr) {  // the table was built ahead of the scan: fetch its shared-memory image
-            const uint4* src = reinterpret_cast<const uint4*>(a.lut_img + (size_t)q * C::LUT_BYTES);
-            uint4* dst = reinterpret_cast<uint4*>(smem + (P.lut - base));
-#pragma unroll 4
-            for (int i = ctid; i < C::LUT_BYTES / 16; i += NCT) dst[i] = __ldg(src + i);
+            // One thread asks the copy engine for the image (bulk copies, completion counted on a barrier): the 64 or
+            // 128 KB arrive at the rate of the L2 -> shared-memory path instead of a few 16-byte loads per thread
+            // and round trip.  Every consumer is past its last look-up in the old table (the barrier that ended the
+            // previous query); the fence orders those reads before the copies' writes.
+            if (ctid == 0) {
+                ctrl->cnt = 0;
+                fence_proxy_async();
+                const uint8_t* src = a.lut_img + (size_t)q * C::LUT_BYTES;
+                const uint32_t bar = smem_u32(&ctrl->lutbar);
+                mbar_arrive_expect_tx(bar, (uint32_t)C::LUT_BYTES);
+                constexpr uint32_t PIECE = 32768;
+                for (uint32_t o = 0; o < (uint32_t)C::LUT_BYTES; o += PIECE)
+                    bulk_g2s(P.lut + o, src + o, (uint32_t)C::LUT_BYTES - o < PIECE ? (uint32_t)C::LUT_BYTES - o : PIECE, bar);
+            }
             inv_scale = __ldg(a.lut_inv + q);
-            if (ctid == 0) ctrl->cnt = 0;
             tau = *reinterpret_cast<volatile unsigned long long*>(&a.qthresh[q]);
+            dead = dead || !mbar_wait(smem_u32(&ctrl->lutbar), lphase, abort_flag, a.err);
+            lphase ^= 1u;
             csync();
             return;
         }
