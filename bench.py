@@ -46,8 +46,8 @@ SECONDARY = ("mid", "flat", "coarse_hyper", "iter")
 # of codes; the capture-size rule) and carries over to the full size because the lists are uniform and no list is
 # shared through L2 at either size; "mid" was captured at full size and is not scaled to other sizes.
 SCAN_TRAFFIC = {
-    "hyper": {"scan_sha": "9b3c1451afed23ae", "dram_per_logical": (15971139328 + 11699456) / 16004289600},   # 0.9987
-    "mid": {"scan_sha": "9b3c1451afed23ae", "dram_per_logical": (33890812160 + 7975936) / 42427363200},      # 0.7990
+    "hyper": {"scan_sha": "90e01c4ea3d00589", "dram_per_logical": (15956357120 + 11520000) / 16004289600},   # 0.9977
+    "mid": {"scan_sha": "90e01c4ea3d00589", "dram_per_logical": (34071503872 + 9443072) / 42427363200},      # 0.8033
 }
 
 
